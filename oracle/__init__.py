@@ -1,0 +1,159 @@
+"""ctypes front end of the CPU oracle (``spec_oracle.c``).
+
+Test infrastructure only: the tests, the smoke check and the bench's CPU legs load it; the
+product package never does.  Inputs are CPU torch tensors (bf16 for Q/K/V, int32 for lengths
+and indices); results come back as fp64 (attention, statistic) or int32 (indices) tensors.
+
+A KV cache is described by any object with the attributes ``k, v`` (bf16 CPU tensors that own
+the storage), ``layer_stride, page_stride, head_stride, slot_stride`` (in elements),
+``n_layers, page_size, page_table`` (int32 CPU tensor ``[batch, max_pages]`` or ``None``),
+``max_pages, batch, n_q_heads, n_kv_heads, head_dim, sm_scale``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "spec_oracle.c")
+_LIB = os.path.join(_HERE, "libspec_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over the independent (layer, batch, KV head) problems)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        )
+    return _LIB
+
+
+class _KV(ctypes.Structure):
+    _fields_ = [
+        ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("layer_stride", ctypes.c_int64), ("page_stride", ctypes.c_int64),
+        ("head_stride", ctypes.c_int64), ("slot_stride", ctypes.c_int64),
+        ("n_layers", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("page_table", ctypes.c_void_p),
+        ("max_pages", ctypes.c_int32), ("batch", ctypes.c_int32),
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("sm_scale", ctypes.c_double),
+    ]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_threads.restype = ctypes.c_int
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle will use."""
+    return int(_load().oracle_threads())
+
+
+def _cpu(t: torch.Tensor, dtype) -> torch.Tensor:
+    assert t.device.type == "cpu" and t.dtype == dtype, (t.device, t.dtype, dtype)
+    assert t.is_contiguous()
+    return t
+
+
+def _kv_struct(kv):
+    k = _cpu(kv.k, torch.bfloat16)
+    v = _cpu(kv.v, torch.bfloat16)
+    pt = None
+    if kv.page_table is not None:
+        pt = _cpu(kv.page_table, torch.int32)
+    s = _KV(
+        k.data_ptr(), v.data_ptr(), kv.layer_stride, kv.page_stride, kv.head_stride,
+        kv.slot_stride, kv.n_layers, kv.page_size, pt.data_ptr() if pt is not None else None,
+        kv.max_pages, kv.batch, kv.n_q_heads, kv.n_kv_heads, kv.head_dim,
+        float(kv.sm_scale or 0.0),
+    )
+    return s, (k, v, pt)
+
+
+def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None):
+    """Full-context verification attention and the Eq. 3 statistic.
+
+    Returns ``(out fp64 [L,B,n_q,Hq,D], lse fp64 [L,B,n_q,Hq], stats fp64 [L,B,Hkv,stat_stride])``.
+    """
+    lib = _load()
+    s, keep = _kv_struct(kv)
+    q = _cpu(q, torch.bfloat16)
+    ctx_len = _cpu(ctx_len, torch.int32)
+    L, B, n_q, Hq, D = q.shape
+    assert (L, B, Hq, D) == (kv.n_layers, kv.batch, kv.n_q_heads, kv.head_dim)
+    if stat_stride is None:
+        stat_stride = int(ctx_len.max())
+    out = torch.zeros(L, B, n_q, Hq, D, dtype=torch.float64)
+    lse = torch.zeros(L, B, n_q, Hq, dtype=torch.float64)
+    stats = torch.zeros(L, B, kv.n_kv_heads, stat_stride, dtype=torch.float64)
+    rc = lib.oracle_verify_attn(
+        ctypes.byref(s), ctypes.c_void_p(q.data_ptr()), ctypes.c_int(n_q),
+        ctypes.c_void_p(ctx_len.data_ptr()), ctypes.c_int(stat_window),
+        ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stat_stride),
+    )
+    if rc != 0:
+        raise ValueError("oracle_verify_attn: invalid arguments")
+    del keep
+    return out, lse, stats
+
+
+def select_recall(stats, sel_len, k_sink, k_recent, k_total):
+    """Eq. 4 index set from fp32 scores ``[L,B,Hkv,stat_stride]``.
+
+    Returns ``(indices int32 [L,B,Hkv,k_total] ascending padded with -1, n_idx int32 [L,B,Hkv])``.
+    """
+    lib = _load()
+    stats = _cpu(stats, torch.float32)
+    sel_len = _cpu(sel_len, torch.int32)
+    L, B, Hkv, stride = stats.shape
+    indices = torch.full((L, B, Hkv, k_total), -7, dtype=torch.int32)
+    n_idx = torch.zeros(L, B, Hkv, dtype=torch.int32)
+    rc = lib.oracle_select_recall(
+        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stride), ctypes.c_int(L),
+        ctypes.c_int(B), ctypes.c_int(Hkv), ctypes.c_void_p(sel_len.data_ptr()),
+        ctypes.c_int(k_sink), ctypes.c_int(k_recent), ctypes.c_int(k_total),
+        ctypes.c_void_p(indices.data_ptr()), ctypes.c_void_p(n_idx.data_ptr()),
+    )
+    if rc != 0:
+        raise ValueError("oracle_select_recall: invalid arguments")
+    return indices, n_idx
+
+
+def sparse_draft_attn(kv, q, indices, n_idx, tail_start, cur_len):
+    """Eq. 5 sparse attention of one drafting query per sequence.
+
+    Returns ``(out fp64 [L,B,Hq,D], lse fp64 [L,B,Hq])``.
+    """
+    lib = _load()
+    s, keep = _kv_struct(kv)
+    q = _cpu(q, torch.bfloat16)
+    indices = _cpu(indices, torch.int32)
+    n_idx = _cpu(n_idx, torch.int32)
+    tail_start = _cpu(tail_start, torch.int32)
+    cur_len = _cpu(cur_len, torch.int32)
+    L, B, Hq, D = q.shape
+    assert (L, B, Hq, D) == (kv.n_layers, kv.batch, kv.n_q_heads, kv.head_dim)
+    k_total = indices.shape[-1]
+    out = torch.zeros(L, B, Hq, D, dtype=torch.float64)
+    lse = torch.zeros(L, B, Hq, dtype=torch.float64)
+    rc = lib.oracle_sparse_draft_attn(
+        ctypes.byref(s), ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(indices.data_ptr()),
+        ctypes.c_void_p(n_idx.data_ptr()), ctypes.c_int(k_total),
+        ctypes.c_void_p(tail_start.data_ptr()), ctypes.c_void_p(cur_len.data_ptr()),
+        ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+    )
+    if rc != 0:
+        raise ValueError("oracle_sparse_draft_attn: invalid arguments")
+    del keep
+    return out, lse

@@ -1,0 +1,276 @@
+"""Pins of the CPU oracle against things other than itself: a library fp64 softmax
+attention, closed forms, limits, brute force, and structural invariants."""
+import math
+
+import pytest
+import torch
+
+import oracle
+from paper_2607_27735_b200 import inputs
+from conftest import dense_rows
+
+
+def torch_verify_reference(case, stat_window=16):
+    """softmax(Q K^T * scale + causal mask) V with torch fp64 ops, one (l, b, h, g) at a time."""
+    kv, cfg = case.kv, case.cfg
+    L, B, n_q, Hq, D = case.q_verify.shape
+    G = Hq // kv.n_kv_heads
+    W = min(stat_window, n_q)
+    smax = int(case.ctx_len.max())
+    out = torch.zeros(L, B, n_q, Hq, D, dtype=torch.float64)
+    lse = torch.zeros(L, B, n_q, Hq, dtype=torch.float64)
+    stats = torch.zeros(L, B, kv.n_kv_heads, smax, dtype=torch.float64)
+    for l in range(L):
+        for b in range(B):
+            T = int(case.ctx_len[b])
+            for h in range(kv.n_kv_heads):
+                K = dense_rows(kv, kv.k, l, b, h, range(T))
+                V = dense_rows(kv, kv.v, l, b, h, range(T))
+                for g in range(G):
+                    q = case.q_verify[l, b, :, h * G + g].to(torch.float64)  # [n_q, D]
+                    s = q @ K.T / math.sqrt(D)
+                    row_pos = torch.arange(T - n_q, T)[:, None]
+                    s = s.masked_fill(torch.arange(T)[None, :] > row_pos, float("-inf"))
+                    p = torch.softmax(s, dim=-1)
+                    out[l, b, :, h * G + g] = p @ V
+                    lse[l, b, :, h * G + g] = torch.logsumexp(s, dim=-1)
+                    stats[l, b, h, :T] += p[n_q - W:].sum(0)
+    return out, lse, stats
+
+
+SHAPES = [
+    dict(n_q_heads=4, n_kv_heads=4, head_dim=64, ctx=(37, 37), n_q=1),
+    dict(n_q_heads=8, n_kv_heads=2, head_dim=64, ctx=(130, 130), n_q=5),
+    dict(n_q_heads=10, n_kv_heads=2, head_dim=128, ctx=(65, 65), n_q=17),
+    dict(n_q_heads=8, n_kv_heads=2, head_dim=128, ctx=(40, 90), n_q=3, batch=3, page_size=16,
+         shuffled_pages=True, n_layers=2),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_verify_matches_library_softmax_attention(shape):
+    cfg = inputs.small_config(planted=3, **shape)
+    case = inputs.make_case(cfg)
+    out, lse, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len)
+    ro, rl, rs = torch_verify_reference(case)
+    assert (out - ro).abs().max() < 1e-12
+    assert (lse - rl).abs().max() < 1e-12
+    assert (stats - rs).abs().max() < 1e-12
+
+
+@pytest.mark.parametrize("n_q,window", [(1, 16), (5, 16), (17, 16), (9, 4)])
+def test_statistic_mass_is_group_times_window_rows(n_q, window):
+    cfg = inputs.small_config(n_q=n_q, ctx=(300, 300), n_q_heads=8, n_kv_heads=2)
+    case = inputs.make_case(cfg)
+    _, _, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, stat_window=window)
+    expect = cfg.group * min(window, n_q)
+    assert (stats.sum(-1) - expect).abs().max() < 1e-9
+    assert stats.min() >= 0.0
+
+
+def test_identical_keys_closed_form():
+    """All keys equal: p = 1/(pos+1), O = running mean of V, statistic = G * sum of 1/(pos_j+1)
+    over the window rows that can see the key.  Pins mask alignment, window rule, GQA sum."""
+    cfg = inputs.small_config(n_q=17, ctx=(50, 50), n_q_heads=6, n_kv_heads=2, head_dim=64,
+                              planted=0)
+    case = inputs.make_case(cfg)
+    kv = case.kv
+    kv.k[:] = kv.k.reshape(-1, 64)[0]  # one key row everywhere
+    out, lse, stats = oracle.verify_attn(kv, case.q_verify, case.ctx_len, stat_window=16)
+    T, n_q, G = 50, 17, 3
+    for h in range(2):
+        V = dense_rows(kv, kv.v, 0, 0, h, range(T))
+        for j in range(n_q):
+            pos = T - n_q + j
+            mean_v = V[: pos + 1].mean(0)
+            for g in range(G):
+                assert (out[0, 0, j, h * G + g] - mean_v).abs().max() < 1e-12
+        expect = torch.zeros(T, dtype=torch.float64)
+        for j in range(1, n_q):  # W=16 of 17 rows: row 0 is outside the window
+            pos = T - n_q + j
+            expect[: pos + 1] += G / (pos + 1)
+        assert (stats[0, 0, h, :T] - expect).abs().max() < 1e-12
+
+
+def test_golden_three_token_example():
+    """tests/golden/identical_keys_T3.txt: hand-computed case (T=3, n_q=2, G=1, identical keys)."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "identical_keys_T3.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    golden = {r[0]: [float(x) for x in r[1:]] for r in rows}
+    cfg = inputs.small_config(n_q=2, ctx=(3, 3), n_q_heads=1, n_kv_heads=1, head_dim=64, planted=0,
+                              draft_steps=0)
+    case = inputs.make_case(cfg)
+    kv = case.kv
+    kv.k[:] = 0.5
+    kv.v[:] = 0
+    for i, val in enumerate(golden["v"]):
+        kv.v[0, 0, 0, i, :] = val
+    out, _, stats = oracle.verify_attn(kv, case.q_verify, case.ctx_len)
+    assert torch.allclose(stats[0, 0, 0, :3], torch.tensor(golden["stats"], dtype=torch.float64),
+                          atol=1e-12)
+    assert torch.allclose(out[0, 0, :, 0, 0], torch.tensor(golden["out"], dtype=torch.float64),
+                          atol=1e-12)
+
+
+def test_one_hot_limit():
+    """A key equal to 50x the (unit) query direction takes all the mass."""
+    cfg = inputs.small_config(n_q=4, ctx=(200, 200), n_q_heads=4, n_kv_heads=1, head_dim=64,
+                              planted=0)
+    case = inputs.make_case(cfg)
+    kv = case.kv
+    qdir = case.direction[0, 0, 0]
+    hot = 77
+    kv.k[0, 0, 0, hot] = (50.0 * qdir / qdir.norm() * math.sqrt(64.0)).to(torch.bfloat16)
+    out, _, stats = oracle.verify_attn(kv, case.q_verify, case.ctx_len)
+    v_hot = kv.v[0, 0, 0, hot].to(torch.float64)
+    assert (out[0, 0] - v_hot).abs().max() < 1e-6
+    assert abs(float(stats[0, 0, 0, hot]) - 16.0) < 1e-6  # R = n_q * G rows
+
+
+def test_prefix_permutation_invariance():
+    """Permuting (K, V) rows that every window row can see permutes the statistic, keeps O."""
+    cfg = inputs.small_config(n_q=3, ctx=(90, 90), head_dim=64)
+    case = inputs.make_case(cfg)
+    out, _, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len)
+    T, n_q = 90, 3
+    perm = torch.randperm(T - n_q, generator=torch.Generator().manual_seed(1))
+    kv = case.kv
+    k2, v2 = kv.k.clone(), kv.v.clone()
+    k2[0, 0, :, : T - n_q] = kv.k[0, 0, :, perm]
+    v2[0, 0, :, : T - n_q] = kv.v[0, 0, :, perm]
+    import dataclasses
+    kvp = dataclasses.replace(kv, k=k2, v=v2)
+    out2, _, stats2 = oracle.verify_attn(kvp, case.q_verify, case.ctx_len)
+    assert (out - out2).abs().max() < 1e-12
+    assert (stats[..., perm] - stats2[..., : T - n_q]).abs().max() < 1e-12
+
+
+# ---------------------------------------------------------------------------------------------
+# select
+
+
+def brute_select(st, T, k_sink, k_recent, k_total):
+    if T <= k_total:
+        return list(range(T))
+    cand = list(range(k_sink, T - k_recent))
+    cand.sort(key=lambda i: (-float(st[i]), i))
+    chosen = cand[: k_total - k_sink - k_recent]
+    return sorted(list(range(k_sink)) + chosen + list(range(T - k_recent, T)))
+
+
+@pytest.mark.parametrize("T,k_sink,k_recent,k_total", [
+    (64, 4, 8, 24), (64, 0, 0, 10), (20, 4, 8, 24), (24, 4, 8, 24), (25, 4, 8, 24),
+    (300, 4, 64, 68), (300, 4, 64, 100), (13, 13, 0, 13), (40, 5, 5, 10),
+])
+def test_select_brute_force_with_ties(T, k_sink, k_recent, k_total):
+    g = torch.Generator().manual_seed(T * 31 + k_total)
+    # few distinct values: many exact ties, including across the selection threshold
+    stats = (torch.randint(0, 5, (2, 2, 3, T + 7), generator=g).float()) * 0.25
+    sel_len = torch.tensor([T, max(1, T - 3)], dtype=torch.int32)
+    idx, n = oracle.select_recall(stats, sel_len, k_sink, k_recent, k_total)
+    for l in range(2):
+        for b in range(2):
+            for h in range(3):
+                want = brute_select(stats[l, b, h], int(sel_len[b]), k_sink, k_recent, k_total)
+                got = idx[l, b, h, : int(n[l, b, h])].tolist()
+                assert got == want
+                assert int(n[l, b, h]) == min(k_total, int(sel_len[b]))
+                assert (idx[l, b, h, int(n[l, b, h]):] == -1).all()
+
+
+def test_select_all_equal_scores_takes_lowest_positions():
+    stats = torch.ones(1, 1, 1, 100)
+    idx, n = oracle.select_recall(stats, torch.tensor([100], dtype=torch.int32), 2, 3, 15)
+    assert idx[0, 0, 0].tolist() == list(range(0, 12)) + [97, 98, 99]
+
+
+def test_select_set_matches_torch_topk_on_distinct_values():
+    g = torch.Generator().manual_seed(5)
+    T, k_sink, k_recent, k_total = 5000, 4, 64, 512
+    stats = torch.rand(1, 2, 4, T, generator=g)
+    idx, n = oracle.select_recall(stats, torch.tensor([T, T], dtype=torch.int32), k_sink,
+                                  k_recent, k_total)
+    k_mid = k_total - k_sink - k_recent
+    for b in range(2):
+        for h in range(4):
+            mid = stats[0, b, h, k_sink:T - k_recent]
+            top = (mid.topk(k_mid).indices + k_sink).sort().values
+            got = idx[0, b, h]
+            assert got[:k_sink].tolist() == list(range(k_sink))
+            assert got[-k_recent:].tolist() == list(range(T - k_recent, T))
+            assert torch.equal(got[k_sink:-k_recent].long(), top)
+            assert len(set(got.tolist())) == k_total  # no duplicates: sink/recent are excluded
+
+
+# ---------------------------------------------------------------------------------------------
+# draft
+
+
+def test_draft_matches_library_softmax_on_explicit_subset():
+    cfg = inputs.small_config(ctx=(300, 300), n_q=2, draft_steps=3, batch=2, n_layers=2,
+                              page_size=16, shuffled_pages=True)
+    case = inputs.make_case(cfg)
+    kv = case.kv
+    g = torch.Generator().manual_seed(9)
+    k_total = 40
+    idx = torch.full((2, 2, 2, k_total), -1, dtype=torch.int32)
+    n_idx = torch.zeros(2, 2, 2, dtype=torch.int32)
+    tail_start = torch.tensor([290, 300], dtype=torch.int32)
+    cur_len = torch.tensor([293, 300], dtype=torch.int32)  # second sequence: empty tail
+    for l in range(2):
+        for b in range(2):
+            for h in range(2):
+                n = int(torch.randint(1, k_total + 1, (1,), generator=g))
+                sel = torch.randperm(int(tail_start[b]), generator=g)[:n].sort().values
+                idx[l, b, h, :n] = sel.int()
+                n_idx[l, b, h] = n
+    q = case.q_draft[0]
+    out, lse = oracle.sparse_draft_attn(kv, q, idx, n_idx, tail_start, cur_len)
+    G = cfg.group
+    for l in range(2):
+        for b in range(2):
+            for h in range(2):
+                keys = idx[l, b, h, : int(n_idx[l, b, h])].tolist() + list(
+                    range(int(tail_start[b]), int(cur_len[b])))
+                K = dense_rows(kv, kv.k, l, b, h, keys)
+                V = dense_rows(kv, kv.v, l, b, h, keys)
+                for gg in range(G):
+                    qq = q[l, b, h * G + gg].to(torch.float64)
+                    s = K @ qq / math.sqrt(cfg.head_dim)
+                    p = torch.softmax(s, 0)
+                    assert (out[l, b, h * G + gg] - p @ V).abs().max() < 1e-12
+                    assert abs(float(lse[l, b, h * G + gg] - torch.logsumexp(s, 0))) < 1e-12
+
+
+def test_budget_at_least_context_reduces_draft_to_dense_attention():
+    """select with k_total >= T' keeps 0..T'-1, and the draft then equals verification with
+    n_q = 1 on the same cache (the query being the last cached position)."""
+    cfg = inputs.small_config(ctx=(150, 150), n_q=1, draft_steps=1, head_dim=64)
+    case = inputs.make_case(cfg)
+    T = 150
+    stats = torch.rand(1, 1, 2, T)
+    idx, n = oracle.select_recall(stats, torch.tensor([T - 1], dtype=torch.int32), 4, 16, 256)
+    assert idx[0, 0, 0, : T - 1].tolist() == list(range(T - 1)) and int(n[0, 0, 0]) == T - 1
+    q1 = case.q_verify[:, :, 0]  # [L, B, Hq, D]
+    d_out, d_lse = oracle.sparse_draft_attn(
+        case.kv, q1, idx, n, torch.tensor([T - 1], dtype=torch.int32),
+        torch.tensor([T], dtype=torch.int32))
+    v_out, v_lse, _ = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len)
+    assert (d_out - v_out[:, :, 0]).abs().max() < 1e-12
+    assert (d_lse - v_lse[:, :, 0]).abs().max() < 1e-12
+
+
+def test_planted_heavy_hitters_are_recalled():
+    """Tiny baseline workload: every planted position outside sink/recent lands in the index
+    set and the planted set carries most of the window's attention mass."""
+    cfg = inputs.baseline_configs()["cfg1_tiny"]
+    case = inputs.make_case(cfg)
+    _, _, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len)
+    idx, _ = oracle.select_recall(stats.float(), case.ctx_len, cfg.k_sink, cfg.k_recent,
+                                  cfg.k_total)
+    for h in range(cfg.n_kv_heads):
+        chosen = set(idx[0, 0, h].tolist())
+        planted = case.planted_pos[0, 0, h].tolist()
+        assert all(p in chosen for p in planted)
+        assert stats[0, 0, h][planted].sum() / stats[0, 0, h].sum() > 0.5
