@@ -1,0 +1,187 @@
+/*
+ * spec_attn.h - C ABI of the B200 (sm_100a) attention hot path of SparseSpec-L
+ * train-free self-speculative decoding.
+ *
+ * One decode iteration of the method drafts k tokens with sparse attention over a
+ * recallable subset of the KV cache and then verifies them in one dense pass
+ * ("Sparse Drafting Stage" / "Full Verification Stage", Sec. 3.1).  This library holds the
+ * three data-parallel attention-side steps of that iteration:
+ *
+ *   spec_verify_attn        dense verification attention of the k+1 speculated rows over the
+ *                           whole cache, with the importance score of Eq. 3 produced in the
+ *                           same pass;
+ *   spec_select_recall      the index set of Eq. 4 (sink + TopK over the middle span + recent);
+ *   spec_sparse_draft_attn  attention over Gather(K, I), Gather(V, I) of Eq. 5, the gather
+ *                           fused into the attention (the gathered copies are never
+ *                           materialised), plus the dense tail of tokens drafted this round.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless it says "host".  The caller owns every buffer,
+ *     including the workspace; the library allocates no device memory, never frees anything
+ *     and never writes K or V (the dense cache stays resident, Sec. 3.2).
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and return without synchronising.  Lengths live in device arrays.
+ *   - Return value: 0 on success, a negative SPEC_ERR_* decided on the host BEFORE anything
+ *     is launched.  Device-side anomalies (an out-of-range recall index, a bounded wait that
+ *     ran out) set a status word at the head of the workspace and the kernel exits cleanly;
+ *     read it with spec_read_status().
+ *   - Positions are 0-based (the paper counts from 1).  bf16 inputs, fp32 accumulation and
+ *     fp32 outputs.
+ *   - GQA: query head hq reads KV head hq / (n_q_heads / n_kv_heads); the Eq. 3 score is kept
+ *     per KV head, summed over the query heads that share it.
+ *   - "problem" = one (layer, sequence, KV head); n_layers > 1 folds independent layers that
+ *     share shapes into one launch.
+ */
+#ifndef SPEC_ATTN_H_
+#define SPEC_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    SPEC_OK = 0,
+    SPEC_ERR_INVALID_ARG = -1,         /* null pointer, negative size, inconsistent fields */
+    SPEC_ERR_UNSUPPORTED_SHAPE = -2,   /* head_dim not 64/128, too many rows per KV head, ... */
+    SPEC_ERR_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < spec_workspace_bytes(...) */
+    SPEC_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed at launch time */
+    SPEC_ERR_TIMEOUT = -5,             /* status word: a bounded device-side wait ran out */
+    SPEC_ERR_BAD_INDEX = -6            /* status word: a recall index was out of range */
+};
+
+/* Which entry point a workspace is sized for. */
+enum { SPEC_WS_VERIFY = 0, SPEC_WS_SELECT = 1, SPEC_WS_DRAFT = 2 };
+
+/* Verification kernel choice for spec_set_verify_impl(). */
+enum { SPEC_VERIFY_AUTO = 0, SPEC_VERIFY_GENERIC = 1, SPEC_VERIFY_TCGEN05 = 2 };
+
+/*
+ * Dense KV cache of one or more layers (the K_{l,h}, V_{l,h} of Eq. 5), READ-ONLY.
+ * Element (layer, b, pos, h, d) of K lives at
+ *     k + layer*layer_stride + phys*page_stride + h*head_stride + slot*slot_stride + d
+ * with page = pos / page_size, slot = pos % page_size and
+ *     phys = page_table ? page_table[b*max_pages + page] : b*max_pages + page.
+ * Strides are in elements; d is contiguous; every stride must be a multiple of 8 elements and
+ * k, v 16-byte aligned.  A contiguous per-sequence cache is the case max_pages == 1.
+ */
+typedef struct {
+    const void* k;                 /* bf16 */
+    const void* v;                 /* bf16 */
+    int64_t layer_stride, page_stride, head_stride, slot_stride;
+    int32_t n_layers;              /* >= 1 */
+    int32_t page_size;             /* tokens per page, >= 1 */
+    const int32_t* page_table;     /* device int32 [batch, max_pages] or NULL */
+    int32_t max_pages, batch, n_q_heads, n_kv_heads;
+    int32_t head_dim;              /* 64 or 128 */
+    float sm_scale;                /* softmax scale; <= 0 means 1/sqrt(head_dim) */
+} spec_kv_t;
+
+/*
+ * Full-context verification attention + importance score (Sec. 3.1 "Full Verification
+ * Stage"; Eq. 3).
+ *
+ * Row j (0 <= j < n_q) of sequence b sits at position ctx_len[b]-n_q+j and attends keys
+ * 0..that position of the whole dense cache (causal inside the window).  out = softmax(q K^T *
+ * sm_scale) V.  stats[layer,b,h,i] = sum over the last min(stat_window, n_q) rows j and over
+ * the query heads of KV head h of the attention probability row j gives key i (0 where
+ * masked).  Probabilities use the global softmax normaliser, so each contributing row adds
+ * exactly 1 to the sum of stats over i.
+ *
+ *   q        bf16 [n_layers, batch, n_q, n_q_heads, head_dim]
+ *   n_q      k+1, 1..32, with n_q * (n_q_heads/n_kv_heads) <= 128
+ *   ctx_len  int32 [batch], each n_q <= ctx_len[b] <= max_ctx_len; INCLUDES the n_q rows, whose
+ *            K/V are already in the cache
+ *   max_ctx_len  host upper bound of ctx_len (sizes the launch)
+ *   stat_window  W of Eq. 3; 0 means 16
+ *   out      fp32 [n_layers, batch, n_q, n_q_heads, head_dim]
+ *   lse      fp32 [n_layers, batch, n_q, n_q_heads] (natural-log softmax denominator) or NULL
+ *   stats    fp32 [n_layers, batch, n_kv_heads, stat_stride]; entries [0, ctx_len[b]) are
+ *            written, the rest left untouched; stat_stride >= max_ctx_len
+ *   workspace  >= spec_workspace_bytes(SPEC_WS_VERIFY, ...) bytes, 256-byte aligned, contents
+ *            need not be initialised; must not be shared by calls that may overlap on the GPU
+ */
+int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                     int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
+                     float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,
+                     void* cuda_stream);
+
+/*
+ * Recall selection (Eq. 4).  For each problem with T' = sel_len[b]:
+ *   T' <= k_total : indices = 0..T'-1, n = T'.
+ *   otherwise     : sink [0,k_sink) U the k_mid = k_total-k_sink-k_recent positions of
+ *                   [k_sink, T'-k_recent) with the largest stats (equal stats: the lower
+ *                   position wins) U recent [T'-k_recent, T'); n = k_total.
+ * Output ascending, padded with -1.  stats must be finite and >= 0 (they are sums of
+ * probabilities), which makes the fp32 bit pattern order-isomorphic to the value; the result
+ * is a pure function of the stats bits, so it is reproducible bit for bit.
+ *
+ *   stats     fp32 [n_layers, batch, n_kv_heads, stat_stride]
+ *   sel_len   int32 [batch], committed length T' (<= stat_stride); positions >= T' are ignored
+ *   indices   int32 [n_layers, batch, n_kv_heads, k_total]
+ *   n_indices int32 [n_layers, batch, n_kv_heads]
+ *   workspace unused at present (may be NULL, 0)
+ */
+int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
+                       int32_t n_kv_heads, const int32_t* sel_len, int32_t k_sink,
+                       int32_t k_recent, int32_t k_total, int32_t* indices, int32_t* n_indices,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Sparse draft attention (Eq. 5; Sec. 3.1 "Sparse Drafting Stage").  One query per sequence.
+ * Key set of (layer, b, KV head h) = indices[layer,b,h,0..n_indices) U the dense tail
+ * [tail_start[b], cur_len[b]) (tokens drafted in the current round, the query's own position
+ * included); softmax is renormalised over exactly that set.  Rows are read straight from the
+ * dense cache by index.
+ *
+ *   q          bf16 [n_layers, batch, n_q_heads, head_dim]
+ *   indices    int32 [n_layers, batch, n_kv_heads, k_total], entries < tail_start[b]; unique
+ *   n_indices  int32 [n_layers, batch, n_kv_heads], 0..k_total
+ *   tail_start int32 [batch]; cur_len int32 [batch], cur_len - tail_start <= max_tail
+ *   max_tail   host upper bound of the tail length (sizes the launch)
+ *   out        fp32 [n_layers, batch, n_q_heads, head_dim]; lse fp32 [n_layers,batch,n_q_heads]
+ *              or NULL
+ *   workspace  >= spec_workspace_bytes(SPEC_WS_DRAFT, ...) bytes, 256-byte aligned
+ * An index outside [0, cur_len[b]) is skipped and sets SPEC_ERR_BAD_INDEX in the status word.
+ * A problem with an empty key set yields out = 0, lse = -inf.
+ */
+int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* indices,
+                           const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
+                           const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Bytes of workspace entry point `which` needs for this cache description.  n_q and
+ * max_ctx_len matter for SPEC_WS_VERIFY, k_total (+ max_tail folded into it by the caller)
+ * for SPEC_WS_DRAFT.  Returns 0 on invalid arguments.
+ */
+size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t max_ctx_len,
+                            int32_t k_total);
+
+/*
+ * Synchronises `cuda_stream` and returns the status word at the head of `workspace`
+ * (SPEC_OK, SPEC_ERR_TIMEOUT or SPEC_ERR_BAD_INDEX), or SPEC_ERR_CUDA if the stream reports
+ * an error.
+ */
+int spec_read_status(const void* workspace, void* cuda_stream);
+
+/* Chooses the verification kernel (process-wide; SPEC_VERIFY_AUTO picks the tcgen05 kernel
+ * when the shape allows it).  Returns the previous setting, or SPEC_ERR_INVALID_ARG. */
+int spec_set_verify_impl(int impl);
+
+/* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC or
+ * SPEC_VERIFY_TCGEN05; 0 before the first call). */
+int spec_last_verify_impl(void);
+
+/* Number of kernels this library has launched since load (host-side counter). */
+int64_t spec_launch_count(void);
+
+const char* spec_strerror(int code);
+int spec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPEC_ATTN_H_ */

@@ -1,0 +1,200 @@
+"""ctypes binding of ``libspec_attn.so``: argument marshalling only.
+
+Every function takes CUDA torch tensors (torch is used for device memory and streams), checks
+dtypes/devices, passes raw pointers through the C ABI of ``include/spec_attn.h`` and raises
+``SpecError`` on a non-zero return code.  There is no CPU fallback: if the library is missing
+or the tensors are not on a CUDA device the call fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspec_attn.so")
+
+WS_VERIFY, WS_SELECT, WS_DRAFT = 0, 1, 2
+VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05 = 0, 1, 2
+
+EXPORTS = [
+    "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
+    "spec_read_status", "spec_set_verify_impl", "spec_last_verify_impl", "spec_launch_count",
+    "spec_strerror", "spec_version",
+]
+
+
+class SpecError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class _KV(ctypes.Structure):
+    _fields_ = [
+        ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("layer_stride", ctypes.c_int64), ("page_stride", ctypes.c_int64),
+        ("head_stride", ctypes.c_int64), ("slot_stride", ctypes.c_int64),
+        ("n_layers", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("page_table", ctypes.c_void_p),
+        ("max_pages", ctypes.c_int32), ("batch", ctypes.c_int32),
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+    ]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads the compiled library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: run `python -m paper_2607_27735_b200.build` "
+                "(there is no fallback implementation)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+        lib.spec_verify_attn.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
+                                         i64, vp, ctypes.c_size_t, vp]
+        lib.spec_select_recall.argtypes = [vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp,
+                                           ctypes.c_size_t, vp]
+        lib.spec_sparse_draft_attn.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
+                                               vp, vp, vp, ctypes.c_size_t, vp]
+        lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
+        lib.spec_workspace_bytes.restype = ctypes.c_size_t
+        lib.spec_read_status.argtypes = [vp, vp]
+        lib.spec_set_verify_impl.argtypes = [ctypes.c_int]
+        lib.spec_launch_count.restype = ctypes.c_int64
+        lib.spec_strerror.argtypes = [ctypes.c_int]
+        lib.spec_strerror.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return load().spec_strerror(code).decode()
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (no CPU path exists)")
+    if t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name}: expected contiguous {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _kv_struct(kv) -> _KV:
+    _dev(kv.k, torch.bfloat16, "kv.k")
+    _dev(kv.v, torch.bfloat16, "kv.v")
+    pt = None if kv.page_table is None else _dev(kv.page_table, torch.int32, "kv.page_table")
+    return _KV(kv.k.data_ptr(), kv.v.data_ptr(), kv.layer_stride, kv.page_stride, kv.head_stride,
+               kv.slot_stride, kv.n_layers, kv.page_size, pt, kv.max_pages, kv.batch,
+               kv.n_q_heads, kv.n_kv_heads, kv.head_dim, float(kv.sm_scale or 0.0))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def workspace_bytes(which: int, kv, n_q: int = 1, max_ctx_len: int = 1, k_total: int = 1) -> int:
+    return int(load().spec_workspace_bytes(which, ctypes.byref(_kv_struct(kv)), n_q, max_ctx_len,
+                                           k_total))
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """A 256-byte aligned byte tensor (torch's caching allocator aligns to 512 bytes)."""
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    assert ws.data_ptr() % 256 == 0
+    return ws
+
+
+def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
+                     stat_stride=None, workspace=None, want_lse=True):
+    """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``."""
+    lib = load()
+    L, B, n_q, Hq, D = q.shape
+    dev = q.device
+    s = _kv_struct(kv)
+    if stat_stride is None:
+        stat_stride = (max_ctx_len + 63) // 64 * 64 if stats is None else stats.shape[-1]
+    if out is None:
+        out = torch.empty(L, B, n_q, Hq, D, dtype=torch.float32, device=dev)
+    if lse is None and want_lse:
+        lse = torch.empty(L, B, n_q, Hq, dtype=torch.float32, device=dev)
+    if stats is None:
+        stats = torch.zeros(L, B, kv.n_kv_heads, stat_stride, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(WS_VERIFY, kv, n_q, max_ctx_len), dev)
+    rc = lib.spec_verify_attn(
+        ctypes.byref(s), _dev(q, torch.bfloat16, "q"), n_q, _dev(ctx_len, torch.int32, "ctx_len"),
+        max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
+        None if lse is None else _dev(lse, torch.float32, "lse"),
+        _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel(),
+        _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_verify_attn")
+    return out, lse, stats, workspace
+
+
+def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, n_indices=None):
+    """Eq. 4 recall selection; returns ``(indices, n_indices)``."""
+    lib = load()
+    L, B, Hkv, stride = stats.shape
+    dev = stats.device
+    if indices is None:
+        indices = torch.empty(L, B, Hkv, k_total, dtype=torch.int32, device=dev)
+    if n_indices is None:
+        n_indices = torch.empty(L, B, Hkv, dtype=torch.int32, device=dev)
+    rc = lib.spec_select_recall(
+        _dev(stats, torch.float32, "stats"), stride, L, B, Hkv,
+        _dev(sel_len, torch.int32, "sel_len"), k_sink, k_recent, k_total,
+        _dev(indices, torch.int32, "indices"), _dev(n_indices, torch.int32, "n_indices"), None, 0,
+        _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_select_recall")
+    return indices, n_indices
+
+
+def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_tail, out=None,
+                           lse=None, workspace=None, want_lse=True):
+    """Eq. 5 sparse draft attention; returns ``(out, lse, workspace)``."""
+    lib = load()
+    L, B, Hq, D = q.shape
+    dev = q.device
+    s = _kv_struct(kv)
+    k_total = indices.shape[-1]
+    if out is None:
+        out = torch.empty(L, B, Hq, D, dtype=torch.float32, device=dev)
+    if lse is None and want_lse:
+        lse = torch.empty(L, B, Hq, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(workspace_bytes(WS_DRAFT, kv, k_total=k_total + max_tail), dev)
+    rc = lib.spec_sparse_draft_attn(
+        ctypes.byref(s), _dev(q, torch.bfloat16, "q"), _dev(indices, torch.int32, "indices"),
+        _dev(n_indices, torch.int32, "n_indices"), k_total,
+        _dev(tail_start, torch.int32, "tail_start"), _dev(cur_len, torch.int32, "cur_len"),
+        max_tail, _dev(out, torch.float32, "out"),
+        None if lse is None else _dev(lse, torch.float32, "lse"), workspace.data_ptr(),
+        workspace.numel(), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_sparse_draft_attn")
+    return out, lse, workspace
+
+
+def read_status(workspace) -> int:
+    return int(load().spec_read_status(workspace.data_ptr(), _stream()))
+
+
+def set_verify_impl(impl: int) -> int:
+    return int(load().spec_set_verify_impl(impl))
+
+
+def last_verify_impl() -> int:
+    return int(load().spec_last_verify_impl())
+
+
+def launch_count() -> int:
+    return int(load().spec_launch_count())

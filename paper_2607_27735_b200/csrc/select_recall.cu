@@ -1,0 +1,159 @@
+// Recall selection of Eq. 4: sink + TopK over the middle span + recent, per (layer, sequence,
+// KV head).  One CTA per problem.  The scores are sums of probabilities (finite, >= 0), so the
+// fp32 bit pattern orders like the value and the K_mid-th largest is found by a three-pass
+// radix select (11 + 11 + 10 bits) on the bit patterns; an ordered compaction then emits, in
+// ascending position, everything above the threshold plus the lowest-position ties.
+#include "spec_common.cuh"
+
+namespace spec {
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kBins = 2048;
+constexpr int kItems = 8;  // consecutive candidates per thread in the compaction sweep
+
+// Exclusive block-wide prefix sum of one int per thread; `total` gets the block sum.
+__device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    __syncthreads();  // warp_tmp may still be read from a previous scan
+    if (lane == 31) warp_tmp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_tmp[lane];
+        int winc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, winc, o);
+            if (lane >= o) winc += y;
+        }
+        warp_tmp[lane] = winc - w;          // exclusive offset of each warp
+        if (lane == 31) warp_tmp[32] = winc;  // block total
+    }
+    __syncthreads();
+    total = warp_tmp[32];
+    return warp_tmp[warp] + inc - x;
+}
+
+__global__ void __launch_bounds__(kThreads)
+select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int batch, int n_kv_heads,
+                     const int32_t* __restrict__ sel_len, int k_sink, int k_recent, int k_total,
+                     int32_t* __restrict__ indices, int32_t* __restrict__ n_indices)
+{
+    __shared__ int hist[kBins];
+    __shared__ int warp_tmp[33];
+    __shared__ int sh_bucket, sh_above;
+
+    const int64_t prob = blockIdx.x;
+    const int b = (int)((prob / n_kv_heads) % batch);
+    const int T = sel_len[b];
+    int32_t* out = indices + prob * k_total;
+    const uint32_t* st = reinterpret_cast<const uint32_t*>(stats + prob * stat_stride);
+    const int tid = threadIdx.x;
+
+    if (T <= k_total) {  // everything fits: keep every position
+        for (int i = tid; i < k_total; i += kThreads) out[i] = i < T ? i : -1;
+        if (tid == 0) n_indices[prob] = T > 0 ? T : 0;
+        return;
+    }
+    const int lo = k_sink, hi = T - k_recent;  // candidate span [lo, hi), holds > k_mid entries
+    const int k_mid = k_total - k_sink - k_recent;
+    for (int i = tid; i < k_sink; i += kThreads) out[i] = i;
+    for (int i = tid; i < k_recent; i += kThreads) out[k_sink + k_mid + i] = hi + i;
+    if (tid == 0) n_indices[prob] = k_total;
+    if (k_mid == 0) return;
+
+    // ---- radix select: bit pattern `thr` of the k_mid-th largest candidate ----
+    uint32_t prefix = 0, mask = 0;
+    int need = k_mid;  // how many to take among candidates matching the decided prefix
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const int nb = pass == 2 ? 1024 : 2048;
+        for (int i = tid; i < kBins; i += kThreads) hist[i] = 0;
+        __syncthreads();
+        for (int i = lo + tid; i < hi; i += kThreads) {
+            const uint32_t u = __ldg(st + i);
+            if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+        }
+        __syncthreads();
+        // walk the buckets from the largest digit down: thread t owns reversed bins 2t, 2t+1
+        const int j0 = 2 * tid, j1 = 2 * tid + 1;
+        const int c0 = j0 < nb ? hist[nb - 1 - j0] : 0;
+        const int c1 = j1 < nb ? hist[nb - 1 - j1] : 0;
+        int total;
+        const int ex = block_exclusive_scan(c0 + c1, warp_tmp, total);
+        if (ex < need && need <= ex + c0) {
+            sh_bucket = nb - 1 - j0;
+            sh_above = ex;
+        } else if (ex + c0 < need && need <= ex + c0 + c1) {
+            sh_bucket = nb - 1 - j1;
+            sh_above = ex + c0;
+        }
+        __syncthreads();
+        prefix |= (uint32_t)sh_bucket << shift;
+        mask |= (uint32_t)(nb - 1) << shift;
+        need -= sh_above;
+        __syncthreads();
+    }
+    const uint32_t thr = prefix;  // take every candidate > thr and the first `need` equal to it
+
+    // ---- ordered compaction over the candidate span ----
+    int written = 0, eq_seen = 0;
+    for (int base = lo; base < hi; base += kThreads * kItems) {
+        const int i0 = base + tid * kItems;
+        uint32_t u[kItems];
+        int n_eq = 0;
+#pragma unroll
+        for (int k = 0; k < kItems; ++k) {
+            u[k] = (i0 + k < hi) ? __ldg(st + i0 + k) : 0u;
+            n_eq += (i0 + k < hi && u[k] == thr) ? 1 : 0;
+        }
+        int eq_total;
+        int eq_rank = eq_seen + block_exclusive_scan(n_eq, warp_tmp, eq_total);
+        int n_take = 0;
+        unsigned take_mask = 0;
+#pragma unroll
+        for (int k = 0; k < kItems; ++k) {
+            if (i0 + k < hi) {
+                bool take = u[k] > thr;
+                if (u[k] == thr) {
+                    take = eq_rank < need;
+                    ++eq_rank;
+                }
+                if (take) {
+                    take_mask |= 1u << k;
+                    ++n_take;
+                }
+            }
+        }
+        int take_total;
+        int dst = written + block_exclusive_scan(n_take, warp_tmp, take_total);
+#pragma unroll
+        for (int k = 0; k < kItems; ++k)
+            if (take_mask & (1u << k)) out[k_sink + dst++] = i0 + k;
+        written += take_total;
+        eq_seen += eq_total;
+    }
+}
+
+}  // namespace
+
+int select_launch(const float* stats, int64_t stat_stride, int n_layers, int batch, int n_kv_heads,
+                  const int32_t* sel_len, int k_sink, int k_recent, int k_total, int32_t* indices,
+                  int32_t* n_indices, cudaStream_t stream)
+{
+    const long probs = (long)n_layers * batch * n_kv_heads;
+    select_recall_kernel<<<(unsigned)probs, kThreads, 0, stream>>>(
+        stats, stat_stride, batch, n_kv_heads, sel_len, k_sink, k_recent, k_total, indices, n_indices);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+}  // namespace spec

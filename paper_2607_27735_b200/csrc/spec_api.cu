@@ -1,0 +1,217 @@
+// C-ABI entry points: argument validation on the host, then kernel launches on the caller's
+// stream.  No device allocation, no synchronisation (except spec_read_status).
+#include <atomic>
+#include <cmath>
+
+#include "spec_common.cuh"
+#include "verify_sm100.cuh"
+
+namespace spec {
+
+static std::atomic<int64_t> g_launches{0};
+static std::atomic<int> g_verify_impl{SPEC_VERIFY_AUTO};
+static std::atomic<int> g_last_verify_impl{0};
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int sm_count()
+{
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            return 148;
+    }
+    return cached;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the cache description and converts it; returns SPEC_OK or an error.
+static int make_view(const spec_kv_t* kv, KvView* out)
+{
+    if (!kv || !kv->k || !kv->v) return SPEC_ERR_INVALID_ARG;
+    if (kv->n_layers < 1 || kv->page_size < 1 || kv->max_pages < 1 || kv->batch < 1 ||
+        kv->n_q_heads < 1 || kv->n_kv_heads < 1)
+        return SPEC_ERR_INVALID_ARG;
+    if (kv->n_q_heads % kv->n_kv_heads != 0) return SPEC_ERR_INVALID_ARG;
+    if (kv->head_dim != 64 && kv->head_dim != 128) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned16(kv->k) || !aligned16(kv->v)) return SPEC_ERR_INVALID_ARG;
+    const int64_t strides[4] = {kv->layer_stride, kv->page_stride, kv->head_stride, kv->slot_stride};
+    for (int64_t s : strides)
+        if (s < 0 || s % 8 != 0) return SPEC_ERR_INVALID_ARG;
+    if (kv->slot_stride < kv->head_dim) return SPEC_ERR_INVALID_ARG;
+    out->k = static_cast<const __nv_bfloat16*>(kv->k);
+    out->v = static_cast<const __nv_bfloat16*>(kv->v);
+    out->layer_stride = kv->layer_stride;
+    out->page_stride = kv->page_stride;
+    out->head_stride = kv->head_stride;
+    out->slot_stride = kv->slot_stride;
+    out->page_table = kv->page_table;
+    out->n_layers = kv->n_layers;
+    out->page_size = kv->page_size;
+    out->max_pages = kv->max_pages;
+    out->batch = kv->batch;
+    out->n_q_heads = kv->n_q_heads;
+    out->n_kv_heads = kv->n_kv_heads;
+    out->head_dim = kv->head_dim;
+    out->scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
+    return SPEC_OK;
+}
+
+static bool use_tcgen05(const KvView& kv, int n_q, int impl)
+{
+    if (impl == SPEC_VERIFY_GENERIC) return false;
+    return verify_sm100_supported(kv, n_q);
+}
+
+}  // namespace spec
+
+using namespace spec;
+
+extern "C" {
+
+int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                     int32_t max_ctx_len, int32_t stat_window, float* out, float* lse, float* stats,
+                     int64_t stat_stride, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    VerifyArgs a;
+    const int rc = make_view(kv, &a.kv);
+    if (rc != SPEC_OK) return rc;
+    if (!q || !ctx_len || !out || !stats || !workspace) return SPEC_ERR_INVALID_ARG;
+    if (n_q < 1 || n_q > 32 || max_ctx_len < n_q || stat_window < 0 || stat_stride < max_ctx_len)
+        return SPEC_ERR_INVALID_ARG;
+    if ((int64_t)kv->max_pages * kv->page_size < max_ctx_len) return SPEC_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return SPEC_ERR_INVALID_ARG;
+    const int G = kv->n_q_heads / kv->n_kv_heads;
+    if (n_q * G > 128) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    const int W = stat_window > 0 ? stat_window : 16;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.n_q = n_q;
+    a.ctx_len = ctx_len;
+    a.max_ctx_len = max_ctx_len;
+    a.first_stat_row = n_q - (W < n_q ? W : n_q);
+    a.out = out;
+    a.lse = lse;
+    a.stats = stats;
+    a.stat_stride = stat_stride;
+    a.workspace = workspace;
+    a.workspace_bytes = workspace_bytes;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int impl = g_verify_impl.load();
+    const bool fast = use_tcgen05(a.kv, n_q, impl);
+    if (impl == SPEC_VERIFY_TCGEN05 && !fast) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    const size_t need = fast ? verify_sm100_workspace(a.kv, n_q, max_ctx_len)
+                             : verify_generic_workspace(a.kv, n_q, max_ctx_len);
+    if (workspace_bytes < need) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+    if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;
+    g_last_verify_impl.store(fast ? SPEC_VERIFY_TCGEN05 : SPEC_VERIFY_GENERIC);
+    return fast ? verify_sm100_launch(a, stream) : verify_generic_launch(a, stream);
+}
+
+int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
+                       int32_t n_kv_heads, const int32_t* sel_len, int32_t k_sink, int32_t k_recent,
+                       int32_t k_total, int32_t* indices, int32_t* n_indices, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream)
+{
+    (void)workspace;
+    (void)workspace_bytes;
+    if (!stats || !sel_len || !indices || !n_indices) return SPEC_ERR_INVALID_ARG;
+    if (n_layers < 1 || batch < 1 || n_kv_heads < 1 || stat_stride < 1) return SPEC_ERR_INVALID_ARG;
+    if (k_sink < 0 || k_recent < 0 || k_total < 1 || k_sink + (int64_t)k_recent > k_total)
+        return SPEC_ERR_INVALID_ARG;
+    return select_launch(stats, stat_stride, n_layers, batch, n_kv_heads, sel_len, k_sink, k_recent,
+                         k_total, indices, n_indices, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* indices,
+                           const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
+                           const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    DraftArgs a;
+    const int rc = make_view(kv, &a.kv);
+    if (rc != SPEC_OK) return rc;
+    if (!q || !indices || !n_indices || !tail_start || !cur_len || !out || !workspace)
+        return SPEC_ERR_INVALID_ARG;
+    if (k_total < 1 || max_tail < 0) return SPEC_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return SPEC_ERR_INVALID_ARG;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.indices = indices;
+    a.n_indices = n_indices;
+    a.k_total = k_total;
+    a.tail_start = tail_start;
+    a.cur_len = cur_len;
+    a.max_tail = max_tail;
+    a.out = out;
+    a.lse = lse;
+    a.workspace = workspace;
+    a.workspace_bytes = workspace_bytes;
+    if (workspace_bytes < draft_workspace(a.kv, k_total + max_tail)) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;
+    return draft_launch(a, stream);
+}
+
+size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t max_ctx_len,
+                            int32_t k_total)
+{
+    if (which == SPEC_WS_SELECT) return kStatusBytes;
+    KvView v;
+    if (make_view(kv, &v) != SPEC_OK) return 0;
+    if (which == SPEC_WS_VERIFY) {
+        if (n_q < 1 || n_q > 32 || max_ctx_len < n_q) return 0;
+        size_t g = verify_generic_workspace(v, n_q, max_ctx_len);
+        size_t f = verify_sm100_supported(v, n_q) ? verify_sm100_workspace(v, n_q, max_ctx_len) : 0;
+        return g > f ? g : f;
+    }
+    if (which == SPEC_WS_DRAFT) {
+        if (k_total < 1) return 0;
+        return draft_workspace(v, k_total);
+    }
+    return 0;
+}
+
+int spec_read_status(const void* workspace, void* cuda_stream)
+{
+    if (!workspace) return SPEC_ERR_INVALID_ARG;
+    int code = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(&code, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return SPEC_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return SPEC_ERR_CUDA;
+    return code;
+}
+
+int spec_set_verify_impl(int impl)
+{
+    if (impl < SPEC_VERIFY_AUTO || impl > SPEC_VERIFY_TCGEN05) return SPEC_ERR_INVALID_ARG;
+    return g_verify_impl.exchange(impl);
+}
+
+int spec_last_verify_impl(void) { return g_last_verify_impl.load(); }
+
+int64_t spec_launch_count(void) { return g_launches.load(); }
+
+const char* spec_strerror(int code)
+{
+    switch (code) {
+        case SPEC_OK: return "ok";
+        case SPEC_ERR_INVALID_ARG: return "invalid argument";
+        case SPEC_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case SPEC_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case SPEC_ERR_CUDA: return "CUDA error";
+        case SPEC_ERR_TIMEOUT: return "device-side wait timed out";
+        case SPEC_ERR_BAD_INDEX: return "recall index out of range";
+        default: return "unknown error";
+    }
+}
+
+int spec_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,98 @@
+// Shared device-side definitions of the attention kernels: cache addressing, bf16 unpacking,
+// warp reductions, and the host-side launcher declarations used by spec_api.cu.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spec_attn.h"
+
+namespace spec {
+
+// Device copy of the cache description (see spec_kv_t for the addressing rule).
+struct KvView {
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    int64_t layer_stride, page_stride, head_stride, slot_stride;
+    const int32_t* page_table;
+    int32_t n_layers, page_size, max_pages, batch, n_q_heads, n_kv_heads, head_dim;
+    float scale;  // resolved softmax scale
+};
+
+__device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, int b, int pos, int h)
+{
+    const int page = pos / kv.page_size;
+    const int slot = pos - page * kv.page_size;
+    const int64_t phys = kv.page_table ? (int64_t)__ldg(kv.page_table + (int64_t)b * kv.max_pages + page)
+                                       : (int64_t)b * kv.max_pages + page;
+    return layer * kv.layer_stride + phys * kv.page_stride + h * kv.head_stride +
+           slot * kv.slot_stride;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ float warp_max(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// The status word lives in the first int of every workspace; errors are sticky until the next
+// call clears it.
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+constexpr int kStatusBytes = 256;  // head of every workspace: status word + padding
+
+// ---- launchers (defined in the kernel files; all enqueue on `stream`, none synchronises) ----
+struct VerifyArgs {
+    KvView kv;
+    const __nv_bfloat16* q;
+    int n_q;
+    const int32_t* ctx_len;
+    int max_ctx_len;
+    int first_stat_row;  // window rows j >= first_stat_row feed the statistic
+    float* out;
+    float* lse;
+    float* stats;
+    int64_t stat_stride;
+    void* workspace;
+    size_t workspace_bytes;
+};
+
+size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);
+int verify_generic_launch(const VerifyArgs& a, cudaStream_t stream);
+
+int select_launch(const float* stats, int64_t stat_stride, int n_layers, int batch, int n_kv_heads,
+                  const int32_t* sel_len, int k_sink, int k_recent, int k_total, int32_t* indices,
+                  int32_t* n_indices, cudaStream_t stream);
+
+struct DraftArgs {
+    KvView kv;
+    const __nv_bfloat16* q;
+    const int32_t* indices;
+    const int32_t* n_indices;
+    int k_total;
+    const int32_t* tail_start;
+    const int32_t* cur_len;
+    int max_tail;
+    float* out;
+    float* lse;
+    void* workspace;
+    size_t workspace_bytes;
+};
+size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
+int draft_launch(const DraftArgs& a, cudaStream_t stream);
+
+void count_launch(int n = 1);
+int sm_count();
+
+}  // namespace spec
