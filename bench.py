@@ -1,0 +1,316 @@
+"""Benchmark of the SparseSpec-L attention hot path on B200.
+
+``python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]``
+
+A step = one speculative iteration of the attention path on a resident KV cache: per layer
+verification attention with the fused Eq. 3 score, Eq. 4 recall selection, then k drafting
+steps of Eq. 5 sparse attention per layer.  Metric: microseconds per step (lower is better) and
+the HBM-roofline fraction of the dominant kernel.  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "us_per_spec_step"
+UNIT = "us"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def pick_config(name: str):
+    from paper_2607_27735_b200 import inputs
+
+    cfgs = inputs.baseline_configs()
+    if name not in cfgs:
+        raise SystemExit(f"unknown config {name}; choose from {list(cfgs)}")
+    return cfgs[name]
+
+
+def config_json(cfg, n_gpus: int) -> dict:
+    return {
+        "workload": f"{cfg.name}: {cfg.n_layers} layers x ({cfg.n_q_heads} q / {cfg.n_kv_heads} kv "
+                    f"heads, head_dim {cfg.head_dim}), batch {cfg.batch} per GPU, context "
+                    f"{cfg.ctx[0]}..{cfg.ctx[1]}, k={cfg.n_q - 1} (n_q={cfg.n_q}), recall budget "
+                    f"{cfg.k_total} (sink {cfg.k_sink} + recent {cfg.k_recent} + top-"
+                    f"{cfg.k_total - cfg.k_sink - cfg.k_recent}), {cfg.draft_steps} draft steps",
+        "global_batch": cfg.batch * n_gpus,
+        "parallelism": f"independent sequences per GPU x{n_gpus} (no collective)",
+        "launch_mode": "one launch per layer (verify, draft), one launch for all layers (select); "
+                       "three CUDA graphs per step",
+        "l2": "inputs larger than L2: every layer streams its own KV (step total >> 126 MB)",
+        "kv_resident": True,
+    }
+
+
+# -------------------------------------------------------------------------------------------------
+# CPU oracle legs
+
+
+def oracle_step_seconds(cfg, sample_layers: int):
+    """Times the oracle on `sample_layers` layers of the workload (host cores)."""
+    import torch
+
+    import oracle
+    from paper_2607_27735_b200 import inputs
+
+    case = inputs.make_case(cfg, device="cpu", n_layers=sample_layers)
+    kv = case.kv
+    t0 = time.perf_counter()
+    out, lse, stats = oracle.verify_attn(kv, case.q_verify, case.ctx_len, cfg.stat_window)
+    idx, n = oracle.select_recall(stats.float(), case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total)
+    for j in range(cfg.draft_steps):
+        oracle.sparse_draft_attn(kv, case.q_draft[j].contiguous(), idx, n, case.ctx_len,
+                                 (case.ctx_len + j + 1).int())
+    dt = time.perf_counter() - t0
+    return dt, oracle.threads()
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle, as it stands, on the same config and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = pick_config(args.config)
+    sample_layers = 1
+    times = []
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        dt, cores = oracle_step_seconds(cfg, sample_layers)
+        if i >= args.warmup:
+            times.append(dt)
+    scale = cfg.n_layers / sample_layers
+    us = statistics.mean(times) * scale * 1e6
+    sample = (f"{sample_layers} of {cfg.n_layers} layers per step (layers are i.i.d. in shape), "
+              f"time scaled x{scale:g}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_json(cfg, args.gpus),
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# -------------------------------------------------------------------------------------------------
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_27735_b200 import binding, inputs, runner
+    from paper_2607_27735_b200.dist_util import init_process_group, max_over_ranks
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        init_process_group("nccl", dev)
+
+    binding.load()
+    cfg = pick_config(args.config)
+    if world > 1:  # every rank serves its own sequences: different seed, same shape
+        import dataclasses
+        cfg = dataclasses.replace(cfg, seed=cfg.seed + 101 * rank)
+    case = inputs.make_case(cfg, device=dev)
+    run = runner.SpecStepRunner(case, fold_layers=args.fold_layers)
+    counts = run.capture()
+    launches_per_step = sum(counts)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        run.replay()
+    barrier()
+
+    # ---- device-timed region: K steps, inputs resident in HBM ----
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    barrier()
+    for s in range(args.steps):
+        run.replay(evs[s])
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = evs[0][0].elapsed_time(evs[-1][3])
+    phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / args.steps for i in range(3)]
+    step_ms = max_over_ranks(total_ms / args.steps, world, dev)
+    phase_ms = [max_over_ranks(p, world, dev) for p in phase_ms]
+
+    # ---- end to end: host Q in, host outputs back, every step ----
+    qv_host = case.q_verify.cpu().pin_memory()
+    qd_host = case.q_draft.cpu().pin_memory()
+    outv_host = torch.empty(run.out_v.shape, dtype=run.out_v.dtype).pin_memory()
+    outd_host = torch.empty(run.out_d.shape, dtype=run.out_d.dtype).pin_memory()
+    h2d = qv_host.numel() * 2 + qd_host.numel() * 2
+    d2h = outv_host.numel() * 4 + outd_host.numel() * 4
+
+    def e2e_step():
+        run.q_verify.copy_(qv_host, non_blocking=True)
+        run.q_draft.copy_(qd_host, non_blocking=True)
+        run.replay()
+        outv_host.copy_(run.out_v, non_blocking=True)
+        outd_host.copy_(run.out_d, non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    L = cfg.n_layers
+    v_launches = 1 if args.fold_layers else L
+    verify_bytes = run.verify_kv_bytes_per_layer() * (L if args.fold_layers else 1)
+    verify_us = phase_ms[0] * 1e3 / v_launches
+    achieved = verify_bytes / (verify_us * 1e-6) / 1e9
+    draft_bytes = sum(run.draft_kv_bytes_per_layer_step(j) for j in range(cfg.draft_steps)) * L
+    draft_gbs = draft_bytes / (phase_ms[2] * 1e-3) / 1e9 if phase_ms[2] > 0 else None
+
+    cpu_layers = 2
+    cpu_dt, cores = oracle_step_seconds(cfg, cpu_layers)
+    cpu_us = cpu_dt * (L / cpu_layers) * 1e6
+
+    line = {
+        "metric": METRIC, "value": step_ms * 1e3, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": config_json(cfg, world),
+        "phases_us": {"verify": phase_ms[0] * 1e3, "select": phase_ms[1] * 1e3,
+                      "draft": phase_ms[2] * 1e3},
+        "verify_impl": {1: "generic", 2: "tcgen05"}.get(binding.last_verify_impl()),
+        "roofline": {
+            "kernel": "verification attention + Eq.3 statistic (per-layer launch)",
+            "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+            "frac_of_8TBs": achieved / 8000.0,
+            "bytes_per_launch": verify_bytes, "us_per_launch": verify_us,
+            "traffic": None,
+        },
+        "draft_roofline": {"achieved": draft_gbs, "frac": draft_gbs / peak if draft_gbs else None,
+                           "bytes_per_step": draft_bytes, "unit": "GB/s"},
+        "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{cpu_layers} of {L} layers, time scaled x{L / cpu_layers:g}"},
+        "e2e": {"value": e2e_ms * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h,
+                "note": "Q in from pinned host memory, attention outputs back to host every step; "
+                        "the dense KV cache stays resident by the method's definition"},
+        "gpu_launches": launches_per_step * args.steps,
+        "launches_per_step": {"verify": counts[0], "select": counts[1], "draft": counts[2]},
+        "clocks": clocks,
+    }
+    traffic_path = os.path.join(ROOT, "profiles", "verify_traffic.json")
+    if os.path.exists(traffic_path):
+        with open(traffic_path) as f:
+            t = json.load(f)
+        if t.get("config") == cfg.name:
+            line["roofline"]["traffic"] = t.get("dram_bytes_per_launch")
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg2_8b_32k")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--fold-layers", action="store_true",
+                    help="issue verify/draft for all layers in one launch (kernel-roofline view)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

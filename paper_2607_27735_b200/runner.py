@@ -1,0 +1,126 @@
+"""One speculative step of the attention hot path on a resident KV cache.
+
+``SpecStepRunner`` owns the output buffers and workspaces of a workload and issues the three
+phases through the C ABI on the current stream:
+
+  verify phase : per layer, ``spec_verify_attn`` (dense attention of the k+1 rows + Eq. 3 score)
+  select phase : ``spec_select_recall`` for every layer in one launch (the index sets are only
+                 needed by the next drafting round, so the layers are independent problems here)
+  draft phase  : per drafting step and layer, ``spec_sparse_draft_attn`` (Eq. 5)
+
+``fold_layers=True`` issues verify and draft with ``n_layers = L`` in one launch instead
+(independent problems; a kernel-roofline view, not the layer-by-layer dependency chain of a
+real decoder).  The phases can be captured into CUDA graphs to take the Python/ctypes launch
+cost out of the timed region.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding
+
+
+class SpecStepRunner:
+    def __init__(self, case, fold_layers: bool = False, want_lse: bool = False):
+        cfg, kv = case.cfg, case.kv
+        self.case, self.cfg, self.kv = case, cfg, kv
+        self.fold = fold_layers
+        dev = kv.k.device
+        L, B = kv.n_layers, kv.batch
+        self.L = L
+        self.max_ctx = int(case.ctx_len.max())
+        self.stat_stride = (self.max_ctx + 127) // 128 * 128
+        self.out_v = torch.empty(L, B, cfg.n_q, kv.n_q_heads, kv.head_dim, device=dev)
+        self.lse_v = torch.empty(L, B, cfg.n_q, kv.n_q_heads, device=dev) if want_lse else None
+        self.stats = torch.zeros(L, B, kv.n_kv_heads, self.stat_stride, device=dev)
+        self.indices = torch.empty(L, B, kv.n_kv_heads, cfg.k_total, dtype=torch.int32, device=dev)
+        self.n_idx = torch.empty(L, B, kv.n_kv_heads, dtype=torch.int32, device=dev)
+        self.out_d = torch.empty(max(cfg.draft_steps, 1), L, B, kv.n_q_heads, kv.head_dim, device=dev)
+        self.q_verify = case.q_verify
+        self.q_draft = case.q_draft
+        self.ctx_len = case.ctx_len
+        self.tail_start = case.ctx_len.clone()
+        self.cur_lens = [(case.ctx_len + j + 1).contiguous() for j in range(cfg.draft_steps)]
+        kvs = kv if fold_layers else kv.layer_slice(0, 1)
+        self.ws_v = binding.alloc_workspace(
+            binding.workspace_bytes(binding.WS_VERIFY, kvs, cfg.n_q, self.max_ctx), dev)
+        self.ws_d = binding.alloc_workspace(
+            binding.workspace_bytes(binding.WS_DRAFT, kvs, k_total=cfg.k_total + cfg.draft_steps), dev)
+        self._layers = [kv.layer_slice(l, l + 1) for l in range(L)]
+        self.graphs = None
+
+    # -- phases ----------------------------------------------------------------------------
+    def verify_phase(self):
+        if self.fold:
+            binding.spec_verify_attn(self.kv, self.q_verify, self.ctx_len, self.max_ctx,
+                                     self.cfg.stat_window, out=self.out_v, lse=self.lse_v,
+                                     stats=self.stats, workspace=self.ws_v, want_lse=False)
+            return
+        for l in range(self.L):
+            binding.spec_verify_attn(
+                self._layers[l], self.q_verify[l:l + 1], self.ctx_len, self.max_ctx,
+                self.cfg.stat_window, out=self.out_v[l:l + 1],
+                lse=None if self.lse_v is None else self.lse_v[l:l + 1],
+                stats=self.stats[l:l + 1], workspace=self.ws_v, want_lse=False)
+
+    def select_phase(self):
+        c = self.cfg
+        binding.spec_select_recall(self.stats, self.ctx_len, c.k_sink, c.k_recent, c.k_total,
+                                   indices=self.indices, n_indices=self.n_idx)
+
+    def draft_phase(self):
+        c = self.cfg
+        for j in range(c.draft_steps):
+            if self.fold:
+                binding.spec_sparse_draft_attn(
+                    self.kv, self.q_draft[j], self.indices, self.n_idx, self.tail_start,
+                    self.cur_lens[j], c.draft_steps, out=self.out_d[j], workspace=self.ws_d,
+                    want_lse=False)
+                continue
+            for l in range(self.L):
+                binding.spec_sparse_draft_attn(
+                    self._layers[l], self.q_draft[j, l:l + 1], self.indices[l:l + 1],
+                    self.n_idx[l:l + 1], self.tail_start, self.cur_lens[j], c.draft_steps,
+                    out=self.out_d[j, l:l + 1], workspace=self.ws_d, want_lse=False)
+
+    def step(self):
+        self.verify_phase()
+        self.select_phase()
+        self.draft_phase()
+
+    # -- CUDA graphs -----------------------------------------------------------------------
+    def capture(self):
+        """Captures the three phases into three CUDA graphs (after one eager warm-up step).
+        Returns the number of kernels each phase launches."""
+        self.step()
+        torch.cuda.synchronize()
+        graphs, counts = [], []
+        for phase in (self.verify_phase, self.select_phase, self.draft_phase):
+            g = torch.cuda.CUDAGraph()
+            before = binding.launch_count()
+            with torch.cuda.graph(g):
+                phase()
+            counts.append(binding.launch_count() - before)
+            graphs.append(g)
+        self.graphs = graphs
+        self.launches_per_phase = counts
+        return counts
+
+    def replay(self, events=None):
+        """Replays the captured step; ``events`` = 4 CUDA events recorded around the phases."""
+        for i, g in enumerate(self.graphs):
+            if events is not None:
+                events[i].record()
+            g.replay()
+        if events is not None:
+            events[3].record()
+
+    # -- algorithmic bytes (what the method must move) ---------------------------------------
+    def verify_kv_bytes_per_layer(self) -> int:
+        kv = self.kv
+        return int(self.ctx_len.sum()) * kv.n_kv_heads * kv.head_dim * 2 * 2
+
+    def draft_kv_bytes_per_layer_step(self, j: int) -> int:
+        kv, c = self.kv, self.cfg
+        rows = sum(min(c.k_total, int(t)) + j + 1 for t in self.ctx_len.tolist())
+        return rows * kv.n_kv_heads * kv.head_dim * 2 * 2
