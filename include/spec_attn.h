@@ -76,6 +76,8 @@ typedef struct {
     const int32_t* page_table;     /* device int32 [batch, max_pages] or NULL */
     int32_t max_pages, batch, n_q_heads, n_kv_heads;
     int32_t head_dim;              /* 64 or 128 */
+    int32_t n_pages;               /* physical pages in the pool (bounds page_table entries);
+                                      0 means batch * max_pages */
     float sm_scale;                /* softmax scale; <= 0 means 1/sqrt(head_dim) */
 } spec_kv_t;
 

@@ -40,7 +40,7 @@ class _KV(ctypes.Structure):
         ("page_table", ctypes.c_void_p),
         ("max_pages", ctypes.c_int32), ("batch", ctypes.c_int32),
         ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
-        ("head_dim", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+        ("head_dim", ctypes.c_int32), ("n_pages", ctypes.c_int32), ("sm_scale", ctypes.c_float),
     ]
 
 
@@ -92,7 +92,8 @@ def _kv_struct(kv) -> _KV:
     pt = None if kv.page_table is None else _dev(kv.page_table, torch.int32, "kv.page_table")
     return _KV(kv.k.data_ptr(), kv.v.data_ptr(), kv.layer_stride, kv.page_stride, kv.head_stride,
                kv.slot_stride, kv.n_layers, kv.page_size, pt, kv.max_pages, kv.batch,
-               kv.n_q_heads, kv.n_kv_heads, kv.head_dim, float(kv.sm_scale or 0.0))
+               kv.n_q_heads, kv.n_kv_heads, kv.head_dim, int(getattr(kv, "n_pages", 0) or 0),
+               float(kv.sm_scale or 0.0))
 
 
 def _stream() -> int:

@@ -58,6 +58,8 @@ static int make_view(const spec_kv_t* kv, KvView* out)
     out->n_q_heads = kv->n_q_heads;
     out->n_kv_heads = kv->n_kv_heads;
     out->head_dim = kv->head_dim;
+    if (kv->n_pages < 0) return SPEC_ERR_INVALID_ARG;
+    out->n_pages = kv->n_pages > 0 ? kv->n_pages : kv->batch * kv->max_pages;
     out->scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
     return SPEC_OK;
 }

@@ -16,7 +16,7 @@ struct KvView {
     const __nv_bfloat16* v;
     int64_t layer_stride, page_stride, head_stride, slot_stride;
     const int32_t* page_table;
-    int32_t n_layers, page_size, max_pages, batch, n_q_heads, n_kv_heads, head_dim;
+    int32_t n_layers, page_size, max_pages, batch, n_q_heads, n_kv_heads, head_dim, n_pages;
     float scale;  // resolved softmax scale
 };
 

@@ -46,6 +46,7 @@ class KVCache:
     n_kv_heads: int
     head_dim: int
     sm_scale: float = 0.0
+    n_pages: int = 0  # physical pages in the pool (0: batch * max_pages)
 
     def to(self, device) -> "KVCache":
         pt = None if self.page_table is None else self.page_table.to(device)
@@ -221,7 +222,7 @@ def make_case(cfg: SpecConfig, device="cpu", n_layers: Optional[int] = None,
         k=k, v=v, layer_stride=n_phys * Hkv * ps * D, page_stride=Hkv * ps * D,
         head_stride=ps * D, slot_stride=D, n_layers=L, page_size=ps,
         page_table=None if page_table is None else page_table.to(dev), max_pages=max_pages,
-        batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, sm_scale=0.0,
+        batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, sm_scale=0.0, n_pages=n_phys,
     )
     return SpecCase(cfg=cfg, kv=kv, ctx_len=ctx.to(dev), q_verify=q_verify.to(torch.bfloat16),
                     q_draft=q_draft.to(torch.bfloat16), planted_pos=planted_pos,

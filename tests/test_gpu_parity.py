@@ -19,7 +19,8 @@ def run_verify(case, stat_window=16, impl=binding.VERIFY_AUTO):
     try:
         out, lse, stats, ws = binding.spec_verify_attn(
             kv, case.q_verify, case.ctx_len, int(case.ctx_len.max()), stat_window)
-        assert binding.read_status(ws) == 0
+        status = binding.read_status(ws)
+        assert status == 0, (status, ws[:16].view(torch.int32).tolist())
     finally:
         binding.set_verify_impl(prev)
     return out, lse, stats
@@ -70,6 +71,39 @@ def test_verify_parity(shape, impl):
     cfg = inputs.small_config(**shape)
     case = inputs.make_case(cfg, device="cuda")
     check_verify(case, impl=impl)
+    if impl == binding.VERIFY_AUTO and cfg.head_dim == 128 and cfg.n_q * cfg.group <= 112:
+        assert binding.last_verify_impl() == binding.VERIFY_TCGEN05  # the fast path really ran
+
+
+TCGEN05_SHAPES = [
+    dict(ctx=(128, 128), n_q=1, planted=0),
+    dict(ctx=(129, 129), n_q=2, planted=0),
+    dict(ctx=(5000, 5000), n_q=9, n_q_heads=32, n_kv_heads=8, planted=50),          # 8B shape
+    dict(ctx=(20000, 20000), n_q=9, n_q_heads=32, n_kv_heads=8, planted=200),       # several tiles per CTA
+    dict(ctx=(9000, 9000), n_q=7, n_q_heads=40, n_kv_heads=8, batch=2, kv_dist="student_t3"),
+    dict(ctx=(3000, 9000), n_q=7, n_q_heads=32, n_kv_heads=8, batch=4, page_size=16,
+         shuffled_pages=True, planted=0, q_mode="iid", q_std=0.09, n_layers=2),
+    dict(ctx=(4100, 4100), n_q=17, n_q_heads=32, n_kv_heads=8, planted=40),         # R=68 > W rows
+    dict(ctx=(2500, 2500), n_q=28, n_q_heads=16, n_kv_heads=4, planted=10),         # R=112
+    dict(ctx=(6000, 6000), n_q=5, n_q_heads=8, n_kv_heads=1, page_size=256, shuffled_pages=True),
+]
+
+
+@pytest.mark.parametrize("shape", TCGEN05_SHAPES)
+def test_verify_tcgen05_parity(shape):
+    cfg = inputs.small_config(**shape)
+    case = inputs.make_case(cfg, device="cuda")
+    check_verify(case, impl=binding.VERIFY_TCGEN05)
+
+
+def test_verify_tcgen05_ignores_garbage_beyond_the_context():
+    """Cache slots past ctx_len may hold anything (NaN included): they must not leak."""
+    cfg = inputs.small_config(ctx=(1000, 1000), n_q=5, planted=5)
+    case = inputs.make_case(cfg, device="cuda")
+    kv = case.kv
+    kv.k[:, :, :, 1000:] = float("nan")
+    kv.v[:, :, :, 1000:] = float("nan")
+    check_verify(case, impl=binding.VERIFY_TCGEN05)
 
 
 @pytest.mark.parametrize("window", [1, 4, 16])
