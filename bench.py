@@ -85,13 +85,18 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
-def pick_config(name: str):
+def pick_config(name: str, layers: int = 0):
+    import dataclasses
+
     from paper_2607_27735_b200 import inputs
 
     cfgs = inputs.baseline_configs()
     if name not in cfgs:
         raise SystemExit(f"unknown config {name}; choose from {list(cfgs)}")
-    return cfgs[name]
+    cfg = cfgs[name]
+    if layers > 0:
+        cfg = dataclasses.replace(cfg, n_layers=layers)
+    return cfg
 
 
 def config_json(cfg, n_gpus: int) -> dict:
@@ -138,7 +143,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg = pick_config(args.config)
+    cfg = pick_config(args.config, args.layers)
     sample_layers = 1
     times = []
     cores = 1
@@ -182,7 +187,7 @@ def run_gpu(args):
         init_process_group("nccl", dev)
 
     binding.load()
-    cfg = pick_config(args.config)
+    cfg = pick_config(args.config, args.layers)
     if world > 1:  # every rank serves its own sequences: different seed, same shape
         import dataclasses
         cfg = dataclasses.replace(cfg, seed=cfg.seed + 101 * rank)
@@ -253,7 +258,7 @@ def run_gpu(args):
     draft_bytes = sum(run.draft_kv_bytes_per_layer_step(j) for j in range(cfg.draft_steps)) * L
     draft_gbs = draft_bytes / (phase_ms[2] * 1e-3) / 1e9 if phase_ms[2] > 0 else None
 
-    cpu_layers = 2
+    cpu_layers = min(2, L)
     cpu_dt, cores = oracle_step_seconds(cfg, cpu_layers)
     cpu_us = cpu_dt * (L / cpu_layers) * 1e6
 
@@ -303,6 +308,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="cfg2_8b_32k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0,
+                    help="use only this many layers of the config (small captures under ncu)")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()

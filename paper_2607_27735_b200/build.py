@@ -29,7 +29,7 @@ def _newest_dep() -> float:
 
 def _compile(src: str, verbose: bool) -> str:
     obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-    cmd = ["nvcc", *NVCC_FLAGS, "-c",
+    cmd = ["nvcc", *NVCC_FLAGS, *os.environ.get("SPEC_EXTRA_NVCC_FLAGS", "").split(), "-c",
            os.path.join(CSRC, src), "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")

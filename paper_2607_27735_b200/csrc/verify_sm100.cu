@@ -39,7 +39,7 @@ constexpr int kD = 128;               // head_dim of the fast path
 constexpr int kSlotBytes = 32768;     // one K or V tile: 2 halves x 128 rows x 128 B (SW128)
 constexpr int kThreads = 384;
 constexpr int kRing = 4;              // partial buffers are recycled every kRing units
-constexpr uint64_t kTimeoutNs = 1000ull * 1000ull * 1000ull;
+constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // about a second of SM clocks
 constexpr uint64_t kEvictFirst = 0x12F0000000000000ull;
 constexpr uint64_t kEvictLast = 0x14F0000000000000ull;
 constexpr int kTmemCols = 512;
@@ -56,6 +56,7 @@ struct FastParams {
     float* o_part;                    // [kRing][HG][cph][R][kD]
     int* status;
     int n_pages;
+    long long* trace;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -146,6 +147,12 @@ __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr)
 {
     return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
+// MN-major operand without swizzle (the P^T tile): 8x8 core matrices of 128 contiguous bytes,
+// K groups 128 B apart (leading offset), 8-row MN blocks 2048 B apart (stride offset).
+__device__ __forceinline__ uint64_t desc_mnmajor_nosw(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (8ull << 16) | (128ull << 32) | (1ull << 46);
+}
 // MN-major operand, 128-byte swizzle: 64-element MN blocks 16 KiB apart (leading offset),
 // 8-row K groups 1024 B apart (stride offset).
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr)
@@ -154,6 +161,14 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr)
 }
 
 // ---------------------------------------------------------------------------------------------
+
+#ifdef SPEC_TRACE
+// Development aid (not compiled by default): per-CTA, per-role clock64 stamps in the workspace.
+#define TRACE(role, slot) do { if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 60) \
+    p.trace[((int64_t)blockIdx.x * 4 + (role)) * 64 + trace_n[role]++] = ((long long)(slot) << 48) | (clock64() & 0xffffffffffffll); } while (0)
+#else
+#define TRACE(role, slot) do { } while (0)
+#endif
 
 struct Ctl {
     volatile int* abort_flag;  // shared
@@ -173,12 +188,12 @@ __device__ __noinline__ void report_timeout(const Ctl& c, int where)
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Ctl& c, int where)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer();
+    const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*c.abort_flag) return false;
-            if (globaltimer() - t0 > kTimeoutNs) {
+            if (clock64() - t0 > kTimeoutCycles) {
                 report_timeout(c, where);
                 return false;
             }
@@ -190,13 +205,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
 __device__ __forceinline__ bool counter_wait(const int* ctr, int target, const Ctl& c, int where)
 {
     if (ld_acquire(ctr) >= target) return true;
-    const uint64_t t0 = globaltimer();
+    const long long t0 = clock64();
     uint32_t spins = 0;
     while (ld_acquire(ctr) < target) {
-        __nanosleep(64);
+        __nanosleep(32);
         if ((++spins & 63u) == 0) {
             if (*c.abort_flag) return false;
-            if (globaltimer() - t0 > kTimeoutNs) {
+            if (clock64() - t0 > kTimeoutCycles) {
                 report_timeout(c, where);
                 return false;
             }
@@ -244,7 +259,7 @@ struct Smem {
 
 struct Bars {  // mbarrier addresses (shared space)
     uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_empty, p_full, p_empty, o_full, o_empty,
-        lse_full, lse_empty, sm_sync, aux_sync;
+        lse_full, lse_empty, sm_sync, aux_sync, stat_full;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -297,15 +312,19 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         B.lse_empty = o; o += 16;
         B.sm_sync = o; o += 8;
         B.aux_sync = o; o += 8;
+        B.stat_full = o; o += 32;
     }
     (void)bar_mem;
     float* lse_s = reinterpret_cast<float*>(misc + 512);                 // [2][128]
-    float* stat_tmp = reinterpret_cast<float*>(misc + 512 + 1024);       // [2][128]
-    float2* red = reinterpret_cast<float2*>(misc + 512 + 2048);          // [8 warps][NH] (m, l)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 512 + 2048 + 8 * 64 * 8);
+    float* stat_tmp = reinterpret_cast<float*>(misc + 512 + 1024);       // [4][128]
+    float2* red = reinterpret_cast<float2*>(misc + 512 + 3072);          // [8 warps][64] (m, l)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 512 + 3072 + 8 * 64 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     Ctl ctl{abort_flag, p.status};
+#ifdef SPEC_TRACE
+    int trace_n[4] = {0, 0, 0, 0};
+#endif
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.n_slots; ++i) {
@@ -326,6 +345,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         mbar_init(B.o_empty, 8);
         mbar_init(B.sm_sync, 8);
         mbar_init(B.aux_sync, 2);
+        for (int i = 0; i < 4; ++i) mbar_init(B.stat_full + 8 * i, 4);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -375,6 +395,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             return true;
         };
         for (int round = 0; round <= U && ok; ++round) {
+            TRACE(0, 1);
             if (round < U) {
                 const Seg sg = get_seg(p, round, head_local, rank);
                 if (sg.t1 > sg.t0) {
@@ -392,6 +413,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t, kEvictLast);
                 }
             }
+            TRACE(0, 2);
             if (round >= 1 && ok) {
                 const Seg sg = get_seg(p, round - 1, head_local, rank);
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
@@ -408,7 +430,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         // =========================== MMA issuer ===========================
         if (lane == 0) {
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
-            const uint32_t idesc_pv = idesc_qk | (1u << 15);  // A = V^T, MN-major
+            const uint32_t idesc_pv = idesc_qk | (1u << 15) | (1u << 16);  // A = V^T and B = P^T, both MN-major
             uint32_t slot_idx = 0, qn = 0, qk_idx = 0, pv_idx = 0, o_phase = 0;
             bool ok = true;
             // pending PV (issued one task late so the next QK^T overlaps the softmax)
@@ -431,7 +453,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const uint64_t a = desc_mnmajor(v_addr + ks * 2048);
-                        const uint64_t b = desc_kmajor(p_addr + (ks >> 2) * (N * 128) + (ks & 3) * 32);
+                        const uint64_t b = desc_mnmajor_nosw(p_addr + ks * 256);
                         tc_mma(d_o, a, b, idesc_pv, (pend_first && part == 0 && ks == 0) ? 0u : 1u);
                     }
                 }
@@ -515,19 +537,22 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
         const int c0 = wg * NH;                  // first column of this warpgroup
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int stat_r0 = p.a.first_stat_row * G;
-        uint32_t qk_idx = 0, pv_idx = 0, slot_idx = 0, lse_n = 0, o_phase = 0, sync_n = 0;
+        const float cs = p.scale_log2;
+        constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
+        uint32_t qk_idx = 0, pv_idx = 0, slot_idx = 0, lse_n = 0, o_phase = 0, sync_n = 0, stat_n = 0;
         bool ok = true;
         int prev_lse_idx = 0;
         bool prev_nonempty = false;
         for (int round = 0; round <= U && ok; ++round) {
             bool cur_nonempty = false;
+            if (warp == 2) TRACE(2, 1);
             if (round < U) {
                 // ------------------------------ P1 ------------------------------
                 const Seg sg = get_seg(p, round, head_local, rank);
                 float m[NH], l[NH];
 #pragma unroll
                 for (int i = 0; i < NH; ++i) {
-                    m[i] = -INFINITY;
+                    m[i] = kNegBig;
                     l[i] = 0.f;
                 }
                 cur_nonempty = sg.t1 > sg.t0;
@@ -543,38 +568,50 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_empty + 8 * sb);
-                    const int key = t * kTile + key_l;
-                    const bool boundary = (t * kTile + kTile > sg.T - p.a.n_q + 1);
+                    float sc[NH];
 #pragma unroll
-                    for (int i = 0; i < NH; ++i) {
-                        const int r = c0 + i;
-                        bool valid = r < R;
-                        if (boundary) valid = valid && (key <= sg.T - p.a.n_q + r / G);
-                        if (valid) {
-                            const float s = __uint_as_float(v[i]) * p.scale_log2;
-                            if (s > m[i] + 8.f) {
-                                l[i] *= ex2(m[i] - s);
-                                m[i] = s;
+                    for (int i = 0; i < NH; ++i) sc[i] = __uint_as_float(v[i]) * cs;
+                    if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
+                        // tile holds keys some window rows may not see (or keys beyond the context)
+                        const int key = t * kTile + key_l;
+                        int j = c0 / G, gg = c0 - j * G;
+#pragma unroll
+                        for (int i = 0; i < NH; ++i) {
+                            if (key > sg.T - p.a.n_q + j) sc[i] = kNegBig;
+                            if (++gg == G) {
+                                gg = 0;
+                                ++j;
                             }
-                            l[i] += ex2(s - m[i]);
                         }
                     }
+                    // running max is refreshed only when some lane's score beats it by 2^8: one
+                    // warp-uniform branch per tile, one ex2 per element otherwise
+                    bool need = false;
+#pragma unroll
+                    for (int i = 0; i < NH; ++i) need |= sc[i] > m[i] + 8.f;
+                    if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+                        for (int i = 0; i < NH; ++i) {
+                            const float mn = fmaxf(m[i], sc[i]);
+                            l[i] *= ex2(m[i] - mn);
+                            m[i] = mn;
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < NH; ++i) l[i] += ex2(sc[i] - m[i]);
                 }
                 if (!ok) break;
-                // reduce (m, l) over the 128 key lanes of this warpgroup's columns
+                if (warp == 2) TRACE(2, 2);
+                // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem
 #pragma unroll
                 for (int i = 0; i < NH; ++i) {
+                    float M = m[i];
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const float m2 = __shfl_xor_sync(0xffffffffu, m[i], o);
-                        const float l2 = __shfl_xor_sync(0xffffffffu, l[i], o);
-                        const float M = fmaxf(m[i], m2);
-                        const float a1 = (m[i] == -INFINITY) ? 0.f : l[i] * ex2(m[i] - M);
-                        const float a2 = (m2 == -INFINITY) ? 0.f : l2 * ex2(m2 - M);
-                        m[i] = M;
-                        l[i] = a1 + a2;
-                    }
-                    if (lane == 0) red[sw * 64 + i] = make_float2(m[i], l[i]);
+                    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                    float L = l[i] * ex2(m[i] - M);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+                    if (lane == 0) red[sw * 64 + i] = make_float2(M, L);
                 }
                 ok = group_sync(B.sm_sync, sync_n, ctl, 26);
                 if (!ok) break;
@@ -582,17 +619,17 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     const int tid = threadIdx.x - 64;  // 0..255
                     const int wgi = tid >> 7, ci = tid & 127;
                     if (ci < NH && wgi * NH + ci < R) {
-                        float M = -INFINITY;
+                        float M = kNegBig;
 #pragma unroll
                         for (int w = 0; w < 4; ++w) M = fmaxf(M, red[(wgi * 4 + w) * 64 + ci].x);
                         float L = 0.f;
 #pragma unroll
                         for (int w = 0; w < 4; ++w) {
                             const float2 ml = red[(wgi * 4 + w) * 64 + ci];
-                            if (ml.x > -INFINITY) L += ml.y * ex2(ml.x - M);
+                            L += ml.y * ex2(ml.x - M);
                         }
                         const int64_t base = (((int64_t)(round % kRing) * p.HG + head_local) * p.cph + rank) * R;
-                        p.ml_part[base + wgi * NH + ci] = make_float2(M, L);
+                        p.ml_part[base + wgi * NH + ci] = make_float2(M, cur_nonempty ? L : 0.f);
                     }
                 }
                 ok = group_sync(B.sm_sync, sync_n, ctl, 27);
@@ -602,6 +639,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     atomicAdd(p.counters + round * p.HG + head_local, 1);
                 }
             }
+            if (warp == 2) TRACE(2, 3);
             if (round >= 1 && ok) {
                 // ------------------------------ P2 ------------------------------
                 const Seg sg = get_seg(p, round - 1, head_local, rank);
@@ -610,7 +648,8 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     const uint32_t lb = prev_lse_idx & 1, lph = (prev_lse_idx >> 1) & 1;
                     ok = mbar_wait(B.lse_full + 8 * lb, lph, ctl, 21);
                     if (!ok) break;
-                    const float* lse2 = lse_s + lb * 128;
+                    const float4* lse4 = reinterpret_cast<const float4*>(lse_s + lb * 128 + c0);
+                    if (warp == 2) TRACE(2, 4);
                     for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                         const uint32_t sb = qk_idx & 1, sbph = (qk_idx >> 1) & 1;
                         ++qk_idx;
@@ -627,29 +666,50 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(B.s_empty + 8 * sb);
-                        ok = mbar_wait(B.p_empty + 8 * pb, pph ^ 1, ctl, 23);
-                        if (!ok) break;
                         const int key = t * kTile + key_l;
-                        const bool boundary = (t * kTile + kTile > sg.T - p.a.n_q + 1);
-                        uint8_t* p_hi = sgen + (s_p - sbase) + (pb * 2 + 0) * p_bytes;
-                        uint8_t* p_lo = sgen + (s_p - sbase) + (pb * 2 + 1) * p_bytes;
-                        const int kh = key_l >> 6, kk = key_l & 63;
-                        const int row_off = kh * (N * 128) + (kk & 7) * 2;
-                        const int chunk = kk >> 3;
+                        float pr[NH];
+#pragma unroll
+                        for (int i = 0; i < NH; i += 4) {
+                            const float4 ls = lse4[i >> 2];
+                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
+                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
+                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
+                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
+                        }
+                        if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
+                            int j = c0 / G, gg = c0 - j * G;
+#pragma unroll
+                            for (int i = 0; i < NH; ++i) {
+                                if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
+                                if (++gg == G) {
+                                    gg = 0;
+                                    ++j;
+                                }
+                            }
+                        }
                         float st = 0.f;
 #pragma unroll
-                        for (int i = 0; i < NH; ++i) {
-                            const int r = c0 + i;
-                            bool valid = r < R;
-                            if (boundary) valid = valid && (key <= sg.T - p.a.n_q + r / G);
-                            float pr = 0.f;
-                            if (valid) pr = ex2(__uint_as_float(v[i]) * p.scale_log2 - lse2[r]);
-                            if (r >= stat_r0) st += pr;
-                            const __nv_bfloat16 hi = __float2bfloat16_rn(pr);
-                            const __nv_bfloat16 lo = __float2bfloat16_rn(pr - __bfloat162float(hi));
-                            const int off = row_off + r * 128 + ((chunk ^ (i & 7)) << 4);
-                            *reinterpret_cast<__nv_bfloat16*>(p_hi + off) = hi;
-                            *reinterpret_cast<__nv_bfloat16*>(p_lo + off) = lo;
+                        for (int i = 0; i < NH; ++i) st += (c0 + i >= stat_r0) ? pr[i] : 0.f;
+                        ok = mbar_wait(B.p_empty + 8 * pb, pph ^ 1, ctl, 23);
+                        if (!ok) break;
+                        // P^T as the B operand, rows contiguous (8 rows = one 16-byte vector per key):
+                        // vector (row block nb, key k) at nb*2048 + (k/8)*128 + (k%8)*16
+                        uint8_t* p_hi = sgen + (s_p - sbase) + (pb * 2 + 0) * p_bytes + (wg * (NH / 8)) * 2048 +
+                                        (key_l >> 3) * 128 + (key_l & 7) * 16;
+                        uint8_t* p_lo = p_hi + p_bytes;
+#pragma unroll
+                        for (int nb = 0; nb < NH / 8; ++nb) {
+                            uint32_t hi[4], lo[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float a = pr[nb * 8 + 2 * q], b = pr[nb * 8 + 2 * q + 1];
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi[q]) : "f"(b), "f"(a));
+                                const float ra = a - __uint_as_float(hi[q] << 16);
+                                const float rb = b - __uint_as_float(hi[q] & 0xffff0000u);
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo[q]) : "f"(rb), "f"(ra));
+                            }
+                            *reinterpret_cast<uint4*>(p_hi + nb * 2048) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<uint4*>(p_lo + nb * 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                         }
                         if (t * kTile + kTile > sg.T) {
                             // ragged last tile: V rows at or beyond T may hold anything; zero them
@@ -666,14 +726,23 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                         __syncwarp();
                         if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
                         // column-split statistic: warpgroup 1 hands its partial sum to warpgroup 0
-                        float* tmp = stat_tmp + (t & 1) * 128;
-                        if (wg == 1) tmp[key_l] = st;
-                        ok = group_sync(B.sm_sync, sync_n, ctl, 28);
-                        if (!ok) break;
-                        if (wg == 0 && key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st + tmp[key_l];
+                        // (4 buffers / barriers: warpgroup 1 can run at most two tiles ahead)
+                        const uint32_t sq = stat_n & 3, sqph = (stat_n >> 2) & 1;
+                        ++stat_n;
+                        if (wg == 1) {
+                            stat_tmp[sq * 128 + key_l] = st;
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(B.stat_full + 8 * sq);
+                        } else {
+                            ok = mbar_wait(B.stat_full + 8 * sq, sqph, ctl, 28);
+                            if (!ok) break;
+                            if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st + stat_tmp[sq * 128 + key_l];
+                        }
                     }
                     if (!ok) break;
+                    __syncwarp();
                     if (lane == 0) mbar_arrive(B.lse_empty + 8 * lb);
+                    if (warp == 2) TRACE(2, 5);
                     // ---- epilogue: O^T (d on lanes, rows on columns) -> partial [r][d] ----
                     ok = mbar_wait(B.o_full, o_phase, ctl, 25);
                     if (!ok) break;
@@ -702,6 +771,7 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
             }
             if (cur_nonempty) prev_lse_idx = lse_n++;
             prev_nonempty = cur_nonempty;
+            if (warp == 2) TRACE(2, 6);
         }
     } else {
         // =========================== aux warps: LSE combine, O reduction ===========================
@@ -718,12 +788,19 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 p.o_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R * kD);
             for (int e = lo + tid; e < hi; e += 64) {
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int k = 0; k < p.cph; ++k) {
-                    const float4 x = __ldcg(src + (int64_t)k * E4 + e);
-                    acc.x += x.x;
-                    acc.y += x.y;
-                    acc.z += x.z;
-                    acc.w += x.w;
+                for (int k0 = 0; k0 < p.cph; k0 += 8) {  // batches of 8 independent loads
+                    float4 x[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        x[u] = (k0 + u < p.cph) ? __ldcg(src + (int64_t)(k0 + u) * E4 + e)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        acc.x += x[u].x;
+                        acc.y += x[u].y;
+                        acc.z += x[u].z;
+                        acc.w += x[u].w;
+                    }
                 }
                 const int r = e / (kD / 4), d4 = e - r * (kD / 4);
                 const int j = r / G, g = r - j * G;
@@ -740,19 +817,31 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                 if (sg.t1 > sg.t0) {
                     const uint32_t lb = lse_n & 1, lph = (lse_n >> 1) & 1;
                     ++lse_n;
+                    if (warp == 10) TRACE(3, 1);
                     ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
                     if (!ok) break;
+                    if (warp == 10) TRACE(3, 2);
                     __threadfence();
                     ok = mbar_wait(B.lse_empty + 8 * lb, lph ^ 1, ctl, 32);
                     if (!ok) break;
                     const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
+                    for (int r = R + tid; r < N; r += 64) lse_s[lb * 128 + r] = 1.0e30f;  // padded rows: P = 0
                     for (int r = tid; r < R; r += 64) {
-                        float M = -INFINITY;
-                        for (int k = 0; k < p.cph; ++k) M = fmaxf(M, __ldcg(src + (int64_t)k * R + r).x);
-                        float L = 0.f;
-                        for (int k = 0; k < p.cph; ++k) {
-                            const float2 ml = __ldcg(src + (int64_t)k * R + r);
-                            if (ml.x > -INFINITY) L += ml.y * exp2f(ml.x - M);
+                        float M = -INFINITY, L = 0.f;
+                        for (int k0 = 0; k0 < p.cph; k0 += 8) {  // batches of 8 independent loads
+                            float2 x[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                x[u] = (k0 + u < p.cph) ? __ldcg(src + (int64_t)(k0 + u) * R + r)
+                                                        : make_float2(0.f, 0.f);
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                if (x[u].y > 0.f) {
+                                    const float Mn = fmaxf(M, x[u].x);
+                                    L = L * exp2f(M - Mn) + x[u].y * exp2f(x[u].x - Mn);
+                                    M = Mn;
+                                }
+                            }
                         }
                         const float lse2 = M + log2f(L);
                         lse_s[lb * 128 + r] = lse2;
@@ -765,9 +854,11 @@ verify_sm100_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_const
                     ok = group_sync(B.aux_sync, sync_n, ctl, 33);
                     if (!ok) break;
                     if (tid == 0) mbar_arrive(B.lse_full + 8 * lb);
+                    if (warp == 10) TRACE(3, 3);
                 }
             }
             if (round >= 2) ok = reduce_unit(round - 2);
+            if (warp == 10) TRACE(3, 4);
         }
     }
 
@@ -803,7 +894,7 @@ EncodeTiledFn encode_fn()
 struct Plan {
     int HG, cph, n_units, N, n_slots, p_bufs, box_rows, boxes;
     size_t smem_bytes;
-    size_t ctr_off, ml_off, o_off, total;
+    size_t ctr_off, ml_off, o_off, total, trace_off;
 };
 
 int box_rows_for(int page_size)
@@ -865,6 +956,10 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, Plan* pl)
     pl->o_off = off;
     off += (size_t)kRing * pl->HG * pl->cph * R * kD * sizeof(float);
     pl->total = (off + 255) & ~(size_t)255;
+#ifdef SPEC_TRACE
+    pl->trace_off = pl->total;
+    pl->total += (size_t)nsm * 4 * 64 * sizeof(long long);
+#endif
     return true;
 }
 
@@ -974,6 +1069,10 @@ int verify_sm100_launch(const VerifyArgs& a, cudaStream_t stream)
     fp.o_part = reinterpret_cast<float*>(ws + pl.o_off);
     fp.status = reinterpret_cast<int*>(ws);
     fp.n_pages = n_pages;
+    fp.trace = nullptr;
+#ifdef SPEC_TRACE
+    fp.trace = reinterpret_cast<long long*>(ws + pl.trace_off);
+#endif
     if (cudaMemsetAsync(ws + pl.ctr_off, 0, (size_t)2 * pl.n_units * pl.HG * sizeof(int), stream) != cudaSuccess)
         return SPEC_ERR_CUDA;
     switch (pl.N / 2) {
