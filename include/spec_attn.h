@@ -56,7 +56,13 @@ enum {
 enum { SPEC_WS_VERIFY = 0, SPEC_WS_SELECT = 1, SPEC_WS_DRAFT = 2 };
 
 /* Verification kernel choice for spec_set_verify_impl(). */
-enum { SPEC_VERIFY_AUTO = 0, SPEC_VERIFY_GENERIC = 1, SPEC_VERIFY_TCGEN05 = 2 };
+enum {
+    SPEC_VERIFY_AUTO = 0,             /* tcgen05 when the shape allows it, else generic */
+    SPEC_VERIFY_GENERIC = 1,          /* plain FP32 CUDA-core kernels, every supported shape */
+    SPEC_VERIFY_TCGEN05 = 2,          /* tcgen05, either variant; unsupported shapes are an error */
+    SPEC_VERIFY_TCGEN05_TWOSWEEP = 3, /* K swept twice (second sweep from L2), any context length */
+    SPEC_VERIFY_TCGEN05_CACHED = 4    /* score tiles cached in tensor memory, K and V read once */
+};
 
 /*
  * Dense KV cache of one or more layers (the K_{l,h}, V_{l,h} of Eq. 5), READ-ONLY.
@@ -173,8 +179,8 @@ int spec_read_status(const void* workspace, void* cuda_stream);
  * when the shape allows it).  Returns the previous setting, or SPEC_ERR_INVALID_ARG. */
 int spec_set_verify_impl(int impl);
 
-/* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC or
- * SPEC_VERIFY_TCGEN05; 0 before the first call). */
+/* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC,
+ * SPEC_VERIFY_TCGEN05_TWOSWEEP or SPEC_VERIFY_TCGEN05_CACHED; 0 before the first call). */
 int spec_last_verify_impl(void);
 
 /* Number of kernels this library has launched since load (host-side counter). */

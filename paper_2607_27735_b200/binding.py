@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libspec_attn.so")
 
 WS_VERIFY, WS_SELECT, WS_DRAFT = 0, 1, 2
-VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05 = 0, 1, 2
+VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCGEN05_CACHED = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",

@@ -1,0 +1,257 @@
+// Shared device-side pieces of the sm_100a verification kernels: PTX wrappers for mbarrier,
+// TMA (cp.async.bulk.tensor, never multicast), tcgen05 (alloc / mma / commit / ld / fences),
+// UMMA shared-memory descriptors, bounded waits, and the work decomposition.
+#pragma once
+
+#include <cuda.h>
+
+#include "spec_common.cuh"
+
+namespace spec {
+namespace sm100 {
+
+constexpr int kTile = 128;            // keys per tile = UMMA M
+constexpr int kD = 128;               // head_dim of the fast path
+constexpr int kSlotBytes = 32768;     // one K or V tile: 2 halves x 128 rows x 128 B (SW128)
+constexpr int kThreads = 384;
+constexpr int kRing = 4;              // partial buffers are recycled every kRing units
+constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // about a second of SM clocks
+constexpr uint64_t kEvictFirst = 0x12F0000000000000ull;
+constexpr uint64_t kEvictLast = 0x14F0000000000000ull;
+constexpr int kTmemCols = 512;
+constexpr int kColS0 = 0, kColS1 = 128, kColO = 256;
+
+struct FastParams {
+    VerifyArgs a;
+    int HG, NHG, cph, n_units, N, R, G;
+    int n_slots, p_bufs;
+    int box_rows, boxes;              // TMA boxes per 64-wide half of a tile
+    float scale_log2;
+    int* counters;                    // [2][n_units * HG]: P1 partials done, O partials done
+    float2* ml_part;                  // [kRing][HG][cph][R]
+    float* o_part;                    // [kRing][HG][cph][R][kD]
+    int* status;
+    int n_pages;
+    int n_cache;                      // S tiles the TMEM cache holds (cached variant)
+    long long* trace;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t globaltimer()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Non-blocking probe (try_wait may suspend the thread for a while; a scheduler loop must not).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* v)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ int ld_acquire(const int* p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4, uint64_t hint)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(hint) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// K-major operand, 128-byte swizzle: rows of 128 B, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand, 128-byte swizzle: 64-element MN blocks 16 KiB apart (leading offset),
+// 8-row K groups 1024 B apart (stride offset).
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1024ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// ---------------------------------------------------------------------------------------------
+
+#ifdef SPEC_TRACE
+// Development aid (not compiled by default): per-CTA, per-role clock64 stamps in the workspace.
+#define TRACE(role, slot) do { if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 60) \
+    p.trace[((int64_t)blockIdx.x * 4 + (role)) * 64 + trace_n[role]++] = ((long long)(slot) << 48) | (clock64() & 0xffffffffffffll); } while (0)
+#define TRACEV(role, slot, val) do { if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 60) \
+    p.trace[((int64_t)blockIdx.x * 4 + (role)) * 64 + trace_n[role]++] = ((long long)(slot) << 48) | ((long long)(val) & 0xffffffffffffll); } while (0)
+#define TCLK() clock64()
+#else
+#define TRACE(role, slot) do { } while (0)
+#define TRACEV(role, slot, val) do { } while (0)
+#define TCLK() 0ll
+#endif
+
+struct Ctl {
+    volatile int* abort_flag;  // shared
+    int* status;               // global status word (+ diagnostics in the following ints)
+};
+
+static __device__ __noinline__ void report_timeout(const Ctl& c, int where)
+{
+    if (atomicCAS(c.status, 0, SPEC_ERR_TIMEOUT) == 0) {
+        c.status[1] = where;
+        c.status[2] = blockIdx.x;
+        c.status[3] = threadIdx.x;
+    }
+    *c.abort_flag = 1;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const Ctl& c, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0) {
+            if (*c.abort_flag) return false;
+            if (clock64() - t0 > kTimeoutCycles) {
+                report_timeout(c, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool counter_wait(const int* ctr, int target, const Ctl& c, int where)
+{
+    if (ld_acquire(ctr) >= target) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (ld_acquire(ctr) < target) {
+        __nanosleep(32);
+        if ((++spins & 63u) == 0) {
+            if (*c.abort_flag) return false;
+            if (clock64() - t0 > kTimeoutCycles) {
+                report_timeout(c, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// Barrier among the warps of one role, built on an mbarrier so that the wait is bounded like
+// every other wait (a hardware named barrier could not be abandoned after a timeout).
+__device__ __forceinline__ bool group_sync(uint32_t bar, uint32_t& n, const Ctl& c, int where)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+    const bool ok = mbar_wait(bar, n & 1, c, where);
+    ++n;
+    return ok;
+}
+
+struct Seg {
+    int layer, b, h, T, t0, t1;
+    int64_t prob;
+};
+
+__device__ __forceinline__ Seg get_seg(const FastParams& p, int unit, int head_local, int rank)
+{
+    Seg s;
+    const int per_layer = p.a.kv.batch * p.NHG;
+    s.layer = unit / per_layer;
+    const int rem = unit - s.layer * per_layer;
+    s.b = rem / p.NHG;
+    s.h = (rem - s.b * p.NHG) * p.HG + head_local;
+    s.T = p.a.ctx_len[s.b];
+    const int nb = (s.T + kTile - 1) / kTile;
+    s.t0 = (int)((int64_t)rank * nb / p.cph);
+    s.t1 = (int)((int64_t)(rank + 1) * nb / p.cph);
+    s.prob = ((int64_t)s.layer * p.a.kv.batch + s.b) * p.a.kv.n_kv_heads + s.h;
+    return s;
+}
+
+// launchers of the two kernel variants (host)
+int launch_twosweep(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
+                    int grid, size_t smem_bytes, cudaStream_t stream);
+int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
+                  int grid, size_t smem_bytes, cudaStream_t stream);
+
+template <int NH>
+__device__ __forceinline__ void load_cols(uint32_t taddr, uint32_t* v)
+{
+#pragma unroll
+    for (int c = 0; c < NH; c += 8) tmem_ld8(taddr + c, v + c);
+    tc_wait_ld();
+}
+
+}  // namespace sm100
+}  // namespace spec

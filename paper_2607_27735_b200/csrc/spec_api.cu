@@ -64,10 +64,9 @@ static int make_view(const spec_kv_t* kv, KvView* out)
     return SPEC_OK;
 }
 
-static bool use_tcgen05(const KvView& kv, int n_q, int impl)
+static int sm100_variant(int impl)
 {
-    if (impl == SPEC_VERIFY_GENERIC) return false;
-    return verify_sm100_supported(kv, n_q);
+    return impl == SPEC_VERIFY_TCGEN05_TWOSWEEP ? 1 : (impl == SPEC_VERIFY_TCGEN05_CACHED ? 2 : 0);
 }
 
 }  // namespace spec
@@ -105,14 +104,21 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
     a.workspace_bytes = workspace_bytes;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int impl = g_verify_impl.load();
-    const bool fast = use_tcgen05(a.kv, n_q, impl);
-    if (impl == SPEC_VERIFY_TCGEN05 && !fast) return SPEC_ERR_UNSUPPORTED_SHAPE;
-    const size_t need = fast ? verify_sm100_workspace(a.kv, n_q, max_ctx_len)
-                             : verify_generic_workspace(a.kv, n_q, max_ctx_len);
-    if (workspace_bytes < need) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+    if (impl != SPEC_VERIFY_GENERIC) {
+        int used = 0;
+        const int rc2 = verify_sm100_launch(a, sm100_variant(impl), stream, &used);
+        if (rc2 == SPEC_OK) {
+            g_last_verify_impl.store(used == 2 ? SPEC_VERIFY_TCGEN05_CACHED : SPEC_VERIFY_TCGEN05_TWOSWEEP);
+            return SPEC_OK;
+        }
+        // an explicit tcgen05 request fails loudly; AUTO falls through to the generic kernels only
+        // when the shape is outside the fast path
+        if (impl != SPEC_VERIFY_AUTO || rc2 != SPEC_ERR_UNSUPPORTED_SHAPE) return rc2;
+    }
+    if (workspace_bytes < verify_generic_workspace(a.kv, n_q, max_ctx_len)) return SPEC_ERR_WORKSPACE_TOO_SMALL;
     if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;
-    g_last_verify_impl.store(fast ? SPEC_VERIFY_TCGEN05 : SPEC_VERIFY_GENERIC);
-    return fast ? verify_sm100_launch(a, stream) : verify_generic_launch(a, stream);
+    g_last_verify_impl.store(SPEC_VERIFY_GENERIC);
+    return verify_generic_launch(a, stream);
 }
 
 int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
@@ -169,7 +175,7 @@ size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t
     if (which == SPEC_WS_VERIFY) {
         if (n_q < 1 || n_q > 32 || max_ctx_len < n_q) return 0;
         size_t g = verify_generic_workspace(v, n_q, max_ctx_len);
-        size_t f = verify_sm100_supported(v, n_q) ? verify_sm100_workspace(v, n_q, max_ctx_len) : 0;
+        size_t f = verify_sm100_workspace(v, n_q, max_ctx_len);
         return g > f ? g : f;
     }
     if (which == SPEC_WS_DRAFT) {
@@ -192,7 +198,7 @@ int spec_read_status(const void* workspace, void* cuda_stream)
 
 int spec_set_verify_impl(int impl)
 {
-    if (impl < SPEC_VERIFY_AUTO || impl > SPEC_VERIFY_TCGEN05) return SPEC_ERR_INVALID_ARG;
+    if (impl < SPEC_VERIFY_AUTO || impl > SPEC_VERIFY_TCGEN05_CACHED) return SPEC_ERR_INVALID_ARG;
     return g_verify_impl.exchange(impl);
 }
 

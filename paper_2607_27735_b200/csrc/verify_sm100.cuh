@@ -1,9 +1,12 @@
-// Interface of the tcgen05 / TMA verification kernel (verify_sm100.cu).
+// Interface of the sm_100a (tcgen05 / TMA) verification path (verify_sm100.cu).
 #pragma once
 #include "spec_common.cuh"
 
 namespace spec {
-bool verify_sm100_supported(const KvView& kv, int n_q);
+// variant: 0 = automatic (score-cache kernel when a CTA's share of keys fits tensor memory,
+// else the two-sweep kernel), 1 = two-sweep only, 2 = score-cache only
+bool verify_sm100_supported(const KvView& kv, int n_q, int variant);
 size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len);
-int verify_sm100_launch(const VerifyArgs& a, cudaStream_t stream);
+// Clears the status word itself; *used_variant gets 1 (two-sweep) or 2 (score-cache).
+int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant);
 }  // namespace spec

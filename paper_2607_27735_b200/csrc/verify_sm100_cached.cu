@@ -1,0 +1,698 @@
+// Verification attention + Eq. 3 statistic for sm_100a, score-cache variant: one persistent,
+// warp-specialised kernel on TMA (no multicast), tcgen05.mma with TMEM accumulators and
+// mbarrier pipelines, in which K and V are each read exactly once from memory.
+//
+// Eq. 3 sums softmax PROBABILITIES over the window rows, so a key's contribution
+// exp(s - LSE_row) needs every row's global normaliser, which is known only after all keys
+// of the head were seen.  Instead of sweeping K twice, every CTA keeps the score tiles
+// S^T = K Q^T of its share of the keys in tensor memory (512 columns per SM hold the output
+// accumulator plus (512 - 2N) / N tiles of 128 keys x N rows):
+//   P1  stream K, S^T tile -> TMEM (kept), per-row running (max, sum) -> partial LSE;
+//   --  partials of the CTAs sharing the head are combined into the row LSE (the only
+//       cross-CTA dependency; V tiles keep streaming into shared memory meanwhile);
+//   P2  stream V, P = exp2(S - LSE) from the cached tile, exactly normalised: column sums ->
+//       stats, O^T += V^T [P_hi | P_lo]^T on the tensor cores (bf16 hi + lo split of P keeps
+//       the 2e-3 bar when one key takes most of the mass).
+// A unit (a group of KV heads of one (layer, sequence)) is cut so that a CTA's share of keys
+// fits the cache; larger shares go to the two-sweep variant.
+//
+// TMEM tile layout: keys on the 128 lanes, the R = n_q * group query rows on the columns, so
+// one thread owns one key: the statistic is a thread-local sum and the P1 row max/sum is
+// thread-local state reduced once per unit.
+//
+// Roles (384 threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer (+ TMEM alloc), warps
+// 2..3 reduce the per-CTA O partials (fixed order: deterministic), warps 4..11 two softmax
+// warpgroups that split the columns.
+//
+// All CTAs must be co-resident (they wait on each other's partials): the grid never exceeds
+// the SM count at one CTA per SM and the launch is cooperative.  Every wait is bounded; on
+// expiry the kernel records SPEC_ERR_TIMEOUT in the status word and drains.
+#include "sm100_common.cuh"
+
+namespace spec {
+namespace sm100 {
+
+namespace {
+
+constexpr int kMaxCache = 32;
+
+struct CBars {  // mbarrier addresses (shared space)
+    uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_free, p_full, p_empty, o_full, o_empty, sm_sync,
+        aux_sync, stat_full;
+};
+
+template <int NH>
+__global__ void __launch_bounds__(kThreads, 1)
+verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                     const __grid_constant__ CUtensorMap tm_q, const FastParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));  // generic pointer to the aligned base
+
+    const int N = p.N, R = p.R, G = p.G;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int head_local = blockIdx.x / p.cph, rank = blockIdx.x % p.cph;
+    const int q_bytes = N * 256;                       // one Q buffer: 2 halves x N rows x 128 B
+    const int p_bytes = ((2 * N + 63) / 64) * 16384;   // one P buffer: [hi | lo] rows, 64-row blocks x 128 keys x 128 B
+
+    const uint32_t s_slots = sbase;
+    const uint32_t s_q = s_slots + p.n_slots * kSlotBytes;
+    const uint32_t s_p = s_q + 2 * q_bytes;
+    const uint32_t s_misc = s_p + p.p_bufs * p_bytes;
+    uint8_t* misc = sgen + (s_misc - sbase);
+    CBars B;
+    {
+        uint32_t o = s_misc;
+        B.slot_full = o; o += 8 * 8;
+        B.slot_empty = o; o += 8 * 8;
+        B.q_full = o; o += 16;
+        B.q_empty = o; o += 16;
+        B.s_full = o; o += 8 * kMaxCache;
+        B.s_free = o; o += 8 * kMaxCache;
+        B.p_full = o; o += 16;
+        B.p_empty = o; o += 16;
+        B.o_full = o; o += 8;
+        B.o_empty = o; o += 8;
+        B.sm_sync = o; o += 8;
+        B.aux_sync = o; o += 8;
+        B.stat_full = o; o += 32;
+    }
+    float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128]
+    float* stat_tmp = reinterpret_cast<float*>(misc + 2048);              // [4][128]
+    float2* red = reinterpret_cast<float2*>(misc + 4096);                 // [8 warps][64] (m, l)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 8192 - 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    Ctl ctl{abort_flag, p.status};
+#ifdef SPEC_TRACE
+    int trace_n[4] = {0, 0, 0, 0};
+#endif
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.n_slots; ++i) {
+            mbar_init(B.slot_full + 8 * i, 1);
+            mbar_init(B.slot_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < kMaxCache; ++i) {
+            mbar_init(B.s_full + 8 * i, 1);
+            mbar_init(B.s_free + 8 * i, 8);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(B.q_full + 8 * i, 1);
+            mbar_init(B.q_empty + 8 * i, 1);
+            mbar_init(B.p_full + 8 * i, 8);
+            mbar_init(B.p_empty + 8 * i, 1);
+        }
+        mbar_init(B.o_full, 1);
+        mbar_init(B.o_empty, 8);
+        mbar_init(B.sm_sync, 8);
+        mbar_init(B.aux_sync, 2);
+        for (int i = 0; i < 4; ++i) mbar_init(B.stat_full + 8 * i, 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // zero the Q buffers once: rows R..N-1 are padding the TMA never writes
+    for (int i = threadIdx.x; i < 2 * q_bytes / 16; i += kThreads)
+        *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
+    for (int r = R + threadIdx.x; r < 128; r += kThreads) lse_s[r] = 1.0e30f;  // padded rows: P = 0
+    fence_proxy_async();
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int U = p.n_units;
+    const uint32_t col_o = 0, col_s = 2 * N;  // O^T (hi | lo) first, then the cached S^T tiles
+
+    if (warp == 0) {
+        // =========================== TMA producer ===========================
+        uint32_t slot_idx = 0, qn = 0;
+        const int boxes = p.boxes, box_rows = p.box_rows;
+        const uint32_t box_bytes = box_rows * 128;
+        bool ok = true;
+        auto load_tile = [&](const CUtensorMap* map, const Seg& sg, int tile) -> bool {
+            const uint32_t s = slot_idx % p.n_slots, ph = (slot_idx / p.n_slots) & 1;
+            ++slot_idx;
+            if (!mbar_wait(B.slot_empty + 8 * s, ph ^ 1, ctl, 1)) return false;
+            // boxes of this tile that hold at least one key < T (pages past the context may not exist)
+            const int key0 = tile * kTile;
+            const int n_box = min(boxes, (sg.T - key0 + box_rows - 1) / box_rows);
+            if (lane == 0) mbar_expect_tx(B.slot_full + 8 * s, 2u * n_box * box_bytes);
+            __syncwarp();
+            for (int i = lane; i < 2 * n_box; i += 32) {
+                const int half = i / n_box, bx = i - half * n_box;
+                const int pos = key0 + bx * box_rows;
+                const int page = pos / p.a.kv.page_size, slot_in_page = pos - page * p.a.kv.page_size;
+                int phys = p.a.kv.page_table ? __ldg(p.a.kv.page_table + (int64_t)sg.b * p.a.kv.max_pages + page)
+                                             : sg.b * p.a.kv.max_pages + page;
+                if (phys < 0 || phys >= p.n_pages) {
+                    set_status(p.status, SPEC_ERR_BAD_INDEX);
+                    phys = 0;
+                }
+                const uint32_t dst = s_slots + s * kSlotBytes + half * 16384 + bx * box_bytes;
+                tma_load_5d(dst, map, B.slot_full + 8 * s, half * 64, slot_in_page, sg.h, phys, sg.layer, kEvictFirst);
+            }
+            __syncwarp();
+            return true;
+        };
+        for (int u = 0; u < U && ok; ++u) {
+            const Seg sg = get_seg(p, u, head_local, rank);
+            if (sg.t1 <= sg.t0) continue;
+            TRACE(0, 1);
+            const uint32_t qb = qn & 1, qph = (qn >> 1) & 1;
+            ++qn;
+            ok = mbar_wait(B.q_empty + 8 * qb, qph ^ 1, ctl, 2);
+            if (!ok) break;
+            if (lane == 0) {
+                mbar_expect_tx(B.q_full + 8 * qb, 2u * R * 128);
+                const int row0 = (sg.layer * p.a.kv.batch + sg.b) * p.a.n_q;
+                tma_load_3d(s_q + qb * q_bytes, &tm_q, B.q_full + 8 * qb, 0, sg.h * G, row0);
+                tma_load_3d(s_q + qb * q_bytes + N * 128, &tm_q, B.q_full + 8 * qb, 64, sg.h * G, row0);
+            }
+            __syncwarp();
+            for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t);
+            TRACE(0, 2);
+            for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_v, sg, t);
+            TRACE(0, 3);
+        }
+        if (!ok) {  // let copies in flight land before the CTA's shared memory is released
+            const long long t0 = clock64();
+            while (clock64() - t0 < 400000ll) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer ===========================
+        if (lane == 0) {
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+            // O^T += V^T [P_hi | P_lo]^T : A = V^T and B = P^T both MN-major, N = 2 * rows
+            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                                      ((uint32_t)((2 * N) >> 3) << 17) | ((128u >> 4) << 24);
+            // Two independent queues, issued in whichever order their inputs become ready: the
+            // QK^T tiles of unit u+1 may overtake the P V tiles of unit u that still wait for P.
+            struct Queue {
+                int u = -1, t = 0, t0 = 0, t1 = 0;
+                uint32_t slot_base = 0;  // ring index of the unit's first K tile
+                uint32_t next_base = 0;  // ring index where the following unit starts
+                uint32_t qn = 0, qb = 0, qph = 0;
+                bool done = false;
+            } qq, pq;
+            auto seek = [&](Queue& c) {  // advance to the next unit with tiles
+                for (;;) {
+                    ++c.u;
+                    if (c.u >= U) {
+                        c.done = true;
+                        return;
+                    }
+                    const Seg sg = get_seg(p, c.u, head_local, rank);
+                    if (sg.t1 > sg.t0) {
+                        c.t0 = sg.t0;
+                        c.t1 = sg.t1;
+                        c.t = sg.t0;
+                        c.slot_base = c.next_base;
+                        c.next_base += 2 * (sg.t1 - sg.t0);
+                        c.qb = c.qn & 1;
+                        c.qph = (c.qn >> 1) & 1;
+                        ++c.qn;
+                        return;
+                    }
+                }
+            };
+            seek(qq);
+            seek(pq);
+            uint32_t sfree_par = 0;  // per cache region: parity of the next "region free" phase
+            uint32_t pv_idx = 0, o_phase = 0;
+            bool ok = true;
+            auto qk_ready = [&]() -> bool {
+                const int c = qq.t - qq.t0;
+                const uint32_t slot = qq.slot_base + c;
+                const uint32_t s = slot % p.n_slots, sph = (slot / p.n_slots) & 1;
+                if (c == 0 && !mbar_test_wait(B.q_full + 8 * qq.qb, qq.qph)) return false;
+                if (!mbar_test_wait(B.slot_full + 8 * s, sph)) return false;
+                return mbar_test_wait(B.s_free + 8 * c, ((sfree_par >> c) & 1) ^ 1);
+            };
+            auto issue_qk = [&]() {
+                const int c = qq.t - qq.t0;
+                const uint32_t slot = qq.slot_base + c;
+                const uint32_t s = slot % p.n_slots;
+                sfree_par ^= 1u << c;
+                tc_fence_after();
+                const uint32_t k_addr = s_slots + s * kSlotBytes;
+                const uint32_t q_addr = s_q + qq.qb * q_bytes;
+                const uint32_t d_s = tmem_base + col_s + c * N;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t a = desc_kmajor(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
+                    const uint64_t b = desc_kmajor(q_addr + (ks >> 2) * (N * 128) + (ks & 3) * 32);
+                    tc_mma(d_s, a, b, idesc_qk, ks ? 1u : 0u);
+                }
+                tc_commit(B.s_full + 8 * c);
+                tc_commit(B.slot_empty + 8 * s);
+                if (qq.t == qq.t1 - 1) tc_commit(B.q_empty + 8 * qq.qb);  // last use of this Q buffer
+                if (++qq.t == qq.t1) seek(qq);
+            };
+            auto pv_ready = [&]() -> bool {
+                const int c = pq.t - pq.t0;
+                const uint32_t slot = pq.slot_base + (pq.t1 - pq.t0) + c;
+                const uint32_t s = slot % p.n_slots, sph = (slot / p.n_slots) & 1;
+                const uint32_t pb = pv_idx % p.p_bufs, pph = (pv_idx / p.p_bufs) & 1;
+                if (!mbar_test_wait(B.p_full + 8 * pb, pph)) return false;
+                if (!mbar_test_wait(B.slot_full + 8 * s, sph)) return false;
+                if (c == 0 && !mbar_test_wait(B.o_empty, o_phase ^ 1)) return false;
+                return true;
+            };
+            auto issue_pv = [&]() {
+                const int c = pq.t - pq.t0;
+                const uint32_t slot = pq.slot_base + (pq.t1 - pq.t0) + c;
+                const uint32_t s = slot % p.n_slots;
+                const uint32_t pb = pv_idx % p.p_bufs;
+                ++pv_idx;
+                const bool first = c == 0, last = pq.t == pq.t1 - 1;
+                tc_fence_after();
+                const uint32_t v_addr = s_slots + s * kSlotBytes;
+                const uint32_t p_addr = s_p + pb * p_bytes;
+                const uint32_t d_o = tmem_base + col_o;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t a = desc_mnmajor(v_addr + ks * 2048);
+                    const uint64_t b = desc_mnmajor(p_addr + ks * 2048);
+                    tc_mma(d_o, a, b, idesc_pv, (first && ks == 0) ? 0u : 1u);
+                }
+                tc_commit(B.slot_empty + 8 * s);
+                tc_commit(B.p_empty + 8 * pb);
+                if (last) {
+                    tc_commit(B.o_full);
+                    o_phase ^= 1;
+                }
+                if (++pq.t == pq.t1) seek(pq);
+            };
+            long long t_idle = clock64();
+            uint32_t spins = 0;
+            while (ok && !(qq.done && pq.done)) {
+                bool progressed = false;
+                // a unit's P V tiles can only follow its own QK^T tiles
+                if (!pq.done && (qq.done || qq.u > pq.u) && pv_ready()) {
+                    issue_pv();
+                    progressed = true;
+                }
+                if (!qq.done && qk_ready()) {
+                    issue_qk();
+                    progressed = true;
+                }
+                if (progressed) {
+                    spins = 0;
+                } else if ((++spins & 63u) == 0) {
+                    if (spins == 64) t_idle = clock64();
+                    if (*ctl.abort_flag) ok = false;
+                    else if (clock64() - t_idle > kTimeoutCycles) {
+                        report_timeout(ctl, 16);
+                        ok = false;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp < 4) {
+        // =========================== O reduction warps ===========================
+        const int tid = threadIdx.x - 64;  // 0..63
+        bool ok = true;
+        for (int unit = 0; unit < U && ok; ++unit) {
+            if (lane == 0) ok = counter_wait(p.counters + U * p.HG + unit * p.HG + head_local, p.cph, ctl, 30);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            __threadfence();
+            if (warp == 2) TRACE(3, 1);
+            const Seg sg = get_seg(p, unit, head_local, rank);
+            const int E4 = R * kD / 4;
+            const int lo = (int)((int64_t)rank * E4 / p.cph), hi = (int)((int64_t)(rank + 1) * E4 / p.cph);
+            const float4* src = reinterpret_cast<const float4*>(
+                p.o_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R * kD);
+            for (int e = lo + tid; e < hi; e += 64) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k0 = 0; k0 < p.cph; k0 += 16) {  // batches of 16 independent loads
+                    float4 x[16];
+#pragma unroll
+                    for (int u = 0; u < 16; ++u)
+                        x[u] = (k0 + u < p.cph) ? __ldcg(src + (int64_t)(k0 + u) * E4 + e)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int u = 0; u < 16; ++u) {
+                        acc.x += x[u].x;
+                        acc.y += x[u].y;
+                        acc.z += x[u].z;
+                        acc.w += x[u].w;
+                    }
+                }
+                const int r = e / (kD / 4), d4 = e - r * (kD / 4);
+                const int j = r / G, g = r - j * G;
+                const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
+                reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
+            }
+            if (warp == 2) TRACE(3, 2);
+        }
+    } else {
+        // =========================== softmax warpgroups ===========================
+        const int sw = warp - 4;                 // 0..7
+        const int wg = sw >> 2;                  // column half
+        const int quarter = warp & 3;            // TMEM lane quarter this warp may touch
+        const int key_l = quarter * 32 + lane;   // key within the tile (P1/P2) or d (epilogue)
+        const int tid_s = threadIdx.x - 128;     // 0..255
+        const int c0 = wg * NH;                  // first column of this warpgroup
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const int stat_r0 = p.a.first_stat_row * G;
+        const float cs = p.scale_log2;
+        constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
+        uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, stat_n = 0, sfull_par = 0;
+        bool ok = true;
+        int pend_unit = -1;                      // unit whose O accumulator still waits for its epilogue
+        bool pend_nonempty = false;
+
+        // O^T (d on lanes, rows on columns, hi and lo parts) -> this CTA's partial [r][d]
+        auto epilogue = [&](int unit, bool nonempty) -> bool {
+            const int64_t obase = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R * kD;
+            if (nonempty) {
+                if (!mbar_wait(B.o_full, o_phase, ctl, 25)) return false;
+                o_phase ^= 1;
+                tc_fence_after();
+                uint32_t v[NH], w[NH];
+                load_cols<NH>(t_lane + col_o + c0, v);
+                load_cols<NH>(t_lane + col_o + N + c0, w);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(B.o_empty);
+#pragma unroll
+                for (int i = 0; i < NH; ++i) {
+                    const int r = c0 + i;
+                    if (r < R) p.o_part[obase + (int64_t)r * kD + key_l] = __uint_as_float(v[i]) + __uint_as_float(w[i]);
+                }
+            } else {
+                for (int i = tid_s; i < R * kD; i += 256) p.o_part[obase + i] = 0.f;
+            }
+            if (!group_sync(B.sm_sync, sync_n, ctl, 29)) return false;
+            if (tid_s == 0) {
+                __threadfence();
+                atomicAdd(p.counters + U * p.HG + unit * p.HG + head_local, 1);
+            }
+            return true;
+        };
+
+        for (int unit = 0; unit < U && ok; ++unit) {
+            const Seg sg = get_seg(p, unit, head_local, rank);
+            const int n_t = sg.t1 - sg.t0;
+            const bool nonempty = n_t > 0;
+            if (warp == 4) TRACE(2, 1);
+            // ------------------------------ P1 ------------------------------
+            float m[NH], l[NH];
+#pragma unroll
+            for (int i = 0; i < NH; ++i) {
+                m[i] = kNegBig;
+                l[i] = 0.f;
+            }
+            for (int c = 0; c < n_t && ok; ++c) {
+                const int t = sg.t0 + c;
+                ok = mbar_wait(B.s_full + 8 * c, (sfull_par >> c) & 1, ctl, 20);
+                if (!ok) break;
+                sfull_par ^= 1u << c;
+                tc_fence_after();
+                uint32_t v[NH];
+                load_cols<NH>(t_lane + col_s + c * N + c0, v);
+                float sc[NH];
+#pragma unroll
+                for (int i = 0; i < NH; ++i) sc[i] = __uint_as_float(v[i]) * cs;
+                if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
+                    // tile holds keys some window rows may not see (or keys beyond the context)
+                    const int key = t * kTile + key_l;
+                    int j = c0 / G, gg = c0 - j * G;
+#pragma unroll
+                    for (int i = 0; i < NH; ++i) {
+                        if (key > sg.T - p.a.n_q + j) sc[i] = kNegBig;
+                        if (++gg == G) {
+                            gg = 0;
+                            ++j;
+                        }
+                    }
+                }
+                // running max is refreshed only when some lane's score beats it by 2^8: one
+                // warp-uniform branch per tile, one ex2 per element otherwise
+                bool need = false;
+#pragma unroll
+                for (int i = 0; i < NH; ++i) need |= sc[i] > m[i] + 8.f;
+                if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+                    for (int i = 0; i < NH; ++i) {
+                        const float mn = fmaxf(m[i], sc[i]);
+                        l[i] *= ex2(m[i] - mn);
+                        m[i] = mn;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < NH; ++i) l[i] += ex2(sc[i] - m[i]);
+            }
+            if (!ok) break;
+            if (warp == 4) TRACE(2, 2);
+            // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem
+#pragma unroll
+            for (int i = 0; i < NH; ++i) {
+                float M = m[i];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                float Ls = l[i] * ex2(m[i] - M);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
+                if (lane == 0) red[sw * 64 + i] = make_float2(M, Ls);
+            }
+            ok = group_sync(B.sm_sync, sync_n, ctl, 26);
+            if (!ok) break;
+            {
+                const int wgi = tid_s >> 7, ci = tid_s & 127;
+                if (ci < NH && wgi * NH + ci < R) {
+                    float M = kNegBig;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) M = fmaxf(M, red[(wgi * 4 + w) * 64 + ci].x);
+                    float Ls = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float2 ml = red[(wgi * 4 + w) * 64 + ci];
+                        Ls += ml.y * ex2(ml.x - M);
+                    }
+                    const int64_t base = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R;
+                    p.ml_part[base + wgi * NH + ci] = make_float2(M, nonempty ? Ls : 0.f);
+                }
+            }
+            ok = group_sync(B.sm_sync, sync_n, ctl, 27);
+            if (!ok) break;
+            if (tid_s == 0) {
+                __threadfence();
+                atomicAdd(p.counters + unit * p.HG + head_local, 1);
+            }
+            if (warp == 4) TRACE(2, 3);
+            // ---- while the other CTAs finish their P1: drain the previous unit's accumulator ----
+            if (pend_unit >= 0) {
+                ok = epilogue(pend_unit, pend_nonempty);
+                if (!ok) break;
+                pend_unit = -1;
+            }
+            if (warp == 4) TRACE(2, 4);
+            if (nonempty) {
+                // ---- row LSE from the partials of the CTAs that share this head ----
+                if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                __threadfence();
+                if (warp == 4) TRACE(2, 5);
+                const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
+                const int tpr = 256 / R;          // threads per row (R <= 128)
+                const int r = tid_s % R, sub = tid_s / R;
+                float M = kNegBig, Ls = 0.f;
+                if (sub < tpr) {
+                    for (int k0 = sub; k0 < p.cph; k0 += 8 * tpr) {  // batches of 8 independent loads
+                        float2 x[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            x[u] = (k0 + u * tpr < p.cph) ? __ldcg(src + (int64_t)(k0 + u * tpr) * R + r)
+                                                          : make_float2(kNegBig, 0.f);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const float Mn = fmaxf(M, x[u].x);
+                            Ls = Ls * ex2(M - Mn) + x[u].y * ex2(x[u].x - Mn);
+                            M = Mn;
+                        }
+                    }
+                    red[sub * R + r] = make_float2(M, Ls);  // tpr * R <= 256 entries
+                }
+                ok = group_sync(B.sm_sync, sync_n, ctl, 21);
+                if (!ok) break;
+                if (tid_s < R) {
+                    float Mx = kNegBig;
+                    for (int s2 = 0; s2 < tpr; ++s2) Mx = fmaxf(Mx, red[s2 * R + tid_s].x);
+                    float Lx = 0.f;
+                    for (int s2 = 0; s2 < tpr; ++s2) {
+                        const float2 ml = red[s2 * R + tid_s];
+                        Lx += ml.y * ex2(ml.x - Mx);
+                    }
+                    const float lse2 = Mx + log2f(Lx);
+                    lse_s[tid_s] = lse2;
+                    if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
+                        const int j = tid_s / G, g = tid_s - j * G;
+                        const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
+                        p.a.lse[row] = lse2 * 0.69314718055994530942f;
+                    }
+                }
+                ok = group_sync(B.sm_sync, sync_n, ctl, 22);
+                if (!ok) break;
+                if (warp == 4) TRACE(2, 6);
+                // ------------------------------ P2 ------------------------------
+                const float4* lse4 = reinterpret_cast<const float4*>(lse_s + c0);
+                for (int c = 0; c < n_t && ok; ++c) {
+                    const int t = sg.t0 + c;
+                    const uint32_t vslot = slot_base + n_t + c;
+                    const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
+                    const uint32_t pb = pv_idx % p.p_bufs, pph = (pv_idx / p.p_bufs) & 1;
+                    ++pv_idx;
+                    uint32_t v[NH];
+                    load_cols<NH>(t_lane + col_s + c * N + c0, v);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(B.s_free + 8 * c);
+                    const int key = t * kTile + key_l;
+                    float pr[NH];
+#pragma unroll
+                    for (int i = 0; i < NH; i += 4) {
+                        const float4 ls = lse4[i >> 2];
+                        pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
+                        pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
+                        pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
+                        pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
+                    }
+                    if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
+                        int j = c0 / G, gg = c0 - j * G;
+#pragma unroll
+                        for (int i = 0; i < NH; ++i) {
+                            if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
+                            if (++gg == G) {
+                                gg = 0;
+                                ++j;
+                            }
+                        }
+                    }
+                    float st = 0.f;
+#pragma unroll
+                    for (int i = 0; i < NH; ++i) st += (c0 + i >= stat_r0) ? pr[i] : 0.f;
+                    ok = mbar_wait(B.p_empty + 8 * pb, pph ^ 1, ctl, 23);
+                    if (!ok) break;
+                    // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, 128-byte swizzle):
+                    // 16-byte chunk j (rows 8j..8j+7 of the concatenation) of key k lives at
+                    // (j/8)*16384 + k*128 + ((j%8) ^ (k%8))*16
+                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + key_l * 128;
+#pragma unroll
+                    for (int nb = 0; nb < NH / 8; ++nb) {
+                        uint32_t hi[4], lo[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float a = pr[nb * 8 + 2 * q], b = pr[nb * 8 + 2 * q + 1];
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi[q]) : "f"(b), "f"(a));
+                            const float ra = a - __uint_as_float(hi[q] << 16);
+                            const float rb = b - __uint_as_float(hi[q] & 0xffff0000u);
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo[q]) : "f"(rb), "f"(ra));
+                        }
+                        const int jh = wg * (NH / 8) + nb, jl = jh + 2 * NH / 8;
+                        *reinterpret_cast<uint4*>(p_row + (jh >> 3) * 16384 + (((jh & 7) ^ (key_l & 7)) << 4)) =
+                            make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                        *reinterpret_cast<uint4*>(p_row + (jl >> 3) * 16384 + (((jl & 7) ^ (key_l & 7)) << 4)) =
+                            make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    }
+                    if (t * kTile + kTile > sg.T) {
+                        // ragged last tile: V rows at or beyond T may hold anything; zero them in
+                        // shared memory so that 0 * garbage never reaches the accumulator
+                        ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
+                        if (!ok) break;
+                        if (key >= sg.T) {
+                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + wg * 16384 + key_l * 128;
+#pragma unroll
+                            for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
+                    // column-split statistic: warpgroup 1 hands its partial sum to warpgroup 0
+                    // (4 buffers / barriers: warpgroup 1 can run at most two tiles ahead)
+                    const uint32_t sq = stat_n & 3, sqph = (stat_n >> 2) & 1;
+                    ++stat_n;
+                    if (wg == 1) {
+                        stat_tmp[sq * 128 + key_l] = st;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(B.stat_full + 8 * sq);
+                    } else {
+                        ok = mbar_wait(B.stat_full + 8 * sq, sqph, ctl, 28);
+                        if (!ok) break;
+                        if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st + stat_tmp[sq * 128 + key_l];
+                    }
+                }
+                if (!ok) break;
+                slot_base += 2 * n_t;
+            }
+            pend_unit = unit;
+            pend_nonempty = nonempty;
+            if (warp == 4) TRACE(2, 7);
+        }
+        if (ok && pend_unit >= 0) ok = epilogue(pend_unit, pend_nonempty);
+        if (warp == 4) TRACE(2, 8);
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+template <int NH>
+int launch_nh(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
+              int grid, size_t smem_bytes, cudaStream_t stream)
+{
+    auto kern = verify_cached_kernel<NH>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+        return SPEC_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they wait on each other
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp) != cudaSuccess) {
+        cudaGetLastError();
+        return SPEC_ERR_CUDA;
+    }
+    count_launch(1);
+    return SPEC_OK;
+}
+
+}  // namespace
+
+int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
+                  int grid, size_t smem_bytes, cudaStream_t stream)
+{
+    switch (fp.N / 2) {
+        case 8: return launch_nh<8>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 16: return launch_nh<16>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 24: return launch_nh<24>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 32: return launch_nh<32>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 40: return launch_nh<40>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 48: return launch_nh<48>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 56: return launch_nh<56>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 64: return launch_nh<64>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        default: return SPEC_ERR_UNSUPPORTED_SHAPE;
+    }
+}
+
+}  // namespace sm100
+}  // namespace spec

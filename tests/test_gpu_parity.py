@@ -72,7 +72,8 @@ def test_verify_parity(shape, impl):
     case = inputs.make_case(cfg, device="cuda")
     check_verify(case, impl=impl)
     if impl == binding.VERIFY_AUTO and cfg.head_dim == 128 and cfg.n_q * cfg.group <= 112:
-        assert binding.last_verify_impl() == binding.VERIFY_TCGEN05  # the fast path really ran
+        # the fast path really ran
+        assert binding.last_verify_impl() in (binding.VERIFY_TCGEN05_TWOSWEEP, binding.VERIFY_TCGEN05_CACHED)
 
 
 TCGEN05_SHAPES = [
@@ -89,11 +90,13 @@ TCGEN05_SHAPES = [
 ]
 
 
+@pytest.mark.parametrize("impl", [binding.VERIFY_TCGEN05_TWOSWEEP, binding.VERIFY_TCGEN05_CACHED])
 @pytest.mark.parametrize("shape", TCGEN05_SHAPES)
-def test_verify_tcgen05_parity(shape):
+def test_verify_tcgen05_parity(shape, impl):
     cfg = inputs.small_config(**shape)
     case = inputs.make_case(cfg, device="cuda")
-    check_verify(case, impl=binding.VERIFY_TCGEN05)
+    check_verify(case, impl=impl)
+    assert binding.last_verify_impl() == impl
 
 
 def test_verify_tcgen05_ignores_garbage_beyond_the_context():
@@ -103,7 +106,8 @@ def test_verify_tcgen05_ignores_garbage_beyond_the_context():
     kv = case.kv
     kv.k[:, :, :, 1000:] = float("nan")
     kv.v[:, :, :, 1000:] = float("nan")
-    check_verify(case, impl=binding.VERIFY_TCGEN05)
+    check_verify(case, impl=binding.VERIFY_TCGEN05_TWOSWEEP)
+    check_verify(case, impl=binding.VERIFY_TCGEN05_CACHED)
 
 
 @pytest.mark.parametrize("window", [1, 4, 16])
