@@ -151,7 +151,10 @@ int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers
  *   max_tail   host upper bound of the tail length (sizes the launch)
  *   out        fp32 [n_layers, batch, n_q_heads, head_dim]; lse fp32 [n_layers,batch,n_q_heads]
  *              or NULL
- *   workspace  >= spec_workspace_bytes(SPEC_WS_DRAFT, ...) bytes, 256-byte aligned
+ *   workspace  >= spec_workspace_bytes(SPEC_WS_DRAFT, ...) bytes, 256-byte aligned.  It holds
+ *              only the status word, which this call never clears (one launch per call, no
+ *              memset): zero it once after allocation; an error stays until
+ *              spec_read_status() returns it.
  * An index outside [0, cur_len[b]) is skipped and sets SPEC_ERR_BAD_INDEX in the status word.
  * A problem with an empty key set yields out = 0, lse = -inf.
  */
@@ -171,7 +174,7 @@ size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t
 /*
  * Synchronises `cuda_stream` and returns the status word at the head of `workspace`
  * (SPEC_OK, SPEC_ERR_TIMEOUT or SPEC_ERR_BAD_INDEX), or SPEC_ERR_CUDA if the stream reports
- * an error.
+ * an error.  A non-zero word is reset to SPEC_OK once it has been returned.
  */
 int spec_read_status(const void* workspace, void* cuda_stream);
 

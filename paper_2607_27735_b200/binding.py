@@ -106,8 +106,8 @@ def workspace_bytes(which: int, kv, n_q: int = 1, max_ctx_len: int = 1, k_total:
 
 
 def alloc_workspace(nbytes: int, device) -> torch.Tensor:
-    """A 256-byte aligned byte tensor (torch's caching allocator aligns to 512 bytes)."""
-    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    """A zeroed, 256-byte aligned byte tensor (torch's caching allocator aligns to 512 bytes)."""
+    ws = torch.zeros(max(int(nbytes), 256), dtype=torch.uint8, device=device)
     assert ws.data_ptr() % 256 == 0
     return ws
 

@@ -1,100 +1,138 @@
 // Sparse draft attention of Eq. 5: one query per sequence attends the recalled rows
 // Gather(K, I), Gather(V, I) plus the dense tail of tokens drafted this round.  The gather is
 // fused: 16-byte cp.async copies pull the indexed 2*D-byte rows straight from the dense cache
-// into shared memory; nothing gathered is written back to global memory.
+// into shared memory (two 160-key tiles, so a few hundred keys per CTA are all in flight at
+// once); nothing gathered is written back to global memory.
 //
-// Split-KV: the key list of a problem is cut into n_splits contiguous ranges, one CTA each,
-// every CTA producing an un-normalised partial (running max, sum, P V); a small second kernel
-// merges the partials in a fixed order (deterministic).
+// The call is latency-bound (a few thousand recalled keys per head), so the kernel is built to
+// be short rather than wide:
+//   - every warp is an independent flash-decoding worker on 16 keys of each tile: q K^T and
+//     P V run on the tensor cores (mma.sync m16n8k16, the G <= 8 query rows of the GQA group
+//     padded to 16; P split into bf16 hi + lo parts), its running (max, sum, O) stay in
+//     registers, and no block-wide barrier is needed inside a tile;
+//   - the warps of a CTA are merged once through shared memory, the CTAs of a problem (a
+//     thread-block cluster that splits the key list) once through distributed shared memory:
+//     each deposits its partial in the first CTA of the cluster, which merges them in rank
+//     order (deterministic) after one cluster barrier.
+// One launch per call, no global scratch, no second kernel.
+#include <cooperative_groups.h>
+
 #include "spec_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace spec {
 
 namespace {
 
-constexpr int kTK = 64;        // keys per tile
-constexpr int kThreads = 128;
+constexpr int kTK = 160;       // keys per tile: ten 16-key chunks dealt to the 8 warps
+constexpr int kStages = 2;     // two tiles (320 keys) can be in flight per CTA
+constexpr int kThreads = 256;
 constexpr int kMaxGroup = 8;   // query heads per KV head
-constexpr int kRPT = 4;        // accumulator rows per thread in the PV step
-
-struct Layout {
-    int n_splits;
-    size_t part_off, total;
-};
-
-Layout make_layout(const KvView& kv, int n_keys_max)
-{
-    Layout lo;
-    const int G = kv.n_q_heads / kv.n_kv_heads;
-    const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
-    const int tiles = n_keys_max > 0 ? (n_keys_max + kTK - 1) / kTK : 1;
-    long want = (2L * 148 + probs - 1) / probs;
-    if (want > tiles) want = tiles;
-    if (want < 1) want = 1;
-    lo.n_splits = (int)want;
-    lo.part_off = kStatusBytes;
-    lo.total = lo.part_off + (size_t)probs * lo.n_splits * G * (kv.head_dim + 2) * sizeof(float);
-    lo.total = (lo.total + 255) & ~(size_t)255;
-    return lo;
-}
+constexpr int kMaxCluster = 8; // portable cluster size
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc)
 {
     const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gsrc) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all()
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_dyn(int pending)
 {
-    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+    if (pending <= 0) asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    else asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* p)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
 template <int D>
-__global__ void __launch_bounds__(kThreads)
-draft_partial_kernel(DraftArgs a, int n_splits, float* __restrict__ part, int* __restrict__ status)
-{
-    constexpr int PITCH = D + 8;  // bf16 elements per shared row: 16 B of padding spreads the banks
-    constexpr int CH = D / 8;     // 16-byte chunks per row
-    __shared__ __align__(16) __nv_bfloat16 Ks[kTK * PITCH];
-    __shared__ __align__(16) __nv_bfloat16 Vs[kTK * PITCH];
-    __shared__ __align__(16) float Qs[kMaxGroup * D];
-    __shared__ float S[kMaxGroup * kTK];
-    __shared__ int keypos[kTK];
-    __shared__ float m_run[kMaxGroup], l_run[kMaxGroup], alpha_s[kMaxGroup];
+struct SmemLayout {
+    static constexpr int PITCH = D + 8;  // bf16 elements per shared row: 16 B of padding spreads the banks
+    static constexpr int kv_tile = kTK * PITCH * 2;  // bytes of one K (or V) tile
+    static constexpr int off_k = 0;
+    static constexpr int off_v = kStages * kv_tile;
+    static constexpr int off_q = 2 * kStages * kv_tile;              // bf16 [16][PITCH], rows >= G zero
+    static constexpr int off_pos = off_q + 16 * PITCH * 2;           // int [kStages][kTK]
+    static constexpr int off_wml = off_pos + kStages * kTK * 4;      // float2 [8 warps][kMaxGroup]
+    static constexpr int off_wo = off_k;  // float [8 warps][kMaxGroup][D]: reuses the K tiles once the loop is over
+    static constexpr int off_comb = off_wml + 8 * kMaxGroup * 8;     // float [kMaxCluster][kMaxGroup][D + 2]
+    static constexpr int total = off_comb + kMaxCluster * kMaxGroup * (D + 2) * 4;
+    static_assert(8 * kMaxGroup * D * 4 <= kStages * kv_tile, "warp partials must fit in the K tiles");
+    static_assert(total <= 227 * 1024, "shared memory budget");
+};
 
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
+{
+    using SL = SmemLayout<D>;
+    constexpr int PITCH = SL::PITCH;
+    constexpr int CH = D / 8;    // 16-byte chunks per row
+    constexpr int NT = D / 8;    // 8-wide output tiles of the P V product
+    constexpr float kLog2e = 1.4426950408889634f;
+    extern __shared__ __align__(16) uint8_t smem[];
+    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_k);
+    __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_v);
+    __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_q);
+    int* keypos = reinterpret_cast<int*>(smem + SL::off_pos);
+    float2* wml = reinterpret_cast<float2*>(smem + SL::off_wml);
+    float* wo = reinterpret_cast<float*>(smem + SL::off_wo);
+    float* comb = reinterpret_cast<float*>(smem + SL::off_comb);
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = gridDim.x;              // the cluster spans the x dimension
+    const int rank = blockIdx.x;
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
-    const int split = blockIdx.x, h = blockIdx.y;
+    const int h = blockIdx.y;
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    const int n_rec = min(max(a.n_indices[prob], 0), a.k_total);
-    const int ts = a.tail_start[b], cl = a.cur_len[b];
+    const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
+    const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
     const int n_tail = min(max(cl - ts, 0), a.max_tail);
     const int n = n_rec + n_tail;
-    const int tiles = (n + kTK - 1) / kTK;
-    const int per = (tiles + n_splits - 1) / n_splits * kTK;
-    const int k0 = split * per;
+    const int per = (n + CS - 1) / CS;
+    const int k0 = min(n, rank * per);
     const int k1 = min(n, k0 + per);
+    const int n_tiles = (k1 - k0 + kTK - 1) / kTK;
     const int32_t* idx = a.indices + prob * a.k_total;
 
-    for (int i = tid; i < G * D; i += kThreads) {
-        const int g = i / D, d = i - g * D;
-        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + g;
-        Qs[i] = __bfloat162float(a.q[row * D + d]);
-    }
-    if (tid < kMaxGroup) {
-        m_run[tid] = -INFINITY;
-        l_run[tid] = 0.f;
-    }
-    constexpr int NG = kThreads / (D / 2);
-    const int dp = tid % (D / 2), rg = tid / (D / 2);
-    float acc[kRPT][2];
-#pragma unroll
-    for (int i = 0; i < kRPT; ++i) acc[i][0] = acc[i][1] = 0.f;
-    __syncthreads();
-
-    for (int base = k0; base < k1; base += kTK) {
+    // positions of a tile, then its rows: every copy of the tile is in flight before any wait
+    auto issue_tile = [&](int tile) {
+        const int buf = tile % kStages;
+        const int base = k0 + tile * kTK;
         const int nk = min(kTK, k1 - base);
+        int* kp = keypos + buf * kTK;
         if (tid < kTK) {
             int pos = -1;
             if (tid < nk) {
@@ -105,152 +143,235 @@ draft_partial_kernel(DraftArgs a, int n_splits, float* __restrict__ part, int* _
                     pos = -1;
                 }
             }
-            keypos[tid] = pos;
+            kp[tid] = pos;
         }
         __syncthreads();
+        __nv_bfloat16* kb = Ks + buf * kTK * PITCH;
+        __nv_bfloat16* vb = Vs + buf * kTK * PITCH;
         for (int c = tid; c < kTK * CH; c += kThreads) {
             const int row = c / CH, ch = c - row * CH;
-            const int pos = keypos[row];
+            const int pos = kp[row];
             if (pos >= 0) {
                 const int64_t off = kv_row_offset(a.kv, layer, b, pos, h) + ch * 8;
-                cp_async16(Ks + row * PITCH + ch * 8, a.kv.k + off);
-                cp_async16(Vs + row * PITCH + ch * 8, a.kv.v + off);
-            } else {
-                *reinterpret_cast<uint4*>(Ks + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(Vs + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
+                cp_async16(kb + row * PITCH + ch * 8, a.kv.k + off);
+                cp_async16(vb + row * PITCH + ch * 8, a.kv.v + off);
+            } else {  // masked rows must still be finite: they meet P = 0 in the P V product
+                *reinterpret_cast<uint4*>(kb + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vb + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
             }
         }
-        cp_async_wait_all();
-        __syncthreads();
-        {  // scores: thread = (key, half of the rows)
-            const int key = tid % kTK, part_id = tid / kTK;
-            const bool ok = keypos[key] >= 0;
-            for (int g = part_id; g < G; g += kThreads / kTK) {
-                float dot = 0.f;
-                const uint4* kr = reinterpret_cast<const uint4*>(Ks + key * PITCH);
-                const float4* qr = reinterpret_cast<const float4*>(Qs + g * D);
-#pragma unroll 4
-                for (int c = 0; c < CH; ++c) {
-                    const uint4 kk = kr[c];
-                    const float4 q0 = qr[2 * c], q1 = qr[2 * c + 1];
-                    dot += q0.x * bf16_lo(kk.x) + q0.y * bf16_hi(kk.x) + q0.z * bf16_lo(kk.y) +
-                           q0.w * bf16_hi(kk.y) + q1.x * bf16_lo(kk.z) + q1.y * bf16_hi(kk.z) +
-                           q1.z * bf16_lo(kk.w) + q1.w * bf16_hi(kk.w);
-                }
-                S[g * kTK + key] = ok ? dot * a.kv.scale : -INFINITY;
-            }
+        cp_async_commit();
+    };
+
+    int issued = 0;
+    for (; issued < min(n_tiles, kStages); ++issued) issue_tile(issued);
+
+    // Q of the group -> bf16 [16][PITCH] in shared memory (rows >= G zero), then A fragments
+    for (int i = tid; i < 16 * CH; i += kThreads) {
+        const int g = i / CH, ch = i - g * CH;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (g < G) {
+            const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + g;
+            val = __ldg(reinterpret_cast<const uint4*>(a.q + row * D) + ch);
         }
+        *reinterpret_cast<uint4*>(Qs + g * PITCH + ch * 8) = val;
+    }
+    __syncthreads();
+    uint32_t qa[D / 16][4];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks)
+        ldmatrix_x4(qa[ks], Qs + ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + ks * 16 + (lane >> 4) * 8);
+
+    // per-warp flash-decoding state: the thread owns row g = lane / 4 (and the padding row g + 8)
+    const int g_row = lane >> 2, quad = lane & 3;
+    const float sc = a.kv.scale * kLog2e;
+    float m_run = -INFINITY, l_run = 0.f;
+    float o[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        const int buf = tile % kStages;
+        cp_async_wait_dyn(issued - tile - 1);
         __syncthreads();
-        for (int g = warp; g < G; g += kThreads / 32) {  // online softmax, one warp per row
-            const float v0 = S[g * kTK + lane], v1 = S[g * kTK + lane + 32];
-            const float mt = warp_max(fmaxf(v0, v1));
-            const float m_old = m_run[g];
-            const float m_new = fmaxf(m_old, mt);
-            float alpha = 1.f, p0 = 0.f, p1 = 0.f;
+        const int nk = min(kTK, k1 - (k0 + tile * kTK));
+        for (int ck = warp * 16; ck < nk; ck += 8 * 16) {  // this warp's 16-key chunks of the tile
+            const int* kp = keypos + buf * kTK;
+            const __nv_bfloat16* kb = Ks + (buf * kTK + ck) * PITCH;
+            const __nv_bfloat16* vb = Vs + (buf * kTK + ck) * PITCH;
+            // ---- S = q K^T for 16 keys: two 8-key output tiles ----
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                uint32_t kf[4];
+                ldmatrix_x4(kf, kb + ((lane & 7) + (lane >> 4) * 8) * PITCH + ks * 16 + ((lane >> 3) & 1) * 8);
+                mma_bf16(s0, qa[ks], kf[0], kf[1]);
+                mma_bf16(s1, qa[ks], kf[2], kf[3]);
+            }
+            // the thread's keys: ck + 2*quad + {0,1} (tile 0) and + 8 (tile 1); rows g_row (real) only
+            const int kA = ck + 2 * quad;
+            float v0 = kp[kA] >= 0 ? s0[0] * sc : -INFINITY;
+            float v1 = kp[kA + 1] >= 0 ? s0[1] * sc : -INFINITY;
+            float v2 = kp[kA + 8] >= 0 ? s1[0] * sc : -INFINITY;
+            float v3 = kp[kA + 9] >= 0 ? s1[1] * sc : -INFINITY;
+            float mt = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+            const float m_new = fmaxf(m_run, mt);
+            float alpha = 1.f, p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
             if (m_new > -INFINITY) {
-                alpha = expf(m_old - m_new);
-                p0 = expf(v0 - m_new);
-                p1 = expf(v1 - m_new);
+                alpha = ex2f(m_run - m_new);
+                p0 = ex2f(v0 - m_new);
+                p1 = ex2f(v1 - m_new);
+                p2 = ex2f(v2 - m_new);
+                p3 = ex2f(v3 - m_new);
             }
-            S[g * kTK + lane] = p0;
-            S[g * kTK + lane + 32] = p1;
-            const float s = warp_sum(p0 + p1);
-            if (lane == 0) {
-                l_run[g] = l_run[g] * alpha + s;
-                m_run[g] = m_new;
-                alpha_s[g] = alpha;
+            m_run = m_new;
+            l_run = l_run * alpha + (p0 + p1) + (p2 + p3);
+            // ---- P (hi + lo bf16) as the A operand of P V; padding rows (g_row + 8) are zero ----
+            uint32_t ph[4], pl[4];
+            ph[0] = pack_bf16x2(p0, p1);
+            ph[2] = pack_bf16x2(p2, p3);
+            ph[1] = ph[3] = 0u;
+            pl[0] = pack_bf16x2(p0 - __uint_as_float(ph[0] << 16), p1 - __uint_as_float(ph[0] & 0xffff0000u));
+            pl[2] = pack_bf16x2(p2 - __uint_as_float(ph[2] << 16), p3 - __uint_as_float(ph[2] & 0xffff0000u));
+            pl[1] = pl[3] = 0u;
+#pragma unroll
+            for (int nt = 0; nt < NT; nt += 2) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(vf, vb + ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + nt * 8 + (lane >> 4) * 8);
+                o[nt][0] *= alpha;
+                o[nt][1] *= alpha;
+                o[nt + 1][0] *= alpha;
+                o[nt + 1][1] *= alpha;
+                mma_bf16(o[nt], ph, vf[0], vf[1]);
+                mma_bf16(o[nt], pl, vf[0], vf[1]);
+                mma_bf16(o[nt + 1], ph, vf[2], vf[3]);
+                mma_bf16(o[nt + 1], pl, vf[2], vf[3]);
             }
         }
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < kRPT; ++i) {
-            const int r = rg + i * NG;
-            if (r < G) {
-                const float al = alpha_s[r];
-                acc[i][0] *= al;
-                acc[i][1] *= al;
-            }
+        __syncthreads();  // the tile's buffer is free again
+        if (issued < n_tiles) {
+            issue_tile(issued);
+            ++issued;
         }
-        for (int key = 0; key < nk; ++key) {
-            const uint32_t w = *reinterpret_cast<const uint32_t*>(Vs + key * PITCH + 2 * dp);
-            const float v0 = bf16_lo(w), v1 = bf16_hi(w);
+    }
+
+    // ---- merge the 8 warps of the CTA ----
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (g_row < G) {
+        if (quad == 0) wml[warp * kMaxGroup + g_row] = make_float2(m_run, l_run);
+        float* dst = wo + (warp * kMaxGroup + g_row) * D + 2 * quad;
 #pragma unroll
-            for (int i = 0; i < kRPT; ++i) {
-                const int r = rg + i * NG;
-                if (r < G) {
-                    const float p = S[r * kTK + key];
-                    acc[i][0] += p * v0;
-                    acc[i][1] += p * v1;
+        for (int nt = 0; nt < NT; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+    }
+    __syncthreads();
+    float* comb0 = CS > 1 ? cluster.map_shared_rank(comb, 0) : comb;
+    float* mine = comb0 + rank * (kMaxGroup * (D + 2));
+    for (int i = tid; i < G * (D / 2); i += kThreads) {
+        const int r = i / (D / 2), dp = i - r * (D / 2);
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) M = fmaxf(M, wml[w * kMaxGroup + r].x);
+        float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
+        if (M > -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                const float2 ml = wml[w * kMaxGroup + r];
+                if (ml.y > 0.f) {
+                    const float wgt = ex2f(ml.x - M);
+                    const float2 ov = *(reinterpret_cast<const float2*>(wo + (w * kMaxGroup + r) * D) + dp);
+                    Lsum += ml.y * wgt;
+                    o0 += ov.x * wgt;
+                    o1 += ov.y * wgt;
                 }
             }
         }
-        __syncthreads();
+        *(reinterpret_cast<float2*>(mine + r * D) + dp) = make_float2(o0, o1);
+        if (dp == 0) {
+            mine[kMaxGroup * D + r] = M;
+            mine[kMaxGroup * D + kMaxGroup + r] = Lsum;
+        }
     }
-    float* dst = part + (prob * n_splits + split) * (int64_t)G * (D + 2);
-#pragma unroll
-    for (int i = 0; i < kRPT; ++i) {
-        const int r = rg + i * NG;
-        if (r < G) *(reinterpret_cast<float2*>(dst + r * D) + dp) = make_float2(acc[i][0], acc[i][1]);
-    }
-    if (tid < G) {
-        dst[G * D + tid] = m_run[tid];
-        dst[G * D + G + tid] = l_run[tid];
+    // ---- merge the CTAs of the cluster in its first CTA ----
+    if (CS > 1) cluster.sync(); else __syncthreads();
+    if (rank != 0) return;
+    for (int i = tid; i < G * (D / 2); i += kThreads) {
+        const int r = i / (D / 2), dp = i - r * (D / 2);
+        float M = -INFINITY;
+        for (int c = 0; c < CS; ++c) M = fmaxf(M, comb[c * (kMaxGroup * (D + 2)) + kMaxGroup * D + r]);
+        float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
+        if (M > -INFINITY) {
+            for (int c = 0; c < CS; ++c) {
+                const float* pc = comb + c * (kMaxGroup * (D + 2));
+                const float lc = pc[kMaxGroup * D + kMaxGroup + r];
+                if (lc > 0.f) {
+                    const float wgt = ex2f(pc[kMaxGroup * D + r] - M);
+                    const float2 ov = *(reinterpret_cast<const float2*>(pc + r * D) + dp);
+                    Lsum += lc * wgt;
+                    o0 += ov.x * wgt;
+                    o1 += ov.y * wgt;
+                }
+            }
+        }
+        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + r;
+        const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+        *(reinterpret_cast<float2*>(a.out + row * D) + dp) = make_float2(o0 * inv, o1 * inv);
+        if (a.lse && dp == 0) a.lse[row] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.69314718055994530942f : -INFINITY;
     }
 }
 
-__global__ void draft_combine_kernel(DraftArgs a, int n_splits, const float* __restrict__ part)
+int pick_cluster(const KvView& kv, int n_keys_max)
 {
-    const int D = a.kv.head_dim, G = a.kv.n_q_heads / a.kv.n_kv_heads;
-    const int64_t prob = blockIdx.x;
-    const int d = threadIdx.x;
-    const int h = prob % a.kv.n_kv_heads;
-    const int64_t lb = prob / a.kv.n_kv_heads;
-    const int64_t stride = (int64_t)G * (D + 2);
-    for (int g = 0; g < G; ++g) {
-        float M = -INFINITY;
-        for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part[(prob * n_splits + s) * stride + G * D + g]);
-        float Lsum = 0.f, o = 0.f;
-        if (M > -INFINITY) {
-            for (int s = 0; s < n_splits; ++s) {
-                const float* p = part + (prob * n_splits + s) * stride;
-                const float l = p[G * D + G + g];
-                if (l > 0.f) {
-                    const float w = expf(p[G * D + g] - M);
-                    Lsum += l * w;
-                    o += p[g * D + d] * w;
-                }
-            }
-        }
-        const int64_t row = lb * a.kv.n_q_heads + h * G + g;
-        a.out[row * D + d] = Lsum > 0.f ? o / Lsum : 0.f;
-        if (a.lse && d == 0) a.lse[row] = Lsum > 0.f ? M + logf(Lsum) : -INFINITY;
+    // enough CTAs to cover the SMs, at most one tile-pair of work each, at most a portable cluster
+    const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
+    const int tiles = n_keys_max > 0 ? (n_keys_max + kTK - 1) / kTK : 1;
+    int cs = 1;
+    while (cs < kMaxCluster && probs * cs < sm_count() && cs * 2 <= tiles) cs *= 2;
+    return cs;
+}
+
+template <int D>
+int launch_d(const DraftArgs& a, int cs, cudaStream_t stream)
+{
+    auto kern = draft_cluster_kernel<D>;
+    const size_t smem = SmemLayout<D>::total;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SPEC_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, a, static_cast<int*>(a.workspace)) != cudaSuccess) {
+        cudaGetLastError();
+        return SPEC_ERR_CUDA;
     }
+    count_launch(1);
+    return SPEC_OK;
 }
 
 }  // namespace
 
-size_t draft_workspace(const KvView& kv, int n_keys_max) { return make_layout(kv, n_keys_max).total; }
+size_t draft_workspace(const KvView&, int) { return kStatusBytes; }
 
 int draft_launch(const DraftArgs& a, cudaStream_t stream)
 {
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     if (G > kMaxGroup) return SPEC_ERR_UNSUPPORTED_SHAPE;
-    const Layout lo = make_layout(a.kv, a.k_total + a.max_tail);
-    if (a.workspace_bytes < lo.total) return SPEC_ERR_WORKSPACE_TOO_SMALL;
-    char* ws = static_cast<char*>(a.workspace);
-    float* part = reinterpret_cast<float*>(ws + lo.part_off);
-    int* status = reinterpret_cast<int*>(ws);
-    const dim3 grid(lo.n_splits, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
-    const long probs = (long)a.kv.n_layers * a.kv.batch * a.kv.n_kv_heads;
-    if (a.kv.head_dim == 128)
-        draft_partial_kernel<128><<<grid, kThreads, 0, stream>>>(a, lo.n_splits, part, status);
-    else if (a.kv.head_dim == 64)
-        draft_partial_kernel<64><<<grid, kThreads, 0, stream>>>(a, lo.n_splits, part, status);
-    else
-        return SPEC_ERR_UNSUPPORTED_SHAPE;
-    draft_combine_kernel<<<(unsigned)probs, a.kv.head_dim, 0, stream>>>(a, lo.n_splits, part);
-    count_launch(2);
-    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+    if (a.workspace_bytes < kStatusBytes) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+    const int cs = pick_cluster(a.kv, a.k_total + a.max_tail);
+    if (a.kv.head_dim == 128) return launch_d<128>(a, cs, stream);
+    if (a.kv.head_dim == 64) return launch_d<64>(a, cs, stream);
+    return SPEC_ERR_UNSUPPORTED_SHAPE;
 }
 
 }  // namespace spec

@@ -161,9 +161,7 @@ int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* in
     a.workspace = workspace;
     a.workspace_bytes = workspace_bytes;
     if (workspace_bytes < draft_workspace(a.kv, k_total + max_tail)) return SPEC_ERR_WORKSPACE_TOO_SMALL;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;
-    return draft_launch(a, stream);
+    return draft_launch(a, static_cast<cudaStream_t>(cuda_stream));
 }
 
 size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t max_ctx_len,
@@ -193,6 +191,11 @@ int spec_read_status(const void* workspace, void* cuda_stream)
     if (cudaMemcpyAsync(&code, workspace, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return SPEC_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return SPEC_ERR_CUDA;
+    if (code != 0) {  // reading an error acknowledges it
+        if (cudaMemsetAsync(const_cast<void*>(workspace), 0, sizeof(int), stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+            return SPEC_ERR_CUDA;
+    }
     return code;
 }
 
