@@ -33,7 +33,9 @@ struct FastParams {
     int* status;
     int n_pages;
     int n_cache;                      // S tiles the TMEM cache holds (cached variant)
+    int q_bufs;                       // Q buffers in shared memory (cached variant: 1)
     long long* trace;
+    int dbg;                          // development knobs (trace builds only)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -134,6 +136,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t saddr)
 {
     return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// MN-major operand without swizzle: 8x8 core matrices of 128 contiguous bytes, K groups 128 B
+// apart (leading offset), 8-row MN blocks 2048 B apart (stride offset).
+__device__ __forceinline__ uint64_t desc_mnmajor_nosw(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (8ull << 16) | (128ull << 32) | (1ull << 46);
 }
 // MN-major operand, 128-byte swizzle: 64-element MN blocks 16 KiB apart (leading offset),
 // 8-row K groups 1024 B apart (stride offset).

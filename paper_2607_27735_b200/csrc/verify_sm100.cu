@@ -103,17 +103,28 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
     pl->N = N;
     pl->box_rows = box_rows;
     pl->boxes = kTile / box_rows;
-    const size_t p_bytes = (size_t)((2 * N + 63) / 64) * 16384;
     const size_t cap = 227 * 1024;
     size_t fixed = 0;
     int slots = 0;
-    const char* env_pb = std::getenv("SPEC_VERIFY_PBUFS");
-    const int pb_hi = env_pb ? std::atoi(env_pb) : 2;
-    for (int pb = (pb_hi == 1 ? 1 : 2); pb >= 1; --pb) {
-        fixed = 1024 /*alignment slack*/ + 2 * (size_t)N * 256 + pb * p_bytes + 8192;
+    if (cached) {
+        // one Q buffer, two P buffers ([hi | lo] rows, 8-row blocks: 2N * 256 B each), 12.25 KB of
+        // barriers and small arrays; the rest is the K/V tile ring
+        pl->p_bufs = 2;
+        fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544;
         slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
-        pl->p_bufs = pb;
-        if (slots >= (cached ? 5 : 4)) break;
+        if (slots < 4) {
+            pl->p_bufs = 1;
+            fixed -= (size_t)(2 * N * 256);
+            slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
+        }
+    } else {
+        const size_t p_bytes = (size_t)((2 * N + 63) / 64) * 16384;
+        for (int pb = 2; pb >= 1; --pb) {  // two P buffers if that still leaves a 4-deep K/V ring
+            fixed = 1024 /*alignment slack*/ + 2 * (size_t)N * 256 + pb * p_bytes + 12544;
+            slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
+            pl->p_bufs = pb;
+            if (slots >= 4) break;
+        }
     }
     if (slots > 8) slots = 8;
     if (slots < 3) return false;
@@ -223,8 +234,10 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.n_pages = n_pages;
     fp.n_cache = pl.n_cache;
     fp.trace = nullptr;
+    fp.dbg = 0;
 #ifdef SPEC_TRACE
     fp.trace = reinterpret_cast<long long*>(ws + pl.trace_off);
+    if (const char* e = std::getenv("SPEC_DBG")) fp.dbg = std::atoi(e);
 #endif
     // one memset clears the status word and the cross-CTA counters that follow it
     if (cudaMemsetAsync(ws, 0, pl.ctr_off + pl.ctr_bytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;

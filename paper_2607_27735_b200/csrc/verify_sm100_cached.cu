@@ -41,8 +41,10 @@ struct CBars {  // mbarrier addresses (shared space)
         aux_sync, stat_full;
 };
 
-template <int NH>
-__global__ void __launch_bounds__(kThreads, 1)
+// NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
+// more, narrower warpgroups hide the latency of the serial softmax sections.
+template <int NC, int CG>
+__global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_q, const FastParams p)
 {
@@ -50,15 +52,18 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));  // generic pointer to the aligned base
 
+    constexpr int NH = NC;                       // columns per thread
+    constexpr int kBlock = 128 + 128 * CG;       // threads per CTA
+    constexpr int kSW = 4 * CG;                  // softmax warps
     const int N = p.N, R = p.R, G = p.G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head_local = blockIdx.x / p.cph, rank = blockIdx.x % p.cph;
     const int q_bytes = N * 256;                       // one Q buffer: 2 halves x N rows x 128 B
-    const int p_bytes = ((2 * N + 63) / 64) * 16384;   // one P buffer: [hi | lo] rows, 64-row blocks x 128 keys x 128 B
+    const int p_bytes = 2 * N * 256;                   // one P buffer: [hi | lo] rows, 8-row blocks x 128 keys x 16 B
 
     const uint32_t s_slots = sbase;
     const uint32_t s_q = s_slots + p.n_slots * kSlotBytes;
-    const uint32_t s_p = s_q + 2 * q_bytes;
+    const uint32_t s_p = s_q + q_bytes;                // one Q buffer: the next unit's Q lands after this unit's last QK^T
     const uint32_t s_misc = s_p + p.p_bufs * p_bytes;
     uint8_t* misc = sgen + (s_misc - sbase);
     CBars B;
@@ -71,7 +76,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.s_full = o; o += 8 * kMaxCache;
         B.s_free = o; o += 8 * kMaxCache;
         B.p_full = o; o += 16;
-        B.p_empty = o; o += 16;
+        B.p_empty = o; o += 32;  // four: indexed by tile sequence number mod 4 (see the P2 loop)
         B.o_full = o; o += 8;
         B.o_empty = o; o += 8;
         B.sm_sync = o; o += 8;
@@ -79,9 +84,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.stat_full = o; o += 32;
     }
     float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128]
-    float* stat_tmp = reinterpret_cast<float*>(misc + 2048);              // [4][128]
-    float2* red = reinterpret_cast<float2*>(misc + 4096);                 // [8 warps][64] (m, l)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 8192 - 16);
+    float2* red = reinterpret_cast<float2*>(misc + 8192);                 // [kSW warps][NC] (m, l), <= 4 KB
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 12288);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     Ctl ctl{abort_flag, p.status};
@@ -96,26 +100,26 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         }
         for (int i = 0; i < kMaxCache; ++i) {
             mbar_init(B.s_full + 8 * i, 1);
-            mbar_init(B.s_free + 8 * i, 8);
+            mbar_init(B.s_free + 8 * i, 4);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(B.q_full + 8 * i, 1);
             mbar_init(B.q_empty + 8 * i, 1);
-            mbar_init(B.p_full + 8 * i, 8);
-            mbar_init(B.p_empty + 8 * i, 1);
+            mbar_init(B.p_full + 8 * i, 4);
         }
+        for (int i = 0; i < 4; ++i) mbar_init(B.p_empty + 8 * i, 1);
         mbar_init(B.o_full, 1);
-        mbar_init(B.o_empty, 8);
-        mbar_init(B.sm_sync, 8);
+        mbar_init(B.o_empty, kSW);
+        mbar_init(B.sm_sync, kSW);
         mbar_init(B.aux_sync, 2);
-        for (int i = 0; i < 4; ++i) mbar_init(B.stat_full + 8 * i, 4);
+        for (int i = 0; i < 4; ++i) mbar_init(B.stat_full + 8 * i, CG > 1 ? 4 * (CG - 1) : 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the Q buffers once: rows R..N-1 are padding the TMA never writes
-    for (int i = threadIdx.x; i < 2 * q_bytes / 16; i += kThreads)
+    for (int i = threadIdx.x; i < q_bytes / 16; i += kBlock)
         *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
-    for (int r = R + threadIdx.x; r < 128; r += kThreads) lse_s[r] = 1.0e30f;  // padded rows: P = 0
+    for (int r = R + threadIdx.x; r < 128; r += kBlock) lse_s[r] = 1.0e30f;  // padded rows: P = 0
     fence_proxy_async();
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -137,7 +141,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         auto load_tile = [&](const CUtensorMap* map, const Seg& sg, int tile) -> bool {
             const uint32_t s = slot_idx % p.n_slots, ph = (slot_idx / p.n_slots) & 1;
             ++slot_idx;
-            if (!mbar_wait(B.slot_empty + 8 * s, ph ^ 1, ctl, 1)) return false;
+            bool got = true;
+            if (lane == 0) got = mbar_wait(B.slot_empty + 8 * s, ph ^ 1, ctl, 1);  // one lane polls
+            if (!__shfl_sync(0xffffffffu, got ? 1 : 0, 0)) return false;
             // boxes of this tile that hold at least one key < T (pages past the context may not exist)
             const int key0 = tile * kTile;
             const int n_box = min(boxes, (sg.T - key0 + box_rows - 1) / box_rows);
@@ -163,7 +169,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             const Seg sg = get_seg(p, u, head_local, rank);
             if (sg.t1 <= sg.t0) continue;
             TRACE(0, 1);
-            const uint32_t qb = qn & 1, qph = (qn >> 1) & 1;
+            const uint32_t qb = 0, qph = qn & 1;
             ++qn;
             ok = mbar_wait(B.q_empty + 8 * qb, qph ^ 1, ctl, 2);
             if (!ok) break;
@@ -176,6 +182,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             __syncwarp();
             for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t);
             TRACE(0, 2);
+#ifdef SPEC_TRACE
+            if (p.dbg & 32) {  // experiment: hold the V prefetch until half of the head's CTAs published P1
+                bool got = true;
+                if (lane == 0) got = counter_wait(p.counters + u * p.HG + head_local, p.cph / 2, ctl, 3);
+                if (!__shfl_sync(0xffffffffu, got ? 1 : 0, 0)) break;
+            }
+#endif
             for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_v, sg, t);
             TRACE(0, 3);
         }
@@ -213,8 +226,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         c.t = sg.t0;
                         c.slot_base = c.next_base;
                         c.next_base += 2 * (sg.t1 - sg.t0);
-                        c.qb = c.qn & 1;
-                        c.qph = (c.qn >> 1) & 1;
+                        c.qb = 0;
+                        c.qph = c.qn & 1;
                         ++c.qn;
                         return;
                     }
@@ -250,6 +263,12 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 }
                 tc_commit(B.s_full + 8 * c);
                 tc_commit(B.slot_empty + 8 * s);
+#ifdef SPEC_TRACE
+                if (p.dbg & 16) {
+                    mbar_wait(B.slot_empty + 8 * s, (slot / p.n_slots) & 1, ctl, 18);
+                    TRACE(1, 4);
+                }
+#endif
                 if (qq.t == qq.t1 - 1) tc_commit(B.q_empty + 8 * qq.qb);  // last use of this Q buffer
                 if (++qq.t == qq.t1) seek(qq);
             };
@@ -268,6 +287,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const uint32_t slot = pq.slot_base + (pq.t1 - pq.t0) + c;
                 const uint32_t s = slot % p.n_slots;
                 const uint32_t pb = pv_idx % p.p_bufs;
+                const uint32_t pe = pv_idx & 3;
                 ++pv_idx;
                 const bool first = c == 0, last = pq.t == pq.t1 - 1;
                 tc_fence_after();
@@ -277,11 +297,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t a = desc_mnmajor(v_addr + ks * 2048);
-                    const uint64_t b = desc_mnmajor(p_addr + ks * 2048);
+                    const uint64_t b = desc_mnmajor_nosw(p_addr + ks * 256);
                     tc_mma(d_o, a, b, idesc_pv, (first && ks == 0) ? 0u : 1u);
                 }
                 tc_commit(B.slot_empty + 8 * s);
-                tc_commit(B.p_empty + 8 * pb);
+                tc_commit(B.p_empty + 8 * pe);
                 if (last) {
                     tc_commit(B.o_full);
                     o_phase ^= 1;
@@ -303,7 +323,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 }
                 if (progressed) {
                     spins = 0;
-                } else if ((++spins & 63u) == 0) {
+                    continue;
+                }
+                __nanosleep(40);  // idle: leave the issue slots of this sub-core to the softmax warps
+                if ((++spins & 63u) == 0) {
                     if (spins == 64) t_idle = clock64();
                     if (*ctl.abort_flag) ok = false;
                     else if (clock64() - t_idle > kTimeoutCycles) {
@@ -354,17 +377,17 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         }
     } else {
         // =========================== softmax warpgroups ===========================
-        const int sw = warp - 4;                 // 0..7
-        const int wg = sw >> 2;                  // column half
+        const int sw = warp - 4;                 // 0..kSW-1
+        const int wg = sw >> 2;                  // column group
         const int quarter = warp & 3;            // TMEM lane quarter this warp may touch
         const int key_l = quarter * 32 + lane;   // key within the tile (P1/P2) or d (epilogue)
-        const int tid_s = threadIdx.x - 128;     // 0..255
+        const int tid_s = threadIdx.x - 128;     // 0..128*CG-1
         const int c0 = wg * NH;                  // first column of this warpgroup
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int stat_r0 = p.a.first_stat_row * G;
         const float cs = p.scale_log2;
         constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
-        uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, stat_n = 0, sfull_par = 0;
+        uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, sfull_par = 0;
         bool ok = true;
         int pend_unit = -1;                      // unit whose O accumulator still waits for its epilogue
         bool pend_nonempty = false;
@@ -388,7 +411,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     if (r < R) p.o_part[obase + (int64_t)r * kD + key_l] = __uint_as_float(v[i]) + __uint_as_float(w[i]);
                 }
             } else {
-                for (int i = tid_s; i < R * kD; i += 256) p.o_part[obase + i] = 0.f;
+                for (int i = tid_s; i < R * kD; i += 128 * CG) p.o_part[obase + i] = 0.f;
             }
             if (!group_sync(B.sm_sync, sync_n, ctl, 29)) return false;
             if (tid_s == 0) {
@@ -461,31 +484,32 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 float Ls = l[i] * ex2(m[i] - M);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
-                if (lane == 0) red[sw * 64 + i] = make_float2(M, Ls);
+                if (lane == 0) red[sw * NC + i] = make_float2(M, Ls);
             }
             ok = group_sync(B.sm_sync, sync_n, ctl, 26);
             if (!ok) break;
-            {
-                const int wgi = tid_s >> 7, ci = tid_s & 127;
-                if (ci < NH && wgi * NH + ci < R) {
+            if (sw == kSW - 1) {
+                // the last softmax warp merges the four lane quarters of every column and publishes
+                // the CTA's partial; the other warps go on (they meet it again at the counter)
+                const int64_t base = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R;
+                for (int col = lane; col < R; col += 32) {
+                    const int wgi = col / NC, ci = col - wgi * NC;
                     float M = kNegBig;
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) M = fmaxf(M, red[(wgi * 4 + w) * 64 + ci].x);
+                    for (int w = 0; w < 4; ++w) M = fmaxf(M, red[(wgi * 4 + w) * NC + ci].x);
                     float Ls = 0.f;
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
-                        const float2 ml = red[(wgi * 4 + w) * 64 + ci];
+                        const float2 ml = red[(wgi * 4 + w) * NC + ci];
                         Ls += ml.y * ex2(ml.x - M);
                     }
-                    const int64_t base = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R;
-                    p.ml_part[base + wgi * NH + ci] = make_float2(M, nonempty ? Ls : 0.f);
+                    p.ml_part[base + col] = make_float2(M, nonempty ? Ls : 0.f);
                 }
-            }
-            ok = group_sync(B.sm_sync, sync_n, ctl, 27);
-            if (!ok) break;
-            if (tid_s == 0) {
-                __threadfence();
-                atomicAdd(p.counters + unit * p.HG + head_local, 1);
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(p.counters + unit * p.HG + head_local, 1);
+                }
             }
             if (warp == 4) TRACE(2, 3);
             // ---- while the other CTAs finish their P1: drain the previous unit's accumulator ----
@@ -498,15 +522,16 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (nonempty) {
                 // ---- row LSE from the partials of the CTAs that share this head ----
                 if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
                 if (!ok) break;
-                __threadfence();
                 if (warp == 4) TRACE(2, 5);
                 const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
-                const int tpr = 256 / R;          // threads per row (R <= 128)
-                const int r = tid_s % R, sub = tid_s / R;
+                // tpr threads of one warp share a row: each folds every tpr-th partial, then shuffles
+                int tpr = 32;
+                while (tpr * R > 128 * CG) tpr >>= 1;
+                const int r = tid_s / tpr, sub = tid_s - r * tpr;
                 float M = kNegBig, Ls = 0.f;
-                if (sub < tpr) {
+                if (r < R) {
                     for (int k0 = sub; k0 < p.cph; k0 += 8 * tpr) {  // batches of 8 independent loads
                         float2 x[8];
 #pragma unroll
@@ -520,22 +545,19 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             M = Mn;
                         }
                     }
-                    red[sub * R + r] = make_float2(M, Ls);  // tpr * R <= 256 entries
                 }
-                ok = group_sync(B.sm_sync, sync_n, ctl, 21);
-                if (!ok) break;
-                if (tid_s < R) {
-                    float Mx = kNegBig;
-                    for (int s2 = 0; s2 < tpr; ++s2) Mx = fmaxf(Mx, red[s2 * R + tid_s].x);
-                    float Lx = 0.f;
-                    for (int s2 = 0; s2 < tpr; ++s2) {
-                        const float2 ml = red[s2 * R + tid_s];
-                        Lx += ml.y * ex2(ml.x - Mx);
-                    }
-                    const float lse2 = Mx + log2f(Lx);
-                    lse_s[tid_s] = lse2;
+                for (int o = tpr >> 1; o > 0; o >>= 1) {
+                    const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
+                    const float L2 = __shfl_xor_sync(0xffffffffu, Ls, o);
+                    const float Mn = fmaxf(M, M2);
+                    Ls = Ls * ex2(M - Mn) + L2 * ex2(M2 - Mn);
+                    M = Mn;
+                }
+                if (sub == 0 && r < R) {
+                    const float lse2 = M + log2f(Ls);
+                    lse_s[r] = lse2;
                     if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
-                        const int j = tid_s / G, g = tid_s - j * G;
+                        const int j = r / G, g = r - j * G;
                         const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
                         p.a.lse[row] = lse2 * 0.69314718055994530942f;
                     }
@@ -544,94 +566,113 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 if (!ok) break;
                 if (warp == 4) TRACE(2, 6);
                 // ------------------------------ P2 ------------------------------
-                const float4* lse4 = reinterpret_cast<const float4*>(lse_s + c0);
-                for (int c = 0; c < n_t && ok; ++c) {
+                // Tile-split: warpgroup wg takes the tiles c = wg, wg + CG, ... whole (all N
+                // columns per thread), so CG tiles are in flight at once, the statistic is a
+                // thread-local sum, and each tile's fixed costs (waits, proxy fence, arrivals)
+                // are paid by one warpgroup instead of by all of them.
+                for (int c = wg; c < n_t && ok; c += CG) {
                     const int t = sg.t0 + c;
                     const uint32_t vslot = slot_base + n_t + c;
                     const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
-                    const uint32_t pb = pv_idx % p.p_bufs, pph = (pv_idx / p.p_bufs) & 1;
-                    ++pv_idx;
-                    uint32_t v[NH];
-                    load_cols<NH>(t_lane + col_s + c * N + c0, v);
+                    const uint32_t pvi = pv_idx + c;
+                    const uint32_t pb = pvi % p.p_bufs;
+                    const int key = t * kTile + key_l;
+                    const bool boundary = t * kTile + kTile > sg.T - p.a.n_q + 1;
+                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + (key_l >> 3) * 128 + (key_l & 7) * 16;
+                    float st = 0.f;
+                    bool waited = false;
+#pragma unroll 1
+                    for (int cb = 0; cb < N; cb += 16) {  // 16 columns at a time keeps the live set small
+                        uint32_t v[16];
+                        tmem_ld8(t_lane + col_s + c * N + cb, v);
+                        tmem_ld8(t_lane + col_s + c * N + cb + 8, v + 8);
+                        tc_wait_ld();
+                        const float4* lse4 = reinterpret_cast<const float4*>(lse_s + cb);
+                        float pr[16];
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            const float4 ls = lse4[i >> 2];
+                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
+                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
+                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
+                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
+                        }
+                        if (boundary) {
+                            int j = cb / G, gg = cb - j * G;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
+                                if (++gg == G) {
+                                    gg = 0;
+                                    ++j;
+                                }
+                            }
+                        }
+                        if (cb >= stat_r0) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) st += pr[i];
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) st += (cb + i >= stat_r0) ? pr[i] : 0.f;
+                        }
+                        if (!waited) {
+                            // the P buffer is free once the P V product p_bufs tiles back is done.  Warpgroups
+                            // run ahead of each other, so the "done" barriers are indexed by the tile's
+                            // sequence number mod 4: a waiter is then never two phases ahead of its barrier.
+                            if (pvi >= (uint32_t)p.p_bufs) {
+                                const uint32_t prev = pvi - p.p_bufs;
+                                ok = mbar_wait(B.p_empty + 8 * (prev & 3), (prev >> 2) & 1, ctl, 23);
+                                if (!ok) break;
+                            }
+                            waited = true;
+                        }
+                        // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, no swizzle): the
+                        // 16-byte vector of row block j (rows 8j..8j+7 of the concatenation) and key k
+                        // lives at j*2048 + (k/8)*128 + (k%8)*16
+#pragma unroll
+                        for (int nb = 0; nb < 2; ++nb) {
+                            uint32_t hi[4], lo[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                // p = hi + lo with both parts cut to bf16 by truncation (plain integer ops, no
+                                // conversion instructions): hi keeps the top 16 bits, lo the top 16 bits of the
+                                // exact remainder, so p - (hi + lo) < 2^-14 p
+                                const uint32_t ua = __float_as_uint(pr[nb * 8 + 2 * q]), ub = __float_as_uint(pr[nb * 8 + 2 * q + 1]);
+                                hi[q] = __byte_perm(ua, ub, 0x7632);
+                                const float ra = __uint_as_float(ua) - __uint_as_float(ua & 0xffff0000u);
+                                const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
+                                lo[q] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+                            }
+                            const int jh = cb / 8 + nb, jl = jh + N / 8;
+                            *reinterpret_cast<uint4*>(p_row + jh * 2048) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<uint4*>(p_row + jl * 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        }
+                    }
+                    if (!ok) break;
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_free + 8 * c);
-                    const int key = t * kTile + key_l;
-                    float pr[NH];
-#pragma unroll
-                    for (int i = 0; i < NH; i += 4) {
-                        const float4 ls = lse4[i >> 2];
-                        pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
-                        pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
-                        pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
-                        pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
-                    }
-                    if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
-                        int j = c0 / G, gg = c0 - j * G;
-#pragma unroll
-                        for (int i = 0; i < NH; ++i) {
-                            if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
-                            if (++gg == G) {
-                                gg = 0;
-                                ++j;
-                            }
-                        }
-                    }
-                    float st = 0.f;
-#pragma unroll
-                    for (int i = 0; i < NH; ++i) st += (c0 + i >= stat_r0) ? pr[i] : 0.f;
-                    ok = mbar_wait(B.p_empty + 8 * pb, pph ^ 1, ctl, 23);
-                    if (!ok) break;
-                    // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, 128-byte swizzle):
-                    // 16-byte chunk j (rows 8j..8j+7 of the concatenation) of key k lives at
-                    // (j/8)*16384 + k*128 + ((j%8) ^ (k%8))*16
-                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + key_l * 128;
-#pragma unroll
-                    for (int nb = 0; nb < NH / 8; ++nb) {
-                        uint32_t hi[4], lo[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            const float a = pr[nb * 8 + 2 * q], b = pr[nb * 8 + 2 * q + 1];
-                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi[q]) : "f"(b), "f"(a));
-                            const float ra = a - __uint_as_float(hi[q] << 16);
-                            const float rb = b - __uint_as_float(hi[q] & 0xffff0000u);
-                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo[q]) : "f"(rb), "f"(ra));
-                        }
-                        const int jh = wg * (NH / 8) + nb, jl = jh + 2 * NH / 8;
-                        *reinterpret_cast<uint4*>(p_row + (jh >> 3) * 16384 + (((jh & 7) ^ (key_l & 7)) << 4)) =
-                            make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                        *reinterpret_cast<uint4*>(p_row + (jl >> 3) * 16384 + (((jl & 7) ^ (key_l & 7)) << 4)) =
-                            make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                    }
                     if (t * kTile + kTile > sg.T) {
                         // ragged last tile: V rows at or beyond T may hold anything; zero them in
                         // shared memory so that 0 * garbage never reaches the accumulator
                         ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
                         if (!ok) break;
                         if (key >= sg.T) {
-                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + wg * 16384 + key_l * 128;
+                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + key_l * 128;
 #pragma unroll
-                            for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
+                            for (int ch = 0; ch < 8; ++ch) {
+                                *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4*>(vrow + 16384 + 16 * ch) = make_uint4(0, 0, 0, 0);
+                            }
                         }
                     }
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
-                    // column-split statistic: warpgroup 1 hands its partial sum to warpgroup 0
-                    // (4 buffers / barriers: warpgroup 1 can run at most two tiles ahead)
-                    const uint32_t sq = stat_n & 3, sqph = (stat_n >> 2) & 1;
-                    ++stat_n;
-                    if (wg == 1) {
-                        stat_tmp[sq * 128 + key_l] = st;
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(B.stat_full + 8 * sq);
-                    } else {
-                        ok = mbar_wait(B.stat_full + 8 * sq, sqph, ctl, 28);
-                        if (!ok) break;
-                        if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st + stat_tmp[sq * 128 + key_l];
-                    }
+                    if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st;
                 }
                 if (!ok) break;
+                pv_idx += n_t;
                 slot_base += 2 * n_t;
             }
             pend_unit = unit;
@@ -651,16 +692,16 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     }
 }
 
-template <int NH>
-int launch_nh(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
-              int grid, size_t smem_bytes, cudaStream_t stream)
+template <int NC, int CG>
+int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
+               int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    auto kern = verify_cached_kernel<NH>;
+    auto kern = verify_cached_kernel<NC, CG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(128 + 128 * CG);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -681,15 +722,15 @@ int launch_nh(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& t
 int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                   int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    switch (fp.N / 2) {
-        case 8: return launch_nh<8>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 16: return launch_nh<16>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 24: return launch_nh<24>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 32: return launch_nh<32>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 40: return launch_nh<40>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 48: return launch_nh<48>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 56: return launch_nh<56>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 64: return launch_nh<64>(tk, tv, tq, fp, grid, smem_bytes, stream);
+    switch (fp.N) {  // (columns per warpgroup, warpgroups)
+        case 16: return launch_cfg<8, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 32: return launch_cfg<8, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 48: return launch_cfg<16, 3>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 64: return launch_cfg<16, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 80: return launch_cfg<40, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 96: return launch_cfg<24, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 112: return launch_cfg<56, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 128: return launch_cfg<32, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
         default: return SPEC_ERR_UNSUPPORTED_SHAPE;
     }
 }

@@ -526,11 +526,21 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                             uint32_t hi[4], lo[4];
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
-                                const float a = pr[nb * 8 + 2 * q], b = pr[nb * 8 + 2 * q + 1];
-                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(hi[q]) : "f"(b), "f"(a));
-                                const float ra = a - __uint_as_float(hi[q] << 16);
-                                const float rb = b - __uint_as_float(hi[q] & 0xffff0000u);
-                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(lo[q]) : "f"(rb), "f"(ra));
+                                // p = hi + lo with both parts cut to bf16 by truncation (plain integer ops, no
+
+                                // conversion instructions): hi keeps the top 16 bits, lo the top 16 bits of the exact
+
+                                // remainder, so p - (hi + lo) < 2^-14 p
+
+                                const uint32_t ua = __float_as_uint(pr[nb * 8 + 2 * q]), ub = __float_as_uint(pr[nb * 8 + 2 * q + 1]);
+
+                                hi[q] = __byte_perm(ua, ub, 0x7632);
+
+                                const float ra = __uint_as_float(ua) - __uint_as_float(ua & 0xffff0000u);
+
+                                const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
+
+                                lo[q] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
                             }
                             const int jh = wg * (NH / 8) + nb, jl = jh + 2 * NH / 8;
                             *reinterpret_cast<uint4*>(p_row + (jh >> 3) * 16384 + (((jh & 7) ^ (key_l & 7)) << 4)) =
