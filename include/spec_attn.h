@@ -24,7 +24,8 @@
  *   - Return value: 0 on success, a negative SPEC_ERR_* decided on the host BEFORE anything
  *     is launched.  Device-side anomalies (an out-of-range recall index, a bounded wait that
  *     ran out) set a status word at the head of the workspace and the kernel exits cleanly;
- *     read it with spec_read_status().
+ *     read it with spec_read_status().  Workspaces must be zero-filled once after allocation;
+ *     no call clears the status word, reading it does.
  *   - Positions are 0-based (the paper counts from 1).  bf16 inputs, fp32 accumulation and
  *     fp32 outputs.
  *   - GQA: query head hq reads KV head hq / (n_q_heads / n_kv_heads); the Eq. 3 score is kept
@@ -108,8 +109,12 @@ typedef struct {
  *   lse      fp32 [n_layers, batch, n_q, n_q_heads] (natural-log softmax denominator) or NULL
  *   stats    fp32 [n_layers, batch, n_kv_heads, stat_stride]; entries [0, ctx_len[b]) are
  *            written, the rest left untouched; stat_stride >= max_ctx_len
- *   workspace  >= spec_workspace_bytes(SPEC_WS_VERIFY, ...) bytes, 256-byte aligned, contents
- *            need not be initialised; must not be shared by calls that may overlap on the GPU
+ *   workspace  >= spec_workspace_bytes(SPEC_WS_VERIFY, ...) bytes, 256-byte aligned, ZERO-FILLED
+ *            once before its first use (cudaMemset); every call leaves it ready for the next one
+ *            (no per-call memset: the kernel's last CTA puts its cross-CTA counters back to
+ *            zero).  The status word is sticky until spec_read_status() returns it; after
+ *            SPEC_ERR_TIMEOUT zero the workspace again.  Must not be shared by calls that may
+ *            overlap on the GPU.
  */
 int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
                      int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,

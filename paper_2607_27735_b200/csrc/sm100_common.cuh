@@ -27,7 +27,8 @@ struct FastParams {
     int n_slots, p_bufs;
     int box_rows, boxes;              // TMA boxes per 64-wide half of a tile
     float scale_log2;
-    int* counters;                    // [2][n_units * HG]: P1 partials done, O partials done
+    int* counters;                    // [2][n_units * HG]: P1 partials done, O partials done; then one
+                                      // "CTAs finished" word.  All zero between calls.
     float2* ml_part;                  // [kRing][HG][cph][R]
     float* o_part;                    // [kRing][HG][cph][R][kD]
     int* status;
@@ -252,6 +253,22 @@ int launch_twosweep(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensor
                     int grid, size_t smem_bytes, cudaStream_t stream);
 int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                   int grid, size_t smem_bytes, cudaStream_t stream);
+
+// End of kernel: the last CTA to get here puts the cross-CTA counters back to zero, so the next
+// call on this workspace needs no memset (a memset node between two kernels of a CUDA graph
+// costs more than the whole prologue of this kernel).  Call after the CTA's last use of them.
+__device__ __forceinline__ void reset_counters_if_last(const FastParams& p, int* smem_flag)
+{
+    const int n = 2 * p.n_units * p.HG;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        *smem_flag = atomicAdd(p.counters + n, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (*smem_flag) {
+        for (int i = threadIdx.x; i <= n; i += blockDim.x) p.counters[i] = 0;
+    }
+}
 
 template <int NH>
 __device__ __forceinline__ void load_cols(uint32_t taddr, uint32_t* v)

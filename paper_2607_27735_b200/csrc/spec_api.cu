@@ -116,7 +116,6 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
         if (impl != SPEC_VERIFY_AUTO || rc2 != SPEC_ERR_UNSUPPORTED_SHAPE) return rc2;
     }
     if (workspace_bytes < verify_generic_workspace(a.kv, n_q, max_ctx_len)) return SPEC_ERR_WORKSPACE_TOO_SMALL;
-    if (cudaMemsetAsync(workspace, 0, kStatusBytes, stream) != cudaSuccess) return SPEC_ERR_CUDA;
     g_last_verify_impl.store(SPEC_VERIFY_GENERIC);
     return verify_generic_launch(a, stream);
 }

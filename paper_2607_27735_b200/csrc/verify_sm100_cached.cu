@@ -83,7 +83,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.aux_sync = o; o += 8;
         B.stat_full = o; o += 32;
     }
-    float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128]
+    float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128] global row LSE (log2 domain)
+    float* loc_s = reinterpret_cast<float*>(misc + 1024 + 512);           // [128] CTA-local row LSE
+    float* fac_s = reinterpret_cast<float*>(misc + 2048);                 // [128] exp2(local - global)
     float2* red = reinterpret_cast<float2*>(misc + 8192);                 // [kSW warps][NC] (m, l), <= 4 KB
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 12288);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -119,7 +121,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     // zero the Q buffers once: rows R..N-1 are padding the TMA never writes
     for (int i = threadIdx.x; i < q_bytes / 16; i += kBlock)
         *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
-    for (int r = R + threadIdx.x; r < 128; r += kBlock) lse_s[r] = 1.0e30f;  // padded rows: P = 0
+    for (int r = R + threadIdx.x; r < 128; r += kBlock) {  // padded rows: P = 0
+        lse_s[r] = 1.0e30f;
+        loc_s[r] = 1.0e30f;
+    }
     fence_proxy_async();
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -389,10 +394,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
         uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, sfull_par = 0;
         bool ok = true;
-        int pend_unit = -1;                      // unit whose O accumulator still waits for its epilogue
-        bool pend_nonempty = false;
 
-        // O^T (d on lanes, rows on columns, hi and lo parts) -> this CTA's partial [r][d]
+        // O^T (d on lanes, rows on columns, hi and lo parts), rescaled from the CTA-local to the
+        // global normaliser -> this CTA's partial [r][d]
         auto epilogue = [&](int unit, bool nonempty) -> bool {
             const int64_t obase = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R * kD;
             if (nonempty) {
@@ -408,7 +412,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
                 for (int i = 0; i < NH; ++i) {
                     const int r = c0 + i;
-                    if (r < R) p.o_part[obase + (int64_t)r * kD + key_l] = __uint_as_float(v[i]) + __uint_as_float(w[i]);
+                    if (r < R)
+                        p.o_part[obase + (int64_t)r * kD + key_l] =
+                            (__uint_as_float(v[i]) + __uint_as_float(w[i])) * fac_s[r];
                 }
             } else {
                 for (int i = tid_s; i < R * kD; i += 128 * CG) p.o_part[obase + i] = 0.f;
@@ -489,8 +495,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             ok = group_sync(B.sm_sync, sync_n, ctl, 26);
             if (!ok) break;
             if (sw == kSW - 1) {
-                // the last softmax warp merges the four lane quarters of every column and publishes
-                // the CTA's partial; the other warps go on (they meet it again at the counter)
+                // the last softmax warp merges the four lane quarters of every column, publishes the
+                // CTA's partial and leaves the CTA-local normaliser for the P V pass
                 const int64_t base = (((int64_t)(unit % kRing) * p.HG + head_local) * p.cph + rank) * R;
                 for (int col = lane; col < R; col += 32) {
                     const int wgi = col / NC, ci = col - wgi * NC;
@@ -503,7 +509,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         const float2 ml = red[(wgi * 4 + w) * NC + ci];
                         Ls += ml.y * ex2(ml.x - M);
                     }
-                    p.ml_part[base + col] = make_float2(M, nonempty ? Ls : 0.f);
+                    const bool has = nonempty && M > 0.5f * kNegBig;  // the row saw at least one key here
+                    p.ml_part[base + col] = make_float2(M, has ? Ls : 0.f);
+                    loc_s[col] = has ? M + log2f(Ls) : 1.0e30f;       // no key: P = exp2(s - big) = 0
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -511,15 +519,110 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     atomicAdd(p.counters + unit * p.HG + head_local, 1);
                 }
             }
+            ok = group_sync(B.sm_sync, sync_n, ctl, 27);
+            if (!ok) break;
             if (warp == 4) TRACE(2, 3);
-            // ---- while the other CTAs finish their P1: drain the previous unit's accumulator ----
-            if (pend_unit >= 0) {
-                ok = epilogue(pend_unit, pend_nonempty);
-                if (!ok) break;
-                pend_unit = -1;
-            }
-            if (warp == 4) TRACE(2, 4);
             if (nonempty) {
+                // ------------------------------ P2a: P V with the CTA-local normaliser ------------------
+                // P~ = exp2(S - lse_local) needs nothing from other CTAs, so V streams and the tensor
+                // cores run while the partials of the other CTAs are still on their way; the partial
+                // O is rescaled by exp2(lse_local - LSE) per row in the epilogue.
+                // Tile-split: warpgroup wg takes the tiles c = wg, wg + CG, ... whole (all N columns
+                // per thread), so CG tiles are in flight at once and each tile's fixed costs (waits,
+                // proxy fence, arrivals) are paid by one warpgroup instead of by all of them.
+                for (int c = wg; c < n_t && ok; c += CG) {
+                    const int t = sg.t0 + c;
+                    const uint32_t vslot = slot_base + n_t + c;
+                    const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
+                    const uint32_t pvi = pv_idx + c;
+                    const uint32_t pb = pvi % p.p_bufs;
+                    const int key = t * kTile + key_l;
+                    const bool boundary = t * kTile + kTile > sg.T - p.a.n_q + 1;
+                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + (key_l >> 3) * 128 + (key_l & 7) * 16;
+                    bool waited = false;
+#pragma unroll 1
+                    for (int cb = 0; cb < N; cb += 16) {  // 16 columns at a time keeps the live set small
+                        uint32_t v[16];
+                        tmem_ld8(t_lane + col_s + c * N + cb, v);
+                        tmem_ld8(t_lane + col_s + c * N + cb + 8, v + 8);
+                        tc_wait_ld();
+                        const float4* loc4 = reinterpret_cast<const float4*>(loc_s + cb);
+                        float pr[16];
+#pragma unroll
+                        for (int i = 0; i < 16; i += 4) {
+                            const float4 ls = loc4[i >> 2];
+                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
+                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
+                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
+                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
+                        }
+                        if (boundary) {
+                            int j = cb / G, gg = cb - j * G;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
+                                if (++gg == G) {
+                                    gg = 0;
+                                    ++j;
+                                }
+                            }
+                        }
+                        if (!waited) {
+                            // the P buffer is free once the P V product p_bufs tiles back is done.  Warpgroups
+                            // run ahead of each other, so the "done" barriers are indexed by the tile's
+                            // sequence number mod 4: a waiter is then never two phases ahead of its barrier.
+                            if (pvi >= (uint32_t)p.p_bufs) {
+                                const uint32_t prev = pvi - p.p_bufs;
+                                ok = mbar_wait(B.p_empty + 8 * (prev & 3), (prev >> 2) & 1, ctl, 23);
+                                if (!ok) break;
+                            }
+                            waited = true;
+                        }
+                        // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, no swizzle): the
+                        // 16-byte vector of row block j (rows 8j..8j+7 of the concatenation) and key k
+                        // lives at j*2048 + (k/8)*128 + (k%8)*16
+#pragma unroll
+                        for (int nb = 0; nb < 2; ++nb) {
+                            uint32_t hi[4], lo[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                // p = hi + lo with both parts cut to bf16 by truncation (plain integer ops, no
+                                // conversion instructions): hi keeps the top 16 bits, lo the top 16 bits of the
+                                // exact remainder, so p - (hi + lo) < 2^-14 p
+                                const uint32_t ua = __float_as_uint(pr[nb * 8 + 2 * q]), ub = __float_as_uint(pr[nb * 8 + 2 * q + 1]);
+                                hi[q] = __byte_perm(ua, ub, 0x7632);
+                                const float ra = __uint_as_float(ua) - __uint_as_float(ua & 0xffff0000u);
+                                const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
+                                lo[q] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
+                            }
+                            const int jh = cb / 8 + nb, jl = jh + N / 8;
+                            *reinterpret_cast<uint4*>(p_row + jh * 2048) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                            *reinterpret_cast<uint4*>(p_row + jl * 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        }
+                    }
+                    if (!ok) break;
+                    if (t * kTile + kTile > sg.T) {
+                        // ragged last tile: V rows at or beyond T may hold anything; zero them in
+                        // shared memory so that 0 * garbage never reaches the accumulator
+                        ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
+                        if (!ok) break;
+                        if (key >= sg.T) {
+                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + key_l * 128;
+#pragma unroll
+                            for (int ch = 0; ch < 8; ++ch) {
+                                *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4*>(vrow + 16384 + 16 * ch) = make_uint4(0, 0, 0, 0);
+                            }
+                        }
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
+                }
+                if (!ok) break;
+                pv_idx += n_t;
+                slot_base += 2 * n_t;
+                if (warp == 4) TRACE(2, 4);
                 // ---- row LSE from the partials of the CTAs that share this head ----
                 if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
@@ -556,6 +659,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 if (sub == 0 && r < R) {
                     const float lse2 = M + log2f(Ls);
                     lse_s[r] = lse2;
+                    const float loc = loc_s[r];
+                    fac_s[r] = loc < 1.0e29f ? ex2(loc - lse2) : 0.f;  // local -> global normaliser
                     if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
                         const int j = r / G, g = r - j * G;
                         const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
@@ -565,24 +670,18 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 ok = group_sync(B.sm_sync, sync_n, ctl, 22);
                 if (!ok) break;
                 if (warp == 4) TRACE(2, 6);
-                // ------------------------------ P2 ------------------------------
-                // Tile-split: warpgroup wg takes the tiles c = wg, wg + CG, ... whole (all N
-                // columns per thread), so CG tiles are in flight at once, the statistic is a
-                // thread-local sum, and each tile's fixed costs (waits, proxy fence, arrivals)
-                // are paid by one warpgroup instead of by all of them.
-                for (int c = wg; c < n_t && ok; c += CG) {
+                // ------------------------------ P2b: the Eq. 3 statistic ------------------------------
+                // second visit of the cached score tiles, now with the global LSE: column sums of the
+                // exactly normalised probabilities.  No shared memory, no tensor cores; the tile's
+                // TMEM region is released afterwards.
+                for (int c = wg; c < n_t; c += CG) {
                     const int t = sg.t0 + c;
-                    const uint32_t vslot = slot_base + n_t + c;
-                    const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
-                    const uint32_t pvi = pv_idx + c;
-                    const uint32_t pb = pvi % p.p_bufs;
                     const int key = t * kTile + key_l;
                     const bool boundary = t * kTile + kTile > sg.T - p.a.n_q + 1;
-                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + (key_l >> 3) * 128 + (key_l & 7) * 16;
                     float st = 0.f;
-                    bool waited = false;
 #pragma unroll 1
-                    for (int cb = 0; cb < N; cb += 16) {  // 16 columns at a time keeps the live set small
+                    for (int cb = 0; cb < N; cb += 16) {
+                        if (cb + 16 <= stat_r0) continue;  // rows outside the statistic window
                         uint32_t v[16];
                         tmem_ld8(t_lane + col_s + c * N + cb, v);
                         tmem_ld8(t_lane + col_s + c * N + cb + 8, v + 8);
@@ -615,72 +714,19 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
                             for (int i = 0; i < 16; ++i) st += (cb + i >= stat_r0) ? pr[i] : 0.f;
                         }
-                        if (!waited) {
-                            // the P buffer is free once the P V product p_bufs tiles back is done.  Warpgroups
-                            // run ahead of each other, so the "done" barriers are indexed by the tile's
-                            // sequence number mod 4: a waiter is then never two phases ahead of its barrier.
-                            if (pvi >= (uint32_t)p.p_bufs) {
-                                const uint32_t prev = pvi - p.p_bufs;
-                                ok = mbar_wait(B.p_empty + 8 * (prev & 3), (prev >> 2) & 1, ctl, 23);
-                                if (!ok) break;
-                            }
-                            waited = true;
-                        }
-                        // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, no swizzle): the
-                        // 16-byte vector of row block j (rows 8j..8j+7 of the concatenation) and key k
-                        // lives at j*2048 + (k/8)*128 + (k%8)*16
-#pragma unroll
-                        for (int nb = 0; nb < 2; ++nb) {
-                            uint32_t hi[4], lo[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                // p = hi + lo with both parts cut to bf16 by truncation (plain integer ops, no
-                                // conversion instructions): hi keeps the top 16 bits, lo the top 16 bits of the
-                                // exact remainder, so p - (hi + lo) < 2^-14 p
-                                const uint32_t ua = __float_as_uint(pr[nb * 8 + 2 * q]), ub = __float_as_uint(pr[nb * 8 + 2 * q + 1]);
-                                hi[q] = __byte_perm(ua, ub, 0x7632);
-                                const float ra = __uint_as_float(ua) - __uint_as_float(ua & 0xffff0000u);
-                                const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
-                                lo[q] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
-                            }
-                            const int jh = cb / 8 + nb, jl = jh + N / 8;
-                            *reinterpret_cast<uint4*>(p_row + jh * 2048) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                            *reinterpret_cast<uint4*>(p_row + jl * 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                        }
                     }
-                    if (!ok) break;
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_free + 8 * c);
-                    if (t * kTile + kTile > sg.T) {
-                        // ragged last tile: V rows at or beyond T may hold anything; zero them in
-                        // shared memory so that 0 * garbage never reaches the accumulator
-                        ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
-                        if (!ok) break;
-                        if (key >= sg.T) {
-                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + key_l * 128;
-#pragma unroll
-                            for (int ch = 0; ch < 8; ++ch) {
-                                *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
-                                *reinterpret_cast<uint4*>(vrow + 16384 + 16 * ch) = make_uint4(0, 0, 0, 0);
-                            }
-                        }
-                    }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
                     if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st;
                 }
-                if (!ok) break;
-                pv_idx += n_t;
-                slot_base += 2 * n_t;
             }
-            pend_unit = unit;
-            pend_nonempty = nonempty;
             if (warp == 4) TRACE(2, 7);
+            // ---- this unit's accumulator: rescale and hand to the reducers ----
+            ok = epilogue(unit, nonempty);
+            if (!ok) break;
+            if (warp == 4) TRACE(2, 8);
         }
-        if (ok && pend_unit >= 0) ok = epilogue(pend_unit, pend_nonempty);
-        if (warp == 4) TRACE(2, 8);
     }
 
     // ---- teardown ----
@@ -690,6 +736,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+    if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
 template <int NC, int CG>
@@ -709,6 +756,9 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+#ifdef SPEC_TRACE
+    if (fp.dbg & 128) cfg.numAttrs = 0;  // timing experiment only
+#endif
     if (cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp) != cudaSuccess) {
         cudaGetLastError();
         return SPEC_ERR_CUDA;

@@ -709,6 +709,7 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+    if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
 template <int NH>
