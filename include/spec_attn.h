@@ -169,6 +169,33 @@ int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* in
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Verification attention without a caller-provided workspace.  The paper has no counterpart;
+ * this entry point exists for hosts that cannot allocate device memory themselves: a plugin
+ * running inside a runtime that owns every device buffer and hands in only inputs and
+ * outputs, or code that starts after a framework's memory pool has taken the whole GPU.
+ *
+ * Same arguments, results and error codes as spec_verify_attn, minus the workspace.  The
+ * scratch is a fixed array inside the library image: spec_noalloc_scratch_bytes() bytes
+ * (16 MiB) on every GPU that loads the library, held until the process exits.  The call
+ * allocates and frees nothing.
+ *   - A shape whose spec_workspace_bytes(SPEC_WS_VERIFY, ...) exceeds that size is refused with
+ *     SPEC_ERR_WORKSPACE_TOO_SMALL before anything is launched.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, with that device current); make that first call before starting any
+ *     stream capture on the device.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents;
+ *     every call re-zeroes the control words it depends on, on `cuda_stream`.  Two calls that
+ *     may overlap on the GPU (different streams, no ordering) race on it: serialise them.
+ *   - spec_noalloc_read_status() is spec_read_status() on that array for the current device.
+ */
+int spec_verify_attn_noalloc(const spec_kv_t* kv, const void* q, int32_t n_q,
+                             const int32_t* ctx_len, int32_t max_ctx_len, int32_t stat_window,
+                             float* out, float* lse, float* stats, int64_t stat_stride,
+                             void* cuda_stream);
+size_t spec_noalloc_scratch_bytes(void);
+int spec_noalloc_read_status(void* cuda_stream);
+
+/*
  * Bytes of workspace entry point `which` needs for this cache description.  n_q and
  * max_ctx_len matter for SPEC_WS_VERIFY, k_total (+ max_tail folded into it by the caller)
  * for SPEC_WS_DRAFT.  Returns 0 on invalid arguments.

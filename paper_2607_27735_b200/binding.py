@@ -21,7 +21,8 @@ VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCG
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
     "spec_read_status", "spec_set_verify_impl", "spec_last_verify_impl", "spec_launch_count",
-    "spec_strerror", "spec_version",
+    "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
+    "spec_noalloc_read_status",
 ]
 
 
@@ -63,6 +64,10 @@ def load() -> ctypes.CDLL:
                                            ctypes.c_size_t, vp]
         lib.spec_sparse_draft_attn.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
                                                vp, vp, vp, ctypes.c_size_t, vp]
+        lib.spec_verify_attn_noalloc.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp,
+                                                 vp, i64, vp]
+        lib.spec_noalloc_scratch_bytes.restype = ctypes.c_size_t
+        lib.spec_noalloc_read_status.argtypes = [vp]
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
         lib.spec_workspace_bytes.restype = ctypes.c_size_t
         lib.spec_read_status.argtypes = [vp, vp]
@@ -138,6 +143,41 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
     if rc != 0:
         raise SpecError(rc, "spec_verify_attn")
     return out, lse, stats, workspace
+
+
+def spec_verify_attn_noalloc(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None,
+                             stats=None, want_lse=True):
+    """spec_verify_attn on the library's built-in scratch, for callers that cannot allocate a
+    workspace (a plugin inside a runtime that owns all device memory).  The output tensors are
+    still the caller's; this wrapper creates them only when they are not passed in.
+    Returns ``(out, lse, stats)``."""
+    lib = load()
+    L, B, n_q, Hq, D = q.shape
+    dev = q.device
+    s = _kv_struct(kv)
+    if out is None:
+        out = torch.empty(L, B, n_q, Hq, D, dtype=torch.float32, device=dev)
+    if lse is None and want_lse:
+        lse = torch.empty(L, B, n_q, Hq, dtype=torch.float32, device=dev)
+    if stats is None:
+        stats = torch.zeros(L, B, kv.n_kv_heads, (max_ctx_len + 63) // 64 * 64,
+                            dtype=torch.float32, device=dev)
+    rc = lib.spec_verify_attn_noalloc(
+        ctypes.byref(s), _dev(q, torch.bfloat16, "q"), n_q, _dev(ctx_len, torch.int32, "ctx_len"),
+        max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
+        None if lse is None else _dev(lse, torch.float32, "lse"),
+        _dev(stats, torch.float32, "stats"), stats.shape[-1], _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_verify_attn_noalloc")
+    return out, lse, stats
+
+
+def noalloc_scratch_bytes() -> int:
+    return int(load().spec_noalloc_scratch_bytes())
+
+
+def noalloc_read_status() -> int:
+    return int(load().spec_noalloc_read_status(_stream()))
 
 
 def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, n_indices=None):
