@@ -1,8 +1,8 @@
 // Sparse draft attention of Eq. 5: one query per sequence attends the recalled rows
 // Gather(K, I), Gather(V, I) plus the dense tail of tokens drafted this round.  The gather is
-// fused: 16-byte cp.async copies pull the indexed 2*D-byte rows straight from the dense cache
-// into shared memory (two 160-key tiles, so a few hundred keys per CTA are all in flight at
-// once); nothing gathered is written back to global memory.
+// fused: one bulk asynchronous copy (cp.async.bulk, completion on an mbarrier) per indexed
+// 2*D-byte row pulls K and V straight from the dense cache into shared memory (two 144-key
+// tiles in flight per CTA); nothing gathered is written back to global memory.
 //
 // The call is latency-bound (a few thousand recalled keys per head), so the kernel is built to
 // be short rather than wide:
@@ -25,22 +25,41 @@ namespace spec {
 
 namespace {
 
-constexpr int kTK = 160;       // keys per tile: ten 16-key chunks dealt to the 8 warps
-constexpr int kStages = 2;     // two tiles (320 keys) can be in flight per CTA
+constexpr int kTK = 144;       // keys per tile: nine 16-key chunks dealt to the 8 warps
+constexpr int kStages = 2;     // two tiles (288 keys) can be in flight per CTA
 constexpr int kThreads = 256;
 constexpr int kMaxGroup = 8;   // query heads per KV head
-constexpr int kMaxCluster = 8; // portable cluster size
+constexpr int kMaxCluster = 8;  // portable cluster size (16 was measured slower: one cluster per GPC)
+constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // bound of the copy wait: about a second
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc)
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gsrc) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_dyn(int pending)
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
-    if (pending <= 0) asm volatile("cp.async.wait_group 0;\n" ::: "memory");
-    else asm volatile("cp.async.wait_group 1;\n" ::: "memory");
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// one row of the cache -> shared memory (16-byte aligned on both sides, size a multiple of 16)
+__device__ __forceinline__ void bulk_copy_row(void* smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(smem_dst)), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p)
 {
@@ -82,11 +101,13 @@ struct SmemLayout {
     static constexpr int off_v = kStages * kv_tile;
     static constexpr int off_q = 2 * kStages * kv_tile;              // bf16 [16][PITCH], rows >= G zero
     static constexpr int off_pos = off_q + 16 * PITCH * 2;           // int [kStages][kTK]
-    static constexpr int off_wml = off_pos + kStages * kTK * 4;      // float2 [8 warps][kMaxGroup]
+    static constexpr int off_bar = off_pos + kStages * kTK * 4;      // mbarrier [kStages]
+    static constexpr int off_wml = off_bar + 64;                     // float2 [8 warps][kMaxGroup]
     static constexpr int off_wo = off_k;  // float [8 warps][kMaxGroup][D]: reuses the K tiles once the loop is over
     static constexpr int off_comb = off_wml + 8 * kMaxGroup * 8;     // float [kMaxCluster][kMaxGroup][D + 2]
     static constexpr int total = off_comb + kMaxCluster * kMaxGroup * (D + 2) * 4;
     static_assert(8 * kMaxGroup * D * 4 <= kStages * kv_tile, "warp partials must fit in the K tiles");
+    static_assert(PITCH * 2 % 16 == 0, "bulk copies need 16-byte aligned rows");
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
@@ -117,55 +138,82 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    // Programmatic dependent launch: the next kernel in the stream may start its own prologue
+    // (index loads, gather of recalled rows) while this one is still computing.  Everything this
+    // kernel reads before griddep_wait() below is immutable during a drafting round (indices,
+    // lengths, recalled rows of the dense cache); Q, the dense tail and the outputs come after.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool dep_waited = false;
+    auto griddep_wait = [&]() {
+        if (!dep_waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            dep_waited = true;
+        }
+    };
+    const uint32_t bar0 = smem_addr(smem + SL::off_bar);
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) mbar_init(bar0 + 8 * i, kTK);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const int32_t* idx = a.indices + prob * a.k_total;
+    // the index of this thread's row in the first tile is fetched before the list length is
+    // known (the tail of the array holds -1 padding, never read past k_total)
+    const int per_guess = ((a.k_total + a.max_tail + CS - 1) / CS + 15) & ~15;
+    int idx_pre = -1;
+    if (tid < kTK && rank * per_guess + tid < a.k_total) idx_pre = __ldg(idx + rank * per_guess + tid);
     const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
     const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
     const int n_tail = min(max(cl - ts, 0), a.max_tail);
     const int n = n_rec + n_tail;
-    const int per = (n + CS - 1) / CS;
+    // contiguous shares in multiples of the 16-key chunk; the share size depends only on host-side
+    // bounds, so every CTA of the cluster agrees on it without exchanging anything
+    const int per = per_guess;
     const int k0 = min(n, rank * per);
     const int k1 = min(n, k0 + per);
     const int n_tiles = (k1 - k0 + kTK - 1) / kTK;
-    const int32_t* idx = a.indices + prob * a.k_total;
+    __syncthreads();  // barriers initialised
 
-    // positions of a tile, then its rows: every copy of the tile is in flight before any wait
+    // one thread per row: position, then one bulk copy each for the K row and the V row; every
+    // copy of the tile is in flight before anything waits
     auto issue_tile = [&](int tile) {
         const int buf = tile % kStages;
         const int base = k0 + tile * kTK;
         const int nk = min(kTK, k1 - base);
-        int* kp = keypos + buf * kTK;
-        if (tid < kTK) {
-            int pos = -1;
-            if (tid < nk) {
-                const int e = base + tid;
-                pos = e < n_rec ? __ldg(idx + e) : ts + (e - n_rec);
-                if (pos < 0 || pos >= cl) {
-                    set_status(status, SPEC_ERR_BAD_INDEX);
-                    pos = -1;
-                }
-            }
-            kp[tid] = pos;
-        }
-        __syncthreads();
-        __nv_bfloat16* kb = Ks + buf * kTK * PITCH;
-        __nv_bfloat16* vb = Vs + buf * kTK * PITCH;
-        for (int c = tid; c < kTK * CH; c += kThreads) {
-            const int row = c / CH, ch = c - row * CH;
-            const int pos = kp[row];
-            if (pos >= 0) {
-                const int64_t off = kv_row_offset(a.kv, layer, b, pos, h) + ch * 8;
-                cp_async16(kb + row * PITCH + ch * 8, a.kv.k + off);
-                cp_async16(vb + row * PITCH + ch * 8, a.kv.v + off);
-            } else {  // masked rows must still be finite: they meet P = 0 in the P V product
-                *reinterpret_cast<uint4*>(kb + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(vb + row * PITCH + ch * 8) = make_uint4(0, 0, 0, 0);
+        if (base + nk > n_rec) griddep_wait();  // the tile reaches into the tail drafted this round
+        if (tid >= kTK) return;
+        const uint32_t bar = bar0 + 8 * buf;
+        int pos = -1;
+        if (tid < nk) {
+            const int e = base + tid;
+            pos = e < n_rec ? (tile == 0 ? idx_pre : __ldg(idx + e)) : ts + (e - n_rec);
+            if (pos < 0 || pos >= cl) {
+                set_status(status, SPEC_ERR_BAD_INDEX);
+                pos = -1;
             }
         }
-        cp_async_commit();
+        keypos[buf * kTK + tid] = pos;
+        __nv_bfloat16* kr = Ks + (buf * kTK + tid) * PITCH;
+        __nv_bfloat16* vr = Vs + (buf * kTK + tid) * PITCH;
+        if (pos >= 0) {
+            const int64_t off = kv_row_offset(a.kv, layer, b, pos, h);
+            mbar_arrive_expect_tx(bar, 2 * D * 2);
+            bulk_copy_row(kr, a.kv.k + off, D * 2, bar);
+            bulk_copy_row(vr, a.kv.v + off, D * 2, bar);
+        } else {  // masked rows must still be finite: they meet P = 0 in the P V product
+#pragma unroll
+            for (int ch = 0; ch < CH; ++ch) {
+                *reinterpret_cast<uint4*>(kr + ch * 8) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vr + ch * 8) = make_uint4(0, 0, 0, 0);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // a later bulk copy reuses the row
+            mbar_arrive(bar);
+        }
     };
 
     int issued = 0;
     for (; issued < min(n_tiles, kStages); ++issued) issue_tile(issued);
 
+    griddep_wait();
     // Q of the group -> bf16 [16][PITCH] in shared memory (rows >= G zero), then A fragments
     for (int i = tid; i < 16 * CH; i += kThreads) {
         const int g = i / CH, ch = i - g * CH;
@@ -192,8 +240,16 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 
     for (int tile = 0; tile < n_tiles; ++tile) {
         const int buf = tile % kStages;
-        cp_async_wait_dyn(issued - tile - 1);
-        __syncthreads();
+        {  // the tile's rows have landed (bounded wait: a stall ends in a status code)
+            const uint32_t bar = bar0 + 8 * buf, parity = (tile / kStages) & 1;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar, parity)) {
+                if (clock64() - t0 > kTimeoutCycles) {
+                    set_status(status, SPEC_ERR_TIMEOUT);
+                    break;
+                }
+            }
+        }
         const int nk = min(kTK, k1 - (k0 + tile * kTK));
         for (int ck = warp * 16; ck < nk; ck += 8 * 16) {  // this warp's 16-key chunks of the tile
             const int* kp = keypos + buf * kTK;
@@ -324,11 +380,11 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 
 int pick_cluster(const KvView& kv, int n_keys_max)
 {
-    // enough CTAs to cover the SMs, at most one tile-pair of work each, at most a portable cluster
+    // enough CTAs to cover the SMs, at most about one tile of work each
     const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
     const int tiles = n_keys_max > 0 ? (n_keys_max + kTK - 1) / kTK : 1;
     int cs = 1;
-    while (cs < kMaxCluster && probs * cs < sm_count() && cs * 2 <= tiles) cs *= 2;
+    while (cs < kMaxCluster && probs * cs < sm_count() && cs < tiles) cs *= 2;
     return cs;
 }
 
@@ -337,26 +393,38 @@ int launch_d(const DraftArgs& a, int cs, cudaStream_t stream)
 {
     auto kern = draft_cluster_kernel<D>;
     const size_t smem = SmemLayout<D>::total;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return SPEC_ERR_CUDA;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cs;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, kern, a, static_cast<int*>(a.workspace)) != cudaSuccess) {
-        cudaGetLastError();
-        return SPEC_ERR_CUDA;
+    static bool configured = false;  // per template instance
+    if (!configured) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return SPEC_ERR_CUDA;
+        // clusters of 16 are outside the portable range: opt in (a refusal just keeps them at 8)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+            cudaGetLastError();
+        configured = true;
     }
-    count_launch(1);
-    return SPEC_OK;
+    for (; cs >= 1; cs /= 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the kernel's prologue
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        if (cudaLaunchKernelEx(&cfg, kern, a, static_cast<int*>(a.workspace)) == cudaSuccess) {
+            count_launch(1);
+            return SPEC_OK;
+        }
+        cudaGetLastError();
+        if (cs <= 8) break;  // a portable size that still fails is a real error
+    }
+    return SPEC_ERR_CUDA;
 }
 
 }  // namespace

@@ -236,7 +236,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.trace = nullptr;
     fp.dbg = 0;
 #ifdef SPEC_TRACE
-    fp.trace = reinterpret_cast<long long*>(ws + pl.trace_off);
+    fp.trace = reinterpret_cast<long long*>(ws + a.workspace_bytes - (size_t)sm_count() * 4 * 64 * sizeof(long long));  // tail of the caller's buffer
     if (const char* e = std::getenv("SPEC_DBG")) fp.dbg = std::atoi(e);
 #endif
     // no memset: the workspace arrives zeroed and the kernel's last CTA re-zeroes the counters
