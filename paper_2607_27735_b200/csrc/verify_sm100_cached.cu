@@ -133,6 +133,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // Programmatic dependent launch: this kernel's prologue above may run while the previous
+    // kernel in the stream drains; nothing before this point touches global memory the stream
+    // produces (the workspace is shared with the previous call).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     const int U = p.n_units;
     const uint32_t col_o = 0, col_s = 2 * N;  // O^T (hi | lo) first, then the cached S^T tiles
@@ -513,14 +518,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     p.ml_part[base + col] = make_float2(M, has ? Ls : 0.f);
                     loc_s[col] = has ? M + log2f(Ls) : 1.0e30f;       // no key: P = exp2(s - big) = 0
                 }
-                __syncwarp();
-                if (lane == 0) {
-                    __threadfence();
-                    atomicAdd(p.counters + unit * p.HG + head_local, 1);
-                }
             }
             ok = group_sync(B.sm_sync, sync_n, ctl, 27);
             if (!ok) break;
+            if (sw == kSW - 1 && lane == 0) {  // publish after the barrier: nobody here waits for the round trip
+                __threadfence();
+                atomicAdd(p.counters + unit * p.HG + head_local, 1);
+            }
             if (warp == 4) TRACE(2, 3);
             if (nonempty) {
                 // ------------------------------ P2a: P V with the CTA-local normaliser ------------------
@@ -751,15 +755,22 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
     cfg.blockDim = dim3(128 + 128 * CG);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they wait on each other
     attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-#ifdef SPEC_TRACE
-    if (fp.dbg & 128) cfg.numAttrs = 0;  // timing experiment only
-#endif
-    if (cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp) != cudaSuccess) {
+    static bool pdl_ok = true;  // a driver that refuses the combination is asked only once
+    cfg.numAttrs = pdl_ok ? 2 : 1;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp);
+    if (err != cudaSuccess && cfg.numAttrs == 2) {
+        cudaGetLastError();
+        pdl_ok = false;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp);
+    }
+    if (err != cudaSuccess) {
         cudaGetLastError();
         return SPEC_ERR_CUDA;
     }
