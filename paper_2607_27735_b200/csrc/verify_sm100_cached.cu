@@ -38,7 +38,7 @@ constexpr int kMaxCache = 32;
 
 struct CBars {  // mbarrier addresses (shared space)
     uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_free, p_full, p_empty, o_full, o_empty, sm_sync,
-        aux_sync, stat_full;
+        pub_p1, pub_o;
 };
 
 // NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
@@ -80,8 +80,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.o_full = o; o += 8;
         B.o_empty = o; o += 8;
         B.sm_sync = o; o += 8;
-        B.aux_sync = o; o += 8;
-        B.stat_full = o; o += 32;
+        B.pub_p1 = o; o += 8;   // the last softmax warp stored this CTA's (max, sum) partial
+        B.pub_o = o; o += 8;    // every softmax warp stored its share of the output partial
     }
     float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128] global row LSE (log2 domain)
     float* loc_s = reinterpret_cast<float*>(misc + 1024 + 512);           // [128] CTA-local row LSE
@@ -113,8 +113,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         mbar_init(B.o_full, 1);
         mbar_init(B.o_empty, kSW);
         mbar_init(B.sm_sync, kSW);
-        mbar_init(B.aux_sync, 2);
-        for (int i = 0; i < 4; ++i) mbar_init(B.stat_full + 8 * i, CG > 1 ? 4 * (CG - 1) : 1);
+        mbar_init(B.pub_p1, 1);
+        mbar_init(B.pub_o, kSW);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -347,22 +347,39 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
         }
         __syncwarp();
-    } else if (warp < 4) {
-        // =========================== O reduction warps ===========================
-        const int tid = threadIdx.x - 64;  // 0..63
+    } else if (warp == 2) {
+        // =========================== publisher warp ===========================
+        // Makes this CTA's partials visible to the other CTAs (device-scope fence + counter), so
+        // that no softmax warp ever waits for that round trip: they only arrive on a CTA barrier.
+        if (lane == 0) {
+            bool ok = true;
+            for (int unit = 0; unit < U && ok; ++unit) {
+                ok = mbar_wait(B.pub_p1, unit & 1, ctl, 34);
+                if (!ok) break;
+                __threadfence();
+                atomicAdd(p.counters + unit * p.HG + head_local, 1);
+                ok = mbar_wait(B.pub_o, unit & 1, ctl, 35);
+                if (!ok) break;
+                __threadfence();
+                atomicAdd(p.counters + U * p.HG + unit * p.HG + head_local, 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 3) {
+        // =========================== O reduction warp ===========================
+        const int tid = lane;
         bool ok = true;
         for (int unit = 0; unit < U && ok; ++unit) {
             if (lane == 0) ok = counter_wait(p.counters + U * p.HG + unit * p.HG + head_local, p.cph, ctl, 30);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-            __threadfence();
-            if (warp == 2) TRACE(3, 1);
+            TRACE(3, 1);
             const Seg sg = get_seg(p, unit, head_local, rank);
             const int E4 = R * kD / 4;
             const int lo = (int)((int64_t)rank * E4 / p.cph), hi = (int)((int64_t)(rank + 1) * E4 / p.cph);
             const float4* src = reinterpret_cast<const float4*>(
                 p.o_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R * kD);
-            for (int e = lo + tid; e < hi; e += 64) {
+            for (int e = lo + tid; e < hi; e += 32) {
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int k0 = 0; k0 < p.cph; k0 += 16) {  // batches of 16 independent loads
                     float4 x[16];
@@ -383,7 +400,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
                 reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
             }
-            if (warp == 2) TRACE(3, 2);
+            TRACE(3, 2);
         }
     } else {
         // =========================== softmax warpgroups ===========================
@@ -424,11 +441,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             } else {
                 for (int i = tid_s; i < R * kD; i += 128 * CG) p.o_part[obase + i] = 0.f;
             }
-            if (!group_sync(B.sm_sync, sync_n, ctl, 29)) return false;
-            if (tid_s == 0) {
-                __threadfence();
-                atomicAdd(p.counters + U * p.HG + unit * p.HG + head_local, 1);
-            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(B.pub_o);  // the publisher warp fences and bumps the counter
             return true;
         };
 
@@ -518,13 +532,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     p.ml_part[base + col] = make_float2(M, has ? Ls : 0.f);
                     loc_s[col] = has ? M + log2f(Ls) : 1.0e30f;       // no key: P = exp2(s - big) = 0
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(B.pub_p1);  // the publisher warp takes it from here
             }
             ok = group_sync(B.sm_sync, sync_n, ctl, 27);
             if (!ok) break;
-            if (sw == kSW - 1 && lane == 0) {  // publish after the barrier: nobody here waits for the round trip
-                __threadfence();
-                atomicAdd(p.counters + unit * p.HG + head_local, 1);
-            }
             if (warp == 4) TRACE(2, 3);
             if (nonempty) {
                 // ------------------------------ P2a: P V with the CTA-local normaliser ------------------
