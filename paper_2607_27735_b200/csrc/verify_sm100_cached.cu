@@ -107,7 +107,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         for (int i = 0; i < 2; ++i) {
             mbar_init(B.q_full + 8 * i, 1);
             mbar_init(B.q_empty + 8 * i, 1);
-            mbar_init(B.p_full + 8 * i, 4);
+            mbar_init(B.p_full + 8 * i, kSW);
         }
         for (int i = 0; i < 4; ++i) mbar_init(B.p_empty + 8 * i, 1);
         mbar_init(B.o_full, 1);
@@ -543,39 +543,41 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 // P~ = exp2(S - lse_local) needs nothing from other CTAs, so V streams and the tensor
                 // cores run while the partials of the other CTAs are still on their way; the partial
                 // O is rescaled by exp2(lse_local - LSE) per row in the epilogue.
-                // Tile-split: warpgroup wg takes the tiles c = wg, wg + CG, ... whole (all N columns
-                // per thread), so CG tiles are in flight at once and each tile's fixed costs (waits,
-                // proxy fence, arrivals) are paid by one warpgroup instead of by all of them.
-                for (int c = wg; c < n_t && ok; c += CG) {
-                    const int t = sg.t0 + c;
-                    const uint32_t vslot = slot_base + n_t + c;
-                    const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
-                    const uint32_t pvi = pv_idx + c;
-                    const uint32_t pb = pvi % p.p_bufs;
-                    const int key = t * kTile + key_l;
-                    const bool boundary = t * kTile + kTile > sg.T - p.a.n_q + 1;
-                    uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + (key_l >> 3) * 128 + (key_l & 7) * 16;
-                    bool waited = false;
-#pragma unroll 1
-                    for (int cb = 0; cb < N; cb += 16) {  // 16 columns at a time keeps the live set small
-                        uint32_t v[16];
-                        tmem_ld8(t_lane + col_s + c * N + cb, v);
-                        tmem_ld8(t_lane + col_s + c * N + cb + 8, v + 8);
-                        tc_wait_ld();
-                        const float4* loc4 = reinterpret_cast<const float4*>(loc_s + cb);
-                        float pr[16];
+                // Column-split like P1: every warpgroup works on the same tile, NC columns each, so
+                // a tile's P is ready after one short pass; the score columns of the next tile are
+                // fetched from tensor memory while the current ones are being turned into P.
+                {
+                    const float4* loc4 = reinterpret_cast<const float4*>(loc_s + c0);
+                    uint32_t v[NH];
+                    if (n_t > 0) {
 #pragma unroll
-                        for (int i = 0; i < 16; i += 4) {
+                        for (int q = 0; q < NH; q += 8) tmem_ld8(t_lane + col_s + c0 + q, v + q);
+                    }
+                    for (int c = 0; c < n_t && ok; ++c) {
+                        const int t = sg.t0 + c;
+                        const uint32_t vslot = slot_base + n_t + c;
+                        const uint32_t vs = vslot % p.n_slots, vsph = (vslot / p.n_slots) & 1;
+                        const uint32_t pvi = pv_idx + c;
+                        const uint32_t pb = pvi % p.p_bufs;
+                        const int key = t * kTile + key_l;
+                        tc_wait_ld();
+                        float pr[NH];
+#pragma unroll
+                        for (int i = 0; i < NH; i += 4) {
                             const float4 ls = loc4[i >> 2];
                             pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
                             pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
                             pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
                             pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
                         }
-                        if (boundary) {
-                            int j = cb / G, gg = cb - j * G;
+                        if (c + 1 < n_t) {  // next tile's columns: in flight during the rest of this tile
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) {
+                            for (int q = 0; q < NH; q += 8) tmem_ld8(t_lane + col_s + (c + 1) * N + c0 + q, v + q);
+                        }
+                        if (t * kTile + kTile > sg.T - p.a.n_q + 1) {
+                            int j = c0 / G, gg = c0 - j * G;
+#pragma unroll
+                            for (int i = 0; i < NH; ++i) {
                                 if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
                                 if (++gg == G) {
                                     gg = 0;
@@ -583,22 +585,19 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                                 }
                             }
                         }
-                        if (!waited) {
-                            // the P buffer is free once the P V product p_bufs tiles back is done.  Warpgroups
-                            // run ahead of each other, so the "done" barriers are indexed by the tile's
-                            // sequence number mod 4: a waiter is then never two phases ahead of its barrier.
-                            if (pvi >= (uint32_t)p.p_bufs) {
-                                const uint32_t prev = pvi - p.p_bufs;
-                                ok = mbar_wait(B.p_empty + 8 * (prev & 3), (prev >> 2) & 1, ctl, 23);
-                                if (!ok) break;
-                            }
-                            waited = true;
+                        // the P buffer is free once the P V product p_bufs tiles back is done ("done"
+                        // barriers are indexed by the tile's sequence number mod 4)
+                        if (pvi >= (uint32_t)p.p_bufs) {
+                            const uint32_t prev = pvi - p.p_bufs;
+                            ok = mbar_wait(B.p_empty + 8 * (prev & 3), (prev >> 2) & 1, ctl, 23);
+                            if (!ok) break;
                         }
                         // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, no swizzle): the
                         // 16-byte vector of row block j (rows 8j..8j+7 of the concatenation) and key k
                         // lives at j*2048 + (k/8)*128 + (k%8)*16
+                        uint8_t* p_row = sgen + (s_p - sbase) + pb * p_bytes + (key_l >> 3) * 128 + (key_l & 7) * 16;
 #pragma unroll
-                        for (int nb = 0; nb < 2; ++nb) {
+                        for (int nb = 0; nb < NH / 8; ++nb) {
                             uint32_t hi[4], lo[4];
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
@@ -611,29 +610,25 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                                 const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
                                 lo[q] = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
                             }
-                            const int jh = cb / 8 + nb, jl = jh + N / 8;
+                            const int jh = wg * (NH / 8) + nb, jl = jh + N / 8;
                             *reinterpret_cast<uint4*>(p_row + jh * 2048) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                             *reinterpret_cast<uint4*>(p_row + jl * 2048) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                         }
-                    }
-                    if (!ok) break;
-                    if (t * kTile + kTile > sg.T) {
-                        // ragged last tile: V rows at or beyond T may hold anything; zero them in
-                        // shared memory so that 0 * garbage never reaches the accumulator
-                        ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
-                        if (!ok) break;
-                        if (key >= sg.T) {
-                            uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + key_l * 128;
+                        if (t * kTile + kTile > sg.T) {
+                            // ragged last tile: V rows at or beyond T may hold anything; zero them in
+                            // shared memory so that 0 * garbage never reaches the accumulator
+                            ok = mbar_wait(B.slot_full + 8 * vs, vsph, ctl, 24);
+                            if (!ok) break;
+                            if (key >= sg.T && wg < 2) {  // warpgroups 0 and 1 clear one 64-wide half each
+                                uint8_t* vrow = sgen + (s_slots - sbase) + vs * kSlotBytes + wg * 16384 + key_l * 128;
 #pragma unroll
-                            for (int ch = 0; ch < 8; ++ch) {
-                                *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
-                                *reinterpret_cast<uint4*>(vrow + 16384 + 16 * ch) = make_uint4(0, 0, 0, 0);
+                                for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(vrow + 16 * ch) = make_uint4(0, 0, 0, 0);
                             }
                         }
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
                     }
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(B.p_full + 8 * pb);
                 }
                 if (!ok) break;
                 pv_idx += n_t;
