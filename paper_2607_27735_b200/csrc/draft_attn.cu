@@ -129,6 +129,12 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     float* wo = reinterpret_cast<float*>(smem + SL::off_wo);
     float* comb = reinterpret_cast<float*>(smem + SL::off_comb);
 
+#ifdef SPEC_TRACE
+#define DSTAMP(i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) reinterpret_cast<long long*>(status)[8 + (i)] = clock64(); } while (0)
+#else
+#define DSTAMP(i) do { } while (0)
+#endif
+    DSTAMP(0);
     cg::cluster_group cluster = cg::this_cluster();
     const int CS = gridDim.x;              // the cluster spans the x dimension
     const int rank = blockIdx.x;
@@ -213,7 +219,9 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     int issued = 0;
     for (; issued < min(n_tiles, kStages); ++issued) issue_tile(issued);
 
+    DSTAMP(1);
     griddep_wait();
+    DSTAMP(2);
     // Q of the group -> bf16 [16][PITCH] in shared memory (rows >= G zero), then A fragments
     for (int i = tid; i < 16 * CH; i += kThreads) {
         const int g = i / CH, ch = i - g * CH;
@@ -230,6 +238,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     for (int ks = 0; ks < D / 16; ++ks)
         ldmatrix_x4(qa[ks], Qs + ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + ks * 16 + (lane >> 4) * 8);
 
+    DSTAMP(3);
     // per-warp flash-decoding state: the thread owns row g = lane / 4 (and the padding row g + 8)
     const int g_row = lane >> 2, quad = lane & 3;
     const float sc = a.kv.scale * kLog2e;
@@ -313,6 +322,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
         }
     }
 
+    DSTAMP(4);
     // ---- merge the 8 warps of the CTA ----
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -351,7 +361,9 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
         }
     }
     // ---- merge the CTAs of the cluster in its first CTA ----
+    DSTAMP(5);
     if (CS > 1) cluster.sync(); else __syncthreads();
+    DSTAMP(6);
     if (rank != 0) return;
     for (int i = tid; i < G * (D / 2); i += kThreads) {
         const int r = i / (D / 2), dp = i - r * (D / 2);
@@ -376,6 +388,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
         *(reinterpret_cast<float2*>(a.out + row * D) + dp) = make_float2(o0 * inv, o1 * inv);
         if (a.lse && dp == 0) a.lse[row] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.69314718055994530942f : -INFINITY;
     }
+    DSTAMP(7);
 }
 
 int pick_cluster(const KvView& kv, int n_keys_max)
