@@ -25,6 +25,13 @@ if ROOT not in sys.path:
 METRIC = "us_per_spec_step"
 UNIT = "us"
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/, for the per-layer launches of the headline workload.  A launch
+# that folds L layers moves L times as much (traffic grows in proportion to the keys streamed).
+NCU_TRAFFIC = {
+    "cfg2_8b_32k": {"verify": 134.39e6 + 3.77e6, "draft": 8.50e6},
+}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -48,7 +55,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -278,9 +285,17 @@ def run_gpu(args):
             "frac_of_8TBs": achieved / 8000.0,
             "bytes_per_launch": verify_bytes, "us_per_launch": verify_us,
             "traffic": None,
+            "share_of_step_time": phase_ms[0] / step_ms,
+            "share_of_step_bytes": verify_bytes * v_launches / (verify_bytes * v_launches + draft_bytes),
         },
-        "draft_roofline": {"achieved": draft_gbs, "frac": draft_gbs / peak if draft_gbs else None,
-                           "bytes_per_step": draft_bytes, "unit": "GB/s"},
+        "draft_roofline": {
+            "kernel": "sparse draft attention (one launch per layer and drafting step; latency-bound "
+                      "at batch 1: 8.4 MB per launch)",
+            "bound": "hbm", "achieved": draft_gbs, "peak": peak, "unit": "GB/s",
+            "frac": draft_gbs / peak if draft_gbs else None, "bytes_per_step": draft_bytes,
+            "us_per_launch": phase_ms[2] * 1e3 / max(1, counts[2]), "traffic": None,
+            "share_of_step_time": phase_ms[2] / step_ms,
+        },
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{cpu_layers} of {L} layers, time scaled x{L / cpu_layers:g}"},
         "e2e": {"value": e2e_ms * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -291,12 +306,11 @@ def run_gpu(args):
         "launches_per_step": {"verify": counts[0], "select": counts[1], "draft": counts[2]},
         "clocks": clocks,
     }
-    traffic_path = os.path.join(ROOT, "profiles", "verify_traffic.json")
-    if os.path.exists(traffic_path):
-        with open(traffic_path) as f:
-            t = json.load(f)
-        if t.get("config") == cfg.name:
-            line["roofline"]["traffic"] = t.get("dram_bytes_per_launch")
+    t = NCU_TRAFFIC.get(cfg.name)
+    if t and cfg.n_layers == pick_config(args.config).n_layers:
+        fold = L if args.fold_layers else 1
+        line["roofline"]["traffic"] = t["verify"] * fold
+        line["draft_roofline"]["traffic"] = t["draft"] * fold
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -305,7 +319,7 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="cfg2_8b_32k")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
