@@ -22,6 +22,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+K3 = 8  # speculation length of the third workload (--k3)
 METRIC = "us_per_spec_step"
 UNIT = "us"
 
@@ -97,7 +98,7 @@ def pick_config(name: str, layers: int = 0):
 
     from paper_2607_27735_b200 import inputs
 
-    cfgs = inputs.baseline_configs()
+    cfgs = inputs.baseline_configs(K3)
     if name not in cfgs:
         raise SystemExit(f"unknown config {name}; choose from {list(cfgs)}")
     cfg = cfgs[name]
@@ -266,7 +267,10 @@ def run_gpu(args):
     draft_gbs = draft_bytes / (phase_ms[2] * 1e-3) / 1e9 if phase_ms[2] > 0 else None
 
     cpu_layers = min(2, L)
-    cpu_dt, cores = oracle_step_seconds(cfg, cpu_layers)
+    if args.no_cpu_baseline:
+        cpu_dt, cores = float("nan"), 0
+    else:
+        cpu_dt, cores = oracle_step_seconds(cfg, cpu_layers)
     cpu_us = cpu_dt * (L / cpu_layers) * 1e6
 
     line = {
@@ -325,9 +329,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0,
                     help="use only this many layers of the config (small captures under ncu)")
+    ap.add_argument("--k3", type=int, default=8,
+                    help="speculation length k of cfg3_8b_128k (its sweep is k in 1, 2, 4, 8, 16)")
+    ap.add_argument("--no-cpu-baseline", action="store_true",
+                    help="skip the oracle timing (sweeps over the other workloads)")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()
+    global K3
+    K3 = args.k3
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -1,21 +1,25 @@
 // Sparse draft attention of Eq. 5: one query per sequence attends the recalled rows
 // Gather(K, I), Gather(V, I) plus the dense tail of tokens drafted this round.  The gather is
-// fused: one bulk asynchronous copy (cp.async.bulk, completion on an mbarrier) per indexed
-// 2*D-byte row pulls K and V straight from the dense cache into shared memory (two 144-key
-// tiles in flight per CTA); nothing gathered is written back to global memory.
+// fused: 16-byte asynchronous copies (cp.async) pull every indexed K and V row straight from the
+// dense cache into shared memory; nothing gathered is written back to global memory.
 //
 // The call is latency-bound (a few thousand recalled keys per head), so the kernel is built to
-// be short rather than wide:
-//   - every warp is an independent flash-decoding worker on 16 keys of each tile: q K^T and
-//     P V run on the tensor cores (mma.sync m16n8k16, the G <= 8 query rows of the GQA group
-//     padded to 16; P split into bf16 hi + lo parts), its running (max, sum, O) stay in
-//     registers, and no block-wide barrier is needed inside a tile;
-//   - the warps of a CTA are merged once through shared memory, the CTAs of a problem (a
-//     thread-block cluster that splits the key list) once through distributed shared memory:
-//     each deposits its partial in the first CTA of the cluster, which merges them in rank
-//     order (deterministic) after one cluster barrier.
+// be short rather than wide.  A thread-block cluster splits the key list of one (sequence, KV
+// head); each CTA keeps its whole share (up to 288 keys) in shared memory and runs three short
+// phases on it, separated by two block barriers:
+//   1. scores: every warp takes 16-key chunks, S^T = K q^T on the tensor cores (mma.sync
+//      m16n8k16 with the keys as the M dimension and the G <= 8 query heads of the group as N),
+//      and publishes its running maximum;
+//   2. probabilities: with the CTA-wide maximum known, P = 2^(S - max) is written once to
+//      shared memory as bf16 hi + lo parts;
+//   3. values: each warp owns a 16-wide slice of the head dimension and accumulates
+//      O^T = V^T P^T over all keys of the share, so no merge between warps is needed.
+// The CTAs of the cluster deposit (max, sum, O) in the first CTA through distributed shared
+// memory; it merges them in rank order (deterministic) after one cluster barrier.
 // One launch per call, no global scratch, no second kernel.
 #include <cooperative_groups.h>
+#include <cstdio>
+#include <cstdlib>
 
 #include "spec_common.cuh"
 
@@ -25,53 +29,36 @@ namespace spec {
 
 namespace {
 
-constexpr int kTK = 144;       // keys per tile: nine 16-key chunks dealt to the 8 warps
-constexpr int kStages = 2;     // two tiles (288 keys) can be in flight per CTA
+constexpr int kCap = 304;      // K rows (and V rows) resident per CTA
+constexpr int kRound = 144;    // keys per round when a share exceeds kCap (two buffers of kRound)
 constexpr int kThreads = 256;
-constexpr int kMaxGroup = 8;   // query heads per KV head
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxCluster = 8;  // portable cluster size (16 was measured slower: one cluster per GPC)
-constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // bound of the copy wait: about a second
+constexpr float kNegBig = -1.0e30f;  // "minus infinity" that stays finite under subtraction
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+// 16 bytes global -> shared; src_bytes = 0 writes zeros instead (masked rows)
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uint32_t src_bytes)
 {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr(smem_dst)), "l"(gsrc), "r"(src_bytes)
+                 : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// one row of the cache -> shared memory (16-byte aligned on both sides, size a multiple of 16)
-__device__ __forceinline__ void bulk_copy_row(void* smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(smem_dst)), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p)
 {
-    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr(p)));
 }
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* p)
 {
-    const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr(p)));
 }
 // D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
@@ -86,28 +73,34 @@ __device__ __forceinline__ float ex2f(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+__device__ __forceinline__ float group_max(float x)  // over the 8 lanes that share lane % 4
 {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
+    x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 4));
+    x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 8));
+    return fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 16));
+}
+__device__ __forceinline__ float group_sum(float x)
+{
+    x += __shfl_xor_sync(0xffffffffu, x, 4);
+    x += __shfl_xor_sync(0xffffffffu, x, 8);
+    return x + __shfl_xor_sync(0xffffffffu, x, 16);
 }
 
 template <int D>
 struct SmemLayout {
-    static constexpr int PITCH = D + 8;  // bf16 elements per shared row: 16 B of padding spreads the banks
-    static constexpr int kv_tile = kTK * PITCH * 2;  // bytes of one K (or V) tile
+    static constexpr int PITCH = D + 8;   // bf16 elements per K/V row: 16 B of padding spreads the banks
+    static constexpr int PP = kCap + 8;   // bf16 elements per row of P (one row per query head)
+    static constexpr int kv_bytes = kCap * PITCH * 2;
     static constexpr int off_k = 0;
-    static constexpr int off_v = kStages * kv_tile;
-    static constexpr int off_q = 2 * kStages * kv_tile;              // bf16 [16][PITCH], rows >= G zero
-    static constexpr int off_pos = off_q + 16 * PITCH * 2;           // int [kStages][kTK]
-    static constexpr int off_bar = off_pos + kStages * kTK * 4;      // mbarrier [kStages]
-    static constexpr int off_wml = off_bar + 64;                     // float2 [8 warps][kMaxGroup]
-    static constexpr int off_wo = off_k;  // float [8 warps][kMaxGroup][D]: reuses the K tiles once the loop is over
-    static constexpr int off_comb = off_wml + 8 * kMaxGroup * 8;     // float [kMaxCluster][kMaxGroup][D + 2]
+    static constexpr int off_v = kv_bytes;
+    static constexpr int off_ph = 2 * kv_bytes;                      // bf16 [kMaxGroup][PP], hi parts
+    static constexpr int off_pl = off_ph + kMaxGroup * PP * 2;       // bf16 [kMaxGroup][PP], lo parts
+    static constexpr int off_pos = off_pl + kMaxGroup * PP * 2;      // int [kCap]
+    static constexpr int off_wmax = off_pos + kCap * 4;              // float [kWarps][kMaxGroup]
+    static constexpr int off_wl = off_wmax + kWarps * kMaxGroup * 4;  // float [kWarps][kMaxGroup]
+    static constexpr int off_comb = off_wl + kWarps * kMaxGroup * 4;  // float [kMaxCluster][kMaxGroup * (D + 2)]
     static constexpr int total = off_comb + kMaxCluster * kMaxGroup * (D + 2) * 4;
-    static_assert(8 * kMaxGroup * D * 4 <= kStages * kv_tile, "warp partials must fit in the K tiles");
-    static_assert(PITCH * 2 % 16 == 0, "bulk copies need 16-byte aligned rows");
+    static_assert(PITCH * 2 % 16 == 0 && off_v % 16 == 0 && off_ph % 16 == 0, "16-byte aligned rows");
     static_assert(total <= 227 * 1024, "shared memory budget");
 };
 
@@ -116,21 +109,29 @@ __global__ void __launch_bounds__(kThreads)
 draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 {
     using SL = SmemLayout<D>;
-    constexpr int PITCH = SL::PITCH;
-    constexpr int CH = D / 8;    // 16-byte chunks per row
-    constexpr int NT = D / 8;    // 8-wide output tiles of the P V product
+    constexpr int PITCH = SL::PITCH, PP = SL::PP;
+    constexpr int CH = D / 8;               // 16-byte pieces per row
+    constexpr int RPP = kThreads / CH;      // rows covered by one pass of the block
+    constexpr int MAXI = (kCap + RPP - 1) / RPP;
+    constexpr int MAXJ = (kCap / 16 + kWarps - 1) / kWarps;  // 16-key chunks per warp and round
+    constexpr int NSL = D / 16;             // 16-wide slices of the head dimension
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) uint8_t smem[];
     __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_k);
     __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_v);
-    __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_q);
+    __nv_bfloat16* Ph = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_ph);
+    __nv_bfloat16* Pl = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_pl);
     int* keypos = reinterpret_cast<int*>(smem + SL::off_pos);
-    float2* wml = reinterpret_cast<float2*>(smem + SL::off_wml);
-    float* wo = reinterpret_cast<float*>(smem + SL::off_wo);
+    float* wmax = reinterpret_cast<float*>(smem + SL::off_wmax);
+    float* wl = reinterpret_cast<float*>(smem + SL::off_wl);
     float* comb = reinterpret_cast<float*>(smem + SL::off_comb);
 
 #ifdef SPEC_TRACE
-#define DSTAMP(i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) reinterpret_cast<long long*>(status)[8 + (i)] = clock64(); } while (0)
+#define DSTAMP(i) do { if (threadIdx.x == 0) { \
+        const size_t blk_ = ((size_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x; \
+        if (a.workspace_bytes >= 256 + (blk_ + 1) * 128) { \
+            unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); \
+            reinterpret_cast<unsigned long long*>(status)[32 + blk_ * 16 + (i)] = t_; } } } while (0)
 #else
 #define DSTAMP(i) do { } while (0)
 #endif
@@ -143,244 +144,309 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = lane >> 2, quad = lane & 3;
 
     // Programmatic dependent launch: the next kernel in the stream may start its own prologue
     // (index loads, gather of recalled rows) while this one is still computing.  Everything this
-    // kernel reads before griddep_wait() below is immutable during a drafting round (indices,
+    // kernel reads before griddepcontrol.wait below is immutable during a drafting round (indices,
     // lengths, recalled rows of the dense cache); Q, the dense tail and the outputs come after.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    bool dep_waited = false;
-    auto griddep_wait = [&]() {
-        if (!dep_waited) {
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            dep_waited = true;
-        }
-    };
-    const uint32_t bar0 = smem_addr(smem + SL::off_bar);
-    if (tid == 0) {
-        for (int i = 0; i < kStages; ++i) mbar_init(bar0 + 8 * i, kTK);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
+
     const int32_t* idx = a.indices + prob * a.k_total;
-    // the index of this thread's row in the first tile is fetched before the list length is
-    // known (the tail of the array holds -1 padding, never read past k_total)
-    const int per_guess = ((a.k_total + a.max_tail + CS - 1) / CS + 15) & ~15;
-    int idx_pre = -1;
-    if (tid < kTK && rank * per_guess + tid < a.k_total) idx_pre = __ldg(idx + rank * per_guess + tid);
-    const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
-    const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
-    const int n_tail = min(max(cl - ts, 0), a.max_tail);
-    const int n = n_rec + n_tail;
     // contiguous shares in multiples of the 16-key chunk; the share size depends only on host-side
     // bounds, so every CTA of the cluster agrees on it without exchanging anything
-    const int per = per_guess;
-    const int k0 = min(n, rank * per);
-    const int k1 = min(n, k0 + per);
-    const int n_tiles = (k1 - k0 + kTK - 1) / kTK;
-    __syncthreads();  // barriers initialised
+    const int per = ((a.k_total + a.max_tail + CS - 1) / CS + 15) & ~15;
+    const int RK = per <= kCap ? per : kRound;  // keys per round
+    const int NB = per <= kCap ? 1 : 2;          // buffers of RK rows
+    const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
+    const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
 
-    // one thread per row: position, then one bulk copy each for the K row and the V row; every
-    // copy of the tile is in flight before anything waits
-    auto issue_tile = [&](int tile) {
-        const int buf = tile % kStages;
-        const int base = k0 + tile * kTK;
-        const int nk = min(kTK, k1 - base);
-        if (base + nk > n_rec) griddep_wait();  // the tile reaches into the tail drafted this round
-        if (tid >= kTK) return;
-        const uint32_t bar = bar0 + 8 * buf;
-        int pos = -1;
-        if (tid < nk) {
-            const int e = base + tid;
-            pos = e < n_rec ? (tile == 0 ? idx_pre : __ldg(idx + e)) : ts + (e - n_rec);
-            if (pos < 0 || pos >= cl) {
+    // Gather of round r into its buffer: CH threads per row, one 16-byte piece of the K row and
+    // one of the V row each.  part 0 = recalled rows and the masked padding of the last chunk
+    // (readable before the dependency wait), 1 = rows of the dense tail, 2 = both.
+    const int slot = tid / CH, piece = tid % CH;
+    const __nv_bfloat16* kbase = a.kv.k + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
+    const __nv_bfloat16* vbase = a.kv.v + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
+    const int32_t* ptab = a.kv.page_table ? a.kv.page_table + (int64_t)b * a.kv.max_pages : nullptr;
+    auto issue_rows = [&](int r, int part, int k0, int k1) {
+        const int base = k0 + r * RK;
+        const int nk = min(RK, k1 - base);
+        const int nrows = (nk + 15) & ~15;
+        const int row0 = NB == 2 ? (r & 1) * kRound : 0;
+        int posv[MAXI];
+#pragma unroll
+        for (int i = 0; i < MAXI; ++i) {  // every index load is in flight before the first is used
+            const int e = base + i * RPP + slot;
+            posv[i] = (part != 1 && i * RPP + slot < RK && e < a.k_total) ? __ldg(idx + e) : -1;
+        }
+        // row offsets next (all page-table loads in flight together), the copies last: the address
+        // arithmetic of different rows overlaps instead of forming one long dependent chain
+        int64_t offv[MAXI];  // -2: not this part's row, -1: masked row (zero fill)
+#pragma unroll
+        for (int i = 0; i < MAXI; ++i) {
+            const int lr = i * RPP + slot;
+            const int e = base + lr;
+            const bool valid = lr < nk;
+            const bool is_tail = valid && e >= n_rec;
+            offv[i] = -2;
+            if (lr >= nrows || (part == 0 ? is_tail : (part == 1 ? !is_tail : false))) continue;
+            int pos = is_tail ? ts + (e - n_rec) : posv[i];
+            if (!valid) pos = -1;
+            else if (pos < 0 || pos >= cl) {
                 set_status(status, SPEC_ERR_BAD_INDEX);
                 pos = -1;
             }
-        }
-        keypos[buf * kTK + tid] = pos;
-        __nv_bfloat16* kr = Ks + (buf * kTK + tid) * PITCH;
-        __nv_bfloat16* vr = Vs + (buf * kTK + tid) * PITCH;
-        if (pos >= 0) {
-            const int64_t off = kv_row_offset(a.kv, layer, b, pos, h);
-            mbar_arrive_expect_tx(bar, 2 * D * 2);
-            bulk_copy_row(kr, a.kv.k + off, D * 2, bar);
-            bulk_copy_row(vr, a.kv.v + off, D * 2, bar);
-        } else {  // masked rows must still be finite: they meet P = 0 in the P V product
-#pragma unroll
-            for (int ch = 0; ch < CH; ++ch) {
-                *reinterpret_cast<uint4*>(kr + ch * 8) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(vr + ch * 8) = make_uint4(0, 0, 0, 0);
+            if (piece == 0) keypos[row0 + lr] = pos;
+            offv[i] = -1;
+            if (pos >= 0) {
+                const int page = page_of(a.kv, pos);
+                const int slot_in = pos - page * a.kv.page_size;
+                const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
+                offv[i] = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // a later bulk copy reuses the row
-            mbar_arrive(bar);
+        }
+#pragma unroll
+        for (int i = 0; i < MAXI; ++i) {
+            if (offv[i] == -2) continue;
+            const int lr = i * RPP + slot;
+            // masked rows are zero-filled: they meet P = 0 in the P V product and must be finite
+            const int64_t off = offv[i] >= 0 ? offv[i] : 0;
+            const uint32_t nbytes = offv[i] >= 0 ? 16u : 0u;
+            cp_async16(Ks + (row0 + lr) * PITCH + piece * 8, kbase + off, nbytes);
+            cp_async16(Vs + (row0 + lr) * PITCH + piece * 8, vbase + off, nbytes);
         }
     };
 
-    int issued = 0;
-    for (; issued < min(n_tiles, kStages); ++issued) issue_tile(issued);
-
+    // the share is known once the list length is; recalled rows never depend on the previous kernel
+    const int n_tail = min(max(cl - ts, 0), a.max_tail);
+    const int n = n_rec + n_tail;
+    const int k0 = min(n, rank * per);
+    const int k1 = min(n, k0 + per);
+    const int n_rounds = (k1 - k0 + RK - 1) / RK;
+    for (int r = 0; r < min(n_rounds, NB); ++r) issue_rows(r, 0, k0, k1);
+    cp_async_commit();
     DSTAMP(1);
-    griddep_wait();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
-    // Q of the group -> bf16 [16][PITCH] in shared memory (rows >= G zero), then A fragments
-    for (int i = tid; i < 16 * CH; i += kThreads) {
-        const int g = i / CH, ch = i - g * CH;
-        uint4 val = make_uint4(0, 0, 0, 0);
-        if (g < G) {
-            const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + g;
-            val = __ldg(reinterpret_cast<const uint4*>(a.q + row * D) + ch);
+    for (int r = 0; r < min(n_rounds, NB); ++r)
+        if (k0 + r * RK + RK > n_rec) issue_rows(r, 1, k0, k1);
+    cp_async_commit();
+
+    // B fragments of q^T (d x g) straight from global memory: the thread holds q[g = grp] at
+    // d = 16 ks + 2 quad + {0, 1} and + {8, 9}; heads beyond the group are zero
+    uint32_t qb[D / 16][2];
+    {
+        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + grp;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + row * D);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            qb[ks][0] = grp < G ? __ldg(qrow + ks * 8 + quad) : 0u;
+            qb[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
         }
-        *reinterpret_cast<uint4*>(Qs + g * PITCH + ch * 8) = val;
     }
+    cp_async_wait<0>();
     __syncthreads();
-    uint32_t qa[D / 16][4];
-#pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks)
-        ldmatrix_x4(qa[ks], Qs + ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + ks * 16 + (lane >> 4) * 8);
-
     DSTAMP(3);
-    // per-warp flash-decoding state: the thread owns row g = lane / 4 (and the padding row g + 8)
-    const int g_row = lane >> 2, quad = lane & 3;
-    const float sc = a.kv.scale * kLog2e;
-    float m_run = -INFINITY, l_run = 0.f;
-    float o[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
 
-    for (int tile = 0; tile < n_tiles; ++tile) {
-        const int buf = tile % kStages;
-        {  // the tile's rows have landed (bounded wait: a stall ends in a status code)
-            const uint32_t bar = bar0 + 8 * buf, parity = (tile / kStages) & 1;
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar, parity)) {
-                if (clock64() - t0 > kTimeoutCycles) {
-                    set_status(status, SPEC_ERR_TIMEOUT);
-                    break;
+    // running state of the share; the thread tracks heads g = 2 quad and 2 quad + 1 (every thread
+    // of the CTA computes the same values for them from shared memory)
+    const float sc = a.kv.scale * kLog2e;
+    float M0 = kNegBig, M1 = kNegBig, L0 = 0.f, L1 = 0.f;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.f;
+
+    for (int r = 0; r < n_rounds; ++r) {
+        if (r > 0) {  // all but the newest group (the round after this one) have landed
+            cp_async_wait<1>();
+            __syncthreads();
+        }
+        const int row0 = NB == 2 ? (r & 1) * kRound : 0;
+        const int nk = min(RK, k1 - (k0 + r * RK));
+        const int nch = (nk + 15) >> 4;
+        const int* kp = keypos + row0;
+
+        // ---- phase 1: S^T = K q^T for this warp's chunks (keys x heads), masked and scaled ----
+        float s[MAXJ][4];
+        float mx0 = kNegBig, mx1 = kNegBig;
+#pragma unroll
+        for (int j = 0; j < MAXJ; ++j) {
+            const int c = warp + kWarps * j;
+            s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+            if (c < nch) {
+                uint32_t kf[D / 16][4];  // all fragments of the chunk are requested before the first MMA
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    ldmatrix_x4(kf[ks], Ks + (row0 + c * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + ks * 16 +
+                                            (lane >> 4) * 8);
+                float s2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ks += 2) {  // two accumulation chains
+                    mma_bf16(s[j], kf[ks], qb[ks][0], qb[ks][1]);
+                    mma_bf16(s2, kf[ks + 1], qb[ks + 1][0], qb[ks + 1][1]);
+                }
+                const bool ka = kp[c * 16 + grp] >= 0, kb = kp[c * 16 + grp + 8] >= 0;
+                s[j][0] = ka ? (s[j][0] + s2[0]) * sc : kNegBig;
+                s[j][1] = ka ? (s[j][1] + s2[1]) * sc : kNegBig;
+                s[j][2] = kb ? (s[j][2] + s2[2]) * sc : kNegBig;
+                s[j][3] = kb ? (s[j][3] + s2[3]) * sc : kNegBig;
+                mx0 = fmaxf(mx0, fmaxf(s[j][0], s[j][2]));
+                mx1 = fmaxf(mx1, fmaxf(s[j][1], s[j][3]));
+            }
+        }
+        mx0 = group_max(mx0);
+        mx1 = group_max(mx1);
+        if (grp == 0) {
+            wmax[warp * kMaxGroup + 2 * quad] = mx0;
+            wmax[warp * kMaxGroup + 2 * quad + 1] = mx1;
+        }
+        __syncthreads();
+
+        // ---- phase 2: P = 2^(S - max) against the CTA-wide maximum, stored as bf16 hi + lo ----
+        float Mn0 = M0, Mn1 = M1;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            Mn0 = fmaxf(Mn0, wmax[w * kMaxGroup + 2 * quad]);
+            Mn1 = fmaxf(Mn1, wmax[w * kMaxGroup + 2 * quad + 1]);
+        }
+        const float alpha0 = ex2f(M0 - Mn0), alpha1 = ex2f(M1 - Mn1);
+        float ls0 = 0.f, ls1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < MAXJ; ++j) {
+            const int c = warp + kWarps * j;
+            if (c < nch) {
+                float p[4];
+                p[0] = s[j][0] > 0.5f * kNegBig ? ex2f(s[j][0] - Mn0) : 0.f;
+                p[1] = s[j][1] > 0.5f * kNegBig ? ex2f(s[j][1] - Mn1) : 0.f;
+                p[2] = s[j][2] > 0.5f * kNegBig ? ex2f(s[j][2] - Mn0) : 0.f;
+                p[3] = s[j][3] > 0.5f * kNegBig ? ex2f(s[j][3] - Mn1) : 0.f;
+                ls0 += p[0] + p[2];
+                ls1 += p[1] + p[3];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int g = 2 * quad + (e & 1), key = c * 16 + grp + (e >> 1) * 8;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(p[e]);
+                    Ph[g * PP + key] = hi;
+                    Pl[g * PP + key] = __float2bfloat16_rn(p[e] - __bfloat162float(hi));
                 }
             }
         }
-        const int nk = min(kTK, k1 - (k0 + tile * kTK));
-        for (int ck = warp * 16; ck < nk; ck += 8 * 16) {  // this warp's 16-key chunks of the tile
-            const int* kp = keypos + buf * kTK;
-            const __nv_bfloat16* kb = Ks + (buf * kTK + ck) * PITCH;
-            const __nv_bfloat16* vb = Vs + (buf * kTK + ck) * PITCH;
-            // ---- S = q K^T for 16 keys: two 8-key output tiles ----
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                uint32_t kf[4];
-                ldmatrix_x4(kf, kb + ((lane & 7) + (lane >> 4) * 8) * PITCH + ks * 16 + ((lane >> 3) & 1) * 8);
-                mma_bf16(s0, qa[ks], kf[0], kf[1]);
-                mma_bf16(s1, qa[ks], kf[2], kf[3]);
-            }
-            // the thread's keys: ck + 2*quad + {0,1} (tile 0) and + 8 (tile 1); rows g_row (real) only
-            const int kA = ck + 2 * quad;
-            float v0 = kp[kA] >= 0 ? s0[0] * sc : -INFINITY;
-            float v1 = kp[kA + 1] >= 0 ? s0[1] * sc : -INFINITY;
-            float v2 = kp[kA + 8] >= 0 ? s1[0] * sc : -INFINITY;
-            float v3 = kp[kA + 9] >= 0 ? s1[1] * sc : -INFINITY;
-            float mt = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
-            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
-            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
-            const float m_new = fmaxf(m_run, mt);
-            float alpha = 1.f, p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
-            if (m_new > -INFINITY) {
-                alpha = ex2f(m_run - m_new);
-                p0 = ex2f(v0 - m_new);
-                p1 = ex2f(v1 - m_new);
-                p2 = ex2f(v2 - m_new);
-                p3 = ex2f(v3 - m_new);
-            }
-            m_run = m_new;
-            l_run = l_run * alpha + (p0 + p1) + (p2 + p3);
-            // ---- P (hi + lo bf16) as the A operand of P V; padding rows (g_row + 8) are zero ----
-            uint32_t ph[4], pl[4];
-            ph[0] = pack_bf16x2(p0, p1);
-            ph[2] = pack_bf16x2(p2, p3);
-            ph[1] = ph[3] = 0u;
-            pl[0] = pack_bf16x2(p0 - __uint_as_float(ph[0] << 16), p1 - __uint_as_float(ph[0] & 0xffff0000u));
-            pl[2] = pack_bf16x2(p2 - __uint_as_float(ph[2] << 16), p3 - __uint_as_float(ph[2] & 0xffff0000u));
-            pl[1] = pl[3] = 0u;
-#pragma unroll
-            for (int nt = 0; nt < NT; nt += 2) {
-                uint32_t vf[4];
-                ldmatrix_x4_trans(vf, vb + ((lane & 7) + ((lane >> 3) & 1) * 8) * PITCH + nt * 8 + (lane >> 4) * 8);
-                o[nt][0] *= alpha;
-                o[nt][1] *= alpha;
-                o[nt + 1][0] *= alpha;
-                o[nt + 1][1] *= alpha;
-                mma_bf16(o[nt], ph, vf[0], vf[1]);
-                mma_bf16(o[nt], pl, vf[0], vf[1]);
-                mma_bf16(o[nt + 1], ph, vf[2], vf[3]);
-                mma_bf16(o[nt + 1], pl, vf[2], vf[3]);
-            }
+        ls0 = group_sum(ls0);
+        ls1 = group_sum(ls1);
+        if (grp == 0) {
+            wl[warp * kMaxGroup + 2 * quad] = ls0;
+            wl[warp * kMaxGroup + 2 * quad + 1] = ls1;
         }
-        __syncthreads();  // the tile's buffer is free again
-        if (issued < n_tiles) {
-            issue_tile(issued);
-            ++issued;
+        __syncthreads();
+        {
+            float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                t0 += wl[w * kMaxGroup + 2 * quad];
+                t1 += wl[w * kMaxGroup + 2 * quad + 1];
+            }
+            L0 = L0 * alpha0 + t0;
+            L1 = L1 * alpha1 + t1;
+            M0 = Mn0;
+            M1 = Mn1;
         }
-    }
 
-    DSTAMP(4);
-    // ---- merge the 8 warps of the CTA ----
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (g_row < G) {
-        if (quad == 0) wml[warp * kMaxGroup + g_row] = make_float2(m_run, l_run);
-        float* dst = wo + (warp * kMaxGroup + g_row) * D + 2 * quad;
+        // ---- phase 3: O^T += V^T P^T on this warp's 16-wide slice of the head dimension ----
+        if (warp < NSL) {
+            if (r > 0) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(o[nt][0], o[nt][1]);
+                for (int i = 0; i < 4; ++i) {
+                    acc[i][0] *= alpha0;
+                    acc[i][1] *= alpha1;
+                    acc[i][2] *= alpha0;
+                    acc[i][3] *= alpha1;
+                }
+            }
+            const __nv_bfloat16* vb = Vs + (row0 + (lane & 7) + ((lane >> 4) & 1) * 8) * PITCH + warp * 16 +
+                                      ((lane >> 3) & 1) * 8;
+            const uint32_t* ph = reinterpret_cast<const uint32_t*>(Ph + grp * PP) + quad;
+            const uint32_t* pl = reinterpret_cast<const uint32_t*>(Pl + grp * PP) + quad;
+            const bool real = grp < G;
+            for (int kc0 = 0; kc0 < nch; kc0 += 4) {  // four chunks requested, then eight MMAs on four chains
+                uint32_t vf[4][4], pb[4][4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int kc = kc0 + u;
+                    if (kc < nch) {
+                        ldmatrix_x4_trans(vf[u], vb + kc * 16 * PITCH);
+                        pb[u][0] = real ? ph[kc * 8] : 0u;
+                        pb[u][1] = real ? ph[kc * 8 + 4] : 0u;
+                        pb[u][2] = real ? pl[kc * 8] : 0u;
+                        pb[u][3] = real ? pl[kc * 8 + 4] : 0u;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (kc0 + u < nch) {
+                        mma_bf16(acc[(u & 1) * 2], vf[u], pb[u][0], pb[u][1]);
+                        mma_bf16(acc[(u & 1) * 2 + 1], vf[u], pb[u][2], pb[u][3]);
+                    }
+                }
+            }
+        }
+        if (NB == 2) {  // refill the buffer just consumed with the round after next
+            __syncthreads();
+            if (r + NB < n_rounds) issue_rows(r + NB, 2, k0, k1);
+            cp_async_commit();
+        }
     }
-    __syncthreads();
+    DSTAMP(4);
+
+    // ---- deposit (max, sum, O) of the share in the first CTA of the cluster ----
     float* comb0 = CS > 1 ? cluster.map_shared_rank(comb, 0) : comb;
     float* mine = comb0 + rank * (kMaxGroup * (D + 2));
-    for (int i = tid; i < G * (D / 2); i += kThreads) {
-        const int r = i / (D / 2), dp = i - r * (D / 2);
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) M = fmaxf(M, wml[w * kMaxGroup + r].x);
-        float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
-        if (M > -INFINITY) {
-#pragma unroll
-            for (int w = 0; w < 8; ++w) {
-                const float2 ml = wml[w * kMaxGroup + r];
-                if (ml.y > 0.f) {
-                    const float wgt = ex2f(ml.x - M);
-                    const float2 ov = *(reinterpret_cast<const float2*>(wo + (w * kMaxGroup + r) * D) + dp);
-                    Lsum += ml.y * wgt;
-                    o0 += ov.x * wgt;
-                    o1 += ov.y * wgt;
-                }
-            }
+    if (warp < NSL) {
+        const int d = warp * 16 + grp, g0 = 2 * quad;
+        if (g0 < G) {
+            mine[g0 * D + d] = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]);
+            mine[g0 * D + d + 8] = (acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]);
         }
-        *(reinterpret_cast<float2*>(mine + r * D) + dp) = make_float2(o0, o1);
-        if (dp == 0) {
-            mine[kMaxGroup * D + r] = M;
-            mine[kMaxGroup * D + kMaxGroup + r] = Lsum;
+        if (g0 + 1 < G) {
+            mine[(g0 + 1) * D + d] = (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]);
+            mine[(g0 + 1) * D + d + 8] = (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]);
         }
     }
-    // ---- merge the CTAs of the cluster in its first CTA ----
+    if (warp == 0 && grp == 0) {
+        mine[kMaxGroup * D + 2 * quad] = M0;
+        mine[kMaxGroup * D + 2 * quad + 1] = M1;
+        mine[kMaxGroup * D + kMaxGroup + 2 * quad] = L0;
+        mine[kMaxGroup * D + kMaxGroup + 2 * quad + 1] = L1;
+    }
     DSTAMP(5);
     if (CS > 1) cluster.sync(); else __syncthreads();
     DSTAMP(6);
     if (rank != 0) return;
+    // ---- merge the CTAs of the cluster, in rank order ----
     for (int i = tid; i < G * (D / 2); i += kThreads) {
         const int r = i / (D / 2), dp = i - r * (D / 2);
-        float M = -INFINITY;
-        for (int c = 0; c < CS; ++c) M = fmaxf(M, comb[c * (kMaxGroup * (D + 2)) + kMaxGroup * D + r]);
-        float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
-        if (M > -INFINITY) {
-            for (int c = 0; c < CS; ++c) {
+        float Mc[kMaxCluster], Lc[kMaxCluster];
+        float2 oc[kMaxCluster];
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) {  // every load is in flight before the first is used
+            if (c < CS) {
                 const float* pc = comb + c * (kMaxGroup * (D + 2));
-                const float lc = pc[kMaxGroup * D + kMaxGroup + r];
-                if (lc > 0.f) {
-                    const float wgt = ex2f(pc[kMaxGroup * D + r] - M);
-                    const float2 ov = *(reinterpret_cast<const float2*>(pc + r * D) + dp);
-                    Lsum += lc * wgt;
-                    o0 += ov.x * wgt;
-                    o1 += ov.y * wgt;
-                }
+                Mc[c] = pc[kMaxGroup * D + r];
+                Lc[c] = pc[kMaxGroup * D + kMaxGroup + r];
+                oc[c] = *(reinterpret_cast<const float2*>(pc + r * D) + dp);
+            }
+        }
+        float M = kNegBig;
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c)
+            if (c < CS) M = fmaxf(M, Mc[c]);
+        float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) {
+            if (c < CS && Lc[c] > 0.f) {
+                const float wgt = ex2f(Mc[c] - M);
+                Lsum += Lc[c] * wgt;
+                o0 += oc[c].x * wgt;
+                o1 += oc[c].y * wgt;
             }
         }
         const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + r;
@@ -393,9 +459,9 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 
 int pick_cluster(const KvView& kv, int n_keys_max)
 {
-    // enough CTAs to cover the SMs, at most about one tile of work each
+    // enough CTAs to cover the SMs, at most about one round of work each
     const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
-    const int tiles = n_keys_max > 0 ? (n_keys_max + kTK - 1) / kTK : 1;
+    const int tiles = n_keys_max > 0 ? (n_keys_max + kRound - 1) / kRound : 1;
     int cs = 1;
     while (cs < kMaxCluster && probs * cs < sm_count() && cs < tiles) cs *= 2;
     return cs;
@@ -415,6 +481,33 @@ int launch_d(const DraftArgs& a, int cs, cudaStream_t stream)
             cudaGetLastError();
         configured = true;
     }
+#ifdef SPEC_TRACE
+    {
+        static bool printed = false;
+        if (!printed) {
+            printed = true;
+            for (int c2 : {4, 5, 6, 7, 8}) {
+                for (size_t sm2 : {smem}) {
+                    cudaLaunchConfig_t q = {};
+                    q.gridDim = dim3(c2, 8, 4);
+                    q.blockDim = dim3(kThreads);
+                    q.dynamicSmemBytes = sm2;
+                    cudaLaunchAttribute at[1];
+                    at[0].id = cudaLaunchAttributeClusterDimension;
+                    at[0].val.clusterDim.x = c2;
+                    at[0].val.clusterDim.y = 1;
+                    at[0].val.clusterDim.z = 1;
+                    q.attrs = at;
+                    q.numAttrs = 1;
+                    int nclu = -1;
+                    cudaError_t e = cudaOccupancyMaxActiveClusters(&nclu, kern, &q);
+                    fprintf(stderr, "max active clusters: size %d smem %zu -> %d (%s)\n", c2, sm2, nclu, cudaGetErrorString(e));
+                }
+            }
+            cudaGetLastError();
+        }
+    }
+#endif
     for (; cs >= 1; cs /= 2) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
@@ -449,7 +542,10 @@ int draft_launch(const DraftArgs& a, cudaStream_t stream)
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     if (G > kMaxGroup) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.workspace_bytes < kStatusBytes) return SPEC_ERR_WORKSPACE_TOO_SMALL;
-    const int cs = pick_cluster(a.kv, a.k_total + a.max_tail);
+    int cs = pick_cluster(a.kv, a.k_total + a.max_tail);
+#ifdef SPEC_TRACE
+    if (const char* e = getenv("SPEC_DRAFT_CS")) cs = atoi(e);
+#endif
     if (a.kv.head_dim == 128) return launch_d<128>(a, cs, stream);
     if (a.kv.head_dim == 64) return launch_d<64>(a, cs, stream);
     return SPEC_ERR_UNSUPPORTED_SHAPE;

@@ -61,6 +61,7 @@ static int make_view(const spec_kv_t* kv, KvView* out)
     if (kv->n_pages < 0) return SPEC_ERR_INVALID_ARG;
     out->n_pages = kv->n_pages > 0 ? kv->n_pages : kv->batch * kv->max_pages;
     out->scale = kv->sm_scale > 0.f ? kv->sm_scale : 1.0f / std::sqrt((float)kv->head_dim);
+    set_page_divisor(out);
     return SPEC_OK;
 }
 

@@ -18,11 +18,35 @@ struct KvView {
     const int32_t* page_table;
     int32_t n_layers, page_size, max_pages, batch, n_q_heads, n_kv_heads, head_dim, n_pages;
     float scale;  // resolved softmax scale
+    // pos / page_size without a division: page = umulhi(pos, page_mul) >> page_sh for 0 <= pos < 2^31
+    // (page_mul = ceil(2^(31 + c) / page_size), page_sh = c - 1, c = ceil(log2 page_size));
+    // page_sh < 0 marks page_size == 1
+    uint32_t page_mul;
+    int32_t page_sh;
 };
+
+inline void set_page_divisor(KvView* kv)
+{
+    const uint32_t d = (uint32_t)kv->page_size;
+    if (d <= 1) {
+        kv->page_mul = 0;
+        kv->page_sh = -1;
+        return;
+    }
+    int c = 0;
+    while ((1ull << c) < d) ++c;
+    kv->page_mul = (uint32_t)(((1ull << (31 + c)) + d - 1) / d);
+    kv->page_sh = c - 1;
+}
+
+__device__ __forceinline__ int page_of(const KvView& kv, int pos)
+{
+    return kv.page_sh < 0 ? pos : (int)(__umulhi((uint32_t)pos, kv.page_mul) >> kv.page_sh);
+}
 
 __device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, int b, int pos, int h)
 {
-    const int page = pos / kv.page_size;
+    const int page = page_of(kv, pos);
     const int slot = pos - page * kv.page_size;
     const int64_t phys = kv.page_table ? (int64_t)__ldg(kv.page_table + (int64_t)b * kv.max_pages + page)
                                        : (int64_t)b * kv.max_pages + page;
