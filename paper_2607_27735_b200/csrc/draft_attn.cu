@@ -29,12 +29,12 @@ namespace spec {
 
 namespace {
 
-constexpr int kCap = 304;      // K rows (and V rows) resident per CTA
+constexpr int kCap = 352;      // most K rows (and V rows) resident per CTA
 constexpr int kRound = 144;    // keys per round when a share exceeds kCap (two buffers of kRound)
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxGroup = 8;    // query heads per KV head
-constexpr int kMaxCluster = 8;  // portable cluster size (16 was measured slower: one cluster per GPC)
+constexpr int kMaxCluster = 8;  // portable cluster size (a GPC cannot hold two clusters of 16)
 constexpr float kNegBig = -1.0e30f;  // "minus infinity" that stays finite under subtraction
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -86,30 +86,28 @@ __device__ __forceinline__ float group_sum(float x)
     return x + __shfl_xor_sync(0xffffffffu, x, 16);
 }
 
-template <int D>
-struct SmemLayout {
-    static constexpr int PITCH = D + 8;   // bf16 elements per K/V row: 16 B of padding spreads the banks
-    static constexpr int PP = kCap + 8;   // bf16 elements per row of P (one row per query head)
-    static constexpr int kv_bytes = kCap * PITCH * 2;
-    static constexpr int off_k = 0;
-    static constexpr int off_v = kv_bytes;
-    static constexpr int off_ph = 2 * kv_bytes;                      // bf16 [kMaxGroup][PP], hi parts
-    static constexpr int off_pl = off_ph + kMaxGroup * PP * 2;       // bf16 [kMaxGroup][PP], lo parts
-    static constexpr int off_pos = off_pl + kMaxGroup * PP * 2;      // int [kCap]
-    static constexpr int off_wmax = off_pos + kCap * 4;              // float [kWarps][kMaxGroup]
-    static constexpr int off_wl = off_wmax + kWarps * kMaxGroup * 4;  // float [kWarps][kMaxGroup]
-    static constexpr int off_comb = off_wl + kWarps * kMaxGroup * 4;  // float [kMaxCluster][kMaxGroup * (D + 2)]
-    static constexpr int total = off_comb + kMaxCluster * kMaxGroup * (D + 2) * 4;
-    static_assert(PITCH * 2 % 16 == 0 && off_v % 16 == 0 && off_ph % 16 == 0, "16-byte aligned rows");
-    static_assert(total <= 227 * 1024, "shared memory budget");
+// How a call is split: CTAs per cluster (one cluster per (layer, sequence, KV head)), keys per
+// CTA, keys per round, K rows resident per CTA.
+struct DraftShape {
+    int cs, per, rk, rows;
 };
+
+// Shared memory of one CTA, in this order (every block 16-byte aligned):
+//   K [rows][D + 8] bf16 | V [rows][D + 8] bf16 | P hi, P lo [8][rk + 8] bf16 each |
+//   key positions int [rows] | per-warp maxima, per-warp sums float [8 warps][8] each |
+//   deposit area float [cs][G * (D + 2)] (used in the first CTA of the cluster)
+// The 16 bytes of padding per K/V row spread the banks for ldmatrix.
+__host__ __device__ inline size_t draft_smem_bytes(int D, int G, const DraftShape& s)
+{
+    return (size_t)2 * s.rows * (D + 8) * 2 + (size_t)2 * kMaxGroup * (s.rk + 8) * 2 + (size_t)s.rows * 4 +
+           (size_t)2 * kWarps * kMaxGroup * 4 + (size_t)s.cs * G * (D + 2) * 4;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads)
-draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
+draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
 {
-    using SL = SmemLayout<D>;
-    constexpr int PITCH = SL::PITCH, PP = SL::PP;
+    constexpr int PITCH = D + 8;
     constexpr int CH = D / 8;               // 16-byte pieces per row
     constexpr int RPP = kThreads / CH;      // rows covered by one pass of the block
     constexpr int MAXI = (kCap + RPP - 1) / RPP;
@@ -117,14 +115,16 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     constexpr int NSL = D / 16;             // 16-wide slices of the head dimension
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) uint8_t smem[];
-    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_k);
-    __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_v);
-    __nv_bfloat16* Ph = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_ph);
-    __nv_bfloat16* Pl = reinterpret_cast<__nv_bfloat16*>(smem + SL::off_pl);
-    int* keypos = reinterpret_cast<int*>(smem + SL::off_pos);
-    float* wmax = reinterpret_cast<float*>(smem + SL::off_wmax);
-    float* wl = reinterpret_cast<float*>(smem + SL::off_wl);
-    float* comb = reinterpret_cast<float*>(smem + SL::off_comb);
+    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+    const int per = shp.per, RK = shp.rk, PP = RK + 8, PS = G * (D + 2);
+    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem);
+    __nv_bfloat16* Vs = Ks + shp.rows * PITCH;
+    __nv_bfloat16* Ph = Vs + shp.rows * PITCH;
+    __nv_bfloat16* Pl = Ph + kMaxGroup * PP;
+    int* keypos = reinterpret_cast<int*>(Pl + kMaxGroup * PP);
+    float* wmax = reinterpret_cast<float*>(keypos + shp.rows);
+    float* wl = wmax + kWarps * kMaxGroup;
+    float* comb = wl + kWarps * kMaxGroup;  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
 
 #ifdef SPEC_TRACE
 #define DSTAMP(i) do { if (threadIdx.x == 0) { \
@@ -139,7 +139,6 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     cg::cluster_group cluster = cg::this_cluster();
     const int CS = gridDim.x;              // the cluster spans the x dimension
     const int rank = blockIdx.x;
-    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     const int h = blockIdx.y;
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
@@ -155,20 +154,18 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     const int32_t* idx = a.indices + prob * a.k_total;
     // contiguous shares in multiples of the 16-key chunk; the share size depends only on host-side
     // bounds, so every CTA of the cluster agrees on it without exchanging anything
-    const int per = ((a.k_total + a.max_tail + CS - 1) / CS + 15) & ~15;
-    const int RK = per <= kCap ? per : kRound;  // keys per round
-    const int NB = per <= kCap ? 1 : 2;          // buffers of RK rows
+    const int NB = RK < per ? 2 : 1;  // buffers of RK rows (two when the share takes several rounds)
     const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
     const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
 
     // Gather of round r into its buffer: CH threads per row, one 16-byte piece of the K row and
-    // one of the V row each.  part 0 = recalled rows and the masked padding of the last chunk
-    // (readable before the dependency wait), 1 = rows of the dense tail, 2 = both.
+    // one of the V row each.  with_tail = false leaves out the rows of the dense tail (the rest
+    // can be read before the dependency wait); masked padding rows of the last chunk are zero-filled.
     const int slot = tid / CH, piece = tid % CH;
     const __nv_bfloat16* kbase = a.kv.k + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
     const __nv_bfloat16* vbase = a.kv.v + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
     const int32_t* ptab = a.kv.page_table ? a.kv.page_table + (int64_t)b * a.kv.max_pages : nullptr;
-    auto issue_rows = [&](int r, int part, int k0, int k1) {
+    auto issue_rows = [&](int r, bool with_tail, int k0, int k1) {
         const int base = k0 + r * RK;
         const int nk = min(RK, k1 - base);
         const int nrows = (nk + 15) & ~15;
@@ -177,11 +174,11 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 #pragma unroll
         for (int i = 0; i < MAXI; ++i) {  // every index load is in flight before the first is used
             const int e = base + i * RPP + slot;
-            posv[i] = (part != 1 && i * RPP + slot < RK && e < a.k_total) ? __ldg(idx + e) : -1;
+            posv[i] = (i * RPP + slot < RK && e < a.k_total) ? __ldg(idx + e) : -1;
         }
         // row offsets next (all page-table loads in flight together), the copies last: the address
         // arithmetic of different rows overlaps instead of forming one long dependent chain
-        int64_t offv[MAXI];  // -2: not this part's row, -1: masked row (zero fill)
+        int64_t offv[MAXI];  // -2: not issued here, -1: masked row (zero fill)
 #pragma unroll
         for (int i = 0; i < MAXI; ++i) {
             const int lr = i * RPP + slot;
@@ -189,7 +186,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
             const bool valid = lr < nk;
             const bool is_tail = valid && e >= n_rec;
             offv[i] = -2;
-            if (lr >= nrows || (part == 0 ? is_tail : (part == 1 ? !is_tail : false))) continue;
+            if (lr >= nrows || (is_tail && !with_tail)) continue;
             int pos = is_tail ? ts + (e - n_rec) : posv[i];
             if (!valid) pos = -1;
             else if (pos < 0 || pos >= cl) {
@@ -223,13 +220,34 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     const int k0 = min(n, rank * per);
     const int k1 = min(n, k0 + per);
     const int n_rounds = (k1 - k0 + RK - 1) / RK;
-    for (int r = 0; r < min(n_rounds, NB); ++r) issue_rows(r, 0, k0, k1);
+    for (int r = 0; r < min(n_rounds, NB); ++r) issue_rows(r, false, k0, k1);
     cp_async_commit();
     DSTAMP(1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
-    for (int r = 0; r < min(n_rounds, NB); ++r)
-        if (k0 + r * RK + RK > n_rec) issue_rows(r, 1, k0, k1);
+    {  // rows of the dense tail that fall into the rounds gathered above: at most max_tail, one short pass
+        const int e0 = max(n_rec, k0), e1 = min(k1, k0 + NB * RK);
+        for (int t = slot; t < e1 - e0; t += RPP) {
+            const int e = e0 + t, lr = e - k0;
+            const int r = lr / RK;
+            const int row = (NB == 2 ? (r & 1) * kRound : 0) + (lr - r * RK);
+            int pos = ts + (e - n_rec);
+            if (pos < 0 || pos >= cl) {
+                set_status(status, SPEC_ERR_BAD_INDEX);
+                pos = -1;
+            }
+            if (piece == 0) keypos[row] = pos;
+            int64_t off = 0;
+            if (pos >= 0) {
+                const int page = page_of(a.kv, pos);
+                const int slot_in = pos - page * a.kv.page_size;
+                const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
+                off = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
+            }
+            cp_async16(Ks + row * PITCH + piece * 8, kbase + off, pos >= 0 ? 16u : 0u);
+            cp_async16(Vs + row * PITCH + piece * 8, vbase + off, pos >= 0 ? 16u : 0u);
+        }
+    }
     cp_async_commit();
 
     // B fragments of q^T (d x g) straight from global memory: the thread holds q[g = grp] at
@@ -301,6 +319,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
             wmax[warp * kMaxGroup + 2 * quad + 1] = mx1;
         }
         __syncthreads();
+        if (r == 0) DSTAMP(8);
 
         // ---- phase 2: P = 2^(S - max) against the CTA-wide maximum, stored as bf16 hi + lo ----
         float Mn0 = M0, Mn1 = M1;
@@ -338,6 +357,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
             wl[warp * kMaxGroup + 2 * quad + 1] = ls1;
         }
         __syncthreads();
+        if (r == 0) DSTAMP(9);
         {
             float t0 = 0.f, t1 = 0.f;
 #pragma unroll
@@ -391,7 +411,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
         }
         if (NB == 2) {  // refill the buffer just consumed with the round after next
             __syncthreads();
-            if (r + NB < n_rounds) issue_rows(r + NB, 2, k0, k1);
+            if (r + NB < n_rounds) issue_rows(r + NB, true, k0, k1);
             cp_async_commit();
         }
     }
@@ -399,7 +419,7 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 
     // ---- deposit (max, sum, O) of the share in the first CTA of the cluster ----
     float* comb0 = CS > 1 ? cluster.map_shared_rank(comb, 0) : comb;
-    float* mine = comb0 + rank * (kMaxGroup * (D + 2));
+    float* mine = comb0 + rank * PS;
     if (warp < NSL) {
         const int d = warp * 16 + grp, g0 = 2 * quad;
         if (g0 < G) {
@@ -412,10 +432,14 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
         }
     }
     if (warp == 0 && grp == 0) {
-        mine[kMaxGroup * D + 2 * quad] = M0;
-        mine[kMaxGroup * D + 2 * quad + 1] = M1;
-        mine[kMaxGroup * D + kMaxGroup + 2 * quad] = L0;
-        mine[kMaxGroup * D + kMaxGroup + 2 * quad + 1] = L1;
+        if (2 * quad < G) {
+            mine[G * D + 2 * quad] = M0;
+            mine[G * D + G + 2 * quad] = L0;
+        }
+        if (2 * quad + 1 < G) {
+            mine[G * D + 2 * quad + 1] = M1;
+            mine[G * D + G + 2 * quad + 1] = L1;
+        }
     }
     DSTAMP(5);
     if (CS > 1) cluster.sync(); else __syncthreads();
@@ -429,9 +453,9 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
 #pragma unroll
         for (int c = 0; c < kMaxCluster; ++c) {  // every load is in flight before the first is used
             if (c < CS) {
-                const float* pc = comb + c * (kMaxGroup * (D + 2));
-                Mc[c] = pc[kMaxGroup * D + r];
-                Lc[c] = pc[kMaxGroup * D + kMaxGroup + r];
+                const float* pc = comb + c * PS;
+                Mc[c] = pc[G * D + r];
+                Lc[c] = pc[G * D + G + r];
                 oc[c] = *(reinterpret_cast<const float2*>(pc + r * D) + dp);
             }
         }
@@ -457,80 +481,118 @@ draft_cluster_kernel(DraftArgs a, int* __restrict__ status)
     DSTAMP(7);
 }
 
-int pick_cluster(const KvView& kv, int n_keys_max)
+constexpr size_t kSmemLimit = 227 * 1024;
+
+DraftShape make_shape(int D, int G, int keys, int cs)
 {
-    // enough CTAs to cover the SMs, at most about one round of work each
-    const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
-    const int tiles = n_keys_max > 0 ? (n_keys_max + kRound - 1) / kRound : 1;
-    int cs = 1;
-    while (cs < kMaxCluster && probs * cs < sm_count() && cs < tiles) cs *= 2;
-    return cs;
+    DraftShape s;
+    s.cs = cs;
+    s.per = ((keys + cs - 1) / cs + 15) & ~15;
+    s.rk = s.rows = s.per;  // the whole share resident: one round
+    if (s.per > kCap || draft_smem_bytes(D, G, s) > kSmemLimit) {
+        s.rk = kRound;  // several rounds through two buffers
+        s.rows = 2 * kRound;
+    }
+    return s;
+}
+
+// Clusters of `cs` CTAs with `smem` bytes each that fit on the GPU at once (cached per size).
+template <int D>
+int max_active_clusters(int cs, size_t smem)
+{
+    static int cached[kMaxCluster + 1];
+    static size_t cached_smem[kMaxCluster + 1];
+    if (cached_smem[cs] == smem && cached[cs] > 0) return cached[cs];
+    cudaLaunchConfig_t q = {};
+    q.gridDim = dim3(cs, 1, sm_count());
+    q.blockDim = dim3(kThreads);
+    q.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = cs;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    q.attrs = at;
+    q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, draft_cluster_kernel<D>, &q) != cudaSuccess) {
+        cudaGetLastError();
+        n = sm_count() / cs;
+    }
+    cached[cs] = n;
+    cached_smem[cs] = smem;
+    return n;
 }
 
 template <int D>
-int launch_d(const DraftArgs& a, int cs, cudaStream_t stream)
+bool set_smem_limit(size_t smem)
 {
-    auto kern = draft_cluster_kernel<D>;
-    const size_t smem = SmemLayout<D>::total;
-    static bool configured = false;  // per template instance
-    if (!configured) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return SPEC_ERR_CUDA;
-        // clusters of 16 are outside the portable range: opt in (a refusal just keeps them at 8)
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
-            cudaGetLastError();
-        configured = true;
+    static size_t configured = 0;  // per template instance: largest size opted in so far
+    if (smem <= configured) return true;
+    if (cudaFuncSetAttribute(draft_cluster_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return false;
+    configured = smem;
+    return true;
+}
+
+// Split of a call.  The cluster grows (1, 2, 4, 8 CTAs) until the CTAs cover the SMs or a CTA
+// would get less than about one round of keys.  A call that fits the GPU in one wave wants the
+// next call's gather to run beside it (programmatic dependent launch), which needs both calls'
+// clusters resident together; a GPC holds at most two clusters of eight and not every GPC
+// does, so where 2 x clusters-per-call does not fit, clusters of six (which pack better) are
+// used if the larger share still fits shared memory in one round.
+template <int D>
+bool draft_plan(const KvView& kv, int n_keys_max, DraftShape* out)
+{
+    const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
+    const int G = kv.n_q_heads / kv.n_kv_heads;
+    const int keys = n_keys_max > 0 ? n_keys_max : 1;
+    const int rounds = (keys + kRound - 1) / kRound;
+    int cs = 1;
+    while (cs < kMaxCluster && probs * cs < sm_count() && cs < rounds) cs *= 2;
+    DraftShape s = make_shape(D, G, keys, cs);
+    if (!set_smem_limit<D>(kSmemLimit)) return false;
+    if (cs == kMaxCluster && probs * cs <= sm_count() &&
+        2 * probs > max_active_clusters<D>(cs, draft_smem_bytes(D, G, s))) {
+        const DraftShape t = make_shape(D, G, keys, 6);
+        if (t.rk == t.per && 2 * probs <= max_active_clusters<D>(6, draft_smem_bytes(D, G, t))) s = t;
     }
+    *out = s;
+    return true;
+}
+
+template <int D>
+int launch_d(const DraftArgs& a, cudaStream_t stream)
+{
+    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+    DraftShape shp;
+    if (!draft_plan<D>(a.kv, a.k_total + a.max_tail, &shp)) return SPEC_ERR_CUDA;
 #ifdef SPEC_TRACE
-    {
-        static bool printed = false;
-        if (!printed) {
-            printed = true;
-            for (int c2 : {4, 5, 6, 7, 8}) {
-                for (size_t sm2 : {smem}) {
-                    cudaLaunchConfig_t q = {};
-                    q.gridDim = dim3(c2, 8, 4);
-                    q.blockDim = dim3(kThreads);
-                    q.dynamicSmemBytes = sm2;
-                    cudaLaunchAttribute at[1];
-                    at[0].id = cudaLaunchAttributeClusterDimension;
-                    at[0].val.clusterDim.x = c2;
-                    at[0].val.clusterDim.y = 1;
-                    at[0].val.clusterDim.z = 1;
-                    q.attrs = at;
-                    q.numAttrs = 1;
-                    int nclu = -1;
-                    cudaError_t e = cudaOccupancyMaxActiveClusters(&nclu, kern, &q);
-                    fprintf(stderr, "max active clusters: size %d smem %zu -> %d (%s)\n", c2, sm2, nclu, cudaGetErrorString(e));
-                }
-            }
-            cudaGetLastError();
-        }
-    }
+    if (const char* e = getenv("SPEC_DRAFT_CS")) shp = make_shape(D, G, a.k_total + a.max_tail, atoi(e));
 #endif
-    for (; cs >= 1; cs /= 2) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
-        cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = cs;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the kernel's prologue
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        if (cudaLaunchKernelEx(&cfg, kern, a, static_cast<int*>(a.workspace)) == cudaSuccess) {
-            count_launch(1);
-            return SPEC_OK;
-        }
+    const size_t smem = draft_smem_bytes(D, G, shp);
+    if (smem > kSmemLimit) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(shp.cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = shp.cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the kernel's prologue
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, draft_cluster_kernel<D>, a, shp, static_cast<int*>(a.workspace)) != cudaSuccess) {
         cudaGetLastError();
-        if (cs <= 8) break;  // a portable size that still fails is a real error
+        return SPEC_ERR_CUDA;
     }
-    return SPEC_ERR_CUDA;
+    count_launch(1);
+    return SPEC_OK;
 }
 
 }  // namespace
@@ -542,12 +604,8 @@ int draft_launch(const DraftArgs& a, cudaStream_t stream)
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     if (G > kMaxGroup) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.workspace_bytes < kStatusBytes) return SPEC_ERR_WORKSPACE_TOO_SMALL;
-    int cs = pick_cluster(a.kv, a.k_total + a.max_tail);
-#ifdef SPEC_TRACE
-    if (const char* e = getenv("SPEC_DRAFT_CS")) cs = atoi(e);
-#endif
-    if (a.kv.head_dim == 128) return launch_d<128>(a, cs, stream);
-    if (a.kv.head_dim == 64) return launch_d<64>(a, cs, stream);
+    if (a.kv.head_dim == 128) return launch_d<128>(a, stream);
+    if (a.kv.head_dim == 64) return launch_d<64>(a, stream);
     return SPEC_ERR_UNSUPPORTED_SHAPE;
 }
 
