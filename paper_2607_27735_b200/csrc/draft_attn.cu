@@ -31,7 +31,7 @@ namespace {
 
 constexpr int kCap = 352;      // most K rows (and V rows) resident per CTA
 constexpr int kRound = 144;    // keys per round when a share exceeds kCap (two buffers of kRound)
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;  // four warps per scheduler: the phases are dependent chains that need interleaving
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxCluster = 8;  // portable cluster size (a GPC cannot hold two clusters of 16)
@@ -43,6 +43,11 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uin
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_addr(smem_dst)), "l"(gsrc), "r"(src_bytes)
                  : "memory");
+}
+// asks L2 for `bytes` (a multiple of 16, from a 16-byte aligned address); nothing waits for it
+__device__ __forceinline__ void prefetch_l2(const void* gsrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -90,17 +95,19 @@ __device__ __forceinline__ float group_sum(float x)
 // CTA, keys per round, K rows resident per CTA.
 struct DraftShape {
     int cs, per, rk, rows;
+    int packed;  // G <= 4: [P hi | P lo] share the eight MMA columns in phase 3
 };
 
 // Shared memory of one CTA, in this order (every block 16-byte aligned):
 //   K [rows][D + 8] bf16 | V [rows][D + 8] bf16 | P hi, P lo [8][rk + 8] bf16 each |
-//   key positions int [rows] | per-warp maxima, per-warp sums float [8 warps][8] each |
+//   row offsets int64 [rows] | key positions int [rows] | per-warp maxima, per-warp sums float [8 warps][8] each |
+//   partial O of the warps that share a head-dim slice float [16 - D/16 warps][32 lanes][4] |
 //   deposit area float [cs][G * (D + 2)] (used in the first CTA of the cluster)
 // The 16 bytes of padding per K/V row spread the banks for ldmatrix.
 __host__ __device__ inline size_t draft_smem_bytes(int D, int G, const DraftShape& s)
 {
-    return (size_t)2 * s.rows * (D + 8) * 2 + (size_t)2 * kMaxGroup * (s.rk + 8) * 2 + (size_t)s.rows * 4 +
-           (size_t)2 * kWarps * kMaxGroup * 4 + (size_t)s.cs * G * (D + 2) * 4;
+    return (size_t)2 * s.rows * (D + 8) * 2 + (size_t)2 * kMaxGroup * (s.rk + 8) * 2 + (size_t)s.rows * 12 +
+           (size_t)2 * kWarps * kMaxGroup * 4 + (size_t)(kWarps - D / 16) * 512 + (size_t)s.cs * G * (D + 2) * 4;
 }
 
 template <int D>
@@ -110,9 +117,9 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     constexpr int PITCH = D + 8;
     constexpr int CH = D / 8;               // 16-byte pieces per row
     constexpr int RPP = kThreads / CH;      // rows covered by one pass of the block
-    constexpr int MAXI = (kCap + RPP - 1) / RPP;
     constexpr int MAXJ = (kCap / 16 + kWarps - 1) / kWarps;  // 16-key chunks per warp and round
     constexpr int NSL = D / 16;             // 16-wide slices of the head dimension
+    constexpr int KH = kWarps / NSL;        // warps per slice: each takes every KH-th chunk in phase 3
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(16) uint8_t smem[];
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
@@ -121,10 +128,12 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     __nv_bfloat16* Vs = Ks + shp.rows * PITCH;
     __nv_bfloat16* Ph = Vs + shp.rows * PITCH;
     __nv_bfloat16* Pl = Ph + kMaxGroup * PP;
-    int* keypos = reinterpret_cast<int*>(Pl + kMaxGroup * PP);
+    int64_t* rowoff = reinterpret_cast<int64_t*>(Pl + kMaxGroup * PP);  // element offset of the row, -1 if masked
+    int* keypos = reinterpret_cast<int*>(rowoff + shp.rows);
     float* wmax = reinterpret_cast<float*>(keypos + shp.rows);
     float* wl = wmax + kWarps * kMaxGroup;
-    float* comb = wl + kWarps * kMaxGroup;  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
+    float* opart = wl + kWarps * kMaxGroup;  // [kWarps - NSL][32][4]
+    float* comb = opart + (kWarps - NSL) * 128;  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
 
 #ifdef SPEC_TRACE
 #define DSTAMP(i) do { if (threadIdx.x == 0) { \
@@ -144,6 +153,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int grp = lane >> 2, quad = lane & 3;
+    const int slice = warp % NSL, kh = warp / NSL;
 
     // Programmatic dependent launch: the next kernel in the stream may start its own prologue
     // (index loads, gather of recalled rows) while this one is still computing.  Everything this
@@ -158,59 +168,54 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
     const int ts = __ldg(a.tail_start + b), cl = __ldg(a.cur_len + b);
 
-    // Gather of round r into its buffer: CH threads per row, one 16-byte piece of the K row and
-    // one of the V row each.  with_tail = false leaves out the rows of the dense tail (the rest
-    // can be read before the dependency wait); masked padding rows of the last chunk are zero-filled.
+    // Gather of round r into its buffer, in two short loops (the code is kept small on purpose:
+    // a kernel this short is paced by instruction fetch when its loops are unrolled into long
+    // straight-line code).  First one thread per row resolves the row: position, validity, offset
+    // in the cache (page-table lookup) -> shared memory.  After a barrier CH threads per row copy
+    // one 16-byte piece of the K row and one of the V row each; masked rows are zero-filled (they
+    // meet P = 0 in the P V product and must be finite).
+    // mode 0: recalled rows and the masked padding of the last chunk (readable before the
+    // dependency wait), 1: rows of the dense tail only, 2: all.
     const int slot = tid / CH, piece = tid % CH;
     const __nv_bfloat16* kbase = a.kv.k + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
     const __nv_bfloat16* vbase = a.kv.v + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
     const int32_t* ptab = a.kv.page_table ? a.kv.page_table + (int64_t)b * a.kv.max_pages : nullptr;
-    auto issue_rows = [&](int r, bool with_tail, int k0, int k1) {
+    auto gather = [&](int r, int mode, int k0, int k1) {
         const int base = k0 + r * RK;
-        const int nk = min(RK, k1 - base);
-        const int nrows = (nk + 15) & ~15;
+        const int nk = max(min(RK, k1 - base), 0);
         const int row0 = NB == 2 ? (r & 1) * kRound : 0;
-        int posv[MAXI];
-#pragma unroll
-        for (int i = 0; i < MAXI; ++i) {  // every index load is in flight before the first is used
-            const int e = base + i * RPP + slot;
-            posv[i] = (i * RPP + slot < RK && e < a.k_total) ? __ldg(idx + e) : -1;
-        }
-        // row offsets next (all page-table loads in flight together), the copies last: the address
-        // arithmetic of different rows overlaps instead of forming one long dependent chain
-        int64_t offv[MAXI];  // -2: not issued here, -1: masked row (zero fill)
-#pragma unroll
-        for (int i = 0; i < MAXI; ++i) {
-            const int lr = i * RPP + slot;
-            const int e = base + lr;
-            const bool valid = lr < nk;
-            const bool is_tail = valid && e >= n_rec;
-            offv[i] = -2;
-            if (lr >= nrows || (is_tail && !with_tail)) continue;
-            int pos = is_tail ? ts + (e - n_rec) : posv[i];
-            if (!valid) pos = -1;
-            else if (pos < 0 || pos >= cl) {
-                set_status(status, SPEC_ERR_BAD_INDEX);
-                pos = -1;
+        const int first_tail = min(max(n_rec - base, 0), nk);  // rows [first_tail, nk) come from the dense tail
+        const int lo = mode == 1 ? first_tail : 0;
+        const int hi = mode == 1 ? nk : ((nk + 15) & ~15);
+        for (int lr = lo + tid; lr < hi; lr += kThreads) {
+            const bool is_tail = lr >= first_tail && lr < nk;
+            if (mode == 0 && is_tail) continue;
+            int pos = -1;
+            if (lr < nk) {
+                pos = is_tail ? ts + (base + lr - n_rec) : __ldg(idx + base + lr);
+                if (pos < 0 || pos >= cl) {
+                    set_status(status, SPEC_ERR_BAD_INDEX);
+                    pos = -1;
+                }
             }
-            if (piece == 0) keypos[row0 + lr] = pos;
-            offv[i] = -1;
+            int64_t off = -1;
             if (pos >= 0) {
                 const int page = page_of(a.kv, pos);
                 const int slot_in = pos - page * a.kv.page_size;
                 const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
-                offv[i] = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
+                off = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
             }
+            keypos[row0 + lr] = pos;
+            rowoff[row0 + lr] = off;
         }
-#pragma unroll
-        for (int i = 0; i < MAXI; ++i) {
-            if (offv[i] == -2) continue;
-            const int lr = i * RPP + slot;
-            // masked rows are zero-filled: they meet P = 0 in the P V product and must be finite
-            const int64_t off = offv[i] >= 0 ? offv[i] : 0;
-            const uint32_t nbytes = offv[i] >= 0 ? 16u : 0u;
-            cp_async16(Ks + (row0 + lr) * PITCH + piece * 8, kbase + off, nbytes);
-            cp_async16(Vs + (row0 + lr) * PITCH + piece * 8, vbase + off, nbytes);
+        __syncthreads();
+#pragma unroll 2
+        for (int lr = lo + slot; lr < hi; lr += RPP) {
+            if (mode == 0 && lr >= first_tail && lr < nk) continue;
+            const int64_t off = rowoff[row0 + lr];
+            const uint32_t nbytes = off >= 0 ? 16u : 0u;
+            cp_async16(Ks + (row0 + lr) * PITCH + piece * 8, kbase + (off >= 0 ? off : 0), nbytes);
+            cp_async16(Vs + (row0 + lr) * PITCH + piece * 8, vbase + (off >= 0 ? off : 0), nbytes);
         }
     };
 
@@ -220,34 +225,28 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     const int k0 = min(n, rank * per);
     const int k1 = min(n, k0 + per);
     const int n_rounds = (k1 - k0 + RK - 1) / RK;
-    for (int r = 0; r < min(n_rounds, NB); ++r) issue_rows(r, false, k0, k1);
+    for (int r = 0; r < min(n_rounds, NB); ++r) gather(r, 0, k0, k1);
     cp_async_commit();
+    // Q and the dense tail are written by earlier kernels of the stream and read after the wait;
+    // asking L2 for their lines now is harmless (L2 is the point of coherence: a later write
+    // lands in the same line) and spares the wait a trip to DRAM when they were not there yet
+    if (tid < G)
+        prefetch_l2(a.q + (((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + tid) * D, D * 2);
+    else if (tid >= 32 && tid < 32 + k1 - max(n_rec, k0)) {
+        const int pos = ts + (max(n_rec, k0) + tid - 32 - n_rec);
+        if (pos >= 0 && pos < cl) {
+            const int page = page_of(a.kv, pos);
+            const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
+            const int64_t off = layer * a.kv.layer_stride + h * a.kv.head_stride + phys * a.kv.page_stride +
+                                (int64_t)(pos - page * a.kv.page_size) * a.kv.slot_stride;
+            prefetch_l2(a.kv.k + off, D * 2);
+            prefetch_l2(a.kv.v + off, D * 2);
+        }
+    }
     DSTAMP(1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
-    {  // rows of the dense tail that fall into the rounds gathered above: at most max_tail, one short pass
-        const int e0 = max(n_rec, k0), e1 = min(k1, k0 + NB * RK);
-        for (int t = slot; t < e1 - e0; t += RPP) {
-            const int e = e0 + t, lr = e - k0;
-            const int r = lr / RK;
-            const int row = (NB == 2 ? (r & 1) * kRound : 0) + (lr - r * RK);
-            int pos = ts + (e - n_rec);
-            if (pos < 0 || pos >= cl) {
-                set_status(status, SPEC_ERR_BAD_INDEX);
-                pos = -1;
-            }
-            if (piece == 0) keypos[row] = pos;
-            int64_t off = 0;
-            if (pos >= 0) {
-                const int page = page_of(a.kv, pos);
-                const int slot_in = pos - page * a.kv.page_size;
-                const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
-                off = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
-            }
-            cp_async16(Ks + row * PITCH + piece * 8, kbase + off, pos >= 0 ? 16u : 0u);
-            cp_async16(Vs + row * PITCH + piece * 8, vbase + off, pos >= 0 ? 16u : 0u);
-        }
-    }
+    for (int r = 0; r < min(n_rounds, NB); ++r) gather(r, 1, k0, k1);
     cp_async_commit();
 
     // B fragments of q^T (d x g) straight from global memory: the thread holds q[g = grp] at
@@ -269,6 +268,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     // running state of the share; the thread tracks heads g = 2 quad and 2 quad + 1 (every thread
     // of the CTA computes the same values for them from shared memory)
     const float sc = a.kv.scale * kLog2e;
+    const bool packed = shp.packed != 0;  // see phase 3
     float M0 = kNegBig, M1 = kNegBig, L0 = 0.f, L1 = 0.f;
     float acc[4][4];
 #pragma unroll
@@ -346,7 +346,8 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
                     const int g = 2 * quad + (e & 1), key = c * 16 + grp + (e >> 1) * 8;
                     const __nv_bfloat16 hi = __float2bfloat16_rn(p[e]);
                     Ph[g * PP + key] = hi;
-                    Pl[g * PP + key] = __float2bfloat16_rn(p[e] - __bfloat162float(hi));
+                    // G <= 4: the lo parts go to rows 4..7 of the hi array (see phase 3)
+                    (packed ? Ph + 4 * PP : Pl)[g * PP + key] = __float2bfloat16_rn(p[e] - __bfloat162float(hi));
                 }
             }
         }
@@ -372,37 +373,64 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
 
         // ---- phase 3: O^T += V^T P^T on this warp's 16-wide slice of the head dimension ----
-        if (warp < NSL) {
+        // With G <= 4 the eight columns of the MMA hold [P hi | P lo] of the four heads side by
+        // side, so one MMA per chunk covers both parts (the two halves are added at the end);
+        // larger groups take one MMA for each part.
+        {
             if (r > 0) {
+                float a0 = alpha0, a1 = alpha1;
+                if (packed) {  // columns 4..7 belong to heads 0..3 again
+                    a0 = __shfl_sync(0xffffffffu, alpha0, (lane & ~3) | (quad & 1));
+                    a1 = __shfl_sync(0xffffffffu, alpha1, (lane & ~3) | (quad & 1));
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    acc[i][0] *= alpha0;
-                    acc[i][1] *= alpha1;
-                    acc[i][2] *= alpha0;
-                    acc[i][3] *= alpha1;
+                    acc[i][0] *= a0;
+                    acc[i][1] *= a1;
+                    acc[i][2] *= a0;
+                    acc[i][3] *= a1;
                 }
             }
-            const __nv_bfloat16* vb = Vs + (row0 + (lane & 7) + ((lane >> 4) & 1) * 8) * PITCH + warp * 16 +
+            const __nv_bfloat16* vb = Vs + (row0 + (lane & 7) + ((lane >> 4) & 1) * 8) * PITCH + slice * 16 +
                                       ((lane >> 3) & 1) * 8;
-            const uint32_t* ph = reinterpret_cast<const uint32_t*>(Ph + grp * PP) + quad;
-            const uint32_t* pl = reinterpret_cast<const uint32_t*>(Pl + grp * PP) + quad;
-            const bool real = grp < G;
-            for (int kc0 = 0; kc0 < nch; kc0 += 4) {  // four chunks requested, then eight MMAs on four chains
-                uint32_t vf[4][4], pb[4][4];
+            // no branches inside the loops: a chunk index past the end is clamped to a valid chunk
+            // and meets P = 0 (uniform branches around the asm blocks cost more than the work)
+            if (packed) {
+                const uint32_t* pp = reinterpret_cast<const uint32_t*>(Ph + grp * PP) + quad;
+                const bool real = (grp & 3) < G;
+                for (int kc0 = kh; kc0 < nch; kc0 += 4 * KH) {  // four chunks requested, then four MMAs on four chains
+                    uint32_t vf[4][4], pb[4][2];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int kc = kc0 + u;
-                    if (kc < nch) {
+                    for (int u = 0; u < 4; ++u) {
+                        const bool ok = kc0 + u * KH < nch;
+                        const int kc = ok ? kc0 + u * KH : kc0;
                         ldmatrix_x4_trans(vf[u], vb + kc * 16 * PITCH);
-                        pb[u][0] = real ? ph[kc * 8] : 0u;
-                        pb[u][1] = real ? ph[kc * 8 + 4] : 0u;
-                        pb[u][2] = real ? pl[kc * 8] : 0u;
-                        pb[u][3] = real ? pl[kc * 8 + 4] : 0u;
+                        const uint32_t v0 = pp[kc * 8], v1 = pp[kc * 8 + 4];
+                        pb[u][0] = real && ok ? v0 : 0u;
+                        pb[u][1] = real && ok ? v1 : 0u;
                     }
-                }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    if (kc0 + u < nch) {
+                    for (int u = 0; u < 4; ++u) mma_bf16(acc[u], vf[u], pb[u][0], pb[u][1]);
+                }
+            } else {
+                const uint32_t* ph = reinterpret_cast<const uint32_t*>(Ph + grp * PP) + quad;
+                const uint32_t* pl = reinterpret_cast<const uint32_t*>(Pl + grp * PP) + quad;
+                const bool real = grp < G;
+                for (int kc0 = kh; kc0 < nch; kc0 += 4 * KH) {  // four chunks requested, then eight MMAs on four chains
+                    uint32_t vf[4][4], pb[4][4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const bool ok = kc0 + u * KH < nch;
+                        const int kc = ok ? kc0 + u * KH : kc0;
+                        ldmatrix_x4_trans(vf[u], vb + kc * 16 * PITCH);
+                        const uint32_t v0 = ph[kc * 8], v1 = ph[kc * 8 + 4], v2 = pl[kc * 8], v3 = pl[kc * 8 + 4];
+                        pb[u][0] = real && ok ? v0 : 0u;
+                        pb[u][1] = real && ok ? v1 : 0u;
+                        pb[u][2] = real && ok ? v2 : 0u;
+                        pb[u][3] = real && ok ? v3 : 0u;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
                         mma_bf16(acc[(u & 1) * 2], vf[u], pb[u][0], pb[u][1]);
                         mma_bf16(acc[(u & 1) * 2 + 1], vf[u], pb[u][2], pb[u][3]);
                     }
@@ -411,7 +439,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
         if (NB == 2) {  // refill the buffer just consumed with the round after next
             __syncthreads();
-            if (r + NB < n_rounds) issue_rows(r + NB, true, k0, k1);
+            if (r + NB < n_rounds) gather(r + NB, 2, k0, k1);
             cp_async_commit();
         }
     }
@@ -420,15 +448,32 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     // ---- deposit (max, sum, O) of the share in the first CTA of the cluster ----
     float* comb0 = CS > 1 ? cluster.map_shared_rank(comb, 0) : comb;
     float* mine = comb0 + rank * PS;
-    if (warp < NSL) {
-        const int d = warp * 16 + grp, g0 = 2 * quad;
+    float o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        o[i] = (acc[0][i] + acc[1][i]) + (acc[2][i] + acc[3][i]);
+        if (packed) o[i] += __shfl_xor_sync(0xffffffffu, o[i], 2);  // hi columns + lo columns
+    }
+    // the warps that share a slice add up through shared memory, in a fixed order
+    if (kh > 0) *reinterpret_cast<float4*>(opart + ((kh - 1) * NSL + slice) * 128 + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
+    __syncthreads();
+    if (kh == 0) {
+#pragma unroll
+        for (int k = 1; k < KH; ++k) {
+            const float4 t = *reinterpret_cast<const float4*>(opart + ((k - 1) * NSL + slice) * 128 + lane * 4);
+            o[0] += t.x;
+            o[1] += t.y;
+            o[2] += t.z;
+            o[3] += t.w;
+        }
+        const int d = slice * 16 + grp, g0 = 2 * quad;
         if (g0 < G) {
-            mine[g0 * D + d] = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]);
-            mine[g0 * D + d + 8] = (acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]);
+            mine[g0 * D + d] = o[0];
+            mine[g0 * D + d + 8] = o[2];
         }
         if (g0 + 1 < G) {
-            mine[(g0 + 1) * D + d] = (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]);
-            mine[(g0 + 1) * D + d + 8] = (acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]);
+            mine[(g0 + 1) * D + d] = o[1];
+            mine[(g0 + 1) * D + d + 8] = o[3];
         }
     }
     if (warp == 0 && grp == 0) {
@@ -487,6 +532,7 @@ DraftShape make_shape(int D, int G, int keys, int cs)
 {
     DraftShape s;
     s.cs = cs;
+    s.packed = G <= 4;
     s.per = ((keys + cs - 1) / cs + 15) & ~15;
     s.rk = s.rows = s.per;  // the whole share resident: one round
     if (s.per > kCap || draft_smem_bytes(D, G, s) > kSmemLimit) {
@@ -570,6 +616,7 @@ int launch_d(const DraftArgs& a, cudaStream_t stream)
     if (!draft_plan<D>(a.kv, a.k_total + a.max_tail, &shp)) return SPEC_ERR_CUDA;
 #ifdef SPEC_TRACE
     if (const char* e = getenv("SPEC_DRAFT_CS")) shp = make_shape(D, G, a.k_total + a.max_tail, atoi(e));
+    if (getenv("SPEC_DRAFT_UNPACKED")) shp.packed = 0;
 #endif
     const size_t smem = draft_smem_bytes(D, G, shp);
     if (smem > kSmemLimit) return SPEC_ERR_UNSUPPORTED_SHAPE;
