@@ -33,6 +33,7 @@ constexpr int kCap = 352;      // most K rows (and V rows) resident per CTA
 constexpr int kRound = 144;    // keys per round when a share exceeds kCap (two buffers of kRound)
 constexpr int kThreads = 512;  // four warps per scheduler: the phases are dependent chains that need interleaving
 constexpr int kWarps = kThreads / 32;
+constexpr int kRedPitch = kWarps + 2;  // float2 per quad row of the per-warp maxima / sums: the 16 B of padding keeps the four rows on different banks
 constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxCluster = 8;  // portable cluster size (a GPC cannot hold two clusters of 16)
 constexpr float kNegBig = -1.0e30f;  // "minus infinity" that stays finite under subtraction
@@ -100,14 +101,14 @@ struct DraftShape {
 
 // Shared memory of one CTA, in this order (every block 16-byte aligned):
 //   K [rows][D + 8] bf16 | V [rows][D + 8] bf16 | P hi, P lo [8][rk + 8] bf16 each |
-//   row offsets int64 [rows] | key positions int [rows] | per-warp maxima, per-warp sums float [8 warps][8] each |
+//   row offsets int64 [rows] | key positions int [rows] | per-warp maxima, per-warp sums float2 [4][16 warps + 2] each |
 //   partial O of the warps that share a head-dim slice float [16 - D/16 warps][32 lanes][4] |
 //   deposit area float [cs][G * (D + 2)] (used in the first CTA of the cluster)
 // The 16 bytes of padding per K/V row spread the banks for ldmatrix.
 __host__ __device__ inline size_t draft_smem_bytes(int D, int G, const DraftShape& s)
 {
     return (size_t)2 * s.rows * (D + 8) * 2 + (size_t)2 * kMaxGroup * (s.rk + 8) * 2 + (size_t)s.rows * 12 +
-           (size_t)2 * kWarps * kMaxGroup * 4 + (size_t)(kWarps - D / 16) * 512 + (size_t)s.cs * G * (D + 2) * 4;
+           (size_t)2 * 8 * kRedPitch * 4 + (size_t)(kWarps - D / 16) * 512 + (size_t)s.cs * G * (D + 2) * 4;
 }
 
 template <int D>
@@ -131,8 +132,8 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     int64_t* rowoff = reinterpret_cast<int64_t*>(Pl + kMaxGroup * PP);  // element offset of the row, -1 if masked
     int* keypos = reinterpret_cast<int*>(rowoff + shp.rows);
     float* wmax = reinterpret_cast<float*>(keypos + shp.rows);
-    float* wl = wmax + kWarps * kMaxGroup;
-    float* opart = wl + kWarps * kMaxGroup;  // [kWarps - NSL][32][4]
+    float* wl = wmax + 8 * kRedPitch;
+    float* opart = wl + 8 * kRedPitch;  // [kWarps - NSL][32][4]
     float* comb = opart + (kWarps - NSL) * 128;  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
 
 #ifdef SPEC_TRACE
@@ -246,9 +247,10 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     DSTAMP(1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
-    for (int r = 0; r < min(n_rounds, NB); ++r) gather(r, 1, k0, k1);
-    cp_async_commit();
-
+    if (k1 > max(n_rec, k0)) {  // this CTA holds rows of the dense tail (the same answer in every thread)
+        for (int r = 0; r < min(n_rounds, NB); ++r) gather(r, 1, k0, k1);
+        cp_async_commit();
+    }
     // B fragments of q^T (d x g) straight from global memory: the thread holds q[g = grp] at
     // d = 16 ks + 2 quad + {0, 1} and + {8, 9}; heads beyond the group are zero
     uint32_t qb[D / 16][2];
@@ -261,6 +263,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
             qb[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
         }
     }
+
     cp_async_wait<0>();
     __syncthreads();
     DSTAMP(3);
@@ -314,19 +317,25 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
         mx0 = group_max(mx0);
         mx1 = group_max(mx1);
-        if (grp == 0) {
-            wmax[warp * kMaxGroup + 2 * quad] = mx0;
-            wmax[warp * kMaxGroup + 2 * quad + 1] = mx1;
-        }
+        if (grp == 0) reinterpret_cast<float2*>(wmax)[quad * kRedPitch + warp] = make_float2(mx0, mx1);
         __syncthreads();
         if (r == 0) DSTAMP(8);
 
         // ---- phase 2: P = 2^(S - max) against the CTA-wide maximum, stored as bf16 hi + lo ----
         float Mn0 = M0, Mn1 = M1;
+        {   // [quad][warp] pairs: two warps per 16-byte load, every lane of a quad reads the same words
+            const float4* wm = reinterpret_cast<const float4*>(wmax) + quad * (kRedPitch / 2);
+            float a0 = kNegBig, a1 = kNegBig, b0 = kNegBig, b1 = kNegBig;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            Mn0 = fmaxf(Mn0, wmax[w * kMaxGroup + 2 * quad]);
-            Mn1 = fmaxf(Mn1, wmax[w * kMaxGroup + 2 * quad + 1]);
+            for (int w = 0; w < kWarps / 2; ++w) {
+                const float4 t = wm[w];
+                a0 = fmaxf(a0, t.x);
+                a1 = fmaxf(a1, t.y);
+                b0 = fmaxf(b0, t.z);
+                b1 = fmaxf(b1, t.w);
+            }
+            Mn0 = fmaxf(Mn0, fmaxf(a0, b0));
+            Mn1 = fmaxf(Mn1, fmaxf(a1, b1));
         }
         const float alpha0 = ex2f(M0 - Mn0), alpha1 = ex2f(M1 - Mn1);
         float ls0 = 0.f, ls1 = 0.f;
@@ -353,19 +362,22 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
         ls0 = group_sum(ls0);
         ls1 = group_sum(ls1);
-        if (grp == 0) {
-            wl[warp * kMaxGroup + 2 * quad] = ls0;
-            wl[warp * kMaxGroup + 2 * quad + 1] = ls1;
-        }
+        if (grp == 0) reinterpret_cast<float2*>(wl)[quad * kRedPitch + warp] = make_float2(ls0, ls1);
         __syncthreads();
         if (r == 0) DSTAMP(9);
         {
-            float t0 = 0.f, t1 = 0.f;
+            const float4* wlp = reinterpret_cast<const float4*>(wl) + quad * (kRedPitch / 2);
+            float t0 = 0.f, t1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) {
-                t0 += wl[w * kMaxGroup + 2 * quad];
-                t1 += wl[w * kMaxGroup + 2 * quad + 1];
+            for (int w = 0; w < kWarps / 2; ++w) {  // fixed order: even warps, odd warps, then both
+                const float4 t = wlp[w];
+                t0 += t.x;
+                t1 += t.y;
+                u0 += t.z;
+                u1 += t.w;
             }
+            t0 += u0;
+            t1 += u1;
             L0 = L0 * alpha0 + t0;
             L1 = L1 * alpha1 + t1;
             M0 = Mn0;
