@@ -229,6 +229,59 @@ def make_case(cfg: SpecConfig, device="cpu", n_layers: Optional[int] = None,
                     direction=direction, capacity=ps * max_pages)
 
 
+def resample_planted(case: SpecCase, prob: float, step: int) -> int:
+    """Move each planted heavy-hitter position with probability ``prob`` (third workload: the
+    important set drifts between speculation rounds, so the index must be rebuilt from the fresh
+    statistic).  The old row gets a fresh background key, the new position (uniform in the
+    context, not planted already) gets ``planted_mult`` x the head's direction (+ noise).
+    Updates ``case.kv.k`` and ``case.planted_pos`` in place; returns how many positions moved.
+    Seeded by (config seed, step)."""
+    cfg = case.cfg
+    assert case.planted_pos is not None and case.direction is not None
+    dev = case.kv.k.device
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7368787 * cfg.seed + 104729 * step + 5)
+    L, B, Hkv, n_pl = case.planted_pos.shape
+    D, ps = cfg.head_dim, case.kv.page_size
+    ptab = case.kv.page_table
+    moved_total = 0
+    for l in range(L):
+        for b in range(B):
+            T = int(case.ctx_len[b])
+            pos = case.planted_pos[l, b]  # [Hkv, n_pl]
+            move = torch.rand((Hkv, n_pl), generator=gen, device=dev) < prob
+            cand = torch.randint(0, T, (Hkv, n_pl), generator=gen, device=dev)
+            taken = torch.zeros((Hkv, T), dtype=torch.bool, device=dev)
+            taken.scatter_(1, pos, True)
+            move &= ~taken.gather(1, cand)  # a candidate that is planted already: stay
+            # two moves of one head to the same candidate: keep the first
+            order = torch.where(move, cand, torch.full_like(cand, T)).sort(dim=1)
+            dup = torch.zeros_like(move)
+            dup.scatter_(1, order.indices[:, 1:], (order.values[:, 1:] == order.values[:, :-1]) &
+                         (order.values[:, 1:] < T))
+            move &= ~dup
+            hh = torch.arange(Hkv, device=dev)[:, None].expand(Hkv, n_pl)
+
+            def rows(p):
+                page, slot = p // ps, p % ps
+                phys = (b * case.kv.max_pages + page) if ptab is None else ptab[b][page].long()
+                return phys, slot
+
+            old_phys, old_slot = rows(pos[move])
+            fresh = _draw_kv((int(move.sum()), D), cfg.kv_dist, gen, dev).to(torch.bfloat16)
+            kview = case.kv.k.view(L, case.kv.n_pages, Hkv, ps, D)
+            kview[l, old_phys, hh[move], old_slot] = fresh
+            key = cfg.planted_mult * case.direction[l, b][:, None, :].expand(Hkv, n_pl, D)[move]
+            if cfg.planted_noise:
+                key = key + torch.randn(key.shape, generator=gen, device=dev, dtype=torch.float32)
+            new_phys, new_slot = rows(cand[move])
+            kview[l, new_phys, hh[move], new_slot] = key.to(torch.bfloat16)
+            pos[move] = cand[move]
+            case.planted_pos[l, b] = pos.sort(dim=1).values
+            moved_total += int(move.sum())
+    return moved_total
+
+
 def small_config(name="small", **kw) -> SpecConfig:
     """A config sized for element-by-element parity against the oracle; fields overridable."""
     base = dict(name=name, n_layers=1, batch=1, n_q_heads=8, n_kv_heads=2, head_dim=128,

@@ -128,3 +128,47 @@ def test_cfg5_32b_shape_student_t_values():
     recent; 4 of the 64 layers."""
     cfg = dataclasses.replace(inputs.baseline_configs()["cfg5_32b_64k"], n_layers=4)
     run_config(cfg, [(0, 0, 0), (3, 3, 7)])
+
+
+def test_128k_index_follows_resampled_heavy_hitters():
+    """Third workload, full context and budget, 2 of its 32 layers: between speculation rounds
+    each planted position moves with probability 0.1.  The index rebuilt from each round's GPU
+    statistic must hold (nearly) all CURRENT planted positions, the ones that just moved in
+    included, and the draft output over that index must match the oracle on a sampled head."""
+    cfg = dataclasses.replace(inputs.baseline_configs(4)["cfg3_8b_128k"], n_layers=2)
+    case = inputs.make_case(cfg, device="cuda")
+    run = runner.SpecStepRunner(case)
+    G = cfg.group
+    for step in range(3):
+        before = case.planted_pos.clone()
+        moved = inputs.resample_planted(case, 0.1, step)
+        assert moved > 0
+        run.step()
+        torch.cuda.synchronize()
+        assert binding.read_status(run.ws_v) == 0 and binding.read_status(run.ws_d) == 0
+        hit_all, n_all, hit_new, n_new = 0, 0, 0, 0
+        for layer in range(cfg.n_layers):
+            for h in range(cfg.n_kv_heads):
+                chosen = set(run.indices[layer, 0, h, :int(run.n_idx[layer, 0, h])].tolist())
+                cur = set(case.planted_pos[layer, 0, h].tolist())
+                new = cur - set(before[layer, 0, h].tolist())
+                hit_all += len(cur & chosen)
+                n_all += len(cur)
+                hit_new += len(new & chosen)
+                n_new += len(new)
+        assert n_new > 0
+        # 3 x the direction plus unit noise: a planted key sits about 5 sigma above the background
+        assert hit_all / n_all > 0.97, (step, hit_all, n_all)
+        assert hit_new / n_new > 0.95, (step, hit_new, n_new)
+    # the last round's draft outputs on one sampled head, against the oracle over the GPU's index
+    layer, b, h = 1, 0, 5
+    T = int(case.ctx_len[b])
+    sub = one_head_cache(case.kv, layer, b, h, T + cfg.draft_steps)
+    idx = run.indices[layer, b, h].cpu().view(1, 1, 1, -1).contiguous()
+    n = run.n_idx[layer, b, h].cpu().view(1, 1, 1).contiguous()
+    for j in range(cfg.draft_steps):
+        q = case.q_draft[j, layer, b, h * G:(h + 1) * G].cpu().contiguous().view(1, 1, G, -1)
+        o_out, _ = oracle.sparse_draft_attn(sub, q, idx, n, torch.tensor([T], dtype=torch.int32),
+                                            torch.tensor([T + j + 1], dtype=torch.int32))
+        g_out = run.out_d[j, layer, b, h * G:(h + 1) * G].cpu().double()
+        assert (g_out - o_out[0, 0]).abs().max().item() < TOL

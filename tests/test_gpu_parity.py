@@ -207,6 +207,12 @@ DRAFT_SHAPES = [
     dict(ctx=(300, 2000), k_total=256, k_recent=64, batch=3, page_size=16, shuffled_pages=True,
          planted=0, q_mode="iid", q_std=0.09, n_layers=2),
     dict(ctx=(700, 700), k_total=100, k_sink=0, k_recent=0, n_q_heads=8, n_kv_heads=8),
+    # 8 problems x 2048 keys: the planner takes clusters of six (two calls resident together)
+    dict(ctx=(4000, 4000), k_total=2048, k_recent=64, n_q_heads=32, n_kv_heads=8, planted=0.01),
+    # 4104-key lists on 2 problems: shares of 528 keys run in rounds through two buffers
+    dict(ctx=(6000, 6000), k_total=4096, k_recent=64, n_q_heads=8, n_kv_heads=2, planted=0.01),
+    # group of 8 query heads: one MMA each for the hi and the lo part of P
+    dict(ctx=(1500, 1500), k_total=512, k_recent=32, n_q_heads=16, n_kv_heads=2),
 ]
 
 

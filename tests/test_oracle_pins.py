@@ -274,3 +274,27 @@ def test_planted_heavy_hitters_are_recalled():
         planted = case.planted_pos[0, 0, h].tolist()
         assert all(p in chosen for p in planted)
         assert stats[0, 0, h][planted].sum() / stats[0, 0, h].sum() > 0.5
+
+
+def test_resampled_heavy_hitters_are_recalled_from_the_fresh_statistic():
+    """Third workload's drift, scaled down: every round some planted positions move; the index
+    rebuilt from that round's statistic holds the CURRENT set, an index kept from the round
+    before misses exactly the positions that moved in."""
+    cfg = inputs.small_config(ctx=(3000, 3000), planted=0.02, k_total=256, k_recent=16,
+                              planted_mult=4.0, planted_noise=False, seed=5)
+    case = inputs.make_case(cfg)
+    prev_idx = None
+    for step in range(3):
+        moved = inputs.resample_planted(case, 0.25, step)
+        assert moved > 0
+        _, _, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len)
+        idx, _ = oracle.select_recall(stats.float(), case.ctx_len, cfg.k_sink, cfg.k_recent,
+                                      cfg.k_total)
+        for h in range(cfg.n_kv_heads):
+            planted = set(case.planted_pos[0, 0, h].tolist())
+            assert len(planted) == case.planted_pos.shape[-1]  # positions stay distinct
+            assert planted <= set(idx[0, 0, h].tolist())
+            if prev_idx is not None:
+                stale = set(prev_idx[0, 0, h].tolist())
+                assert len(planted - stale) > 0  # the drift is visible to a stale index
+        prev_idx = idx
