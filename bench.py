@@ -177,6 +177,41 @@ def run_reference(args):
 # -------------------------------------------------------------------------------------------------
 
 
+def drift_recall(case, run, n_rounds, prob=0.1):
+    """After the timed region: ``n_rounds`` more speculation rounds in which every planted position
+    moves with probability ``prob`` first (third workload's drift).  Reports, per round, which
+    fraction of the CURRENT planted set, and of the positions that just moved in, the index rebuilt
+    from that round's statistic holds."""
+    import torch
+
+    from paper_2607_27735_b200 import inputs
+    cfg = case.cfg
+    per_round, per_round_new, stale, prev_chosen = [], [], [], None
+    for step in range(n_rounds):
+        before = case.planted_pos.clone()
+        inputs.resample_planted(case, prob, step)
+        run.step()
+        torch.cuda.synchronize()
+        idx = run.indices.long()                                       # [L, B, Hkv, k_total], -1 padded
+        T = int(case.ctx_len.max()) + cfg.draft_steps + 1
+        chosen = torch.zeros(idx.shape[:3] + (T + 1,), dtype=torch.bool, device=idx.device)
+        chosen.scatter_(3, torch.where(idx >= 0, idx, torch.full_like(idx, T)), True)
+        chosen[..., T] = False
+        was = torch.zeros_like(chosen)
+        was.scatter_(3, before, True)
+        hit = chosen.gather(3, case.planted_pos)
+        new = ~was.gather(3, case.planted_pos)
+        per_round.append(hit.float().mean().item())
+        per_round_new.append((hit & new).sum().item() / max(1, int(new.sum())))
+        if prev_chosen is not None:  # what an index kept from the round before would have held
+            stale.append(prev_chosen.gather(3, case.planted_pos).float().mean().item())
+        prev_chosen = chosen
+    return {"rounds": n_rounds, "move_prob": prob,
+            "recall_current_by_previous_rounds_index_mean": sum(stale) / max(1, len(stale)),
+            "recall_current_min": min(per_round), "recall_current_mean": sum(per_round) / n_rounds,
+            "recall_moved_min": min(per_round_new), "recall_moved_mean": sum(per_round_new) / n_rounds}
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -315,6 +350,8 @@ def run_gpu(args):
         fold = L if args.fold_layers else 1
         line["roofline"]["traffic"] = t["verify"] * fold
         line["draft_roofline"]["traffic"] = t["draft"] * fold
+    if args.recall_steps > 0 and case.planted_pos is not None:
+        line["recall"] = drift_recall(case, run, args.recall_steps)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -333,6 +370,8 @@ def main():
                     help="speculation length k of cfg3_8b_128k (its sweep is k in 1, 2, 4, 8, 16)")
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the oracle timing (sweeps over the other workloads)")
+    ap.add_argument("--recall-steps", type=int, default=0,
+                    help="after timing, run this many rounds with drifting planted positions and report recall")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()
