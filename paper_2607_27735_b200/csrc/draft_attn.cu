@@ -247,7 +247,42 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     DSTAMP(1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
-    if (k1 > max(n_rec, k0)) {  // this CTA holds rows of the dense tail (the same answer in every thread)
+    // Rows of the dense tail.  A share that is resident in one round: the warp that owns a tail row's
+    // chunk in phase 1 copies the row itself and waits for it only when it reaches that chunk, so the
+    // fetch runs beside the Q loads instead of in front of the block barrier.  Shares that take
+    // several rounds use the common gather.
+    const int t0 = max(n_rec, k0) - k0, t1 = k1 - k0;  // local rows [t0, t1) of the share come from the tail
+    if (NB == 1) {
+        constexpr int LPR = 2 * CH;  // lanes per row: CH pieces of K, CH pieces of V
+        for (int c = t0 >> 4; c * 16 < t1; ++c) {
+            if (c % kWarps != warp) continue;
+            const int lo = max(c * 16, t0), n = min(c * 16 + 16, t1) - lo;  // n <= 16 rows, one lane resolves each
+            int64_t off = -1;
+            if (lane < n) {
+                int pos = ts + (k0 + lo + lane - n_rec);
+                if (pos < 0 || pos >= cl) {
+                    set_status(status, SPEC_ERR_BAD_INDEX);
+                    pos = -1;
+                }
+                keypos[lo + lane] = pos;
+                if (pos >= 0) {
+                    const int page = page_of(a.kv, pos);
+                    const int slot_in = pos - page * a.kv.page_size;
+                    const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
+                    off = phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride;
+                }
+            }
+            const bool is_v = (lane % LPR) >= CH;  // kbase / vbase already point at this lane's piece (lane % CH)
+            for (int i = 0; i < n; i += 32 / LPR) {
+                const int row = i + lane / LPR;
+                const int64_t o = __shfl_sync(0xffffffffu, off, row & 31);
+                if (row < n)
+                    cp_async16((is_v ? Vs : Ks) + (lo + row) * PITCH + piece * 8, (is_v ? vbase : kbase) + (o >= 0 ? o : 0),
+                               o >= 0 ? 16u : 0u);
+            }
+        }
+        cp_async_commit();
+    } else if (t1 > t0) {  // the same answer in every thread
         for (int r = 0; r < min(n_rounds, NB); ++r) gather(r, 1, k0, k1);
         cp_async_commit();
     }
@@ -264,7 +299,8 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
     }
 
-    cp_async_wait<0>();
+    if (NB == 1) cp_async_wait<1>();  // everything but the tail rows just requested
+    else cp_async_wait<0>();
     __syncthreads();
     DSTAMP(3);
 
@@ -295,6 +331,10 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
             const int c = warp + kWarps * j;
             s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
             if (c < nch) {
+                if (NB == 1 && c * 16 + 16 > t0 && c * 16 < t1) {  // this warp copied the chunk's tail rows
+                    cp_async_wait<0>();
+                    __syncwarp();
+                }
                 uint32_t kf[D / 16][4];  // all fragments of the chunk are requested before the first MMA
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
@@ -318,6 +358,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         mx0 = group_max(mx0);
         mx1 = group_max(mx1);
         if (grp == 0) reinterpret_cast<float2*>(wmax)[quad * kRedPitch + warp] = make_float2(mx0, mx1);
+        cp_async_wait<0>();  // tail rows of V: seen by every warp after the barrier
         __syncthreads();
         if (r == 0) DSTAMP(8);
 
