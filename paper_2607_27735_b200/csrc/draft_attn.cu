@@ -15,15 +15,13 @@
 //   3. values: each warp owns a 16-wide slice of the head dimension and accumulates
 //      O^T = V^T P^T over all keys of the share, so no merge between warps is needed.
 // The CTAs of the cluster deposit (max, sum, O) in the first CTA through distributed shared
-// memory; it merges them in rank order (deterministic) after one cluster barrier.
+// memory (asynchronous stores counted on an mbarrier there); it merges them in rank order
+// (deterministic) once every byte has landed.
 // One launch per call, no global scratch, no second kernel.
-#include <cooperative_groups.h>
 #include <cstdio>
 #include <cstdlib>
 
 #include "spec_common.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace spec {
 
@@ -37,6 +35,7 @@ constexpr int kRedPitch = kWarps + 2;  // float2 per quad row of the per-warp ma
 constexpr int kMaxGroup = 8;    // query heads per KV head
 constexpr int kMaxCluster = 8;  // portable cluster size (a GPC cannot hold two clusters of 16)
 constexpr float kNegBig = -1.0e30f;  // "minus infinity" that stays finite under subtraction
+constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // bound of the deposit wait: about a second
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 // 16 bytes global -> shared; src_bytes = 0 writes zeros instead (masked rows)
@@ -49,6 +48,37 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uin
 __device__ __forceinline__ void prefetch_l2(const void* gsrc, uint32_t bytes)
 {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
+}
+// 4 bytes into the shared memory of another CTA of the cluster; the bytes are counted on that
+// CTA's mbarrier when they have landed (no fence, no cluster barrier needed on either side)
+__device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint32_t remote_bar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(remote_addr), "r"(__float_as_uint(v)), "r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -103,12 +133,12 @@ struct DraftShape {
 //   K [rows][D + 8] bf16 | V [rows][D + 8] bf16 | P hi, P lo [8][rk + 8] bf16 each |
 //   row offsets int64 [rows] | key positions int [rows] | per-warp maxima, per-warp sums float2 [4][16 warps + 2] each |
 //   partial O of the warps that share a head-dim slice float [16 - D/16 warps][32 lanes][4] |
-//   deposit area float [cs][G * (D + 2)] (used in the first CTA of the cluster)
+//   deposit barrier (16 B) | deposit area float [cs][G * (D + 2)] (used in the first CTA of the cluster)
 // The 16 bytes of padding per K/V row spread the banks for ldmatrix.
 __host__ __device__ inline size_t draft_smem_bytes(int D, int G, const DraftShape& s)
 {
     return (size_t)2 * s.rows * (D + 8) * 2 + (size_t)2 * kMaxGroup * (s.rk + 8) * 2 + (size_t)s.rows * 12 +
-           (size_t)2 * 8 * kRedPitch * 4 + (size_t)(kWarps - D / 16) * 512 + (size_t)s.cs * G * (D + 2) * 4;
+           (size_t)2 * 8 * kRedPitch * 4 + (size_t)(kWarps - D / 16) * 512 + 16 + (size_t)s.cs * G * (D + 2) * 4;
 }
 
 template <int D>
@@ -134,7 +164,8 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     float* wmax = reinterpret_cast<float*>(keypos + shp.rows);
     float* wl = wmax + 8 * kRedPitch;
     float* opart = wl + 8 * kRedPitch;  // [kWarps - NSL][32][4]
-    float* comb = opart + (kWarps - NSL) * 128;  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
+    uint64_t* dep_bar = reinterpret_cast<uint64_t*>(opart + (kWarps - NSL) * 128);  // first CTA: counts deposited bytes
+    float* comb = reinterpret_cast<float*>(dep_bar + 2);  // [CS][PS]: O rows [G][D], then the maxima [G], then the sums [G]
 
 #ifdef SPEC_TRACE
 #define DSTAMP(i) do { if (threadIdx.x == 0) { \
@@ -146,7 +177,6 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
 #define DSTAMP(i) do { } while (0)
 #endif
     DSTAMP(0);
-    cg::cluster_group cluster = cg::this_cluster();
     const int CS = gridDim.x;              // the cluster spans the x dimension
     const int rank = blockIdx.x;
     const int h = blockIdx.y;
@@ -161,6 +191,17 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     // kernel reads before griddepcontrol.wait below is immutable during a drafting round (indices,
     // lengths, recalled rows of the dense cache); Q, the dense tail and the outputs come after.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // The first CTA of the cluster counts the bytes the others deposit at the end on an mbarrier.
+    // It is armed here; the cluster barrier that tells the others so is split around the gather.
+    if (CS > 1) {
+        if (rank == 0 && tid == 0) {
+            mbar_init(smem_addr(dep_bar), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            mbar_arrive_expect_tx(smem_addr(dep_bar), (uint32_t)(CS - 1) * PS * 4);
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
 
     const int32_t* idx = a.indices + prob * a.k_total;
     // contiguous shares in multiples of the 16-key chunk; the share size depends only on host-side
@@ -245,6 +286,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
     }
     DSTAMP(1);
+    if (CS > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     DSTAMP(2);
     // Rows of the dense tail.  A share that is resident in one round: the warp that owns a tail row's
@@ -499,8 +541,6 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     DSTAMP(4);
 
     // ---- deposit (max, sum, O) of the share in the first CTA of the cluster ----
-    float* comb0 = CS > 1 ? cluster.map_shared_rank(comb, 0) : comb;
-    float* mine = comb0 + rank * PS;
     float o[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -510,6 +550,16 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     // the warps that share a slice add up through shared memory, in a fixed order
     if (kh > 0) *reinterpret_cast<float4*>(opart + ((kh - 1) * NSL + slice) * 128 + lane * 4) = make_float4(o[0], o[1], o[2], o[3]);
     __syncthreads();
+    // the first CTA writes its own slot; the others send theirs with asynchronous stores that
+    // count on its mbarrier, and are done: no fence, no closing cluster barrier
+    const bool remote = rank != 0;
+    float* mine = comb + rank * PS;
+    const uint32_t mine_r = remote ? map_to_rank(smem_addr(mine), 0) : 0u;
+    const uint32_t bar_r = remote ? map_to_rank(smem_addr(dep_bar), 0) : 0u;
+    auto put = [&](int i, float v) {
+        if (remote) st_async_f32(mine_r + 4 * i, v, bar_r);
+        else mine[i] = v;
+    };
     if (kh == 0) {
 #pragma unroll
         for (int k = 1; k < KH; ++k) {
@@ -521,28 +571,37 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
         const int d = slice * 16 + grp, g0 = 2 * quad;
         if (g0 < G) {
-            mine[g0 * D + d] = o[0];
-            mine[g0 * D + d + 8] = o[2];
+            put(g0 * D + d, o[0]);
+            put(g0 * D + d + 8, o[2]);
         }
         if (g0 + 1 < G) {
-            mine[(g0 + 1) * D + d] = o[1];
-            mine[(g0 + 1) * D + d + 8] = o[3];
+            put((g0 + 1) * D + d, o[1]);
+            put((g0 + 1) * D + d + 8, o[3]);
         }
     }
     if (warp == 0 && grp == 0) {
         if (2 * quad < G) {
-            mine[G * D + 2 * quad] = M0;
-            mine[G * D + G + 2 * quad] = L0;
+            put(G * D + 2 * quad, M0);
+            put(G * D + G + 2 * quad, L0);
         }
         if (2 * quad + 1 < G) {
-            mine[G * D + 2 * quad + 1] = M1;
-            mine[G * D + G + 2 * quad + 1] = L1;
+            put(G * D + 2 * quad + 1, M1);
+            put(G * D + G + 2 * quad + 1, L1);
         }
     }
     DSTAMP(5);
-    if (CS > 1) cluster.sync(); else __syncthreads();
+    if (remote) return;
+    if (CS > 1) {  // every byte of the other CTAs has landed (bounded: a stall ends in a status code)
+        const long long t_start = clock64();
+        while (!mbar_try_wait(smem_addr(dep_bar), 0)) {
+            if (clock64() - t_start > kTimeoutCycles) {
+                set_status(status, SPEC_ERR_TIMEOUT);
+                break;
+            }
+        }
+    }
+    __syncthreads();  // this CTA's own slot
     DSTAMP(6);
-    if (rank != 0) return;
     // ---- merge the CTAs of the cluster, in rank order ----
     for (int i = tid; i < G * (D / 2); i += kThreads) {
         const int r = i / (D / 2), dp = i - r * (D / 2);
