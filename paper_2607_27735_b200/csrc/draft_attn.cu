@@ -28,7 +28,7 @@ namespace spec {
 namespace {
 
 constexpr int kCap = 352;      // most K rows (and V rows) resident per CTA
-constexpr int kRound = 144;    // keys per round when a share exceeds kCap (two buffers of kRound)
+constexpr int kRound = 176;    // keys per round when a share exceeds kCap (two buffers of kRound = kCap rows)
 constexpr int kThreads = 512;  // four warps per scheduler: the phases are dependent chains that need interleaving
 constexpr int kWarps = kThreads / 32;
 constexpr int kRedPitch = kWarps + 2;  // float2 per quad row of the per-warp maxima / sums: the 16 B of padding keeps the four rows on different banks
@@ -694,8 +694,8 @@ bool set_smem_limit(size_t smem)
     return true;
 }
 
-// Split of a call.  The cluster grows (1, 2, 4, 8 CTAs) until the CTAs cover the SMs or a CTA
-// would get less than about one round of keys.  A call that fits the GPU in one wave wants the
+// Split of a call.  The cluster grows (1, 2, 4, 8 CTAs) while all CTAs still fit the SMs in one wave
+// (a second wave could not start its gather under the first) and a CTA keeps about a round of keys.  A call that fits the GPU in one wave wants the
 // next call's gather to run beside it (programmatic dependent launch), which needs both calls'
 // clusters resident together; a GPC holds at most two clusters of eight and not every GPC
 // does, so where 2 x clusters-per-call does not fit, clusters of six (which pack better) are
@@ -708,7 +708,7 @@ bool draft_plan(const KvView& kv, int n_keys_max, DraftShape* out)
     const int keys = n_keys_max > 0 ? n_keys_max : 1;
     const int rounds = (keys + kRound - 1) / kRound;
     int cs = 1;
-    while (cs < kMaxCluster && probs * cs < sm_count() && cs < rounds) cs *= 2;
+    while (cs < kMaxCluster && probs * cs * 2 <= sm_count() && cs < rounds) cs *= 2;  // one wave of CTAs at most
     DraftShape s = make_shape(D, G, keys, cs);
     if (!set_smem_limit<D>(kSmemLimit)) return false;
     if (cs == kMaxCluster && probs * cs <= sm_count() &&
