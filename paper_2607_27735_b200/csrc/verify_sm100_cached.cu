@@ -124,6 +124,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     for (int r = R + threadIdx.x; r < 128; r += kBlock) {  // padded rows: P = 0
         lse_s[r] = 1.0e30f;
         loc_s[r] = 1.0e30f;
+        fac_s[r] = 0.f;
     }
     fence_proxy_async();
     if (warp == 1) {
@@ -585,6 +586,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                                 }
                             }
                         }
+                        // P~ replaces the tile's scores in tensor memory: the statistic pass then only
+                        // weights it with exp2(lse_local - LSE) per row, no second exponential
+#pragma unroll
+                        for (int q = 0; q < NH; q += 8)
+                            tmem_st8(t_lane + col_s + c * N + c0 + q, reinterpret_cast<const uint32_t*>(pr) + q);
                         // the P buffer is free once the P V product p_bufs tiles back is done ("done"
                         // barriers are indexed by the tile's sequence number mod 4)
                         if (pvi >= (uint32_t)p.p_bufs) {
@@ -631,6 +637,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     }
                 }
                 if (!ok) break;
+                tc_wait_st();
+                tc_fence_before();
                 pv_idx += n_t;
                 slot_base += 2 * n_t;
                 if (warp == 4) TRACE(2, 4);
@@ -680,15 +688,16 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 }
                 ok = group_sync(B.sm_sync, sync_n, ctl, 22);
                 if (!ok) break;
+                tc_fence_after();  // the P~ stores of the other warps, ordered by the barrier
                 if (warp == 4) TRACE(2, 6);
                 // ------------------------------ P2b: the Eq. 3 statistic ------------------------------
-                // second visit of the cached score tiles, now with the global LSE: column sums of the
-                // exactly normalised probabilities.  No shared memory, no tensor cores; the tile's
-                // TMEM region is released afterwards.
+                // second visit of the cached tiles, which hold P~ = exp2(S - lse_local) by now (masked
+                // entries are 0): weighted with exp2(lse_local - LSE) per row they are the exactly
+                // normalised probabilities, whose column sums are the statistic.  No exponential, no
+                // shared memory, no tensor cores; the tile's TMEM region is released afterwards.
                 for (int c = wg; c < n_t; c += CG) {
                     const int t = sg.t0 + c;
                     const int key = t * kTile + key_l;
-                    const bool boundary = t * kTile + kTile > sg.T - p.a.n_q + 1;
                     float st = 0.f;
 #pragma unroll 1
                     for (int cb = 0; cb < N; cb += 16) {
@@ -697,26 +706,15 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         tmem_ld8(t_lane + col_s + c * N + cb, v);
                         tmem_ld8(t_lane + col_s + c * N + cb + 8, v + 8);
                         tc_wait_ld();
-                        const float4* lse4 = reinterpret_cast<const float4*>(lse_s + cb);
+                        const float4* fac4 = reinterpret_cast<const float4*>(fac_s + cb);
                         float pr[16];
 #pragma unroll
                         for (int i = 0; i < 16; i += 4) {
-                            const float4 ls = lse4[i >> 2];
-                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
-                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
-                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
-                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
-                        }
-                        if (boundary) {
-                            int j = cb / G, gg = cb - j * G;
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                if (key > sg.T - p.a.n_q + j) pr[i] = 0.f;  // select, so NaN-safe
-                                if (++gg == G) {
-                                    gg = 0;
-                                    ++j;
-                                }
-                            }
+                            const float4 f = fac4[i >> 2];
+                            pr[i + 0] = __uint_as_float(v[i + 0]) * f.x;
+                            pr[i + 1] = __uint_as_float(v[i + 1]) * f.y;
+                            pr[i + 2] = __uint_as_float(v[i + 2]) * f.z;
+                            pr[i + 3] = __uint_as_float(v[i + 3]) * f.w;
                         }
                         if (cb >= stat_r0) {
 #pragma unroll
