@@ -35,15 +35,17 @@ namespace sm100 {
 namespace {
 
 constexpr int kMaxCache = 32;
+constexpr int kLsePubMax = 48;  // CTAs per head up to which the publisher warp alone combines the LSE partials
 
 struct CBars {  // mbarrier addresses (shared space)
     uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_free, p_full, p_empty, o_full, o_empty, sm_sync,
-        pub_p1, pub_o;
+        pub_p1, pub_o, lse_ready;
 };
 
 // NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
 // more, narrower warpgroups hide the latency of the serial softmax sections.
-template <int NC, int CG>
+// LP: the publisher warp combines the LSE partials (few CTAs per head); otherwise the softmax warps do.
+template <int NC, int CG, bool LP>
 __global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_q, const FastParams p)
@@ -82,6 +84,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.sm_sync = o; o += 8;
         B.pub_p1 = o; o += 8;   // the last softmax warp stored this CTA's (max, sum) partial
         B.pub_o = o; o += 8;    // every softmax warp stored its share of the output partial
+        B.lse_ready = o; o += 8;  // the publisher warp left the row LSE and the rescale factors in shared memory
     }
     float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128] global row LSE (log2 domain)
     float* loc_s = reinterpret_cast<float*>(misc + 1024 + 512);           // [128] CTA-local row LSE
@@ -115,6 +118,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         mbar_init(B.sm_sync, kSW);
         mbar_init(B.pub_p1, 1);
         mbar_init(B.pub_o, kSW);
+        mbar_init(B.lse_ready, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -352,20 +356,77 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // =========================== publisher warp ===========================
         // Makes this CTA's partials visible to the other CTAs (device-scope fence + counter), so
         // that no softmax warp ever waits for that round trip: they only arrive on a CTA barrier.
-        if (lane == 0) {
-            bool ok = true;
-            for (int unit = 0; unit < U && ok; ++unit) {
+        // It also combines the (max, sum) partials of the CTAs that share the head into the row
+        // LSE while the softmax warps are busy with the P V pass.
+        bool ok = true;
+        for (int unit = 0; unit < U && ok; ++unit) {
+            if (lane == 0) {
                 ok = mbar_wait(B.pub_p1, unit & 1, ctl, 34);
-                if (!ok) break;
-                __threadfence();
-                atomicAdd(p.counters + unit * p.HG + head_local, 1);
-                ok = mbar_wait(B.pub_o, unit & 1, ctl, 35);
-                if (!ok) break;
-                __threadfence();
-                atomicAdd(p.counters + U * p.HG + unit * p.HG + head_local, 1);
+                if (ok) {
+                    __threadfence();
+                    atomicAdd(p.counters + unit * p.HG + head_local, 1);
+                }
             }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            const Seg sg = get_seg(p, unit, head_local, rank);
+            if (LP && sg.t1 > sg.t0) {
+                // ---- row LSE from the partials of the CTAs that share this head ----
+                if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
+                if (!ok) break;
+                const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
+                // two lanes per row, 16 rows per pass: each lane folds every other partial, 20 loads in flight
+                const int sub = lane & 1;
+                for (int r0 = 0; r0 < R; r0 += 16) {
+                    const int r = r0 + (lane >> 1);
+                    float M = -1.0e30f, Ls = 0.f;
+                    if (r < R) {
+                        for (int k0 = sub; k0 < p.cph; k0 += 40) {
+                            float2 x[20];
+#pragma unroll
+                            for (int u = 0; u < 20; ++u)
+                                x[u] = (k0 + 2 * u < p.cph) ? __ldcg(src + (int64_t)(k0 + 2 * u) * R + r)
+                                                            : make_float2(-1.0e30f, 0.f);
+#pragma unroll
+                            for (int u = 0; u < 20; ++u) {
+                                const float Mn = fmaxf(M, x[u].x);
+                                Ls = Ls * ex2(M - Mn) + x[u].y * ex2(x[u].x - Mn);
+                                M = Mn;
+                            }
+                        }
+                    }
+                    const float M2 = __shfl_xor_sync(0xffffffffu, M, 1);
+                    const float L2 = __shfl_xor_sync(0xffffffffu, Ls, 1);
+                    const float Mn = fmaxf(M, M2);
+                    Ls = Ls * ex2(M - Mn) + L2 * ex2(M2 - Mn);
+                    M = Mn;
+                    if (sub == 0 && r < R) {
+                        const float lse2 = M + log2f(Ls);
+                        lse_s[r] = lse2;
+                        const float loc = loc_s[r];
+                        fac_s[r] = loc < 1.0e29f ? ex2(loc - lse2) : 0.f;  // local -> global normaliser
+                        if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
+                            const int j = r / G, g = r - j * G;
+                            const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
+                            p.a.lse[row] = lse2 * 0.69314718055994530942f;
+                        }
+                    }
+                }
+            }
+            // signalled for every unit, empty ones too: the softmax warps wait for it before they go
+            // on, so they are never more than one barrier phase ahead of this warp
+            __syncwarp();
+            if (lane == 0) mbar_arrive(B.lse_ready);
+            if (lane == 0) {
+                ok = mbar_wait(B.pub_o, unit & 1, ctl, 35);
+                if (ok) {
+                    __threadfence();
+                    atomicAdd(p.counters + U * p.HG + unit * p.HG + head_local, 1);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
-        __syncwarp();
     } else if (warp == 3) {
         // =========================== O reduction warp ===========================
         const int tid = lane;
@@ -642,51 +703,55 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 pv_idx += n_t;
                 slot_base += 2 * n_t;
                 if (warp == 4) TRACE(2, 4);
-                // ---- row LSE from the partials of the CTAs that share this head ----
-                if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
+                // ---- the row LSE and the rescale factors, combined by the publisher warp meanwhile ----
+                ok = mbar_wait(B.lse_ready, unit & 1, ctl, 31);
                 if (!ok) break;
                 if (warp == 4) TRACE(2, 5);
-                const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
-                // tpr threads of one warp share a row: each folds every tpr-th partial, then shuffles
-                int tpr = 32;
-                while (tpr * R > 128 * CG) tpr >>= 1;
-                const int r = tid_s / tpr, sub = tid_s - r * tpr;
-                float M = kNegBig, Ls = 0.f;
-                if (r < R) {
-                    for (int k0 = sub; k0 < p.cph; k0 += 8 * tpr) {  // batches of 8 independent loads
-                        float2 x[8];
+                if (!LP) {  // many CTAs per head: too many partials for one warp, all softmax threads fold them
+                    if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 33);
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
+                    if (!ok) break;
+                    const float2* src = p.ml_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R;
+                    // tpr threads of one warp share a row: each folds every tpr-th partial, then shuffles
+                    int tpr = 32;
+                    while (tpr * R > 128 * CG) tpr >>= 1;
+                    const int r = tid_s / tpr, sub = tid_s - r * tpr;
+                    float M = kNegBig, Ls = 0.f;
+                    if (r < R) {
+                        for (int k0 = sub; k0 < p.cph; k0 += 8 * tpr) {  // batches of 8 independent loads
+                            float2 x[8];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            x[u] = (k0 + u * tpr < p.cph) ? __ldcg(src + (int64_t)(k0 + u * tpr) * R + r)
-                                                          : make_float2(kNegBig, 0.f);
+                            for (int u = 0; u < 8; ++u)
+                                x[u] = (k0 + u * tpr < p.cph) ? __ldcg(src + (int64_t)(k0 + u * tpr) * R + r)
+                                                              : make_float2(kNegBig, 0.f);
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const float Mn = fmaxf(M, x[u].x);
-                            Ls = Ls * ex2(M - Mn) + x[u].y * ex2(x[u].x - Mn);
-                            M = Mn;
+                            for (int u = 0; u < 8; ++u) {
+                                const float Mn = fmaxf(M, x[u].x);
+                                Ls = Ls * ex2(M - Mn) + x[u].y * ex2(x[u].x - Mn);
+                                M = Mn;
+                            }
+                        }
+                    }
+                    for (int o = tpr >> 1; o > 0; o >>= 1) {
+                        const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
+                        const float L2 = __shfl_xor_sync(0xffffffffu, Ls, o);
+                        const float Mn = fmaxf(M, M2);
+                        Ls = Ls * ex2(M - Mn) + L2 * ex2(M2 - Mn);
+                        M = Mn;
+                    }
+                    if (sub == 0 && r < R) {
+                        const float lse2 = M + log2f(Ls);
+                        lse_s[r] = lse2;
+                        const float loc = loc_s[r];
+                        fac_s[r] = loc < 1.0e29f ? ex2(loc - lse2) : 0.f;  // local -> global normaliser
+                        if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
+                            const int j = r / G, g = r - j * G;
+                            const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
+                            p.a.lse[row] = lse2 * 0.69314718055994530942f;
                         }
                     }
                 }
-                for (int o = tpr >> 1; o > 0; o >>= 1) {
-                    const float M2 = __shfl_xor_sync(0xffffffffu, M, o);
-                    const float L2 = __shfl_xor_sync(0xffffffffu, Ls, o);
-                    const float Mn = fmaxf(M, M2);
-                    Ls = Ls * ex2(M - Mn) + L2 * ex2(M2 - Mn);
-                    M = Mn;
-                }
-                if (sub == 0 && r < R) {
-                    const float lse2 = M + log2f(Ls);
-                    lse_s[r] = lse2;
-                    const float loc = loc_s[r];
-                    fac_s[r] = loc < 1.0e29f ? ex2(loc - lse2) : 0.f;  // local -> global normaliser
-                    if (rank == p.cph - 1 && p.a.lse) {  // the last rank always owns at least one tile
-                        const int j = r / G, g = r - j * G;
-                        const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
-                        p.a.lse[row] = lse2 * 0.69314718055994530942f;
-                    }
-                }
-                ok = group_sync(B.sm_sync, sync_n, ctl, 22);
+                ok = group_sync(B.sm_sync, sync_n, ctl, 22);  // every warp is done with the P V pass
                 if (!ok) break;
                 tc_fence_after();  // the P~ stores of the other warps, ordered by the barrier
                 if (warp == 4) TRACE(2, 6);
@@ -730,6 +795,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st;
                 }
             }
+            else {
+                ok = mbar_wait(B.lse_ready, unit & 1, ctl, 32);  // keeps step with the publisher warp (see there)
+                if (!ok) break;
+            }
             if (warp == 4) TRACE(2, 7);
             // ---- this unit's accumulator: rescale and hand to the reducers ----
             ok = epilogue(unit, nonempty);
@@ -748,11 +817,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
-template <int NC, int CG>
+template <int NC, int CG, bool LP>
 int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    auto kern = verify_cached_kernel<NC, CG>;
+    auto kern = verify_cached_kernel<NC, CG, LP>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -788,15 +857,24 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
 int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                   int grid, size_t smem_bytes, cudaStream_t stream)
 {
+    const bool lp = fp.cph <= kLsePubMax;
     switch (fp.N) {  // (columns per warpgroup, warpgroups)
-        case 16: return launch_cfg<8, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 32: return launch_cfg<8, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 48: return launch_cfg<16, 3>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 64: return launch_cfg<16, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 80: return launch_cfg<40, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 96: return launch_cfg<24, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 112: return launch_cfg<56, 2>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 128: return launch_cfg<32, 4>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 16: return lp ? launch_cfg<8, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<8, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 32: return lp ? launch_cfg<8, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<8, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 48: return lp ? launch_cfg<16, 3, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<16, 3, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 64: return lp ? launch_cfg<16, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<16, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 80: return lp ? launch_cfg<40, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<40, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 96: return lp ? launch_cfg<24, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<24, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 112: return lp ? launch_cfg<56, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<56, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        case 128: return lp ? launch_cfg<32, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
+                              : launch_cfg<32, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
         default: return SPEC_ERR_UNSUPPORTED_SHAPE;
     }
 }
