@@ -1,0 +1,72 @@
+"""Randomised shapes through the whole path (verify + statistic, select, draft) against the oracle.
+
+Every case draws batch, head counts, head dimension, ragged context lengths, speculation length,
+page layout, layer count and budget from a seeded generator; the draws are bounded so that the
+oracle finishes each case in about a second.  The fixed lists in test_gpu_parity.py aim at known
+edges; this file looks for the ones nobody thought of (ragged batches with units that are empty
+for some CTAs, odd group sizes, budgets around the cluster and round boundaries)."""
+import random
+
+import pytest
+import torch
+
+import oracle
+from paper_2607_27735_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-3
+
+
+def draw_shape(seed):
+    rng = random.Random(9176 + 31 * seed)
+    n_kv = rng.choice([1, 2, 4, 8])
+    group = rng.choice([1, 2, 4, 5, 8])
+    n_q = rng.choice([1, 2, 3, 5, 7, 9, 12, 17])
+    while n_q * group > 96:  # the tcgen05 path takes up to 96 rows per KV head, the rest falls back: keep both in play
+        n_q = max(1, n_q // 2)
+    batch = rng.choice([1, 1, 2, 3])
+    hi = rng.choice([200, 900, 2500])
+    lo = rng.choice([n_q, hi // 4, hi])
+    page = rng.choice([0, 0, 16, 64, 128])
+    k_recent = rng.choice([0, 8, 64])
+    k_sink = rng.choice([0, 4])
+    k_total = k_sink + k_recent + rng.choice([16, 100, 300, 1200])
+    return dict(ctx=(max(lo, n_q), max(hi, n_q)), n_q=n_q, n_q_heads=n_kv * group, n_kv_heads=n_kv,
+                head_dim=rng.choice([64, 128, 128]), batch=batch, n_layers=rng.choice([1, 2]),
+                page_size=page, shuffled_pages=page > 0 and rng.random() < 0.7,
+                k_total=k_total, k_sink=k_sink, k_recent=k_recent, draft_steps=rng.choice([1, 3]),
+                planted=rng.choice([0, 3]), kv_dist=rng.choice(["normal", "normal", "student_t3"]),
+                seed=100 + seed)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shape_end_to_end(seed):
+    shape = draw_shape(seed)
+    if shape["planted"] == 0:
+        shape.update(q_mode="iid", q_std=0.3)
+    cfg = inputs.small_config(name=f"fuzz{seed}", **shape)
+    case = inputs.make_case(cfg, device="cuda")
+    kv, ctx = case.kv, case.ctx_len
+    # verify + statistic
+    out, lse, stats, ws = binding.spec_verify_attn(kv, case.q_verify, ctx, int(ctx.max()))
+    assert binding.read_status(ws) == 0, shape
+    o_out, o_lse, o_stats = oracle.verify_attn(kv.cpu(), case.q_verify.cpu(), ctx.cpu(), 16, stats.shape[-1])
+    assert (out.cpu().double() - o_out).abs().max().item() <= TOL, shape
+    assert (lse.cpu().double() - o_lse).abs().max().item() <= TOL, shape
+    for b in range(cfg.batch):
+        T = int(ctx[b])
+        assert (stats[:, b, :, :T].cpu().double() - o_stats[:, b, :, :T]).abs().max().item() <= TOL, shape
+    # select: bit-exact on the GPU's own statistic
+    idx, n = binding.spec_select_recall(stats, ctx, cfg.k_sink, cfg.k_recent, cfg.k_total)
+    o_idx, o_n = oracle.select_recall(stats.cpu(), ctx.cpu(), cfg.k_sink, cfg.k_recent, cfg.k_total)
+    assert torch.equal(idx.cpu(), o_idx) and torch.equal(n.cpu(), o_n), shape
+    # draft over that index, every drafting step
+    for step in range(cfg.draft_steps):
+        cur = ctx + step + 1
+        q = case.q_draft[step].contiguous()
+        d_out, d_lse, wd = binding.spec_sparse_draft_attn(kv, q, idx, n, ctx, cur, step + 1)
+        assert binding.read_status(wd) == 0, shape
+        r_out, r_lse = oracle.sparse_draft_attn(kv.cpu(), q.cpu(), idx.cpu(), n.cpu(), ctx.cpu(), cur.cpu())
+        assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL, shape
+        fin = torch.isfinite(r_lse)
+        assert ((d_lse.cpu().double() - r_lse)[fin]).abs().max().item() <= TOL, shape
