@@ -161,6 +161,8 @@ int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers
  *              memset): zero it once after allocation; an error stays until
  *              spec_read_status() returns it.
  * An index outside [0, cur_len[b]) is skipped and sets SPEC_ERR_BAD_INDEX in the status word.
+ * The one device-side wait (the first CTA of a cluster waiting for the partial results of the
+ * others) is bounded; if it runs out the status word gets SPEC_ERR_TIMEOUT.
  * A problem with an empty key set yields out = 0, lse = -inf.
  */
 int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* indices,

@@ -7,12 +7,16 @@
 // of the head were seen.  Instead of sweeping K twice, every CTA keeps the score tiles
 // S^T = K Q^T of its share of the keys in tensor memory (512 columns per SM hold the output
 // accumulator plus (512 - 2N) / N tiles of 128 keys x N rows):
-//   P1  stream K, S^T tile -> TMEM (kept), per-row running (max, sum) -> partial LSE;
-//   --  partials of the CTAs sharing the head are combined into the row LSE (the only
-//       cross-CTA dependency; V tiles keep streaming into shared memory meanwhile);
-//   P2  stream V, P = exp2(S - LSE) from the cached tile, exactly normalised: column sums ->
-//       stats, O^T += V^T [P_hi | P_lo]^T on the tensor cores (bf16 hi + lo split of P keeps
-//       the 2e-3 bar when one key takes most of the mass).
+//   P1   stream K, S^T tile -> TMEM (kept), per-row running (max, sum) -> this CTA's partial,
+//        published to the CTAs that share the head;
+//   P2a  stream V, P~ = exp2(S - lse_local) from the cached tile (needs nothing from other CTAs,
+//        so the exchange of the partials hides behind it): O^T += V^T [P~_hi | P~_lo]^T on the
+//        tensor cores (bf16 hi + lo split of P~ keeps the 2e-3 bar when one key takes most of the
+//        mass); P~ replaces the scores in tensor memory;
+//   --   the partials of the head's CTAs are combined into the row LSE (the only cross-CTA
+//        dependency), by the publisher warp during P2a when few CTAs share the head;
+//   P2b  cached P~ weighted per row with exp2(lse_local - LSE): column sums -> stats;
+//   --   the accumulator, rescaled per row the same way, is this CTA's partial output.
 // A unit (a group of KV heads of one (layer, sequence)) is cut so that a CTA's share of keys
 // fits the cache; larger shares go to the two-sweep variant.
 //
@@ -20,9 +24,9 @@
 // one thread owns one key: the statistic is a thread-local sum and the P1 row max/sum is
 // thread-local state reduced once per unit.
 //
-// Roles (384 threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer (+ TMEM alloc), warps
-// 2..3 reduce the per-CTA O partials (fixed order: deterministic), warps 4..11 two softmax
-// warpgroups that split the columns.
+// Roles (128 + 128 CG threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer (+ TMEM alloc),
+// warp 2 publisher (fences, counters, LSE combine), warp 3 reduces the per-CTA O partials (fixed
+// order: deterministic), warps 4.. CG softmax warpgroups that split the columns.
 //
 // All CTAs must be co-resident (they wait on each other's partials): the grid never exceeds
 // the SM count at one CTA per SM and the launch is cooperative.  Every wait is bounded; on
