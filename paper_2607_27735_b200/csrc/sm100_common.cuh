@@ -37,7 +37,29 @@ struct FastParams {
     int q_bufs;                       // Q buffers in shared memory (cached variant: 1)
     long long* trace;
     int dbg;                          // development knobs (trace builds only)
+    // divisions of get_seg() as multiply-high + shift (x / d = umulhi(x, mul) >> sh for 0 <= x < 2^31;
+    // sh < 0 marks d == 1): by units per layer, by head groups per sequence, by CTAs per head
+    uint32_t div_mul[3];
+    int32_t div_sh[3];
 };
+
+// Host side: magic numbers of an exact division by d >= 1 (see FastParams::div_mul).
+inline void set_divisor(FastParams* p, int which, int d)
+{
+    if (d <= 1) {
+        p->div_mul[which] = 0;
+        p->div_sh[which] = -1;
+        return;
+    }
+    int c = 0;
+    while ((1ull << c) < (unsigned)d) ++c;
+    p->div_mul[which] = (uint32_t)(((1ull << (31 + c)) + d - 1) / d);
+    p->div_sh[which] = c - 1;
+}
+__device__ __forceinline__ int fast_div(const FastParams& p, int which, int x)
+{
+    return p.div_sh[which] < 0 ? x : (int)(__umulhi((uint32_t)x, p.div_mul[which]) >> p.div_sh[which]);
+}
 
 // ---------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -243,14 +265,14 @@ __device__ __forceinline__ Seg get_seg(const FastParams& p, int unit, int head_l
 {
     Seg s;
     const int per_layer = p.a.kv.batch * p.NHG;
-    s.layer = unit / per_layer;
+    s.layer = fast_div(p, 0, unit);
     const int rem = unit - s.layer * per_layer;
-    s.b = rem / p.NHG;
+    s.b = fast_div(p, 1, rem);
     s.h = (rem - s.b * p.NHG) * p.HG + head_local;
     s.T = p.a.ctx_len[s.b];
     const int nb = (s.T + kTile - 1) / kTile;
-    s.t0 = (int)((int64_t)rank * nb / p.cph);
-    s.t1 = (int)((int64_t)(rank + 1) * nb / p.cph);
+    s.t0 = fast_div(p, 2, rank * nb);        // rank < SMs, nb < 2^20: the products stay far below 2^31
+    s.t1 = fast_div(p, 2, (rank + 1) * nb);
     s.prob = ((int64_t)s.layer * p.a.kv.batch + s.b) * p.a.kv.n_kv_heads + s.h;
     return s;
 }

@@ -218,6 +218,9 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.HG = pl.HG;
     fp.NHG = a.kv.n_kv_heads / pl.HG;
     fp.cph = pl.cph;
+    set_divisor(&fp, 0, a.kv.batch * fp.NHG);
+    set_divisor(&fp, 1, fp.NHG);
+    set_divisor(&fp, 2, fp.cph);
     fp.n_units = pl.n_units;
     fp.N = pl.N;
     fp.R = a.n_q * G;
