@@ -38,9 +38,10 @@ struct FastParams {
     long long* trace;
     int dbg;                          // development knobs (trace builds only)
     // divisions of get_seg() as multiply-high + shift (x / d = umulhi(x, mul) >> sh for 0 <= x < 2^31;
-    // sh < 0 marks d == 1): by units per layer, by head groups per sequence, by CTAs per head
-    uint32_t div_mul[3];
-    int32_t div_sh[3];
+    // sh < 0 marks d == 1): by units per layer, by head groups per sequence, by CTAs per head, by the
+    // group size G
+    uint32_t div_mul[4];
+    int32_t div_sh[4];
 };
 
 // Host side: magic numbers of an exact division by d >= 1 (see FastParams::div_mul).

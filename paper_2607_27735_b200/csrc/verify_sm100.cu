@@ -221,6 +221,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     set_divisor(&fp, 0, a.kv.batch * fp.NHG);
     set_divisor(&fp, 1, fp.NHG);
     set_divisor(&fp, 2, fp.cph);
+    set_divisor(&fp, 3, a.kv.n_q_heads / a.kv.n_kv_heads);
     fp.n_units = pl.n_units;
     fp.N = pl.N;
     fp.R = a.n_q * G;

@@ -63,7 +63,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     constexpr int kSW = 4 * CG;                  // softmax warps
     const int N = p.N, R = p.R, G = p.G;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int head_local = blockIdx.x / p.cph, rank = blockIdx.x % p.cph;
+    const int head_local = fast_div(p, 2, blockIdx.x), rank = blockIdx.x - head_local * p.cph;
     const int q_bytes = N * 256;                       // one Q buffer: 2 halves x N rows x 128 B
     const int p_bytes = 2 * N * 256;                   // one P buffer: [hi | lo] rows, 8-row blocks x 128 keys x 16 B
 
@@ -442,7 +442,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             TRACE(3, 1);
             const Seg sg = get_seg(p, unit, head_local, rank);
             const int E4 = R * kD / 4;
-            const int lo = (int)((int64_t)rank * E4 / p.cph), hi = (int)((int64_t)(rank + 1) * E4 / p.cph);
+            const int lo = fast_div(p, 2, rank * E4), hi = fast_div(p, 2, (rank + 1) * E4);  // products far below 2^31
             const float4* src = reinterpret_cast<const float4*>(
                 p.o_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R * kD);
             for (int e = lo + tid; e < hi; e += 32) {
