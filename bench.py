@@ -315,7 +315,8 @@ def run_gpu(args):
         "data": "synthetic", "config": config_json(cfg, world),
         "phases_us": {"verify": phase_ms[0] * 1e3, "select": phase_ms[1] * 1e3,
                       "draft": phase_ms[2] * 1e3},
-        "verify_impl": {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache"}.get(
+        "verify_impl": {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
+                        5: "tcgen05 score-cache, rows in two passes"}.get(
             binding.last_verify_impl()),
         "roofline": {
             "kernel": "verification attention + Eq.3 statistic (per-layer launch)",

@@ -62,7 +62,9 @@ enum {
     SPEC_VERIFY_GENERIC = 1,          /* plain FP32 CUDA-core kernels, every supported shape */
     SPEC_VERIFY_TCGEN05 = 2,          /* tcgen05, either variant; unsupported shapes are an error */
     SPEC_VERIFY_TCGEN05_TWOSWEEP = 3, /* K swept twice (second sweep from L2), any context length */
-    SPEC_VERIFY_TCGEN05_CACHED = 4    /* score tiles cached in tensor memory, K and V read once */
+    SPEC_VERIFY_TCGEN05_CACHED = 4,   /* score tiles cached in tensor memory, K and V read once */
+    SPEC_VERIFY_TCGEN05_CACHED_2PASS = 5 /* reported only (spec_last_verify_impl): AUTO ran the score-cache kernel
+                                            on two halves of the rows because all rows did not fit the cache */
 };
 
 /*
@@ -217,7 +219,8 @@ int spec_read_status(const void* workspace, void* cuda_stream);
 int spec_set_verify_impl(int impl);
 
 /* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC,
- * SPEC_VERIFY_TCGEN05_TWOSWEEP or SPEC_VERIFY_TCGEN05_CACHED; 0 before the first call). */
+ * SPEC_VERIFY_TCGEN05_TWOSWEEP, SPEC_VERIFY_TCGEN05_CACHED or SPEC_VERIFY_TCGEN05_CACHED_2PASS; 0 before the
+ * first call). */
 int spec_last_verify_impl(void);
 
 /* Number of kernels this library has launched since load (host-side counter). */

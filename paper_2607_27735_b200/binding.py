@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libspec_attn.so")
 
 WS_VERIFY, WS_SELECT, WS_DRAFT = 0, 1, 2
 VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCGEN05_CACHED = 0, 1, 2, 3, 4
+VERIFY_TCGEN05_CACHED_2PASS = 5  # reported by last_verify_impl() only: the score-cache kernel on two halves of the rows
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",

@@ -109,7 +109,9 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
         int used = 0;
         const int rc2 = verify_sm100_launch(a, sm100_variant(impl), stream, &used);
         if (rc2 == SPEC_OK) {
-            g_last_verify_impl.store(used == 2 ? SPEC_VERIFY_TCGEN05_CACHED : SPEC_VERIFY_TCGEN05_TWOSWEEP);
+            g_last_verify_impl.store(used == 3   ? SPEC_VERIFY_TCGEN05_CACHED_2PASS
+                                     : used == 2 ? SPEC_VERIFY_TCGEN05_CACHED
+                                                 : SPEC_VERIFY_TCGEN05_TWOSWEEP);
             return SPEC_OK;
         }
         // an explicit tcgen05 request fails loudly; AUTO falls through to the generic kernels only

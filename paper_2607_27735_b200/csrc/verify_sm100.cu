@@ -181,6 +181,52 @@ bool encode_q_map(CUtensorMap* map, const void* q, const KvView& kv, int n_q, in
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// ---- rows in two passes ----------------------------------------------------------------------
+// A single (layer, sequence) whose n_q * G rows do not fit the score cache at its context length
+// (many speculated rows at a very long context) is verified as two calls of the score-cache kernel:
+// rows [0, nA) against the context shortened by the nB rows that follow them, then rows [nA, n_q)
+// against the whole context.  Both are ordinary causal verifications of the same cache; their
+// statistics add up (the window rule is applied to each part's own rows).  K and V are read
+// twice, which still beats the two-sweep kernel at these shapes.
+struct SplitPlan {
+    int nA, nB;
+    size_t main_bytes, ctx_off, stat_off, total;
+    int64_t stat_stride;
+};
+
+bool make_split_plan(const KvView& kv, int n_q, int max_ctx_len, SplitPlan* sp)
+{
+    if (kv.n_layers * kv.batch != 1 || n_q < 2) return false;
+    Plan full;
+    if (make_plan(kv, n_q, max_ctx_len, 2, &full)) return false;  // fits in one pass
+    sp->nA = (n_q + 1) / 2;
+    sp->nB = n_q - sp->nA;
+    Plan pa, pb;
+    if (!make_plan(kv, sp->nA, max_ctx_len, 2, &pa) || !make_plan(kv, sp->nB, max_ctx_len, 2, &pb)) return false;
+    sp->main_bytes = pa.total > pb.total ? pa.total : pb.total;
+    sp->ctx_off = sp->main_bytes;
+    sp->stat_off = sp->ctx_off + 256;
+    sp->stat_stride = ((int64_t)max_ctx_len + 63) / 64 * 64;
+    sp->total = sp->stat_off + (size_t)kv.n_kv_heads * sp->stat_stride * sizeof(float);
+    sp->total = (sp->total + 255) & ~(size_t)255;
+    return true;
+}
+
+__global__ void shorten_ctx_kernel(const int32_t* ctx_len, int by, int32_t* out) { out[0] = ctx_len[0] - by; }
+
+// stats <- (first part's value where it wrote one) + second part's value
+__global__ void add_stats_kernel(float* stats, int64_t stat_stride, const float* second, int64_t second_stride,
+                                 const int32_t* ctx_len, int nB, int n_kv_heads)
+{
+    const int T = ctx_len[0];
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < (int64_t)n_kv_heads * T;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int h = (int)(i / T), key = (int)(i - (int64_t)h * T);
+        const float first = key < T - nB ? stats[h * stat_stride + key] : 0.f;
+        stats[h * stat_stride + key] = first + second[h * second_stride + key];
+    }
+}
+
 }  // namespace
 
 bool verify_sm100_supported(const KvView& kv, int n_q, int variant)
@@ -198,11 +244,47 @@ size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
         Plan pl;
         if (make_plan(kv, n_q, max_ctx_len, variant, &pl) && pl.total > best) best = pl.total;
     }
+    SplitPlan sp;
+    if (make_split_plan(kv, n_q, max_ctx_len, &sp) && sp.total > best) best = sp.total;
     return best;
 }
 
 int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant)
 {
+    SplitPlan sp;
+    if (variant == 0 && make_split_plan(a.kv, a.n_q, a.max_ctx_len, &sp)) {
+        if (a.workspace_bytes < sp.total) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+        char* ws = static_cast<char*>(a.workspace);
+        int32_t* ctx_a = reinterpret_cast<int32_t*>(ws + sp.ctx_off);
+        float* second = reinterpret_cast<float*>(ws + sp.stat_off);
+        const int64_t row_elems = (int64_t)a.kv.n_q_heads * a.kv.head_dim;
+        shorten_ctx_kernel<<<1, 1, 0, stream>>>(a.ctx_len, sp.nB, ctx_a);
+        count_launch(1);
+        VerifyArgs pa = a;  // rows [0, nA): the context ends where the other rows begin
+        pa.n_q = sp.nA;
+        pa.ctx_len = ctx_a;
+        pa.first_stat_row = a.first_stat_row < sp.nA ? a.first_stat_row : sp.nA;
+        pa.workspace_bytes = sp.main_bytes;
+        int rc = verify_sm100_launch(pa, 2, stream, nullptr);
+        if (rc != SPEC_OK) return rc;
+        VerifyArgs pb = a;  // rows [nA, n_q) against the whole context; their statistic goes to scratch
+        pb.n_q = sp.nB;
+        pb.q = a.q + sp.nA * row_elems;
+        pb.out = a.out + sp.nA * row_elems;
+        pb.lse = a.lse ? a.lse + (int64_t)sp.nA * a.kv.n_q_heads : nullptr;
+        pb.first_stat_row = a.first_stat_row > sp.nA ? a.first_stat_row - sp.nA : 0;
+        pb.stats = second;
+        pb.stat_stride = sp.stat_stride;
+        pb.workspace_bytes = sp.main_bytes;
+        rc = verify_sm100_launch(pb, 2, stream, nullptr);
+        if (rc != SPEC_OK) return rc;
+        add_stats_kernel<<<sm_count(), 256, 0, stream>>>(a.stats, a.stat_stride, second, sp.stat_stride, a.ctx_len, sp.nB,
+                                                         a.kv.n_kv_heads);
+        count_launch(1);
+        if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+        if (used_variant) *used_variant = 3;
+        return SPEC_OK;
+    }
     Plan pl;
     if (!make_plan(a.kv, a.n_q, a.max_ctx_len, variant, &pl)) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.workspace_bytes < pl.total) return SPEC_ERR_WORKSPACE_TOO_SMALL;

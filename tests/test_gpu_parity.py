@@ -119,6 +119,24 @@ def test_verify_stat_window(window):
     assert (mass - cfg.group * min(window, 9)).abs().max() < 1e-2
 
 
+@pytest.mark.parametrize("shape,window", [
+    (dict(ctx=(40000, 40000), n_q=32, n_q_heads=4, n_kv_heads=1, planted=0.001), 16),  # 128 rows x 313 tiles: over the cache
+    (dict(ctx=(77000, 77000), n_q=17, n_q_heads=4, n_kv_heads=1, planted=0.001), 16),  # 9 + 8 rows, window drops row 0
+    (dict(ctx=(77000, 77000), n_q=17, n_q_heads=4, n_kv_heads=1, planted=0.001), 4),   # window inside the second pass only
+    (dict(ctx=(40100, 40100), n_q=31, n_q_heads=4, n_kv_heads=1, page_size=64, shuffled_pages=True, planted=0.001), 20),
+])
+def test_verify_rows_in_two_passes(shape, window):
+    """One (layer, sequence) whose rows do not fit the score cache: AUTO verifies the two halves of
+    the rows separately with the score-cache kernel and adds their statistics."""
+    cfg = inputs.small_config(**shape)
+    case = inputs.make_case(cfg, device="cuda")
+    _, _, stats = check_verify(case, stat_window=window)
+    assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED_2PASS
+    T = int(case.ctx_len[0])
+    mass = stats[0, 0, :, :T].sum(-1)
+    assert (mass - cfg.group * min(window, cfg.n_q)).abs().max() < 1e-2
+
+
 def test_verify_is_deterministic_and_leaves_padding_untouched():
     cfg = inputs.small_config(ctx=(300, 1000), batch=2, n_q=5, planted=0, q_mode="iid")
     case = inputs.make_case(cfg, device="cuda")
