@@ -28,9 +28,9 @@
 // warp 2 publisher (fences, counters, LSE combine), warp 3 reduces the per-CTA O partials (fixed
 // order: deterministic), warps 4.. CG softmax warpgroups that split the columns.
 //
-// All CTAs must be co-resident (they wait on each other's partials): the grid never exceeds
-// the SM count at one CTA per SM and the launch is cooperative.  Every wait is bounded; on
-// expiry the kernel records SPEC_ERR_TIMEOUT in the status word and drains.
+// All CTAs must become co-resident (they wait on each other's partials): the grid never exceeds
+// the SM count at one CTA per SM (see the launcher).  Every wait is bounded; on expiry the kernel
+// records SPEC_ERR_TIMEOUT in the status word and drains.
 #include "sm100_common.cuh"
 
 namespace spec {
@@ -833,19 +833,25 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
     cfg.blockDim = dim3(128 + 128 * CG);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeCooperative;  // all CTAs must be co-resident: they wait on each other
-    attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    // All CTAs must become co-resident (they wait on each other's partials).  The grid never exceeds
+    // the SM count at one CTA per SM, so that follows as soon as the previous kernel's CTAs have left:
+    // the launch only asks for programmatic stream serialisation, which lets each CTA take an SM the
+    // moment the previous layer's CTA on it exits (a cooperative launch would wait for the whole
+    // previous grid first: 1.4 us per layer).  A CTA whose peers cannot become resident (SMs held by
+    // an unrelated long kernel) ends in SPEC_ERR_TIMEOUT like any other stall.  If the driver refuses
+    // the attribute the launch falls back to a cooperative one.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static bool pdl_ok = true;  // a driver that refuses the combination is asked only once
-    cfg.numAttrs = pdl_ok ? 2 : 1;
-    cudaError_t err = cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp);
-    if (err != cudaSuccess && cfg.numAttrs == 2) {
-        cudaGetLastError();
+    cfg.numAttrs = 1;
+    static bool pdl_ok = true;  // a driver that refuses it is asked only once
+    cudaError_t err = pdl_ok ? cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp) : cudaErrorNotSupported;
+    if (err != cudaSuccess) {
+        if (pdl_ok) cudaGetLastError();
         pdl_ok = false;
-        cfg.numAttrs = 1;
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
         err = cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp);
     }
     if (err != cudaSuccess) {
