@@ -115,6 +115,32 @@ class SpecStepRunner:
         if events is not None:
             events[3].record()
 
+    def replay_host_io(self, q_verify_host, q_draft_host, out_v_host, out_d_host):
+        """One captured step fed from and drained to pinned host buffers.  The copies that a phase
+        does not wait for travel on a second stream: the drafting Q arrives under the verification
+        phase, the verification outputs leave under selection and drafting.  Every copy of the step
+        is finished (in stream order) when the current stream reaches the end of this call."""
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_side"):
+            self._side = torch.cuda.Stream()
+        side = self._side
+        self.q_verify.copy_(q_verify_host, non_blocking=True)
+        side.wait_stream(main)  # the previous step's drafting phase has read q_draft
+        with torch.cuda.stream(side):
+            self.q_draft.copy_(q_draft_host, non_blocking=True)
+            q_draft_in = side.record_event()
+        self.graphs[0].replay()
+        verified = main.record_event()
+        with torch.cuda.stream(side):
+            side.wait_event(verified)
+            out_v_host.copy_(self.out_v, non_blocking=True)
+            out_v_gone = side.record_event()
+        self.graphs[1].replay()
+        main.wait_event(q_draft_in)
+        self.graphs[2].replay()
+        out_d_host.copy_(self.out_d, non_blocking=True)
+        main.wait_event(out_v_gone)
+
     # -- algorithmic bytes (what the method must move) ---------------------------------------
     def verify_kv_bytes_per_layer(self) -> int:
         kv = self.kv

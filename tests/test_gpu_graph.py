@@ -72,3 +72,29 @@ def test_graph_replay_with_changing_lengths(shape):
         r_out, r_lse = oracle.sparse_draft_attn(kv.cpu(), q_d.cpu(), idx.cpu(), n_idx.cpu(), ctx.cpu(), cur.cpu())
         assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL
         assert (d_lse.cpu().double() - r_lse).abs().max().item() <= TOL
+
+
+def test_runner_step_with_host_buffers_matches_the_resident_step():
+    """runner.replay_host_io overlaps the host copies with the phases on a second stream; the
+    bytes that come back must be those of the plain replay, step after step."""
+    import dataclasses
+
+    from paper_2607_27735_b200 import runner
+    cfg = dataclasses.replace(inputs.baseline_configs()["cfg2_8b_32k"], n_layers=2, ctx=(4096, 4096))
+    case = inputs.make_case(cfg, device="cuda")
+    run = runner.SpecStepRunner(case)
+    run.capture()
+    run.replay()
+    torch.cuda.synchronize()
+    ref_v, ref_d = run.out_v.cpu(), run.out_d.cpu()
+    qv, qd = case.q_verify.cpu().pin_memory(), case.q_draft.cpu().pin_memory()
+    ov = torch.empty(run.out_v.shape).pin_memory()
+    od = torch.empty(run.out_d.shape).pin_memory()
+    run.q_verify.zero_()
+    run.q_draft.zero_()
+    for _ in range(3):
+        ov.zero_()
+        od.zero_()
+        run.replay_host_io(qv, qd, ov, od)
+        torch.cuda.synchronize()
+        assert torch.equal(ov, ref_v) and torch.equal(od, ref_d)
