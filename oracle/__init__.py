@@ -19,15 +19,17 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "spec_oracle.c")
+_SRC_CTRL = os.path.join(_HERE, "controller_oracle.c")
 _LIB = os.path.join(_HERE, "libspec_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP over the independent (layer, batch, KV head) problems)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_CTRL))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, _SRC_CTRL, "-lm"]
         )
     return _LIB
 
@@ -157,3 +159,54 @@ def sparse_draft_attn(kv, q, indices, n_idx, tail_start, cur_len):
         raise ValueError("oracle_sparse_draft_attn: invalid arguments")
     del keep
     return out, lse
+
+
+# ---- entropy-guided length controller (controller_oracle.c) ------------------------------------
+
+
+def token_entropy(logits):
+    """Shannon entropy (nats) of softmax(logits[r, :]) per row; fp32 or bf16 CPU tensor ``[rows, V]``
+    (rows may be strided).  Returns fp64 ``[rows]``."""
+    lib = _load()
+    assert logits.dim() == 2 and logits.stride(1) == 1 and not logits.is_cuda
+    dtype = {torch.float32: 0, torch.bfloat16: 1}[logits.dtype]
+    n_rows, vocab = logits.shape
+    out = torch.zeros(n_rows, dtype=torch.float64)
+    rc = lib.oracle_token_entropy(
+        ctypes.c_void_p(logits.data_ptr()), ctypes.c_int(dtype), ctypes.c_int(n_rows), ctypes.c_int(vocab),
+        ctypes.c_int64(logits.stride(0)), ctypes.c_void_p(out.data_ptr()))
+    if rc != 0:
+        raise ValueError("oracle_token_entropy: invalid arguments")
+    return out
+
+
+def controller_update(state, entropy, n_accepted, beta):
+    """Eq. "ema": returns the new (mean accepted entropy, mean rejected entropy) as fp64 ``[2]``."""
+    lib = _load()
+    state = torch.as_tensor(state, dtype=torch.float64).clone().contiguous()
+    entropy = torch.as_tensor(entropy, dtype=torch.float64).contiguous()
+    rc = lib.oracle_controller_update(
+        ctypes.c_void_p(state.data_ptr()), ctypes.c_void_p(entropy.data_ptr()), ctypes.c_int(entropy.numel()),
+        ctypes.c_int(int(n_accepted)), ctypes.c_double(float(beta)))
+    if rc != 0:
+        raise ValueError("oracle_controller_update: invalid arguments")
+    return state
+
+
+def controller_select(state, entropy, cand, c_d, c_v):
+    """Eq. "prob" + Eq. "optimal_k": returns ``(k_star, p fp64 [n], score fp64 [n_cand])``."""
+    lib = _load()
+    state = torch.as_tensor(state, dtype=torch.float64).contiguous()
+    entropy = torch.as_tensor(entropy, dtype=torch.float64).contiguous()
+    cand = torch.as_tensor(cand, dtype=torch.int32).contiguous()
+    k_star = torch.zeros(1, dtype=torch.int32)
+    p = torch.zeros(entropy.numel(), dtype=torch.float64)
+    score = torch.zeros(cand.numel(), dtype=torch.float64)
+    rc = lib.oracle_controller_select(
+        ctypes.c_void_p(state.data_ptr()), ctypes.c_void_p(entropy.data_ptr()), ctypes.c_int(entropy.numel()),
+        ctypes.c_void_p(cand.data_ptr()), ctypes.c_int(cand.numel()), ctypes.c_double(float(c_d)),
+        ctypes.c_double(float(c_v)), ctypes.c_void_p(k_star.data_ptr()), ctypes.c_void_p(p.data_ptr()),
+        ctypes.c_void_p(score.data_ptr()))
+    if rc != 0:
+        raise ValueError("oracle_controller_select: invalid arguments")
+    return int(k_star[0]), p, score

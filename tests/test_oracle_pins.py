@@ -298,3 +298,84 @@ def test_resampled_heavy_hitters_are_recalled_from_the_fresh_statistic():
                 stale = set(prev_idx[0, 0, h].tolist())
                 assert len(planted - stale) > 0  # the drift is visible to a stale index
         prev_idx = idx
+
+
+# ---- entropy-guided length controller -----------------------------------------------------------
+
+
+def test_entropy_closed_forms():
+    """Uniform logits -> ln V; two equal peaks far above the rest -> ln 2; one dominant logit -> 0;
+    adding a constant to a row changes nothing."""
+    V = 1000
+    z = torch.zeros(4, V)
+    z[1, :2] = 80.0
+    z[2, 7] = 200.0
+    z[3] = torch.linspace(-3, 3, V)
+    h = oracle.token_entropy(z)
+    assert abs(h[0].item() - math.log(V)) < 1e-12
+    assert abs(h[1].item() - math.log(2)) < 1e-9
+    assert h[2].item() < 1e-12
+    h_shift = oracle.token_entropy(z + 5.0)
+    assert (h - h_shift).abs().max().item() < 1e-5  # fp32 inputs: the shift itself rounds
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_entropy_matches_library_softmax(dtype):
+    gen = torch.Generator().manual_seed(3)
+    z = (3.0 * torch.randn(5, 4099, generator=gen)).to(dtype)
+    p = torch.softmax(z.double(), dim=-1)
+    ref = -(p * torch.log(p.clamp_min(1e-300))).sum(-1)
+    view = z[:, :4000]  # strided rows
+    p2 = torch.softmax(view.double(), dim=-1)
+    ref2 = -(p2 * torch.log(p2.clamp_min(1e-300))).sum(-1)
+    assert (oracle.token_entropy(z) - ref).abs().max().item() < 1e-10
+    assert (oracle.token_entropy(view) - ref2).abs().max().item() < 1e-10
+
+
+def test_controller_update_and_select_closed_forms():
+    # equal centres => p = 1/2 for every token => expected length 1 + sum 2^-m
+    k_star, p, score = oracle.controller_select([1.0, 1.0], [0.3, 2.0, 5.0, 0.1], [1, 2, 4], 0.1, 1.0)
+    assert (p - 0.5).abs().max().item() < 1e-15
+    want = [(1 + 0.5) / 1.1, (1 + 0.75) / 1.2, (1 + 0.9375) / 1.4]
+    assert max(abs(a - b) for a, b in zip(score.tolist(), want)) < 1e-14
+    assert k_star == 2
+    # entropies on the accepted centre, rejected centre far away => p -> 1: longer is better while C_d < C_v
+    k_star, p, _ = oracle.controller_select([0.5, 40.0], [0.5] * 8, [2, 4, 8], 0.05, 1.0)
+    assert (1 - p).max().item() < 1e-15 and k_star == 8
+    # ... and the other way round: nothing is expected to pass, the shortest candidate wins
+    k_star, p, _ = oracle.controller_select([40.0, 0.5], [0.5] * 8, [2, 4, 8], 0.05, 1.0)
+    assert p.max().item() < 1e-15 and k_star == 2
+    # exact tie (C_d = 0, p = 0): the smaller candidate
+    k_star, _, score = oracle.controller_select([40.0, 0.5], [0.5] * 8, [4, 2], 0.0, 1.0)
+    assert score[0] == score[1] and k_star == 2
+    # Eq. "ema": 3 of 5 accepted
+    s = oracle.controller_update([1.0, 2.0], [0.2, 0.4, 0.6, 3.0, 5.0], 3, 0.9)
+    assert abs(s[0].item() - (0.9 * 1.0 + 0.1 * 0.4)) < 1e-15 and abs(s[1].item() - (0.9 * 2.0 + 0.1 * 4.0)) < 1e-15
+    # an empty class leaves its mean alone
+    s = oracle.controller_update([1.0, 2.0], [0.2, 0.4], 2, 0.5)
+    assert abs(s[0].item() - 0.65) < 1e-15 and s[1].item() == 2.0
+    s = oracle.controller_update([1.0, 2.0], [0.2, 0.4], 0, 0.5)
+    assert s[0].item() == 1.0 and abs(s[1].item() - 1.15) < 1e-15
+
+
+def test_controller_select_against_plain_python():
+    rng = __import__("random").Random(11)
+    for _ in range(50):
+        n = rng.randint(1, 20)
+        ent = [rng.uniform(0, 6) for _ in range(n)]
+        state = [rng.uniform(0, 3), rng.uniform(1, 6)]
+        cand = sorted(rng.sample(range(1, n + 1), rng.randint(1, min(5, n))))
+        c_d, c_v = rng.uniform(0.01, 0.5), rng.uniform(0.5, 2.0)
+        k_star, p, score = oracle.controller_select(state, ent, cand, c_d, c_v)
+        ps = [math.exp(-abs(h - state[0])) / (math.exp(-abs(h - state[0])) + math.exp(-abs(h - state[1]))) for h in ent]
+        best, best_k = -1.0, None
+        for k in cand:
+            exp_len, pref = 1.0, 1.0
+            for i in range(k):
+                pref *= ps[i]
+                exp_len += pref
+            sc = exp_len / (k * c_d + c_v)
+            if sc > best:
+                best, best_k = sc, k
+        assert k_star == best_k
+        assert max(abs(a - b) for a, b in zip(p.tolist(), ps)) < 1e-14
