@@ -200,6 +200,39 @@ size_t spec_noalloc_scratch_bytes(void);
 int spec_noalloc_read_status(void* cuda_stream);
 
 /*
+ * Speculation-length controller (Sec. "Entropy-Based Acceptance Prediction" and "Optimal
+ * Length Selection").  Every pointer except `cuda_stream` is DEVICE memory owned by the
+ * caller; nothing is allocated, nothing synchronises, results stay on the device (a captured
+ * graph can hold all three calls).  Arithmetic is fp32.
+ *
+ * spec_token_entropy: entropy[r] = Shannon entropy in nats of softmax(logits[r, 0:vocab]) at
+ *   temperature 1: the H_i of each drafted token.  dtype 0 = fp32 logits, 1 = bf16 logits; row
+ *   r starts `row_stride` ELEMENTS after row r - 1 (>= vocab).  One pass over the logits.
+ *   Errors: SPEC_ERR_INVALID_ARG (null pointer, vocab < 1, n_rows < 0, stride < vocab, dtype).
+ *
+ * spec_controller_update: Eq. "ema".  entropy[0:k] are the entropies of the k tokens drafted
+ *   in the step that was just verified, *n_accepted (clamped to 0..k) how many of them were
+ *   accepted.  state[0] (tracked mean of accepted tokens) moves to
+ *   beta * state[0] + (1 - beta) * mean(entropy[0:m]) when m > 0; state[1] (rejected tokens)
+ *   likewise with entropy[m:k] when m < k.  Tokens after the first rejection count as rejected.
+ *
+ * spec_controller_select: Eq. "prob" and Eq. "optimal_k".  p_i = e^-|H_i - state[0]| /
+ *   (e^-|H_i - state[0]| + e^-|H_i - state[1]|) for the n <= 256 entropies given;
+ *   score(k) = (1 + sum_{m=1..k} prod_{i<=m} p_i) / (k * c_d + c_v) for each of the n_cand
+ *   candidate lengths cand[c] in 1..n (a candidate outside that range scores -1 and never
+ *   wins); *k_star = the candidate with the largest score, the smaller one on equal scores
+ *   (0 if no candidate is valid).  p_out (n floats) and score_out (n_cand floats) may be NULL.
+ *   Errors: SPEC_ERR_INVALID_ARG, SPEC_ERR_UNSUPPORTED_SHAPE (n > 256).
+ */
+int spec_token_entropy(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                       int64_t row_stride, float* entropy, void* cuda_stream);
+int spec_controller_update(float* state, const float* entropy, int32_t k,
+                           const int32_t* n_accepted, float beta, void* cuda_stream);
+int spec_controller_select(const float* state, const float* entropy, int32_t n,
+                           const int32_t* cand, int32_t n_cand, float c_d, float c_v,
+                           int32_t* k_star, float* p_out, float* score_out, void* cuda_stream);
+
+/*
  * Bytes of workspace entry point `which` needs for this cache description.  n_q and
  * max_ctx_len matter for SPEC_WS_VERIFY, k_total (+ max_tail folded into it by the caller)
  * for SPEC_WS_DRAFT.  Returns 0 on invalid arguments.

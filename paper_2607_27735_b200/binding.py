@@ -23,7 +23,7 @@ EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
     "spec_read_status", "spec_set_verify_impl", "spec_last_verify_impl", "spec_launch_count",
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
-    "spec_noalloc_read_status",
+    "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
 ]
 
 
@@ -69,6 +69,10 @@ def load() -> ctypes.CDLL:
                                                  vp, i64, vp]
         lib.spec_noalloc_scratch_bytes.restype = ctypes.c_size_t
         lib.spec_noalloc_read_status.argtypes = [vp]
+        f32 = ctypes.c_float
+        lib.spec_token_entropy.argtypes = [vp, i32, i32, i32, i64, vp, vp]
+        lib.spec_controller_update.argtypes = [vp, vp, i32, vp, f32, vp]
+        lib.spec_controller_select.argtypes = [vp, vp, i32, vp, i32, f32, f32, vp, vp, vp, vp]
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
         lib.spec_workspace_bytes.restype = ctypes.c_size_t
         lib.spec_read_status.argtypes = [vp, vp]
@@ -224,6 +228,53 @@ def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_t
     if rc != 0:
         raise SpecError(rc, "spec_sparse_draft_attn")
     return out, lse, workspace
+
+
+def spec_token_entropy(logits, entropy=None):
+    """Entropy (nats) of softmax(logits[r]) per row; ``logits`` is [rows, vocab] fp32 or bf16 with a
+    unit inner stride (rows may be strided).  Returns ``entropy`` ([rows] fp32)."""
+    if not logits.is_cuda or logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits: expected a CUDA [rows, vocab] tensor with unit inner stride")
+    if logits.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"logits: expected fp32 or bf16, got {logits.dtype}")
+    rows, vocab = logits.shape
+    if entropy is None:
+        entropy = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    rc = load().spec_token_entropy(logits.data_ptr(), 1 if logits.dtype == torch.bfloat16 else 0, rows, vocab,
+                                   logits.stride(0) if rows > 1 else max(logits.stride(0), vocab),
+                                   _dev(entropy, torch.float32, "entropy"), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_token_entropy")
+    return entropy
+
+
+def spec_controller_update(state, entropy, n_accepted, beta):
+    """Eq. "ema" in place on ``state`` ([2] fp32: accepted mean, rejected mean); ``n_accepted`` is a
+    device int32 scalar tensor."""
+    rc = load().spec_controller_update(_dev(state, torch.float32, "state"), _dev(entropy, torch.float32, "entropy"),
+                                       entropy.numel(), _dev(n_accepted, torch.int32, "n_accepted"), float(beta),
+                                       _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_controller_update")
+    return state
+
+
+def spec_controller_select(state, entropy, cand, c_d, c_v, k_star=None, p=None, score=None):
+    """Eq. "prob" + Eq. "optimal_k"; returns device tensors ``(k_star, p, score)``."""
+    dev = entropy.device
+    if k_star is None:
+        k_star = torch.empty(1, dtype=torch.int32, device=dev)
+    if p is None:
+        p = torch.empty(entropy.numel(), dtype=torch.float32, device=dev)
+    if score is None:
+        score = torch.empty(cand.numel(), dtype=torch.float32, device=dev)
+    rc = load().spec_controller_select(
+        _dev(state, torch.float32, "state"), _dev(entropy, torch.float32, "entropy"), entropy.numel(),
+        _dev(cand, torch.int32, "cand"), cand.numel(), float(c_d), float(c_v), _dev(k_star, torch.int32, "k_star"),
+        _dev(p, torch.float32, "p"), _dev(score, torch.float32, "score"), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_controller_select")
+    return k_star, p, score
 
 
 def read_status(workspace) -> int:

@@ -1,0 +1,273 @@
+// Entropy-guided speculation-length controller (Sec. "Entropy-Based Acceptance Prediction" and
+// "Optimal Length Selection"): the entropy of each drafted token's output distribution, the two
+// tracked class means (Eq. "ema"), the soft acceptance probabilities (Eq. "prob") and the length
+// that maximises the expected tokens per unit cost (Eq. "optimal_k").
+//
+// The entropy is the only part with real data behind it: one pass over rows x vocabulary logits
+// (HBM-bound; 256 KB per row at a 128K vocabulary in bf16).  A row is split over a thread-block
+// cluster when there are few rows, so that a single drafted token still uses several SMs; every
+// thread keeps a running (max, sum e^(z-max), sum e^(z-max) z) and H = max + ln S - T / S.
+// The two controller steps are a handful of scalars: one warp each, results stay in device
+// memory so that a captured graph can branch on them without a host round trip.
+#include <cooperative_groups.h>
+
+#include "spec_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace spec {
+
+namespace {
+
+constexpr int kEntThreads = 512;
+constexpr int kMaxDrafted = 256;  // drafted tokens the controller looks at in one call
+
+struct Mst {  // running maximum, sum of e^(z - m), sum of e^(z - m) * z
+    float m, s, t;
+};
+
+__device__ __forceinline__ Mst merge(const Mst& a, const Mst& b)
+{
+    const float m = fmaxf(a.m, b.m);
+    const float fa = __expf(a.m - m), fb = __expf(b.m - m);
+    return Mst{m, a.s * fa + b.s * fb, a.t * fa + b.t * fb};
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kUnroll = 4;  // 16-byte loads a thread keeps in flight
+
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void fold8(Mst& acc, const float (&z)[8], float cm)
+{
+    const float mn = fmaxf(acc.m, cm), mb = mn * kLog2e;
+    const float f = ex2(fmaf(acc.m, kLog2e, -mb));
+    float s = acc.s * f, t = acc.t * f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float e = ex2(fmaf(z[i], kLog2e, -mb));
+        s += e;
+        t = fmaf(e, z[i], t);
+    }
+    acc = Mst{mn, s, t};
+}
+
+__device__ __forceinline__ void fold1(Mst& acc, float z)
+{
+    const float mn = fmaxf(acc.m, z), mb = mn * kLog2e;
+    const float f = ex2(fmaf(acc.m, kLog2e, -mb)), e = ex2(fmaf(z, kLog2e, -mb));
+    acc = Mst{mn, fmaf(acc.s, f, e), fmaf(acc.t, f, e * z)};
+}
+
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
+{
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+__device__ __forceinline__ void fold_words(Mst& acc, const uint4& w)  // eight bf16 logits
+{
+    const uint32_t mx = bf16x2_max(bf16x2_max(w.x, w.y), bf16x2_max(w.z, w.w));
+    const float z[8] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y),
+                        bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
+    fold8(acc, z, fmaxf(bf16_lo(mx), bf16_hi(mx)));
+}
+
+__device__ __forceinline__ void fold_words(Mst& acc, const float4& a, const float4& b)  // eight fp32 logits
+{
+    const float z[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    fold8(acc, z, fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w))));
+}
+
+template <int DT>
+__device__ __forceinline__ float load_logit(const void* base, int v)
+{
+    return DT == 1 ? __bfloat162float(static_cast<const __nv_bfloat16*>(base)[v]) : static_cast<const float*>(base)[v];
+}
+
+// One cluster (gridDim.x CTAs) per row.  DT = 0: fp32 logits, 1: bf16 logits.
+template <int DT>
+__global__ void __launch_bounds__(kEntThreads) entropy_kernel(const void* __restrict__ logits, int vocab,
+                                                              int64_t row_stride, float* __restrict__ entropy)
+{
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ Mst warp_part[kEntThreads / 32];
+    __shared__ Mst cta_part;
+    const int CS = gridDim.x, rank = blockIdx.x, row = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const char* base = static_cast<const char*>(logits) + (int64_t)row * row_stride * (DT == 1 ? 2 : 4);
+    Mst acc{-3.0e38f, 0.f, 0.f};
+    if ((reinterpret_cast<uintptr_t>(base) & 15) == 0) {
+        // whole groups of 8 logits, a contiguous share per CTA; the ragged end goes to the last CTA
+        const int groups = vocab / 8;
+        const int g_per = (groups + CS - 1) / CS;
+        const int g0 = min(groups, rank * g_per), g1 = min(groups, g0 + g_per);
+        for (int g = g0 + tid; g < g1; g += kUnroll * kEntThreads) {
+            if (DT == 1) {
+                uint4 w[kUnroll];
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (g + j * kEntThreads < g1)
+                        w[j] = __ldg(reinterpret_cast<const uint4*>(base) + g + j * kEntThreads);
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (g + j * kEntThreads < g1) fold_words(acc, w[j]);
+            } else {
+                float4 w[kUnroll][2];
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (g + j * kEntThreads < g1) {
+                        w[j][0] = __ldg(reinterpret_cast<const float4*>(base) + 2 * (g + j * kEntThreads));
+                        w[j][1] = __ldg(reinterpret_cast<const float4*>(base) + 2 * (g + j * kEntThreads) + 1);
+                    }
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (g + j * kEntThreads < g1) fold_words(acc, w[j][0], w[j][1]);
+            }
+        }
+        if (rank == CS - 1 && groups * 8 + tid < vocab) fold1(acc, load_logit<DT>(base, groups * 8 + tid));
+    } else {
+        // a row that does not start on a 16-byte boundary: element by element
+        const int per = (vocab + CS - 1) / CS;
+        const int v0 = min(vocab, rank * per), v1 = min(vocab, v0 + per);
+        for (int v = v0 + tid; v < v1; v += kEntThreads) fold1(acc, load_logit<DT>(base, v));
+    }
+    // warp, CTA, cluster: merged in a fixed order
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Mst other{__shfl_xor_sync(0xffffffffu, acc.m, o), __shfl_xor_sync(0xffffffffu, acc.s, o),
+                  __shfl_xor_sync(0xffffffffu, acc.t, o)};
+        acc = merge(acc, other);
+    }
+    if (lane == 0) warp_part[warp] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        Mst a = warp_part[0];
+        for (int w = 1; w < kEntThreads / 32; ++w) a = merge(a, warp_part[w]);
+        cta_part = a;
+    }
+    if (CS > 1) cluster.sync(); else __syncthreads();
+    if (rank == 0 && tid == 0) {
+        Mst a = cta_part;
+        for (int c = 1; c < CS; ++c) a = merge(a, *cluster.map_shared_rank(&cta_part, c));
+        entropy[row] = a.s > 0.f ? a.m + __logf(a.s) - a.t / a.s : 0.f;
+    }
+    if (CS > 1) cluster.sync();  // nobody leaves while its partial may still be read
+}
+
+// Eq. "ema": state[0] <- beta state[0] + (1 - beta) mean(H_1..H_m), state[1] likewise with H_{m+1}..H_k
+__global__ void controller_update_kernel(float* state, const float* __restrict__ entropy, int k,
+                                         const int32_t* __restrict__ n_accepted, float beta)
+{
+    const int lane = threadIdx.x;
+    const int m = min(max(*n_accepted, 0), k);
+    float sa = 0.f, sr = 0.f;
+    for (int i = lane; i < k; i += 32) {
+        const float h = entropy[i];
+        if (i < m) sa += h; else sr += h;
+    }
+    sa = warp_sum(sa);
+    sr = warp_sum(sr);
+    if (lane == 0) {
+        if (m > 0) state[0] = beta * state[0] + (1.f - beta) * (sa / m);
+        if (m < k) state[1] = beta * state[1] + (1.f - beta) * (sr / (k - m));
+    }
+}
+
+// Eq. "prob" and Eq. "optimal_k"; ties go to the smaller candidate
+__global__ void controller_select_kernel(const float* __restrict__ state, const float* __restrict__ entropy, int n,
+                                         const int32_t* __restrict__ cand, int n_cand, float c_d, float c_v,
+                                         int32_t* k_star, float* p_out, float* score_out)
+{
+    __shared__ float expected[kMaxDrafted];  // 1 + sum_{m <= k} prod_{i <= m} p_i at k = index + 1
+    const int lane = threadIdx.x;
+    const float acc_c = state[0], rej_c = state[1];
+    for (int i = lane; i < n; i += 32) {
+        const float a = __expf(-fabsf(entropy[i] - acc_c)), b = __expf(-fabsf(entropy[i] - rej_c));
+        const float p = a / (a + b);
+        expected[i] = p;
+        if (p_out) p_out[i] = p;
+    }
+    __syncwarp();
+    if (lane == 0) {
+        float prefix = 1.f, e = 1.f;
+        for (int i = 0; i < n; ++i) {
+            prefix *= expected[i];
+            e += prefix;
+            expected[i] = e;
+        }
+        int best = 0;
+        float best_score = -1.f;
+        for (int c = 0; c < n_cand; ++c) {
+            const int k = cand[c];
+            float score = -1.f;  // a candidate outside 1..n never wins
+            if (k >= 1 && k <= n) score = expected[k - 1] / (k * c_d + c_v);
+            if (score_out) score_out[c] = score;
+            if (score >= 0.f && (score > best_score || (score == best_score && k < best))) {
+                best_score = score;
+                best = k;
+            }
+        }
+        *k_star = best;
+    }
+}
+
+}  // namespace
+
+int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
+                   cudaStream_t stream)
+{
+    // a row per cluster; the cluster shrinks as the rows alone fill the SMs
+    // up to four CTAs per SM (about 128 KB of loads in flight per SM), and no CTA without a full
+    // sweep of its threads
+    int cs = 8;
+    while (cs > 1 && (long)n_rows * cs > 4L * sm_count()) cs /= 2;
+    while (cs > 1 && vocab < cs * 8 * kEntThreads) cs /= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cs, n_rows);
+    cfg.blockDim = dim3(kEntThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = dtype == 1 ? cudaLaunchKernelEx(&cfg, entropy_kernel<1>, logits, vocab, row_stride, entropy)
+                                       : cudaLaunchKernelEx(&cfg, entropy_kernel<0>, logits, vocab, row_stride, entropy);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        return SPEC_ERR_CUDA;
+    }
+    count_launch(1);
+    return SPEC_OK;
+}
+
+int controller_update_launch(float* state, const float* entropy, int k, const int32_t* n_accepted, float beta,
+                             cudaStream_t stream)
+{
+    controller_update_kernel<<<1, 32, 0, stream>>>(state, entropy, k, n_accepted, beta);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    count_launch(1);
+    return SPEC_OK;
+}
+
+int controller_select_launch(const float* state, const float* entropy, int n, const int32_t* cand, int n_cand,
+                             float c_d, float c_v, int32_t* k_star, float* p_out, float* score_out,
+                             cudaStream_t stream)
+{
+    if (n > kMaxDrafted) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    controller_select_kernel<<<1, 32, 0, stream>>>(state, entropy, n, cand, n_cand, c_d, c_v, k_star, p_out, score_out);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    count_launch(1);
+    return SPEC_OK;
+}
+
+}  // namespace spec

@@ -185,6 +185,34 @@ size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t
     return 0;
 }
 
+int spec_token_entropy(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride,
+                       float* entropy, void* cuda_stream)
+{
+    if (!logits || !entropy || n_rows < 0 || vocab < 1 || row_stride < vocab || (dtype != 0 && dtype != 1))
+        return SPEC_ERR_INVALID_ARG;
+    if (n_rows == 0) return SPEC_OK;
+    if (n_rows > 65535) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    return entropy_launch(logits, dtype, n_rows, vocab, row_stride, entropy, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_controller_update(float* state, const float* entropy, int32_t k, const int32_t* n_accepted, float beta,
+                           void* cuda_stream)
+{
+    if (!state || !entropy || !n_accepted || k < 0 || !(beta >= 0.f && beta <= 1.f)) return SPEC_ERR_INVALID_ARG;
+    if (k == 0) return SPEC_OK;
+    return controller_update_launch(state, entropy, k, n_accepted, beta, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_controller_select(const float* state, const float* entropy, int32_t n, const int32_t* cand, int32_t n_cand,
+                           float c_d, float c_v, int32_t* k_star, float* p_out, float* score_out, void* cuda_stream)
+{
+    if (!state || !entropy || !cand || !k_star || n < 1 || n_cand < 1 || !(c_d >= 0.f) || !(c_v >= 0.f) ||
+        !(c_d + c_v > 0.f))
+        return SPEC_ERR_INVALID_ARG;
+    return controller_select_launch(state, entropy, n, cand, n_cand, c_d, c_v, k_star, p_out, score_out,
+                                    static_cast<cudaStream_t>(cuda_stream));
+}
+
 int spec_read_status(const void* workspace, void* cuda_stream)
 {
     if (!workspace) return SPEC_ERR_INVALID_ARG;

@@ -116,6 +116,14 @@ struct DraftArgs {
 size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
 int draft_launch(const DraftArgs& a, cudaStream_t stream);
 
+int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
+                   cudaStream_t stream);
+int controller_update_launch(float* state, const float* entropy, int k, const int32_t* n_accepted, float beta,
+                             cudaStream_t stream);
+int controller_select_launch(const float* state, const float* entropy, int n, const int32_t* cand, int n_cand,
+                             float c_d, float c_v, int32_t* k_star, float* p_out, float* score_out,
+                             cudaStream_t stream);
+
 void count_launch(int n = 1);
 int sm_count();
 

@@ -289,3 +289,24 @@ def small_config(name="small", **kw) -> SpecConfig:
                 planted=6, planted_mult=3.0, planted_noise=True, seed=11)
     base.update(kw)
     return SpecConfig(**base)
+
+
+def make_logits(rows: int, vocab: int, dtype=torch.bfloat16, seed: int = 0, device="cpu",
+                row_stride: Optional[int] = None, offset: int = 0) -> torch.Tensor:
+    """Seeded draft-model logits ``[rows, vocab]`` for the speculation-length controller: a
+    Gaussian background whose spread differs per row (confident rows to near-uniform rows) plus
+    a few boosted tokens per row, the shape of a language model's next-token logits.  Holds no
+    arithmetic of the method.  ``row_stride`` > vocab leaves padding between rows and ``offset``
+    shifts the first element (to exercise strided and unaligned rows)."""
+    gen = torch.Generator().manual_seed(7000 + seed)
+    stride = row_stride or vocab
+    buf = torch.zeros(rows * stride + offset + 8, dtype=torch.float32)
+    view = buf[offset:offset + rows * stride].view(rows, stride)[:, :vocab]
+    spread = torch.empty(rows).uniform_(0.2, 4.0, generator=gen)
+    view.copy_(torch.randn(rows, vocab, generator=gen) * spread[:, None])
+    n_boost = min(4, vocab)
+    cols = torch.randint(0, vocab, (rows, n_boost), generator=gen)
+    boost = torch.empty(rows, n_boost).uniform_(0.0, 14.0, generator=gen)
+    view.scatter_add_(1, cols, boost)
+    buf = buf.to(dtype).to(device)
+    return buf[offset:offset + rows * stride].view(rows, stride)[:, :vocab]
