@@ -212,6 +212,67 @@ def drift_recall(case, run, n_rounds, prob=0.1):
             "recall_moved_min": min(per_round_new), "recall_moved_mean": sum(per_round_new) / n_rounds}
 
 
+def controller_bench(cfg, dev, peak):
+    """After the timed region: the speculation-length controller (not part of the step metric).
+    Token entropy over a 128256-entry bf16 vocabulary for the k rows one sequence drafts and for a
+    1024-row batch (buffers cycled so that every launch reads more than L2 holds since its last
+    visit), and the update + select pair, all replayed from captured graphs."""
+    import torch
+
+    from paper_2607_27735_b200 import binding, inputs
+    vocab = 128256
+    out = {"vocab": vocab, "dtype": "bf16"}
+
+    def timed(graph, launches, reps=5):
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * launches)
+
+    for rows in (cfg.draft_steps * cfg.batch, 1024):
+        n_buf = min(64, max(2, int(300e6 // (rows * vocab * 2)) + 1))
+        base = inputs.make_logits(min(rows, 64), vocab, seed=rows, device=dev)
+        bufs = [base.repeat((rows + base.shape[0] - 1) // base.shape[0], 1)[:rows].roll(i, 0).contiguous()
+                for i in range(n_buf)]
+        ent = torch.empty(rows, device=dev)
+        for b in bufs[:2]:
+            binding.spec_token_entropy(b, entropy=ent)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for b in bufs:
+                binding.spec_token_entropy(b, entropy=ent)
+        us = timed(g, n_buf)
+        gbs = rows * vocab * 2 / us / 1e3
+        out[f"entropy_{rows}_rows"] = {"us_per_launch": us, "GB/s": gbs, "frac": gbs / peak,
+                                       "bytes_per_launch": rows * vocab * 2, "buffers_cycled": n_buf}
+    k = cfg.draft_steps
+    state = torch.tensor([1.0, 4.0], device=dev)
+    ent = torch.rand(k, device=dev) * 5
+    n_acc = torch.tensor([k // 2], dtype=torch.int32, device=dev)
+    cand = torch.arange(1, k + 1, dtype=torch.int32, device=dev)
+    k_star = torch.zeros(1, dtype=torch.int32, device=dev)
+    p, score = torch.empty(k, device=dev), torch.empty(k, device=dev)
+
+    def pair():
+        binding.spec_controller_update(state, ent, n_acc, 0.9)
+        binding.spec_controller_select(state, ent, cand, 0.05, 1.0, k_star=k_star, p=p, score=score)
+
+    pair()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(50):
+            pair()
+    out["update_plus_select_us"] = timed(g, 50)
+    return out
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -351,6 +412,8 @@ def run_gpu(args):
         line["draft_roofline"]["traffic"] = t["draft"] * fold
     if args.recall_steps > 0 and case.planted_pos is not None:
         line["recall"] = drift_recall(case, run, args.recall_steps)
+    if not args.no_controller:
+        line["controller"] = controller_bench(cfg, dev, peak)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -371,6 +434,8 @@ def main():
                     help="skip the oracle timing (sweeps over the other workloads)")
     ap.add_argument("--recall-steps", type=int, default=0,
                     help="after timing, run this many rounds with drifting planted positions and report recall")
+    ap.add_argument("--no-controller", action="store_true",
+                    help="skip the speculation-length controller's own timing (reported beside the step)")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()

@@ -11,6 +11,8 @@
 // memory so that a captured graph can branch on them without a host round trip.
 #include <cooperative_groups.h>
 
+#include <cstdlib>
+
 #include "spec_common.cuh"
 
 namespace cg = cooperative_groups;
@@ -224,11 +226,16 @@ int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t
                    cudaStream_t stream)
 {
     // a row per cluster; the cluster shrinks as the rows alone fill the SMs
-    // up to four CTAs per SM (about 128 KB of loads in flight per SM), and no CTA without a full
-    // sweep of its threads
+    // A row is worth splitting only while the rows alone leave SMs idle: one SM needs about 4 us
+    // for the 128K exponentials of a row (16 per clock), but a cluster costs a few hundred
+    // nanoseconds of barriers, which shows once every SM has two CTAs anyway.  No CTA without a
+    // full sweep of its threads.
     int cs = 8;
-    while (cs > 1 && (long)n_rows * cs > 4L * sm_count()) cs /= 2;
+    while (cs > 1 && (long)n_rows * cs > 2L * sm_count()) cs /= 2;
     while (cs > 1 && vocab < cs * 8 * kEntThreads) cs /= 2;
+#ifdef SPEC_TRACE
+    if (const char* e = getenv("SPEC_ENT_CS")) cs = atoi(e);
+#endif
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cs, n_rows);
     cfg.blockDim = dim3(kEntThreads);
