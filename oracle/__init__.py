@@ -20,16 +20,18 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "spec_oracle.c")
 _SRC_CTRL = os.path.join(_HERE, "controller_oracle.c")
+_SRC_ACC = os.path.join(_HERE, "accept_oracle.c")
 _LIB = os.path.join(_HERE, "libspec_oracle.so")
 _lib = None
 
 
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (OpenMP over the independent (layer, batch, KV head) problems)."""
-    newest = max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_CTRL))
+    newest = max(os.path.getmtime(p) for p in (_SRC, _SRC_CTRL, _SRC_ACC))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         subprocess.check_call(
-            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, _SRC_CTRL, "-lm"]
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, _SRC_CTRL, _SRC_ACC,
+             "-lm"]
         )
     return _LIB
 
@@ -210,3 +212,26 @@ def controller_select(state, entropy, cand, c_d, c_v):
     if rc != 0:
         raise ValueError("oracle_controller_select: invalid arguments")
     return int(k_star[0]), p, score
+
+
+def accept_greedy(logits, draft, n_draft=None):
+    """Greedy prefix acceptance (Sec. "The Draft-Verification Paradigm").  ``logits``: fp32 or bf16 CPU
+    tensor ``[batch, k + 1, V]`` (contiguous); ``draft``: int32 ``[batch, k]``; ``n_draft``: int32
+    ``[batch]`` or None.  Returns ``(target [batch, k + 1], n_accepted [batch], next_token [batch])``."""
+    lib = _load()
+    assert logits.dim() == 3 and logits.is_contiguous() and not logits.is_cuda
+    dtype = {torch.float32: 0, torch.bfloat16: 1}[logits.dtype]
+    batch, k1, vocab = logits.shape
+    draft = torch.as_tensor(draft, dtype=torch.int32).contiguous().view(batch, k1 - 1)
+    nd = None if n_draft is None else torch.as_tensor(n_draft, dtype=torch.int32).contiguous()
+    target = torch.zeros(batch, k1, dtype=torch.int32)
+    n_acc = torch.zeros(batch, dtype=torch.int32)
+    nxt = torch.zeros(batch, dtype=torch.int32)
+    rc = lib.oracle_accept_greedy(
+        ctypes.c_void_p(logits.data_ptr()), ctypes.c_int(dtype), ctypes.c_int(batch), ctypes.c_int(k1),
+        ctypes.c_int(vocab), ctypes.c_int64(vocab), ctypes.c_void_p(draft.data_ptr() if draft.numel() else None),
+        ctypes.c_void_p(None if nd is None else nd.data_ptr()), ctypes.c_void_p(target.data_ptr()),
+        ctypes.c_void_p(n_acc.data_ptr()), ctypes.c_void_p(nxt.data_ptr()))
+    if rc != 0:
+        raise ValueError("oracle_accept_greedy: invalid arguments")
+    return target, n_acc, nxt

@@ -379,3 +379,51 @@ def test_controller_select_against_plain_python():
                 best, best_k = sc, k
         assert k_star == best_k
         assert max(abs(a - b) for a, b in zip(p.tolist(), ps)) < 1e-14
+
+
+# ---- prefix acceptance (Sec. "The Draft-Verification Paradigm", greedy reading) ----
+
+def test_accept_argmax_matches_library_and_breaks_ties_low():
+    gen = torch.Generator().manual_seed(4)
+    logits = torch.randn(3, 5, 777, generator=gen)
+    draft = torch.zeros(3, 4, dtype=torch.int32)
+    target, _, _ = oracle.accept_greedy(logits, draft)
+    assert torch.equal(target.long(), logits.argmax(dim=-1))          # tie-free rows: any argmax agrees
+    tied = torch.zeros(1, 2, 50)
+    tied[0, 0, [7, 30, 31]] = 2.5                                       # equal maxima: the smallest index
+    tied[0, 1, :] = -1.0                                                # a constant row: index 0
+    target, _, _ = oracle.accept_greedy(tied.to(torch.bfloat16), torch.zeros(1, 1, dtype=torch.int32))
+    assert target.tolist() == [[7, 0]]
+
+
+def test_accept_prefix_rule_on_constructed_cases():
+    k, V = 6, 64
+    want = torch.tensor([[5, 9, 9, 40, 63, 0, 17]])                     # the target model's greedy tokens
+
+    def logits_for(tokens):
+        lg = torch.zeros(tokens.shape[0], tokens.shape[1], V)
+        lg.scatter_(2, tokens.long().unsqueeze(-1), 3.0)
+        return lg
+
+    lg = logits_for(want)
+    # every drafted token right: m = k, the corrected token is the bonus row's
+    t, m, nxt = oracle.accept_greedy(lg, want[:, :k].int())
+    assert t.tolist() == want.tolist() and m.tolist() == [6] and nxt.tolist() == [17]
+    # first one wrong: nothing accepted, the corrected token is row 0's
+    d = want[:, :k].clone().int()
+    d[0, 0] = 6
+    _, m, nxt = oracle.accept_greedy(lg, d)
+    assert m.tolist() == [0] and nxt.tolist() == [5]
+    # mismatch at j = 3; the matches after it must not count
+    d = want[:, :k].clone().int()
+    d[0, 3] = 41
+    _, m, nxt = oracle.accept_greedy(lg, d)
+    assert m.tolist() == [3] and nxt.tolist() == [40]
+    # ragged speculation lengths: only n_draft tokens are looked at
+    batch = logits_for(want.repeat(3, 1))
+    d3 = want[:, :k].repeat(3, 1).int()
+    _, m, nxt = oracle.accept_greedy(batch, d3, n_draft=[0, 2, 6])
+    assert m.tolist() == [0, 2, 6] and nxt.tolist() == [5, 9, 17]
+    # k = 0 (plain decoding step): one row, no draft
+    _, m, nxt = oracle.accept_greedy(lg[:, :1].contiguous(), torch.zeros(1, 0, dtype=torch.int32))
+    assert m.tolist() == [0] and nxt.tolist() == [5]
