@@ -226,6 +226,29 @@ int spec_noalloc_read_status(void* cuda_stream);
  */
 int spec_token_entropy(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
                        int64_t row_stride, float* entropy, void* cuda_stream);
+/*
+ * spec_token_argmax: token[r] = the smallest index of the largest logit of row r (greedy
+ *   decoding of that row); if `entropy` is not NULL it also receives spec_token_entropy's value
+ *   from the same pass over the logits (a drafting step needs both).  Same layout and errors as
+ *   spec_token_entropy; n_rows <= 65535.
+ *
+ * spec_accept_greedy: the verification stage's prefix acceptance (Sec. "The Draft-Verification
+ *   Paradigm") under greedy matching.  logits: [batch][k1][vocab], rows `row_stride` elements
+ *   apart across the whole batch, row i of a sequence being the target model's output after
+ *   drafted token i (row 0 after the last committed token).  draft: [batch][k1 - 1] drafted
+ *   tokens; n_draft: [batch] drafted tokens actually present per sequence (clamped to
+ *   0..k1 - 1), or NULL for k1 - 1 everywhere.  Outputs: target[batch][k1] = greedy token of
+ *   every row; n_accepted[b] = m = length of the longest prefix with draft[b][i] == target[b][i];
+ *   next_token[b] = target[b][m], the corrected token the step commits after the prefix.
+ *   Integer results, bit-exact.  Two launches (row argmax, prefix scan) on `cuda_stream`.
+ *   Errors: SPEC_ERR_INVALID_ARG; SPEC_ERR_UNSUPPORTED_SHAPE if batch * k1 > 65535.
+ */
+int spec_token_argmax(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab,
+                      int64_t row_stride, int32_t* token, float* entropy, void* cuda_stream);
+int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t k1, int32_t vocab,
+                       int64_t row_stride, const int32_t* draft, const int32_t* n_draft,
+                       int32_t* target, int32_t* n_accepted, int32_t* next_token,
+                       void* cuda_stream);
 int spec_controller_update(float* state, const float* entropy, int32_t k,
                            const int32_t* n_accepted, float beta, void* cuda_stream);
 int spec_controller_select(const float* state, const float* entropy, int32_t n,

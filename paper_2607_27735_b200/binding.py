@@ -24,6 +24,7 @@ EXPORTS = [
     "spec_read_status", "spec_set_verify_impl", "spec_last_verify_impl", "spec_launch_count",
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
+    "spec_token_argmax", "spec_accept_greedy",
 ]
 
 
@@ -71,6 +72,8 @@ def load() -> ctypes.CDLL:
         lib.spec_noalloc_read_status.argtypes = [vp]
         f32 = ctypes.c_float
         lib.spec_token_entropy.argtypes = [vp, i32, i32, i32, i64, vp, vp]
+        lib.spec_token_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp, vp]
+        lib.spec_accept_greedy.argtypes = [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
         lib.spec_controller_update.argtypes = [vp, vp, i32, vp, f32, vp]
         lib.spec_controller_select.argtypes = [vp, vp, i32, vp, i32, f32, f32, vp, vp, vp, vp]
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
@@ -246,6 +249,55 @@ def spec_token_entropy(logits, entropy=None):
     if rc != 0:
         raise SpecError(rc, "spec_token_entropy")
     return entropy
+
+
+def _logits_2d(logits):
+    if not logits.is_cuda or logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits: expected a CUDA [rows, vocab] tensor with unit inner stride")
+    if logits.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"logits: expected fp32 or bf16, got {logits.dtype}")
+    rows, vocab = logits.shape
+    return rows, vocab, 1 if logits.dtype == torch.bfloat16 else 0, max(logits.stride(0), vocab)
+
+
+def spec_token_argmax(logits, token=None, entropy=None, want_entropy=False):
+    """Greedy token per row (smallest index of the largest logit), optionally with the row's entropy
+    from the same pass.  Returns ``(token, entropy or None)``."""
+    rows, vocab, dt, stride = _logits_2d(logits)
+    if token is None:
+        token = torch.empty(rows, dtype=torch.int32, device=logits.device)
+    if entropy is None and want_entropy:
+        entropy = torch.empty(rows, dtype=torch.float32, device=logits.device)
+    rc = load().spec_token_argmax(logits.data_ptr(), dt, rows, vocab, stride, _dev(token, torch.int32, "token"),
+                                  None if entropy is None else _dev(entropy, torch.float32, "entropy"), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_token_argmax")
+    return token, entropy
+
+
+def spec_accept_greedy(logits, draft, n_draft=None, target=None, n_accepted=None, next_token=None):
+    """Greedy prefix acceptance; ``logits`` is a contiguous CUDA ``[batch, k + 1, vocab]`` tensor, ``draft``
+    int32 ``[batch, k]``.  Returns device tensors ``(target, n_accepted, next_token)``."""
+    if not logits.is_cuda or logits.dim() != 3 or not logits.is_contiguous():
+        raise ValueError("logits: expected a contiguous CUDA [batch, k + 1, vocab] tensor")
+    if logits.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError(f"logits: expected fp32 or bf16, got {logits.dtype}")
+    batch, k1, vocab = logits.shape
+    dev = logits.device
+    if target is None:
+        target = torch.empty(batch, k1, dtype=torch.int32, device=dev)
+    if n_accepted is None:
+        n_accepted = torch.empty(batch, dtype=torch.int32, device=dev)
+    if next_token is None:
+        next_token = torch.empty(batch, dtype=torch.int32, device=dev)
+    rc = load().spec_accept_greedy(
+        logits.data_ptr(), 1 if logits.dtype == torch.bfloat16 else 0, batch, k1, vocab, vocab,
+        _dev(draft, torch.int32, "draft") if k1 > 1 else None,
+        None if n_draft is None else _dev(n_draft, torch.int32, "n_draft"), _dev(target, torch.int32, "target"),
+        _dev(n_accepted, torch.int32, "n_accepted"), _dev(next_token, torch.int32, "next_token"), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_accept_greedy")
+    return target, n_accepted, next_token
 
 
 def spec_controller_update(state, entropy, n_accepted, beta):

@@ -37,6 +37,17 @@ __device__ __forceinline__ Mst merge(const Mst& a, const Mst& b)
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kUnroll = 4;  // 16-byte loads a thread keeps in flight
+constexpr float kNegInf = -__builtin_huge_valf();
+
+struct Arg {  // largest logit seen and the smallest index that holds it
+    float v;
+    int i;
+};
+
+__device__ __forceinline__ Arg merge(const Arg& a, const Arg& b)
+{
+    return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
+}
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -45,25 +56,39 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
-__device__ __forceinline__ void fold8(Mst& acc, const float (&z)[8], float cm)
+// eight logits z (group maximum cm) starting at vocabulary index v0
+template <bool ENT, bool ARG>
+__device__ __forceinline__ void fold8(Mst& acc, Arg& arg, const float (&z)[8], float cm, int v0)
 {
-    const float mn = fmaxf(acc.m, cm), mb = mn * kLog2e;
-    const float f = ex2(fmaf(acc.m, kLog2e, -mb));
-    float s = acc.s * f, t = acc.t * f;
+    if (ARG && cm > arg.v) {  // rare after the first groups: the running maximum seldom moves
+        int first = 7;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float e = ex2(fmaf(z[i], kLog2e, -mb));
-        s += e;
-        t = fmaf(e, z[i], t);
+        for (int i = 6; i >= 0; --i) first = z[i] == cm ? i : first;
+        arg = Arg{cm, v0 + first};
     }
-    acc = Mst{mn, s, t};
+    if (ENT) {
+        const float mn = fmaxf(acc.m, cm), mb = mn * kLog2e;
+        const float f = ex2(fmaf(acc.m, kLog2e, -mb));
+        float s = acc.s * f, t = acc.t * f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float e = ex2(fmaf(z[i], kLog2e, -mb));
+            s += e;
+            t = fmaf(e, z[i], t);
+        }
+        acc = Mst{mn, s, t};
+    }
 }
 
-__device__ __forceinline__ void fold1(Mst& acc, float z)
+template <bool ENT, bool ARG>
+__device__ __forceinline__ void fold1(Mst& acc, Arg& arg, float z, int v)
 {
-    const float mn = fmaxf(acc.m, z), mb = mn * kLog2e;
-    const float f = ex2(fmaf(acc.m, kLog2e, -mb)), e = ex2(fmaf(z, kLog2e, -mb));
-    acc = Mst{mn, fmaf(acc.s, f, e), fmaf(acc.t, f, e * z)};
+    if (ARG && z > arg.v) arg = Arg{z, v};
+    if (ENT) {
+        const float mn = fmaxf(acc.m, z), mb = mn * kLog2e;
+        const float f = ex2(fmaf(acc.m, kLog2e, -mb)), e = ex2(fmaf(z, kLog2e, -mb));
+        acc = Mst{mn, fmaf(acc.s, f, e), fmaf(acc.t, f, e * z)};
+    }
 }
 
 __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
@@ -73,18 +98,21 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b)
     return r;
 }
 
-__device__ __forceinline__ void fold_words(Mst& acc, const uint4& w)  // eight bf16 logits
+template <bool ENT, bool ARG>
+__device__ __forceinline__ void fold_words(Mst& acc, Arg& arg, const uint4& w, int v0)  // eight bf16 logits
 {
     const uint32_t mx = bf16x2_max(bf16x2_max(w.x, w.y), bf16x2_max(w.z, w.w));
     const float z[8] = {bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y),
                         bf16_lo(w.z), bf16_hi(w.z), bf16_lo(w.w), bf16_hi(w.w)};
-    fold8(acc, z, fmaxf(bf16_lo(mx), bf16_hi(mx)));
+    fold8<ENT, ARG>(acc, arg, z, fmaxf(bf16_lo(mx), bf16_hi(mx)), v0);
 }
 
-__device__ __forceinline__ void fold_words(Mst& acc, const float4& a, const float4& b)  // eight fp32 logits
+template <bool ENT, bool ARG>
+__device__ __forceinline__ void fold_words(Mst& acc, Arg& arg, const float4& a, const float4& b, int v0)  // eight fp32
 {
     const float z[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    fold8(acc, z, fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w))));
+    fold8<ENT, ARG>(acc, arg, z,
+                    fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w))), v0);
 }
 
 template <int DT>
@@ -93,18 +121,22 @@ __device__ __forceinline__ float load_logit(const void* base, int v)
     return DT == 1 ? __bfloat162float(static_cast<const __nv_bfloat16*>(base)[v]) : static_cast<const float*>(base)[v];
 }
 
-// One cluster (gridDim.x CTAs) per row.  DT = 0: fp32 logits, 1: bf16 logits.
-template <int DT>
-__global__ void __launch_bounds__(kEntThreads) entropy_kernel(const void* __restrict__ logits, int vocab,
-                                                              int64_t row_stride, float* __restrict__ entropy)
+// One cluster (gridDim.x CTAs) per row.  DT = 0: fp32 logits, 1: bf16 logits.  ENT: entropy[row];
+// ARG: token[row] = the smallest index of the largest logit.
+template <int DT, bool ENT, bool ARG>
+__global__ void __launch_bounds__(kEntThreads) row_kernel(const void* __restrict__ logits, int vocab, int64_t row_stride,
+                                                          float* __restrict__ entropy, int32_t* __restrict__ token)
 {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ Mst warp_part[kEntThreads / 32];
+    __shared__ Arg warp_arg[kEntThreads / 32];
     __shared__ Mst cta_part;
+    __shared__ Arg cta_arg;
     const int CS = gridDim.x, rank = blockIdx.x, row = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const char* base = static_cast<const char*>(logits) + (int64_t)row * row_stride * (DT == 1 ? 2 : 4);
     Mst acc{-3.0e38f, 0.f, 0.f};
+    Arg arg{kNegInf, 0x7fffffff};
     if ((reinterpret_cast<uintptr_t>(base) & 15) == 0) {
         // whole groups of 8 logits, a contiguous share per CTA; the ragged end goes to the last CTA
         const int groups = vocab / 8;
@@ -119,7 +151,7 @@ __global__ void __launch_bounds__(kEntThreads) entropy_kernel(const void* __rest
                         w[j] = __ldg(reinterpret_cast<const uint4*>(base) + g + j * kEntThreads);
 #pragma unroll
                 for (int j = 0; j < kUnroll; ++j)
-                    if (g + j * kEntThreads < g1) fold_words(acc, w[j]);
+                    if (g + j * kEntThreads < g1) fold_words<ENT, ARG>(acc, arg, w[j], (g + j * kEntThreads) * 8);
             } else {
                 float4 w[kUnroll][2];
 #pragma unroll
@@ -130,37 +162,73 @@ __global__ void __launch_bounds__(kEntThreads) entropy_kernel(const void* __rest
                     }
 #pragma unroll
                 for (int j = 0; j < kUnroll; ++j)
-                    if (g + j * kEntThreads < g1) fold_words(acc, w[j][0], w[j][1]);
+                    if (g + j * kEntThreads < g1)
+                        fold_words<ENT, ARG>(acc, arg, w[j][0], w[j][1], (g + j * kEntThreads) * 8);
             }
         }
-        if (rank == CS - 1 && groups * 8 + tid < vocab) fold1(acc, load_logit<DT>(base, groups * 8 + tid));
+        if (rank == CS - 1 && groups * 8 + tid < vocab)
+            fold1<ENT, ARG>(acc, arg, load_logit<DT>(base, groups * 8 + tid), groups * 8 + tid);
     } else {
         // a row that does not start on a 16-byte boundary: element by element
         const int per = (vocab + CS - 1) / CS;
         const int v0 = min(vocab, rank * per), v1 = min(vocab, v0 + per);
-        for (int v = v0 + tid; v < v1; v += kEntThreads) fold1(acc, load_logit<DT>(base, v));
+        for (int v = v0 + tid; v < v1; v += kEntThreads) fold1<ENT, ARG>(acc, arg, load_logit<DT>(base, v), v);
     }
     // warp, CTA, cluster: merged in a fixed order
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        Mst other{__shfl_xor_sync(0xffffffffu, acc.m, o), __shfl_xor_sync(0xffffffffu, acc.s, o),
-                  __shfl_xor_sync(0xffffffffu, acc.t, o)};
-        acc = merge(acc, other);
+        if (ENT) {
+            Mst other{__shfl_xor_sync(0xffffffffu, acc.m, o), __shfl_xor_sync(0xffffffffu, acc.s, o),
+                      __shfl_xor_sync(0xffffffffu, acc.t, o)};
+            acc = merge(acc, other);
+        }
+        if (ARG) {
+            Arg other{__shfl_xor_sync(0xffffffffu, arg.v, o), __shfl_xor_sync(0xffffffffu, arg.i, o)};
+            arg = merge(arg, other);
+        }
     }
-    if (lane == 0) warp_part[warp] = acc;
+    if (lane == 0) {
+        warp_part[warp] = acc;
+        warp_arg[warp] = arg;
+    }
     __syncthreads();
     if (tid == 0) {
         Mst a = warp_part[0];
-        for (int w = 1; w < kEntThreads / 32; ++w) a = merge(a, warp_part[w]);
+        Arg g = warp_arg[0];
+        for (int w = 1; w < kEntThreads / 32; ++w) {
+            if (ENT) a = merge(a, warp_part[w]);
+            if (ARG) g = merge(g, warp_arg[w]);
+        }
         cta_part = a;
+        cta_arg = g;
     }
     if (CS > 1) cluster.sync(); else __syncthreads();
     if (rank == 0 && tid == 0) {
         Mst a = cta_part;
-        for (int c = 1; c < CS; ++c) a = merge(a, *cluster.map_shared_rank(&cta_part, c));
-        entropy[row] = a.s > 0.f ? a.m + __logf(a.s) - a.t / a.s : 0.f;
+        Arg g = cta_arg;
+        for (int c = 1; c < CS; ++c) {
+            if (ENT) a = merge(a, *cluster.map_shared_rank(&cta_part, c));
+            if (ARG) g = merge(g, *cluster.map_shared_rank(&cta_arg, c));
+        }
+        if (ENT) entropy[row] = a.s > 0.f ? a.m + __logf(a.s) - a.t / a.s : 0.f;
+        if (ARG) token[row] = g.i == 0x7fffffff ? 0 : g.i;
     }
     if (CS > 1) cluster.sync();  // nobody leaves while its partial may still be read
+}
+
+// Greedy prefix acceptance: drafted token i of a sequence is accepted iff every earlier one was and
+// it equals the target's token for that position; one thread per sequence.
+__global__ void accept_kernel(const int32_t* __restrict__ target, const int32_t* __restrict__ draft,
+                              const int32_t* __restrict__ n_draft, int batch, int k1,
+                              int32_t* __restrict__ n_accepted, int32_t* __restrict__ next_token)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int nd = n_draft ? min(max(n_draft[b], 0), k1 - 1) : k1 - 1;
+    int m = 0;
+    while (m < nd && draft[b * (k1 - 1) + m] == target[b * k1 + m]) ++m;
+    n_accepted[b] = m;
+    next_token[b] = target[b * k1 + m];
 }
 
 // Eq. "ema": state[0] <- beta state[0] + (1 - beta) mean(H_1..H_m), state[1] likewise with H_{m+1}..H_k
@@ -222,10 +290,17 @@ __global__ void controller_select_kernel(const float* __restrict__ state, const 
 
 }  // namespace
 
-int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
-                   cudaStream_t stream)
+template <int DT, bool ENT, bool ARG>
+static cudaError_t launch_rows(const cudaLaunchConfig_t& cfg, const void* logits, int vocab, int64_t row_stride,
+                               float* entropy, int32_t* token)
 {
-    // a row per cluster; the cluster shrinks as the rows alone fill the SMs
+    return cudaLaunchKernelEx(&cfg, row_kernel<DT, ENT, ARG>, logits, vocab, row_stride, entropy, token);
+}
+
+// entropy and/or token may be null (not both)
+int rows_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
+                int32_t* token, cudaStream_t stream)
+{
     // A row is worth splitting only while the rows alone leave SMs idle: one SM needs about 4 us
     // for the 128K exponentials of a row (16 per clock), but a cluster costs a few hundred
     // nanoseconds of barriers, which shows once every SM has two CTAs anyway.  No CTA without a
@@ -247,12 +322,29 @@ int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = dtype == 1 ? cudaLaunchKernelEx(&cfg, entropy_kernel<1>, logits, vocab, row_stride, entropy)
-                                       : cudaLaunchKernelEx(&cfg, entropy_kernel<0>, logits, vocab, row_stride, entropy);
+    cudaError_t err;
+    if (entropy && token)
+        err = dtype == 1 ? launch_rows<1, true, true>(cfg, logits, vocab, row_stride, entropy, token)
+                         : launch_rows<0, true, true>(cfg, logits, vocab, row_stride, entropy, token);
+    else if (entropy)
+        err = dtype == 1 ? launch_rows<1, true, false>(cfg, logits, vocab, row_stride, entropy, token)
+                         : launch_rows<0, true, false>(cfg, logits, vocab, row_stride, entropy, token);
+    else
+        err = dtype == 1 ? launch_rows<1, false, true>(cfg, logits, vocab, row_stride, entropy, token)
+                         : launch_rows<0, false, true>(cfg, logits, vocab, row_stride, entropy, token);
     if (err != cudaSuccess) {
         cudaGetLastError();
         return SPEC_ERR_CUDA;
     }
+    count_launch(1);
+    return SPEC_OK;
+}
+
+int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_draft, int batch, int k1,
+                  int32_t* n_accepted, int32_t* next_token, cudaStream_t stream)
+{
+    accept_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(target, draft, n_draft, batch, k1, n_accepted, next_token);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     count_launch(1);
     return SPEC_OK;
 }

@@ -192,7 +192,34 @@ int spec_token_entropy(const void* logits, int32_t dtype, int32_t n_rows, int32_
         return SPEC_ERR_INVALID_ARG;
     if (n_rows == 0) return SPEC_OK;
     if (n_rows > 65535) return SPEC_ERR_UNSUPPORTED_SHAPE;
-    return entropy_launch(logits, dtype, n_rows, vocab, row_stride, entropy, static_cast<cudaStream_t>(cuda_stream));
+    return rows_launch(logits, dtype, n_rows, vocab, row_stride, entropy, nullptr,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_token_argmax(const void* logits, int32_t dtype, int32_t n_rows, int32_t vocab, int64_t row_stride,
+                      int32_t* token, float* entropy, void* cuda_stream)
+{
+    if (!logits || !token || n_rows < 0 || vocab < 1 || row_stride < vocab || (dtype != 0 && dtype != 1))
+        return SPEC_ERR_INVALID_ARG;
+    if (n_rows == 0) return SPEC_OK;
+    if (n_rows > 65535) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    return rows_launch(logits, dtype, n_rows, vocab, row_stride, entropy, token,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t k1, int32_t vocab,
+                       int64_t row_stride, const int32_t* draft, const int32_t* n_draft, int32_t* target,
+                       int32_t* n_accepted, int32_t* next_token, void* cuda_stream)
+{
+    if (!logits || !target || !n_accepted || !next_token || batch < 0 || k1 < 1 || vocab < 1 ||
+        row_stride < vocab || (dtype != 0 && dtype != 1) || (k1 > 1 && !draft))
+        return SPEC_ERR_INVALID_ARG;
+    if (batch == 0) return SPEC_OK;
+    if ((int64_t)batch * k1 > 65535) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int rc = rows_launch(logits, dtype, batch * k1, vocab, row_stride, nullptr, target, stream);
+    if (rc != SPEC_OK) return rc;
+    return accept_launch(target, draft, n_draft, batch, k1, n_accepted, next_token, stream);
 }
 
 int spec_controller_update(float* state, const float* entropy, int32_t k, const int32_t* n_accepted, float beta,

@@ -116,8 +116,10 @@ struct DraftArgs {
 size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
 int draft_launch(const DraftArgs& a, cudaStream_t stream);
 
-int entropy_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
-                   cudaStream_t stream);
+int rows_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t row_stride, float* entropy,
+                int32_t* token, cudaStream_t stream);
+int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_draft, int batch, int k1,
+                  int32_t* n_accepted, int32_t* next_token, cudaStream_t stream);
 int controller_update_launch(float* state, const float* entropy, int k, const int32_t* n_accepted, float beta,
                              cudaStream_t stream);
 int controller_select_launch(const float* state, const float* entropy, int n, const int32_t* cand, int n_cand,
