@@ -251,6 +251,30 @@ def controller_bench(cfg, dev, peak):
         gbs = rows * vocab * 2 / us / 1e3
         out[f"entropy_{rows}_rows"] = {"us_per_launch": us, "GB/s": gbs, "frac": gbs / peak,
                                        "bytes_per_launch": rows * vocab * 2, "buffers_cycled": n_buf}
+    # prefix acceptance over the verification pass's logits: this workload's batch and a 64-sequence batch
+    for batch in sorted({cfg.batch, 64}):
+        k1 = cfg.n_q
+        rows = batch * k1
+        n_buf = min(32, max(2, int(300e6 // (rows * vocab * 2)) + 1))
+        base = inputs.make_logits(min(rows, 64), vocab, seed=rows, device=dev)
+        bufs = [base.repeat((rows + base.shape[0] - 1) // base.shape[0], 1)[:rows].roll(i, 0).contiguous()
+                .view(batch, k1, vocab) for i in range(n_buf)]
+        draft = torch.zeros(batch, k1 - 1, dtype=torch.int32, device=dev)
+        tgt = torch.empty(batch, k1, dtype=torch.int32, device=dev)
+        m = torch.empty(batch, dtype=torch.int32, device=dev)
+        nxt = torch.empty(batch, dtype=torch.int32, device=dev)
+        for b in bufs[:2]:
+            binding.spec_accept_greedy(b, draft, target=tgt, n_accepted=m, next_token=nxt)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for b in bufs:
+                binding.spec_accept_greedy(b, draft, target=tgt, n_accepted=m, next_token=nxt)
+        us = timed(g, n_buf)
+        gbs = rows * vocab * 2 / us / 1e3
+        out[f"accept_batch{batch}_x{k1}_rows"] = {"us_per_call": us, "GB/s": gbs, "frac": gbs / peak,
+                                                  "bytes_per_call": rows * vocab * 2, "launches_per_call": 2,
+                                                  "buffers_cycled": n_buf}
     k = cfg.draft_steps
     state = torch.tensor([1.0, 4.0], device=dev)
     ent = torch.rand(k, device=dev) * 5

@@ -41,6 +41,57 @@ namespace {
 constexpr int kMaxCache = 32;
 constexpr int kLsePubMax = 48;  // CTAs per head up to which the publisher warp alone combines the LSE partials
 
+// Cross-lane reduction of per-column (max, sum of exp2(x - max)) pairs.  While the number of
+// columns a lane carries is even, partners exchange halves (the lane with bit `o` set keeps the
+// upper half), so the traffic halves at every step; an odd count is reduced in place on both
+// partners.  Afterwards a lane holds ml_final_n(NH) columns starting at `col`, and lanes that
+// differ only in the bits of ml_dupmask(NH) hold the same ones.
+__host__ __device__ constexpr int ml_final_n(int n)
+{
+    for (int o = 16; o >= 1; o >>= 1)
+        if (n % 2 == 0) n /= 2;
+    return n;
+}
+__host__ __device__ constexpr uint32_t ml_dupmask(int n)
+{
+    uint32_t d = 0;
+    for (int o = 16; o >= 1; o >>= 1) {
+        if (n % 2 == 0) n /= 2;
+        else d |= (uint32_t)o;
+    }
+    return d;
+}
+template <int NHT, int n, int o>
+__device__ __forceinline__ void ml_step(float (&m)[NHT], float (&l)[NHT], int lane, int& col)
+{
+    if constexpr (o >= 1) {
+        if constexpr (n % 2 == 0) {
+            constexpr int h = n / 2;
+            const bool up = (lane & o) != 0;
+#pragma unroll
+            for (int j = 0; j < h; ++j) {
+                const float sm = up ? m[j] : m[j + h], sl = up ? l[j] : l[j + h];
+                const float km = up ? m[j + h] : m[j], kl = up ? l[j + h] : l[j];
+                const float rm = __shfl_xor_sync(0xffffffffu, sm, o), rl = __shfl_xor_sync(0xffffffffu, sl, o);
+                const float M = fmaxf(km, rm);
+                m[j] = M;
+                l[j] = kl * ex2(km - M) + rl * ex2(rm - M);
+            }
+            col += up ? h : 0;
+            ml_step<NHT, h, o / 2>(m, l, lane, col);
+        } else {
+#pragma unroll
+            for (int j = 0; j < n; ++j) {
+                const float rm = __shfl_xor_sync(0xffffffffu, m[j], o), rl = __shfl_xor_sync(0xffffffffu, l[j], o);
+                const float M = fmaxf(m[j], rm);
+                l[j] = l[j] * ex2(m[j] - M) + rl * ex2(rm - M);
+                m[j] = M;
+            }
+            ml_step<NHT, n, o / 2>(m, l, lane, col);
+        }
+    }
+}
+
 struct CBars {  // mbarrier addresses (shared space)
     uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_free, p_full, p_empty, o_full, o_empty, sm_sync,
         pub_p1, pub_o, lse_ready;
@@ -392,12 +443,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             for (int u = 0; u < 20; ++u)
                                 x[u] = (k0 + 2 * u < p.cph) ? __ldcg(src + (int64_t)(k0 + 2 * u) * R + r)
                                                             : make_float2(-1.0e30f, 0.f);
+                            float Mn = M;
 #pragma unroll
-                            for (int u = 0; u < 20; ++u) {
-                                const float Mn = fmaxf(M, x[u].x);
-                                Ls = Ls * ex2(M - Mn) + x[u].y * ex2(x[u].x - Mn);
-                                M = Mn;
-                            }
+                            for (int u = 0; u < 20; ++u) Mn = fmaxf(Mn, x[u].x);
+                            Ls *= ex2(M - Mn);
+#pragma unroll
+                            for (int u = 0; u < 20; ++u) Ls = fmaf(x[u].y, ex2(x[u].x - Mn), Ls);
+                            M = Mn;
                         }
                     }
                     const float M2 = __shfl_xor_sync(0xffffffffu, M, 1);
@@ -566,16 +618,17 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
             if (!ok) break;
             if (warp == 4) TRACE(2, 2);
-            // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem
+            // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem:
+            // a butterfly that halves the columns a lane carries at every step (see ml_step)
+            {
+                int col = 0;
+                ml_step<NH, NH, 16>(m, l, lane, col);
+                constexpr uint32_t kDup = ml_dupmask(NH);
+                constexpr int kLeft = ml_final_n(NH);
+                if ((lane & kDup) == 0) {
 #pragma unroll
-            for (int i = 0; i < NH; ++i) {
-                float M = m[i];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-                float Ls = l[i] * ex2(m[i] - M);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) Ls += __shfl_xor_sync(0xffffffffu, Ls, o);
-                if (lane == 0) red[sw * NC + i] = make_float2(M, Ls);
+                    for (int j = 0; j < kLeft; ++j) red[sw * NC + col + j] = make_float2(m[j], l[j]);
+                }
             }
             ok = group_sync(B.sm_sync, sync_n, ctl, 26);
             if (!ok) break;
