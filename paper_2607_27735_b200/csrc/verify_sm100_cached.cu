@@ -153,21 +153,22 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     int trace_n[4] = {0, 0, 0, 0};
 #endif
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < p.n_slots; ++i) {
+    if (threadIdx.x < kMaxCache) {  // one region's pair of barriers per thread
+        mbar_init(B.s_full + 8 * threadIdx.x, 1);
+        mbar_init(B.s_free + 8 * threadIdx.x, 4);
+    } else if (threadIdx.x < kMaxCache + 8) {
+        const int i = threadIdx.x - kMaxCache;
+        if (i < p.n_slots) {
             mbar_init(B.slot_full + 8 * i, 1);
             mbar_init(B.slot_empty + 8 * i, 1);
         }
-        for (int i = 0; i < kMaxCache; ++i) {
-            mbar_init(B.s_full + 8 * i, 1);
-            mbar_init(B.s_free + 8 * i, 4);
-        }
-        for (int i = 0; i < 2; ++i) {
+        if (i < 2) {
             mbar_init(B.q_full + 8 * i, 1);
             mbar_init(B.q_empty + 8 * i, 1);
             mbar_init(B.p_full + 8 * i, kSW);
         }
-        for (int i = 0; i < 4; ++i) mbar_init(B.p_empty + 8 * i, 1);
+        if (i < 4) mbar_init(B.p_empty + 8 * i, 1);
+    } else if (threadIdx.x == kMaxCache + 8) {
         mbar_init(B.o_full, 1);
         mbar_init(B.o_empty, kSW);
         mbar_init(B.sm_sync, kSW);
@@ -175,8 +176,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         mbar_init(B.pub_o, kSW);
         mbar_init(B.lse_ready, 1);
         *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // zero the Q buffers once: rows R..N-1 are padding the TMA never writes
     for (int i = threadIdx.x; i < q_bytes / 16; i += kBlock)
         *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
@@ -220,9 +221,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (lane == 0) mbar_expect_tx(B.slot_full + 8 * s, 2u * n_box * box_bytes);
             __syncwarp();
             for (int i = lane; i < 2 * n_box; i += 32) {
-                const int half = i / n_box, bx = i - half * n_box;
+                const int half = i >= n_box ? 1 : 0, bx = i - half * n_box;  // i < 2 * n_box
                 const int pos = key0 + bx * box_rows;
-                const int page = pos / p.a.kv.page_size, slot_in_page = pos - page * p.a.kv.page_size;
+                const int page = page_of(p.a.kv, pos), slot_in_page = pos - page * p.a.kv.page_size;
                 int phys = p.a.kv.page_table ? __ldg(p.a.kv.page_table + (int64_t)sg.b * p.a.kv.max_pages + page)
                                              : sg.b * p.a.kv.max_pages + page;
                 if (phys < 0 || phys >= p.n_pages) {
@@ -439,10 +440,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     if (r < R) {
                         for (int k0 = sub; k0 < p.cph; k0 += 40) {
                             float2 x[20];
+                            const float2* q = src + (int64_t)k0 * R + r;
+                            const int n_ld = (p.cph - k0 + 1) >> 1;  // partials k0, k0 + 2, ... below cph
 #pragma unroll
-                            for (int u = 0; u < 20; ++u)
-                                x[u] = (k0 + 2 * u < p.cph) ? __ldcg(src + (int64_t)(k0 + 2 * u) * R + r)
-                                                            : make_float2(-1.0e30f, 0.f);
+                            for (int u = 0; u < 20; ++u) {
+                                x[u] = make_float2(-1.0e30f, 0.f);
+                                if (u < n_ld) x[u] = __ldcg(q + u * 2 * R);
+                            }
                             float Mn = M;
 #pragma unroll
                             for (int u = 0; u < 20; ++u) Mn = fmaxf(Mn, x[u].x);
@@ -501,10 +505,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int k0 = 0; k0 < p.cph; k0 += 16) {  // batches of 16 independent loads
                     float4 x[16];
+                    const float4* q = src + (int64_t)k0 * E4 + e;
+                    const int n_ld = p.cph - k0;
 #pragma unroll
-                    for (int u = 0; u < 16; ++u)
-                        x[u] = (k0 + u < p.cph) ? __ldcg(src + (int64_t)(k0 + u) * E4 + e)
-                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int u = 0; u < 16; ++u) {
+                        x[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (u < n_ld) x[u] = __ldcg(q + u * E4);
+                    }
 #pragma unroll
                     for (int u = 0; u < 16; ++u) {
                         acc.x += x[u].x;
