@@ -112,6 +112,13 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         pl->p_bufs = 2;
         fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544;
         slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
+        if (slots > 8) slots = 8;
+        // more P buffers (up to four) where they cost no K/V slot: the P V product of a tile then has two tiles
+        // of softmax work to hide behind
+        while (slots >= 4 && pl->p_bufs < 4 && fixed + (size_t)(2 * N * 256) + (size_t)slots * kSlotBytes <= cap) {
+            ++pl->p_bufs;
+            fixed += (size_t)(2 * N * 256);
+        }
         if (slots < 4) {
             pl->p_bufs = 1;
             fixed -= (size_t)(2 * N * 256);

@@ -132,7 +132,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.q_empty = o; o += 16;
         B.s_full = o; o += 8 * kMaxCache;
         B.s_free = o; o += 8 * kMaxCache;
-        B.p_full = o; o += 16;
+        B.p_full = o; o += 32;  // up to four P buffers
         B.p_empty = o; o += 32;  // four: indexed by tile sequence number mod 4 (see the P2 loop)
         B.o_full = o; o += 8;
         B.o_empty = o; o += 8;
@@ -165,9 +165,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         if (i < 2) {
             mbar_init(B.q_full + 8 * i, 1);
             mbar_init(B.q_empty + 8 * i, 1);
-            mbar_init(B.p_full + 8 * i, kSW);
         }
-        if (i < 4) mbar_init(B.p_empty + 8 * i, 1);
+        if (i < 4) {
+            mbar_init(B.p_full + 8 * i, kSW);
+            mbar_init(B.p_empty + 8 * i, 1);
+        }
     } else if (threadIdx.x == kMaxCache + 8) {
         mbar_init(B.o_full, 1);
         mbar_init(B.o_empty, kSW);
