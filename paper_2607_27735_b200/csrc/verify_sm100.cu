@@ -111,6 +111,9 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         // barriers and small arrays; the rest is the K/V tile ring
         pl->p_bufs = 2;
         fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544;
+#ifdef SPEC_TRACE
+        fixed += 1536;  // stamps of the development trace
+#endif
         slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
         if (slots > 8) slots = 8;
         // more P buffers (up to four) where they cost no K/V slot: the P V product of a tile then has two tiles
