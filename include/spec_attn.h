@@ -124,6 +124,22 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
                      void* cuda_stream);
 
 /*
+ * spec_verify_attn with option flags.  SPEC_VERIFY_ACCUMULATE_STATS: the statistic of this call
+ * is ADDED to what stats[layer, b, h, 0:ctx_len[b]) already holds instead of replacing it, so that
+ * the window of Eq. 3 can span the rows of several verification passes when one pass has fewer
+ * than W rows (the caller keeps the running sums: zero-fill before the first pass, and subtract or
+ * restart when rows leave the window; positions appended since the previous pass must hold 0).
+ * Two passes over the same cache whose rows are consecutive, the second with the flag set,
+ * give the statistic of one pass over all their rows (with W >= the total).  flags == 0 is
+ * spec_verify_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
+ */
+enum { SPEC_VERIFY_ACCUMULATE_STATS = 1 };
+int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                        int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
+                        float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,
+                        uint32_t flags, void* cuda_stream);
+
+/*
  * Recall selection (Eq. 4).  For each problem with T' = sel_len[b]:
  *   T' <= k_total : indices = 0..T'-1, n = T'.
  *   otherwise     : sink [0,k_sink) U the k_mid = k_total-k_sink-k_recent positions of

@@ -17,14 +17,16 @@ LIB_PATH = os.path.join(_HERE, "libspec_attn.so")
 
 WS_VERIFY, WS_SELECT, WS_DRAFT = 0, 1, 2
 VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCGEN05_CACHED = 0, 1, 2, 3, 4
-VERIFY_TCGEN05_CACHED_2PASS = 5  # reported by last_verify_impl() only: the score-cache kernel on two halves of the rows
+VERIFY_TCGEN05_CACHED_2PASS = 5
+# ^ reported by last_verify_impl() only: the score-cache kernel on two halves of the rows
+VERIFY_ACCUMULATE_STATS = 1  # flag of spec_verify_attn_ex: add to the statistic instead of replacing it
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
     "spec_read_status", "spec_set_verify_impl", "spec_last_verify_impl", "spec_launch_count",
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
-    "spec_token_argmax", "spec_accept_greedy",
+    "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
 ]
 
 
@@ -62,6 +64,8 @@ def load() -> ctypes.CDLL:
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
         lib.spec_verify_attn.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
                                          i64, vp, ctypes.c_size_t, vp]
+        lib.spec_verify_attn_ex.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
+                                            i64, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
         lib.spec_select_recall.argtypes = [vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp,
                                            ctypes.c_size_t, vp]
         lib.spec_sparse_draft_attn.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
@@ -126,8 +130,9 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 
 def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
-                     stat_stride=None, workspace=None, want_lse=True):
-    """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``."""
+                     stat_stride=None, workspace=None, want_lse=True, accumulate=False):
+    """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``.
+    ``accumulate`` adds this call's statistic to the given ``stats`` (spec_verify_attn_ex)."""
     lib = load()
     L, B, n_q, Hq, D = q.shape
     dev = q.device
@@ -142,12 +147,16 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
         stats = torch.zeros(L, B, kv.n_kv_heads, stat_stride, dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(WS_VERIFY, kv, n_q, max_ctx_len), dev)
-    rc = lib.spec_verify_attn(
-        ctypes.byref(s), _dev(q, torch.bfloat16, "q"), n_q, _dev(ctx_len, torch.int32, "ctx_len"),
-        max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
-        None if lse is None else _dev(lse, torch.float32, "lse"),
-        _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel(),
-        _stream())
+    if accumulate and stats is None:
+        raise ValueError("accumulate needs the stats tensor that holds the running sums")
+    args = (ctypes.byref(s), _dev(q, torch.bfloat16, "q"), n_q, _dev(ctx_len, torch.int32, "ctx_len"),
+            max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
+            None if lse is None else _dev(lse, torch.float32, "lse"),
+            _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel())
+    if accumulate:
+        rc = lib.spec_verify_attn_ex(*args, VERIFY_ACCUMULATE_STATS, _stream())
+    else:
+        rc = lib.spec_verify_attn(*args, _stream())
     if rc != 0:
         raise SpecError(rc, "spec_verify_attn")
     return out, lse, stats, workspace

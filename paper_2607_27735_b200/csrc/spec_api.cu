@@ -80,6 +80,16 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
                      int32_t max_ctx_len, int32_t stat_window, float* out, float* lse, float* stats,
                      int64_t stat_stride, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
+    return spec_verify_attn_ex(kv, q, n_q, ctx_len, max_ctx_len, stat_window, out, lse, stats, stat_stride, workspace,
+                               workspace_bytes, 0u, cuda_stream);
+}
+
+int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                        int32_t max_ctx_len, int32_t stat_window, float* out, float* lse, float* stats,
+                        int64_t stat_stride, void* workspace, size_t workspace_bytes, uint32_t flags,
+                        void* cuda_stream)
+{
+    if (flags & ~(uint32_t)SPEC_VERIFY_ACCUMULATE_STATS) return SPEC_ERR_INVALID_ARG;
     VerifyArgs a;
     const int rc = make_view(kv, &a.kv);
     if (rc != SPEC_OK) return rc;
@@ -103,6 +113,7 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
     a.stat_stride = stat_stride;
     a.workspace = workspace;
     a.workspace_bytes = workspace_bytes;
+    a.stat_accumulate = (flags & SPEC_VERIFY_ACCUMULATE_STATS) ? 1 : 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int impl = g_verify_impl.load();
     if (impl != SPEC_VERIFY_GENERIC) {

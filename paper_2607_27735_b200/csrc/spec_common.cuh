@@ -90,6 +90,7 @@ struct VerifyArgs {
     int64_t stat_stride;
     void* workspace;
     size_t workspace_bytes;
+    int stat_accumulate;  // add this call's statistic to what stats[] holds instead of overwriting it
 };
 
 size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);

@@ -230,7 +230,8 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
         if (threadIdx.x < kTK && key0 + threadIdx.x < T) {
             float cs = 0.f;
             for (int r = stat_r0; r < R; ++r) cs += S[r * kSP + threadIdx.x];
-            a.stats[prob * a.stat_stride + key0 + threadIdx.x] = cs;
+            float* dst = a.stats + prob * a.stat_stride + key0 + threadIdx.x;
+            *dst = a.stat_accumulate ? *dst + cs : cs;
         }
         const int nk = min(kTK, T - key0);
         for (int kl = 0; kl < nk; kl += 4) {

@@ -226,13 +226,13 @@ __global__ void shorten_ctx_kernel(const int32_t* ctx_len, int by, int32_t* out)
 
 // stats <- (first part's value where it wrote one) + second part's value
 __global__ void add_stats_kernel(float* stats, int64_t stat_stride, const float* second, int64_t second_stride,
-                                 const int32_t* ctx_len, int nB, int n_kv_heads)
+                                 const int32_t* ctx_len, int nB, int n_kv_heads, int accumulate)
 {
     const int T = ctx_len[0];
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < (int64_t)n_kv_heads * T;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int h = (int)(i / T), key = (int)(i - (int64_t)h * T);
-        const float first = key < T - nB ? stats[h * stat_stride + key] : 0.f;
+        const float first = (key < T - nB || accumulate) ? stats[h * stat_stride + key] : 0.f;  // the first part wrote keys < T - nB
         stats[h * stat_stride + key] = first + second[h * second_stride + key];
     }
 }
@@ -285,11 +285,12 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
         pb.first_stat_row = a.first_stat_row > sp.nA ? a.first_stat_row - sp.nA : 0;
         pb.stats = second;
         pb.stat_stride = sp.stat_stride;
+        pb.stat_accumulate = 0;
         pb.workspace_bytes = sp.main_bytes;
         rc = verify_sm100_launch(pb, 2, stream, nullptr);
         if (rc != SPEC_OK) return rc;
         add_stats_kernel<<<sm_count(), 256, 0, stream>>>(a.stats, a.stat_stride, second, sp.stat_stride, a.ctx_len, sp.nB,
-                                                         a.kv.n_kv_heads);
+                                                         a.kv.n_kv_heads, a.stat_accumulate);
         count_launch(1);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
         if (used_variant) *used_variant = 3;

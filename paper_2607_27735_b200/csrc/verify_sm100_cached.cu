@@ -871,7 +871,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_free + 8 * c);
-                    if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st;
+                    if (key < sg.T) {
+                        float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
+                        *dst = p.a.stat_accumulate ? *dst + st : st;
+                    }
                 }
             }
             else {

@@ -575,7 +575,11 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                             ok = mbar_wait(B.stat_full + 8 * sq, sqph, ctl, 28);
                             if (!ok) break;
                             w_stat += TCLK() - tw2;
-                            if (key < sg.T) p.a.stats[sg.prob * p.a.stat_stride + key] = st + stat_tmp[sq * 128 + key_l];
+                            if (key < sg.T) {
+                                float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
+                                const float v = st + stat_tmp[sq * 128 + key_l];
+                                *dst = p.a.stat_accumulate ? *dst + v : v;
+                            }
                         }
                     }
                     if (!ok) break;

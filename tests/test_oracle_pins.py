@@ -427,3 +427,26 @@ def test_accept_prefix_rule_on_constructed_cases():
     # k = 0 (plain decoding step): one row, no draft
     _, m, nxt = oracle.accept_greedy(lg[:, :1].contiguous(), torch.zeros(1, 0, dtype=torch.int32))
     assert m.tolist() == [0] and nxt.tolist() == [5]
+
+
+# ---- the statistic is additive over consecutive verification passes (Eq. 3 as a sum over rows) ----
+
+def test_statistic_of_two_consecutive_passes_adds_up():
+    """Rows a then b, verified in two passes (the first against the context that ends where the
+    second one's rows begin), give the attention outputs and the Eq. 3 sums of one pass over a + b
+    rows: the window is a sum over query rows, each row's probabilities depend on its own prefix
+    only.  Catches a window or causal-offset mistake in the oracle without retyping its formula."""
+    from paper_2607_27735_b200 import inputs
+    a, b = 3, 4
+    cfg = inputs.small_config(ctx=(300, 300), n_q=a + b, n_q_heads=8, n_kv_heads=2, planted=3, seed=21)
+    case = inputs.make_case(cfg)
+    T = int(case.ctx_len[0])
+    out, lse, stats = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16)
+    qa = case.q_verify[:, :, :a].contiguous()
+    qb = case.q_verify[:, :, a:].contiguous()
+    out_a, lse_a, st_a = oracle.verify_attn(case.kv, qa, case.ctx_len - b, 16, stat_stride=T)
+    out_b, lse_b, st_b = oracle.verify_attn(case.kv, qb, case.ctx_len, 16, stat_stride=T)
+    assert (out[:, :, :a] - out_a).abs().max().item() < 1e-12 and (out[:, :, a:] - out_b).abs().max().item() < 1e-12
+    assert (lse[:, :, :a] - lse_a).abs().max().item() < 1e-12 and (lse[:, :, a:] - lse_b).abs().max().item() < 1e-12
+    assert (stats - (st_a + st_b)).abs().max().item() < 1e-12
+    assert st_a[..., T - b:].abs().max().item() == 0.0   # the first pass cannot see the second one's keys
