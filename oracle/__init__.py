@@ -84,10 +84,11 @@ def _kv_struct(kv):
     return s, (k, v, pt)
 
 
-def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None):
+def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None, per_head=False):
     """Full-context verification attention and the Eq. 3 statistic.
 
-    Returns ``(out fp64 [L,B,n_q,Hq,D], lse fp64 [L,B,n_q,Hq], stats fp64 [L,B,Hkv,stat_stride])``.
+    Returns ``(out fp64 [L,B,n_q,Hq,D], lse fp64 [L,B,n_q,Hq], stats fp64 [L,B,Hkv,stat_stride])``;
+    with ``per_head`` the statistic is kept per attention head: ``[L,B,Hq,stat_stride]``.
     """
     lib = _load()
     s, keep = _kv_struct(kv)
@@ -99,12 +100,12 @@ def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None):
         stat_stride = int(ctx_len.max())
     out = torch.zeros(L, B, n_q, Hq, D, dtype=torch.float64)
     lse = torch.zeros(L, B, n_q, Hq, dtype=torch.float64)
-    stats = torch.zeros(L, B, kv.n_kv_heads, stat_stride, dtype=torch.float64)
-    rc = lib.oracle_verify_attn(
+    stats = torch.zeros(L, B, Hq if per_head else kv.n_kv_heads, stat_stride, dtype=torch.float64)
+    rc = lib.oracle_verify_attn_ex(
         ctypes.byref(s), ctypes.c_void_p(q.data_ptr()), ctypes.c_int(n_q),
         ctypes.c_void_p(ctx_len.data_ptr()), ctypes.c_int(stat_window),
         ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
-        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stat_stride),
+        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stat_stride), ctypes.c_int(1 if per_head else 0),
     )
     if rc != 0:
         raise ValueError("oracle_verify_attn: invalid arguments")
@@ -134,8 +135,9 @@ def select_recall(stats, sel_len, k_sink, k_recent, k_total):
     return indices, n_idx
 
 
-def sparse_draft_attn(kv, q, indices, n_idx, tail_start, cur_len):
-    """Eq. 5 sparse attention of one drafting query per sequence.
+def sparse_draft_attn(kv, q, indices, n_idx, tail_start, cur_len, per_head=False):
+    """Eq. 5 sparse attention of one drafting query per sequence; ``indices`` is ``[L,B,Hkv,k_total]``,
+    or ``[L,B,Hq,k_total]`` with ``per_head`` (every attention head gathers its own set).
 
     Returns ``(out fp64 [L,B,Hq,D], lse fp64 [L,B,Hq])``.
     """
@@ -151,11 +153,12 @@ def sparse_draft_attn(kv, q, indices, n_idx, tail_start, cur_len):
     k_total = indices.shape[-1]
     out = torch.zeros(L, B, Hq, D, dtype=torch.float64)
     lse = torch.zeros(L, B, Hq, dtype=torch.float64)
-    rc = lib.oracle_sparse_draft_attn(
+    assert indices.shape[2] == (Hq if per_head else kv.n_kv_heads)
+    rc = lib.oracle_sparse_draft_attn_ex(
         ctypes.byref(s), ctypes.c_void_p(q.data_ptr()), ctypes.c_void_p(indices.data_ptr()),
         ctypes.c_void_p(n_idx.data_ptr()), ctypes.c_int(k_total),
         ctypes.c_void_p(tail_start.data_ptr()), ctypes.c_void_p(cur_len.data_ptr()),
-        ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
+        ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()), ctypes.c_int(1 if per_head else 0),
     )
     if rc != 0:
         raise ValueError("oracle_sparse_draft_attn: invalid arguments")

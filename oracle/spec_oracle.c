@@ -97,9 +97,12 @@ static double logit(const oracle_kv_t *kv, const uint16_t *qrow, int layer, int 
  * Row j attends keys 0..pos_j (causal, bottom-right aligned).  The statistic sums the
  * probabilities of the last min(W, n_q) rows and of the G query heads that share a KV head.
  */
-int oracle_verify_attn(const oracle_kv_t *kv, const uint16_t *q, int n_q, const int32_t *ctx_len,
-                       int stat_window, double *out, double *lse, double *stats,
-                       int64_t stat_stride)
+/* per_head = 0: stats [L, B, Hkv, stat_stride], the score summed over the query heads of a KV head
+ * (the reading used by the hot path).  per_head = 1: stats [L, B, Hq, stat_stride], one score per
+ * attention head, Eq. 3 as printed ("per-head" indices). */
+int oracle_verify_attn_ex(const oracle_kv_t *kv, const uint16_t *q, int n_q, const int32_t *ctx_len,
+                          int stat_window, double *out, double *lse, double *stats,
+                          int64_t stat_stride, int per_head)
 {
     const int L = kv->n_layers, B = kv->batch, Hq = kv->n_q_heads, Hkv = kv->n_kv_heads;
     const int D = kv->head_dim, G = Hq / Hkv;
@@ -115,12 +118,17 @@ int oracle_verify_attn(const oracle_kv_t *kv, const uint16_t *q, int n_q, const 
         for (int b = 0; b < B; ++b)
             for (int h = 0; h < Hkv; ++h) {
                 const int64_t T = ctx_len[b];
-                double *st = stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
                 double *p = (double *)malloc(sizeof(double) * (size_t)T);
-                for (int64_t i = 0; i < T; ++i) st[i] = 0.0;
+                for (int g = 0; g < (per_head ? G : 1); ++g) {
+                    double *z = per_head ? stats + (((int64_t)layer * B + b) * Hq + h * G + g) * stat_stride
+                                         : stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
+                    for (int64_t i = 0; i < T; ++i) z[i] = 0.0;
+                }
                 for (int j = 0; j < n_q; ++j)
                     for (int g = 0; g < G; ++g) {
                         const int qh = h * G + g;
+                        double *st = per_head ? stats + (((int64_t)layer * B + b) * Hq + qh) * stat_stride
+                                              : stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
                         const int64_t pos = T - n_q + j; /* last visible key */
                         const int64_t row = (((int64_t)layer * B + b) * n_q + j) * Hq + qh;
                         const uint16_t *qrow = q + row * D;
@@ -147,6 +155,13 @@ int oracle_verify_attn(const oracle_kv_t *kv, const uint16_t *q, int n_q, const 
                 free(p);
             }
     return 0;
+}
+
+int oracle_verify_attn(const oracle_kv_t *kv, const uint16_t *q, int n_q, const int32_t *ctx_len,
+                       int stat_window, double *out, double *lse, double *stats,
+                       int64_t stat_stride)
+{
+    return oracle_verify_attn_ex(kv, q, n_q, ctx_len, stat_window, out, lse, stats, stat_stride, 0);
 }
 
 /* ---- Eq. 4: recall selection ------------------------------------------------------------- */
@@ -224,9 +239,12 @@ int oracle_select_recall(const float *stats, int64_t stat_stride, int n_layers, 
  *   tail [tail_start[b], cur_len[b]); softmax is renormalised over exactly that set.
  *   out fp64 [n_layers, batch, Hq, D]; lse fp64 [n_layers, batch, Hq] or NULL
  */
-int oracle_sparse_draft_attn(const oracle_kv_t *kv, const uint16_t *q, const int32_t *indices,
-                             const int32_t *n_idx, int k_total, const int32_t *tail_start,
-                             const int32_t *cur_len, double *out, double *lse)
+/* per_head = 0: indices [L, B, Hkv, k_total], one set per KV head shared by its query heads.
+ * per_head = 1: indices [L, B, Hq, k_total], every attention head gathers its own set (Eq. 5 as
+ * printed); K and V still come from the head's KV head. */
+int oracle_sparse_draft_attn_ex(const oracle_kv_t *kv, const uint16_t *q, const int32_t *indices,
+                                const int32_t *n_idx, int k_total, const int32_t *tail_start,
+                                const int32_t *cur_len, double *out, double *lse, int per_head)
 {
     const int L = kv->n_layers, B = kv->batch, Hq = kv->n_q_heads, Hkv = kv->n_kv_heads;
     const int D = kv->head_dim, G = Hq / Hkv;
@@ -236,17 +254,17 @@ int oracle_sparse_draft_attn(const oracle_kv_t *kv, const uint16_t *q, const int
     for (int layer = 0; layer < L; ++layer)
         for (int b = 0; b < B; ++b)
             for (int h = 0; h < Hkv; ++h) {
-                const int64_t prob = ((int64_t)layer * B + b) * Hkv + h;
-                const int32_t *idx = indices + prob * k_total;
-                const int n_rec = n_idx[prob];
                 const int n_tail = cur_len[b] > tail_start[b] ? cur_len[b] - tail_start[b] : 0;
-                const int n = n_rec + n_tail;
-                int32_t *keys = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
-                double *p = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
-                for (int i = 0; i < n_rec; ++i) keys[i] = idx[i];
-                for (int i = 0; i < n_tail; ++i) keys[n_rec + i] = tail_start[b] + i;
+                int32_t *keys = (int32_t *)malloc(sizeof(int32_t) * (size_t)(k_total + n_tail + 1));
+                double *p = (double *)malloc(sizeof(double) * (size_t)(k_total + n_tail + 1));
                 for (int g = 0; g < G; ++g) {
                     const int64_t row = ((int64_t)layer * B + b) * Hq + h * G + g;
+                    const int64_t prob = per_head ? row : ((int64_t)layer * B + b) * Hkv + h;
+                    const int32_t *idx = indices + prob * k_total;
+                    const int n_rec = n_idx[prob];
+                    const int n = n_rec + n_tail;
+                    for (int i = 0; i < n_rec; ++i) keys[i] = idx[i];
+                    for (int i = 0; i < n_tail; ++i) keys[n_rec + i] = tail_start[b] + i;
                     const uint16_t *qrow = q + row * D;
                     double m = -INFINITY, denom = 0.0;
                     for (int i = 0; i < n; ++i) {
@@ -270,4 +288,11 @@ int oracle_sparse_draft_attn(const oracle_kv_t *kv, const uint16_t *q, const int
                 free(p);
             }
     return 0;
+}
+
+int oracle_sparse_draft_attn(const oracle_kv_t *kv, const uint16_t *q, const int32_t *indices,
+                             const int32_t *n_idx, int k_total, const int32_t *tail_start,
+                             const int32_t *cur_len, double *out, double *lse)
+{
+    return oracle_sparse_draft_attn_ex(kv, q, indices, n_idx, k_total, tail_start, cur_len, out, lse, 0);
 }

@@ -450,3 +450,48 @@ def test_statistic_of_two_consecutive_passes_adds_up():
     assert (lse[:, :, :a] - lse_a).abs().max().item() < 1e-12 and (lse[:, :, a:] - lse_b).abs().max().item() < 1e-12
     assert (stats - (st_a + st_b)).abs().max().item() < 1e-12
     assert st_a[..., T - b:].abs().max().item() == 0.0   # the first pass cannot see the second one's keys
+
+
+# ---- per-attention-head form of Eq. 3 / Eq. 5 (the paper's literal "per-head" indices) ----
+
+def test_per_head_statistic_sums_to_the_group_statistic():
+    from paper_2607_27735_b200 import inputs
+    cfg = inputs.small_config(ctx=(200, 260), batch=2, n_q=5, n_q_heads=8, n_kv_heads=2, planted=2, seed=31)
+    case = inputs.make_case(cfg)
+    out, lse, st = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16)
+    out_h, lse_h, st_h = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16, per_head=True)
+    L, B, Hq, S = st_h.shape
+    assert torch.equal(out, out_h) and torch.equal(lse, lse_h)
+    assert (st_h.view(L, B, 2, 4, S).sum(dim=3) - st).abs().max().item() < 1e-12
+    # every head's last-row probabilities sum to 1 over the keys, so each head's statistic sums to n_q
+    for b in range(B):
+        T = int(case.ctx_len[b])
+        assert (st_h[:, b, :, :T].sum(dim=-1) - cfg.n_q).abs().max().item() < 1e-9
+    # one query head per KV head: the two forms are the same thing
+    cfg1 = inputs.small_config(ctx=(150, 150), n_q=3, n_q_heads=2, n_kv_heads=2, seed=32)
+    c1 = inputs.make_case(cfg1)
+    assert torch.equal(oracle.verify_attn(c1.kv, c1.q_verify, c1.ctx_len, 16)[2],
+                       oracle.verify_attn(c1.kv, c1.q_verify, c1.ctx_len, 16, per_head=True)[2])
+
+
+def test_per_head_draft_with_shared_sets_is_the_group_draft():
+    from paper_2607_27735_b200 import inputs
+    cfg = inputs.small_config(ctx=(300, 300), n_q=3, n_q_heads=8, n_kv_heads=2, k_total=64, k_recent=8, seed=33)
+    case = inputs.make_case(cfg)
+    _, _, st = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16)
+    idx, n = oracle.select_recall(st.float(), case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total)
+    cur = case.ctx_len + 1
+    q = case.q_draft[0].contiguous()
+    ref_out, ref_lse = oracle.sparse_draft_attn(case.kv, q, idx, n, case.ctx_len, cur)
+    idx_h = idx.repeat_interleave(4, dim=2).contiguous()     # every head of a group gets the group's set
+    n_h = n.repeat_interleave(4, dim=2).contiguous()
+    out_h, lse_h = oracle.sparse_draft_attn(case.kv, q, idx_h, n_h, case.ctx_len, cur, per_head=True)
+    assert torch.equal(ref_out, out_h) and torch.equal(ref_lse, lse_h)
+    # a head whose own set is the whole context attends densely: equals the verification row at that position
+    full = torch.arange(300, dtype=torch.int32).view(1, 1, 1, 300).expand(1, 1, 8, 300).contiguous()
+    n_full = torch.full((1, 1, 8), 300, dtype=torch.int32)
+    dense, _ = oracle.sparse_draft_attn(case.kv, q, full, n_full, case.ctx_len, case.ctx_len, per_head=True)
+    kv_plus = case.kv
+    qv = q.view(1, 1, 1, 8, -1).contiguous()
+    ver, _, _ = oracle.verify_attn(kv_plus, qv, case.ctx_len, 16)
+    assert (dense - ver[:, :, 0]).abs().max().item() < 1e-12
