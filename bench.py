@@ -320,7 +320,7 @@ def run_gpu(args):
         import dataclasses
         cfg = dataclasses.replace(cfg, seed=cfg.seed + 101 * rank)
     case = inputs.make_case(cfg, device=dev)
-    run = runner.SpecStepRunner(case, fold_layers=args.fold_layers)
+    run = runner.SpecStepRunner(case, fold_layers=args.fold_layers, per_head=args.per_head)
     counts = run.capture()
     launches_per_step = sum(counts)
 
@@ -434,7 +434,11 @@ def run_gpu(args):
         fold = L if args.fold_layers else 1
         line["roofline"]["traffic"] = t["verify"] * fold
         line["draft_roofline"]["traffic"] = t["draft"] * fold
-    if args.recall_steps > 0 and case.planted_pos is not None:
+    if args.per_head:
+        line["config"]["index_sets"] = "per attention head"
+        line["roofline"]["traffic"] = None
+        line["draft_roofline"]["traffic"] = None
+    if args.recall_steps > 0 and case.planted_pos is not None and not args.per_head:
         line["recall"] = drift_recall(case, run, args.recall_steps)
     if not args.no_controller:
         line["controller"] = controller_bench(cfg, dev, peak)
@@ -460,6 +464,9 @@ def main():
                     help="after timing, run this many rounds with drifting planted positions and report recall")
     ap.add_argument("--no-controller", action="store_true",
                     help="skip the speculation-length controller's own timing (reported beside the step)")
+    ap.add_argument("--per-head", action="store_true",
+                    help="one score and one index set per attention head (Eq. 3 / Eq. 5 as printed) instead of "
+                         "per KV head: the draft gathers group-size times the rows")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()

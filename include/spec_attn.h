@@ -132,8 +132,16 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
  * Two passes over the same cache whose rows are consecutive, the second with the flag set,
  * give the statistic of one pass over all their rows (with W >= the total).  flags == 0 is
  * spec_verify_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
+ *
+ * SPEC_VERIFY_STATS_PER_QUERY_HEAD: Eq. 3 as printed, one score per attention head: stats is
+ * fp32 [n_layers, batch, n_q_heads, stat_stride] and head hq's entry sums the probabilities of
+ * hq's own window rows only (the default sums them over the query heads of a KV head).  The
+ * per-KV-head statistic is the sum of its group's per-head statistics.  Served by the score-cache
+ * tcgen05 kernel when the group size divides 8 and the shape fits its cache, else by the generic
+ * kernels.  spec_select_recall then runs with n_kv_heads = n_q_heads, and the draft call takes
+ * SPEC_DRAFT_INDICES_PER_QUERY_HEAD.
  */
-enum { SPEC_VERIFY_ACCUMULATE_STATS = 1 };
+enum { SPEC_VERIFY_ACCUMULATE_STATS = 1, SPEC_VERIFY_STATS_PER_QUERY_HEAD = 2 };
 int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
                         int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
                         float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,
@@ -270,6 +278,20 @@ int spec_controller_update(float* state, const float* entropy, int32_t k,
 int spec_controller_select(const float* state, const float* entropy, int32_t n,
                            const int32_t* cand, int32_t n_cand, float c_d, float c_v,
                            int32_t* k_star, float* p_out, float* score_out, void* cuda_stream);
+
+/*
+ * spec_sparse_draft_attn with option flags.  SPEC_DRAFT_INDICES_PER_QUERY_HEAD: Eq. 5 as printed,
+ * every attention head gathers its own index set: indices is int32 [n_layers, batch, n_q_heads,
+ * k_total] and n_indices int32 [n_layers, batch, n_q_heads]; K and V rows still come from the
+ * head's KV head (hq / group).  The gathered bytes grow by the group size.  flags == 0 is
+ * spec_sparse_draft_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
+ */
+enum { SPEC_DRAFT_INDICES_PER_QUERY_HEAD = 1 };
+int spec_sparse_draft_attn_ex(const spec_kv_t* kv, const void* q, const int32_t* indices,
+                              const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
+                              const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
+                              void* workspace, size_t workspace_bytes, uint32_t flags,
+                              void* cuda_stream);
 
 /*
  * Bytes of workspace entry point `which` needs for this cache description.  n_q and

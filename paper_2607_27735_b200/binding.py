@@ -20,6 +20,8 @@ VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCG
 VERIFY_TCGEN05_CACHED_2PASS = 5
 # ^ reported by last_verify_impl() only: the score-cache kernel on two halves of the rows
 VERIFY_ACCUMULATE_STATS = 1  # flag of spec_verify_attn_ex: add to the statistic instead of replacing it
+VERIFY_STATS_PER_QUERY_HEAD = 2  # flag of spec_verify_attn_ex: one score per attention head
+DRAFT_INDICES_PER_QUERY_HEAD = 1  # flag of spec_sparse_draft_attn_ex: one index set per attention head
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
@@ -27,6 +29,7 @@ EXPORTS = [
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
     "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
+    "spec_sparse_draft_attn_ex",
 ]
 
 
@@ -66,6 +69,8 @@ def load() -> ctypes.CDLL:
                                          i64, vp, ctypes.c_size_t, vp]
         lib.spec_verify_attn_ex.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
                                             i64, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
+        lib.spec_sparse_draft_attn_ex.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
+                                                  vp, vp, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
         lib.spec_select_recall.argtypes = [vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp,
                                            ctypes.c_size_t, vp]
         lib.spec_sparse_draft_attn.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
@@ -130,9 +135,10 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 
 def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
-                     stat_stride=None, workspace=None, want_lse=True, accumulate=False):
+                     stat_stride=None, workspace=None, want_lse=True, accumulate=False, per_head=False):
     """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``.
-    ``accumulate`` adds this call's statistic to the given ``stats`` (spec_verify_attn_ex)."""
+    ``accumulate`` adds this call's statistic to the given ``stats``; ``per_head`` keeps one score per
+    attention head (``stats`` is ``[L, B, n_q_heads, stride]``); both go through spec_verify_attn_ex."""
     lib = load()
     L, B, n_q, Hq, D = q.shape
     dev = q.device
@@ -144,7 +150,8 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
     if lse is None and want_lse:
         lse = torch.empty(L, B, n_q, Hq, dtype=torch.float32, device=dev)
     if stats is None:
-        stats = torch.zeros(L, B, kv.n_kv_heads, stat_stride, dtype=torch.float32, device=dev)
+        stats = torch.zeros(L, B, kv.n_q_heads if per_head else kv.n_kv_heads, stat_stride,
+                            dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(WS_VERIFY, kv, n_q, max_ctx_len), dev)
     if accumulate and stats is None:
@@ -153,8 +160,11 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
             max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
             None if lse is None else _dev(lse, torch.float32, "lse"),
             _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel())
-    if accumulate:
-        rc = lib.spec_verify_attn_ex(*args, VERIFY_ACCUMULATE_STATS, _stream())
+    if stats.shape[2] != (kv.n_q_heads if per_head else kv.n_kv_heads):
+        raise ValueError("stats: wrong head count for this mode")
+    if accumulate or per_head:
+        flags = (VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0)
+        rc = lib.spec_verify_attn_ex(*args, flags, _stream())
     else:
         rc = lib.spec_verify_attn(*args, _stream())
     if rc != 0:
@@ -217,8 +227,9 @@ def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, 
 
 
 def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_tail, out=None,
-                           lse=None, workspace=None, want_lse=True):
-    """Eq. 5 sparse draft attention; returns ``(out, lse, workspace)``."""
+                           lse=None, workspace=None, want_lse=True, per_head=False):
+    """Eq. 5 sparse draft attention; returns ``(out, lse, workspace)``.  ``per_head``: ``indices`` is
+    ``[L, B, n_q_heads, k_total]``, one set per attention head (spec_sparse_draft_attn_ex)."""
     lib = load()
     L, B, Hq, D = q.shape
     dev = q.device
@@ -230,13 +241,18 @@ def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_t
         lse = torch.empty(L, B, Hq, dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = alloc_workspace(workspace_bytes(WS_DRAFT, kv, k_total=k_total + max_tail), dev)
-    rc = lib.spec_sparse_draft_attn(
-        ctypes.byref(s), _dev(q, torch.bfloat16, "q"), _dev(indices, torch.int32, "indices"),
-        _dev(n_indices, torch.int32, "n_indices"), k_total,
-        _dev(tail_start, torch.int32, "tail_start"), _dev(cur_len, torch.int32, "cur_len"),
-        max_tail, _dev(out, torch.float32, "out"),
-        None if lse is None else _dev(lse, torch.float32, "lse"), workspace.data_ptr(),
-        workspace.numel(), _stream())
+    if indices.shape[2] != (kv.n_q_heads if per_head else kv.n_kv_heads):
+        raise ValueError("indices: wrong head count for this mode")
+    args = (ctypes.byref(s), _dev(q, torch.bfloat16, "q"), _dev(indices, torch.int32, "indices"),
+            _dev(n_indices, torch.int32, "n_indices"), k_total,
+            _dev(tail_start, torch.int32, "tail_start"), _dev(cur_len, torch.int32, "cur_len"),
+            max_tail, _dev(out, torch.float32, "out"),
+            None if lse is None else _dev(lse, torch.float32, "lse"), workspace.data_ptr(),
+            workspace.numel())
+    if per_head:
+        rc = lib.spec_sparse_draft_attn_ex(*args, DRAFT_INDICES_PER_QUERY_HEAD, _stream())
+    else:
+        rc = lib.spec_sparse_draft_attn(*args, _stream())
     if rc != 0:
         raise SpecError(rc, "spec_sparse_draft_attn")
     return out, lse, workspace

@@ -219,8 +219,9 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
     // mode 0: recalled rows and the masked padding of the last chunk (readable before the
     // dependency wait), 1: rows of the dense tail only, 2: all.
     const int slot = tid / CH, piece = tid % CH;
-    const __nv_bfloat16* kbase = a.kv.k + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
-    const __nv_bfloat16* vbase = a.kv.v + layer * a.kv.layer_stride + h * a.kv.head_stride + piece * 8;
+    const int hm = a.head_div > 1 ? h / a.head_div : h;  // the cache head this problem's rows come from
+    const __nv_bfloat16* kbase = a.kv.k + layer * a.kv.layer_stride + hm * a.kv.head_stride + piece * 8;
+    const __nv_bfloat16* vbase = a.kv.v + layer * a.kv.layer_stride + hm * a.kv.head_stride + piece * 8;
     const int32_t* ptab = a.kv.page_table ? a.kv.page_table + (int64_t)b * a.kv.max_pages : nullptr;
     auto gather = [&](int r, int mode, int k0, int k1) {
         const int base = k0 + r * RK;
@@ -279,7 +280,7 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         if (pos >= 0 && pos < cl) {
             const int page = page_of(a.kv, pos);
             const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
-            const int64_t off = layer * a.kv.layer_stride + h * a.kv.head_stride + phys * a.kv.page_stride +
+            const int64_t off = layer * a.kv.layer_stride + hm * a.kv.head_stride + phys * a.kv.page_stride +
                                 (int64_t)(pos - page * a.kv.page_size) * a.kv.slot_stride;
             prefetch_l2(a.kv.k + off, D * 2);
             prefetch_l2(a.kv.v + off, D * 2);

@@ -91,6 +91,7 @@ struct VerifyArgs {
     void* workspace;
     size_t workspace_bytes;
     int stat_accumulate;  // add this call's statistic to what stats[] holds instead of overwriting it
+    int stat_per_head;    // stats is [layers, batch, n_q_heads, stride]: one score per attention head
 };
 
 size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);
@@ -113,6 +114,8 @@ struct DraftArgs {
     float* lse;
     void* workspace;
     size_t workspace_bytes;
+    int head_div;  // K/V of problem head h are read from cache head h / head_div (1 unless every
+                   // attention head carries its own index set)
 };
 size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
 int draft_launch(const DraftArgs& a, cudaStream_t stream);

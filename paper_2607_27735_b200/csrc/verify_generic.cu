@@ -228,10 +228,19 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
         }
         __syncthreads();
         if (threadIdx.x < kTK && key0 + threadIdx.x < T) {
-            float cs = 0.f;
-            for (int r = stat_r0; r < R; ++r) cs += S[r * kSP + threadIdx.x];
-            float* dst = a.stats + prob * a.stat_stride + key0 + threadIdx.x;
-            *dst = a.stat_accumulate ? *dst + cs : cs;
+            if (a.stat_per_head) {  // one score per attention head: rows j * G + g with the same g
+                for (int g = 0; g < G; ++g) {
+                    float cs = 0.f;
+                    for (int r = stat_r0 + g; r < R; r += G) cs += S[r * kSP + threadIdx.x];
+                    float* dst = a.stats + (prob * G + g) * a.stat_stride + key0 + threadIdx.x;
+                    *dst = a.stat_accumulate ? *dst + cs : cs;
+                }
+            } else {
+                float cs = 0.f;
+                for (int r = stat_r0; r < R; ++r) cs += S[r * kSP + threadIdx.x];
+                float* dst = a.stats + prob * a.stat_stride + key0 + threadIdx.x;
+                *dst = a.stat_accumulate ? *dst + cs : cs;
+            }
         }
         const int nk = min(kTK, T - key0);
         for (int kl = 0; kl < nk; kl += 4) {

@@ -111,7 +111,9 @@ struct CBars {  // mbarrier addresses (shared space)
 // NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
 // more, narrower warpgroups hide the latency of the serial softmax sections.
 // LP: the publisher warp combines the LSE partials (few CTAs per head); otherwise the softmax warps do.
-template <int NC, int CG, bool LP>
+// PH: one Eq. 3 score per attention head (stats [.., n_q_heads, stride]) instead of per KV head;
+// the group size must then divide 8.
+template <int NC, int CG, bool LP, bool PH>
 __global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_q, const FastParams p)
@@ -843,6 +845,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     const int t = sg.t0 + c;
                     const int key = t * kTile + key_l;
                     float st = 0.f;
+                    float sth[PH ? 8 : 1];  // PH: column i belongs to head i mod G, and G divides 8
+#pragma unroll
+                    for (int i = 0; i < (PH ? 8 : 1); ++i) sth[i] = 0.f;
 #pragma unroll 1
                     for (int cb = 0; cb < N; cb += 16) {
                         if (cb + 16 <= stat_r0) continue;  // rows outside the statistic window
@@ -860,7 +865,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             pr[i + 2] = __uint_as_float(v[i + 2]) * f.z;
                             pr[i + 3] = __uint_as_float(v[i + 3]) * f.w;
                         }
-                        if (cb >= stat_r0) {
+                        if (PH) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) sth[i & 7] += (cb + i >= stat_r0) ? pr[i] : 0.f;
+                        } else if (cb >= stat_r0) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) st += pr[i];
                         } else {
@@ -871,7 +879,27 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_free + 8 * c);
-                    if (key < sg.T) {
+                    if (PH) {
+                        // fold the eight residues mod 8 down to the G residues mod G
+                        if (G <= 4) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) sth[i] += sth[i + 4];
+                        }
+                        if (G <= 2) {
+                            sth[0] += sth[2];
+                            sth[1] += sth[3];
+                        }
+                        if (G == 1) sth[0] += sth[1];
+                        if (key < sg.T) {
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) {
+                                if (g < G) {
+                                    float* dst = p.a.stats + (sg.prob * G + g) * p.a.stat_stride + key;
+                                    *dst = p.a.stat_accumulate ? *dst + sth[g] : sth[g];
+                                }
+                            }
+                        }
+                    } else if (key < sg.T) {
                         float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
                         *dst = p.a.stat_accumulate ? *dst + st : st;
                     }
@@ -903,11 +931,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
-template <int NC, int CG, bool LP>
+template <int NC, int CG, bool LP, bool PH>
 int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    auto kern = verify_cached_kernel<NC, CG, LP>;
+    auto kern = verify_cached_kernel<NC, CG, LP, PH>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -949,26 +977,25 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
 int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                   int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    const bool lp = fp.cph <= kLsePubMax;
+    const bool lp = fp.cph <= kLsePubMax, ph = fp.a.stat_per_head != 0;
+#define SPEC_CASE(n, nc, cg)                                                                              \
+    case n:                                                                                               \
+        if (ph) return lp ? launch_cfg<nc, cg, true, true>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
+                          : launch_cfg<nc, cg, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
+        return lp ? launch_cfg<nc, cg, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream)             \
+                  : launch_cfg<nc, cg, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
     switch (fp.N) {  // (columns per warpgroup, warpgroups)
-        case 16: return lp ? launch_cfg<8, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<8, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 32: return lp ? launch_cfg<8, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<8, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 48: return lp ? launch_cfg<16, 3, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<16, 3, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 64: return lp ? launch_cfg<16, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<16, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 80: return lp ? launch_cfg<40, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<40, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 96: return lp ? launch_cfg<24, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<24, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 112: return lp ? launch_cfg<56, 2, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<56, 2, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
-        case 128: return lp ? launch_cfg<32, 4, true>(tk, tv, tq, fp, grid, smem_bytes, stream)
-                              : launch_cfg<32, 4, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+        SPEC_CASE(16, 8, 2)
+        SPEC_CASE(32, 8, 4)
+        SPEC_CASE(48, 16, 3)
+        SPEC_CASE(64, 16, 4)
+        SPEC_CASE(80, 40, 2)
+        SPEC_CASE(96, 24, 4)
+        SPEC_CASE(112, 56, 2)
+        SPEC_CASE(128, 32, 4)
         default: return SPEC_ERR_UNSUPPORTED_SHAPE;
     }
+#undef SPEC_CASE
 }
 
 }  // namespace sm100

@@ -21,10 +21,12 @@ from . import binding
 
 
 class SpecStepRunner:
-    def __init__(self, case, fold_layers: bool = False, want_lse: bool = False):
+    def __init__(self, case, fold_layers: bool = False, want_lse: bool = False, per_head: bool = False):
         cfg, kv = case.cfg, case.kv
         self.case, self.cfg, self.kv = case, cfg, kv
         self.fold = fold_layers
+        self.per_head = per_head  # one score and one index set per attention head (Eq. 3 / Eq. 5 as printed)
+        n_sets = kv.n_q_heads if per_head else kv.n_kv_heads
         dev = kv.k.device
         L, B = kv.n_layers, kv.batch
         self.L = L
@@ -32,9 +34,9 @@ class SpecStepRunner:
         self.stat_stride = (self.max_ctx + 127) // 128 * 128
         self.out_v = torch.empty(L, B, cfg.n_q, kv.n_q_heads, kv.head_dim, device=dev)
         self.lse_v = torch.empty(L, B, cfg.n_q, kv.n_q_heads, device=dev) if want_lse else None
-        self.stats = torch.zeros(L, B, kv.n_kv_heads, self.stat_stride, device=dev)
-        self.indices = torch.empty(L, B, kv.n_kv_heads, cfg.k_total, dtype=torch.int32, device=dev)
-        self.n_idx = torch.empty(L, B, kv.n_kv_heads, dtype=torch.int32, device=dev)
+        self.stats = torch.zeros(L, B, n_sets, self.stat_stride, device=dev)
+        self.indices = torch.empty(L, B, n_sets, cfg.k_total, dtype=torch.int32, device=dev)
+        self.n_idx = torch.empty(L, B, n_sets, dtype=torch.int32, device=dev)
         self.out_d = torch.empty(max(cfg.draft_steps, 1), L, B, kv.n_q_heads, kv.head_dim, device=dev)
         self.q_verify = case.q_verify
         self.q_draft = case.q_draft
@@ -54,14 +56,15 @@ class SpecStepRunner:
         if self.fold:
             binding.spec_verify_attn(self.kv, self.q_verify, self.ctx_len, self.max_ctx,
                                      self.cfg.stat_window, out=self.out_v, lse=self.lse_v,
-                                     stats=self.stats, workspace=self.ws_v, want_lse=False)
+                                     stats=self.stats, workspace=self.ws_v, want_lse=False,
+                                     per_head=self.per_head)
             return
         for l in range(self.L):
             binding.spec_verify_attn(
                 self._layers[l], self.q_verify[l:l + 1], self.ctx_len, self.max_ctx,
                 self.cfg.stat_window, out=self.out_v[l:l + 1],
                 lse=None if self.lse_v is None else self.lse_v[l:l + 1],
-                stats=self.stats[l:l + 1], workspace=self.ws_v, want_lse=False)
+                stats=self.stats[l:l + 1], workspace=self.ws_v, want_lse=False, per_head=self.per_head)
 
     def select_phase(self):
         c = self.cfg
@@ -75,13 +78,13 @@ class SpecStepRunner:
                 binding.spec_sparse_draft_attn(
                     self.kv, self.q_draft[j], self.indices, self.n_idx, self.tail_start,
                     self.cur_lens[j], c.draft_steps, out=self.out_d[j], workspace=self.ws_d,
-                    want_lse=False)
+                    want_lse=False, per_head=self.per_head)
                 continue
             for l in range(self.L):
                 binding.spec_sparse_draft_attn(
                     self._layers[l], self.q_draft[j, l:l + 1], self.indices[l:l + 1],
                     self.n_idx[l:l + 1], self.tail_start, self.cur_lens[j], c.draft_steps,
-                    out=self.out_d[j, l:l + 1], workspace=self.ws_d, want_lse=False)
+                    out=self.out_d[j, l:l + 1], workspace=self.ws_d, want_lse=False, per_head=self.per_head)
 
     def step(self):
         self.verify_phase()
@@ -149,4 +152,4 @@ class SpecStepRunner:
     def draft_kv_bytes_per_layer_step(self, j: int) -> int:
         kv, c = self.kv, self.cfg
         rows = sum(min(c.k_total, int(t)) + j + 1 for t in self.ctx_len.tolist())
-        return rows * kv.n_kv_heads * kv.head_dim * 2 * 2
+        return rows * (kv.n_q_heads if self.per_head else kv.n_kv_heads) * kv.head_dim * 2 * 2
