@@ -137,7 +137,7 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
  * fp32 [n_layers, batch, n_q_heads, stat_stride] and head hq's entry sums the probabilities of
  * hq's own window rows only (the default sums them over the query heads of a KV head).  The
  * per-KV-head statistic is the sum of its group's per-head statistics.  Served by the score-cache
- * tcgen05 kernel when the group size divides 8 and the shape fits its cache, else by the generic
+ * tcgen05 kernel for groups of up to 8 heads whose shape fits its cache, else by the generic
  * kernels.  spec_select_recall then runs with n_kv_heads = n_q_heads, and the draft call takes
  * SPEC_DRAFT_INDICES_PER_QUERY_HEAD.
  */

@@ -262,11 +262,11 @@ size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
 int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant)
 {
     if (a.stat_per_head) {
-        // only the score-cache kernel keeps one score per attention head, for groups that divide 8;
+        // only the score-cache kernel keeps one score per attention head, for groups of up to 8;
         // everything else goes to the generic kernels
         const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
         Plan pl;
-        if (variant == 1 || (8 % G) != 0 || !make_plan(a.kv, a.n_q, a.max_ctx_len, 2, &pl))
+        if (variant == 1 || G > 8 || !make_plan(a.kv, a.n_q, a.max_ctx_len, 2, &pl))
             return SPEC_ERR_UNSUPPORTED_SHAPE;
         variant = 2;
     }

@@ -111,8 +111,8 @@ struct CBars {  // mbarrier addresses (shared space)
 // NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
 // more, narrower warpgroups hide the latency of the serial softmax sections.
 // LP: the publisher warp combines the LSE partials (few CTAs per head); otherwise the softmax warps do.
-// PH: one Eq. 3 score per attention head (stats [.., n_q_heads, stride]) instead of per KV head;
-// the group size must then divide 8.
+// PH: one Eq. 3 score per attention head (stats [.., n_q_heads, stride]) instead of per KV head,
+// for groups of at most 8 heads (a short statistic pass when the group size divides 8).
 template <int NC, int CG, bool LP, bool PH>
 __global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -554,6 +554,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         const int c0 = wg * NH;                  // first column of this warpgroup
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int stat_r0 = p.a.first_stat_row * G;
+        const bool ph_fast = (8 % G) == 0;  // per-head statistic: column i of a 16-column chunk is head i mod 8 mod G
         const float cs = p.scale_log2;
         constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
         uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, sfull_par = 0;
@@ -865,9 +866,19 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             pr[i + 2] = __uint_as_float(v[i + 2]) * f.z;
                             pr[i + 3] = __uint_as_float(v[i + 3]) * f.w;
                         }
-                        if (PH) {
+                        if (PH && ph_fast) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) sth[i & 7] += (cb + i >= stat_r0) ? pr[i] : 0.f;
+                        } else if (PH) {
+                            // any group size up to 8: accumulator g takes the columns r with r mod G == g
+                            int g = cb % G;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const float val = (cb + i >= stat_r0) ? pr[i] : 0.f;
+#pragma unroll
+                                for (int t = 0; t < 8; ++t) sth[t] += (g == t) ? val : 0.f;
+                                g = (g + 1 == G) ? 0 : g + 1;
+                            }
                         } else if (cb >= stat_r0) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) st += pr[i];
@@ -880,16 +891,16 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.s_free + 8 * c);
                     if (PH) {
-                        // fold the eight residues mod 8 down to the G residues mod G
-                        if (G <= 4) {
+                        // fast path: fold the eight residues mod 8 down to the G residues mod G
+                        if (ph_fast && G <= 4) {
 #pragma unroll
                             for (int i = 0; i < 4; ++i) sth[i] += sth[i + 4];
                         }
-                        if (G <= 2) {
+                        if (ph_fast && G <= 2) {
                             sth[0] += sth[2];
                             sth[1] += sth[3];
                         }
-                        if (G == 1) sth[0] += sth[1];
+                        if (ph_fast && G == 1) sth[0] += sth[1];
                         if (key < sg.T) {
 #pragma unroll
                             for (int g = 0; g < 8; ++g) {
