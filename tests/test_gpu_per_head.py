@@ -86,3 +86,34 @@ def test_per_head_draft_at_the_8b_shape():
     r_out, r_lse = oracle.sparse_draft_attn(kv.cpu(), q.cpu(), idx.cpu(), n.cpu(), ctx.cpu(), cur.cpu(), per_head=True)
     assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL
     assert (d_lse.cpu().double() - r_lse).abs().max().item() <= TOL
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_per_head_random_shapes(seed):
+    """The randomised shapes of test_gpu_fuzz.py through the per-head calls (score-cache kernel where
+    the shape allows it, generic kernels otherwise)."""
+    from test_gpu_fuzz import draw_shape
+    shape = draw_shape(1000 + seed)
+    if shape["planted"] == 0:
+        shape.update(q_mode="iid", q_std=0.3)
+    cfg = inputs.small_config(name=f"ph{seed}", **shape)
+    case = inputs.make_case(cfg, device="cuda")
+    kv, ctx = case.kv, case.ctx_len
+    out, lse, stats, ws = binding.spec_verify_attn(kv, case.q_verify, ctx, int(ctx.max()), per_head=True)
+    assert binding.read_status(ws) == 0, shape
+    o_out, _, o_stats = oracle.verify_attn(kv.cpu(), case.q_verify.cpu(), ctx.cpu(), 16, stats.shape[-1], per_head=True)
+    assert (out.cpu().double() - o_out).abs().max().item() <= TOL, shape
+    for b in range(cfg.batch):
+        T = int(ctx[b])
+        assert (stats[:, b, :, :T].cpu().double() - o_stats[:, b, :, :T]).abs().max().item() <= TOL, shape
+    idx, n = binding.spec_select_recall(stats, ctx, cfg.k_sink, cfg.k_recent, cfg.k_total)
+    o_idx, o_n = oracle.select_recall(stats.cpu(), ctx.cpu(), cfg.k_sink, cfg.k_recent, cfg.k_total)
+    assert torch.equal(idx.cpu(), o_idx) and torch.equal(n.cpu(), o_n), shape
+    cur = ctx + 1
+    q = case.q_draft[0].contiguous()
+    d_out, d_lse, wd = binding.spec_sparse_draft_attn(kv, q, idx, n, ctx, cur, 1, per_head=True)
+    assert binding.read_status(wd) == 0, shape
+    r_out, r_lse = oracle.sparse_draft_attn(kv.cpu(), q.cpu(), idx.cpu(), n.cpu(), ctx.cpu(), cur.cpu(), per_head=True)
+    assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL, shape
+    fin = torch.isfinite(r_lse)
+    assert ((d_lse.cpu().double() - r_lse)[fin]).abs().max().item() <= TOL, shape
