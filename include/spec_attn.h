@@ -273,6 +273,17 @@ int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t
                        int64_t row_stride, const int32_t* draft, const int32_t* n_draft,
                        int32_t* target, int32_t* n_accepted, int32_t* next_token,
                        void* cuda_stream);
+/*
+ * spec_advance_lengths: the bookkeeping between two speculation rounds, on the device so that a
+ * captured graph can run round after round (Sec. "The Draft-Verification Paradigm": a step commits
+ * the m accepted tokens and one corrected token).  committed[b] += clamp(n_accepted[b], 0, k) + 1
+ * (n_accepted == NULL: committed is left as it is); then, for the round that follows with k drafted
+ * tokens, ctx_verify[b] = committed[b] + k + 1 (the ctx_len of its verification pass, rows included)
+ * and cur_len[j][b] = committed[b] + j + 1 for j < k (the cur_len of its j-th drafting step, whose
+ * tail starts at committed[b]).  ctx_verify and cur_len (int32 [k][batch]) may be NULL.
+ */
+int spec_advance_lengths(int32_t* committed, const int32_t* n_accepted, int32_t batch, int32_t k,
+                         int32_t* ctx_verify, int32_t* cur_len, void* cuda_stream);
 int spec_controller_update(float* state, const float* entropy, int32_t k,
                            const int32_t* n_accepted, float beta, void* cuda_stream);
 int spec_controller_select(const float* state, const float* entropy, int32_t n,

@@ -29,7 +29,7 @@ EXPORTS = [
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
     "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
-    "spec_sparse_draft_attn_ex",
+    "spec_sparse_draft_attn_ex", "spec_advance_lengths",
 ]
 
 
@@ -83,6 +83,7 @@ def load() -> ctypes.CDLL:
         lib.spec_token_entropy.argtypes = [vp, i32, i32, i32, i64, vp, vp]
         lib.spec_token_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp, vp]
         lib.spec_accept_greedy.argtypes = [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
+        lib.spec_advance_lengths.argtypes = [vp, vp, i32, i32, vp, vp, vp]
         lib.spec_controller_update.argtypes = [vp, vp, i32, vp, f32, vp]
         lib.spec_controller_select.argtypes = [vp, vp, i32, vp, i32, f32, f32, vp, vp, vp, vp]
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
@@ -323,6 +324,19 @@ def spec_accept_greedy(logits, draft, n_draft=None, target=None, n_accepted=None
     if rc != 0:
         raise SpecError(rc, "spec_accept_greedy")
     return target, n_accepted, next_token
+
+
+def spec_advance_lengths(committed, n_accepted, k, ctx_verify=None, cur_len=None):
+    """committed += n_accepted + 1 on the device (``n_accepted=None``: unchanged), then the lengths of the
+    next round: ``ctx_verify`` [batch] and ``cur_len`` [k, batch] (both optional, int32)."""
+    rc = load().spec_advance_lengths(
+        _dev(committed, torch.int32, "committed"),
+        None if n_accepted is None else _dev(n_accepted, torch.int32, "n_accepted"), committed.numel(), k,
+        None if ctx_verify is None else _dev(ctx_verify, torch.int32, "ctx_verify"),
+        None if cur_len is None else _dev(cur_len, torch.int32, "cur_len"), _stream())
+    if rc != 0:
+        raise SpecError(rc, "spec_advance_lengths")
+    return committed
 
 
 def spec_controller_update(state, entropy, n_accepted, beta):

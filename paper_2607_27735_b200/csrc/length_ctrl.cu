@@ -288,6 +288,21 @@ __global__ void controller_select_kernel(const float* __restrict__ state, const 
     }
 }
 
+// Lengths of the next round, on the device: committed += accepted + 1 (the corrected token), the
+// verification context of a round with k drafted tokens, and the draft step lengths.
+__global__ void advance_lengths_kernel(int32_t* __restrict__ committed, const int32_t* __restrict__ n_accepted,
+                                       int batch, int k, int32_t* __restrict__ ctx_verify,
+                                       int32_t* __restrict__ cur_len)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    const int t = committed[b] + (n_accepted ? min(max(n_accepted[b], 0), k) + 1 : 0);
+    committed[b] = t;
+    if (ctx_verify) ctx_verify[b] = t + k + 1;
+    if (cur_len)
+        for (int j = 0; j < k; ++j) cur_len[j * batch + b] = t + j + 1;
+}
+
 }  // namespace
 
 template <int DT, bool ENT, bool ARG>
@@ -344,6 +359,15 @@ int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_
                   int32_t* n_accepted, int32_t* next_token, cudaStream_t stream)
 {
     accept_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(target, draft, n_draft, batch, k1, n_accepted, next_token);
+    if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
+    count_launch(1);
+    return SPEC_OK;
+}
+
+int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int32_t* ctx_verify,
+                           int32_t* cur_len, cudaStream_t stream)
+{
+    advance_lengths_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(committed, n_accepted, batch, k, ctx_verify, cur_len);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     count_launch(1);
     return SPEC_OK;

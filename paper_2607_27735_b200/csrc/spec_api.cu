@@ -251,6 +251,15 @@ int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t
     return accept_launch(target, draft, n_draft, batch, k1, n_accepted, next_token, stream);
 }
 
+int spec_advance_lengths(int32_t* committed, const int32_t* n_accepted, int32_t batch, int32_t k,
+                         int32_t* ctx_verify, int32_t* cur_len, void* cuda_stream)
+{
+    if (!committed || batch < 0 || k < 0) return SPEC_ERR_INVALID_ARG;
+    if (batch == 0) return SPEC_OK;
+    return advance_lengths_launch(committed, n_accepted, batch, k, ctx_verify, cur_len,
+                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
 int spec_controller_update(float* state, const float* entropy, int32_t k, const int32_t* n_accepted, float beta,
                            void* cuda_stream)
 {

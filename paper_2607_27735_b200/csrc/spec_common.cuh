@@ -124,6 +124,8 @@ int rows_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t ro
                 int32_t* token, cudaStream_t stream);
 int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_draft, int batch, int k1,
                   int32_t* n_accepted, int32_t* next_token, cudaStream_t stream);
+int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int32_t* ctx_verify,
+                           int32_t* cur_len, cudaStream_t stream);
 int controller_update_launch(float* state, const float* entropy, int k, const int32_t* n_accepted, float beta,
                              cudaStream_t stream);
 int controller_select_launch(const float* state, const float* entropy, int n, const int32_t* cand, int n_cand,

@@ -153,3 +153,94 @@ class SpecStepRunner:
         kv, c = self.kv, self.cfg
         rows = sum(min(c.k_total, int(t)) + j + 1 for t in self.ctx_len.tolist())
         return rows * (kv.n_q_heads if self.per_head else kv.n_kv_heads) * kv.head_dim * 2 * 2
+
+
+class SpecLoopRunner:
+    """Speculation rounds chained on the device: draft k steps -> verify -> greedy prefix acceptance
+    -> speculation-length controller -> commit m + 1 tokens -> rebuild the recall index, with every
+    length in device memory, so that one captured graph is replayed round after round.  The model
+    around the attention is absent: the caller supplies each round's verification logits and drafted
+    tokens (``logits``, ``draft_tokens`` are overwritten between replays); K/V of every position the
+    loop can reach already sit in the cache.  All layers go in one launch per call."""
+
+    def __init__(self, case, committed, vocab: int, c_d: float = 0.05, c_v: float = 1.0, beta: float = 0.9):
+        cfg, kv = case.cfg, case.kv
+        assert cfg.n_q == cfg.draft_steps + 1, "a round verifies the k drafted tokens plus one"
+        self.case, self.cfg, self.kv = case, cfg, kv
+        dev = kv.k.device
+        L, B, k = kv.n_layers, kv.batch, cfg.draft_steps
+        self.k, self.beta, self.c_d, self.c_v = k, beta, c_d, c_v
+        self.max_ctx = kv.max_pages * kv.page_size if kv.page_table is not None else int(case.ctx_len.max()) + k + 1
+        self.committed = committed.to(device=dev, dtype=torch.int32).clone()
+        self.ctx_verify = torch.empty(B, dtype=torch.int32, device=dev)
+        self.cur_len = torch.empty(k, B, dtype=torch.int32, device=dev)
+        self.stat_stride = (self.max_ctx + 127) // 128 * 128
+        self.stats = torch.zeros(L, B, kv.n_kv_heads, self.stat_stride, device=dev)
+        self.indices = torch.empty(L, B, kv.n_kv_heads, cfg.k_total, dtype=torch.int32, device=dev)
+        self.n_idx = torch.empty(L, B, kv.n_kv_heads, dtype=torch.int32, device=dev)
+        self.out_v = torch.empty(L, B, cfg.n_q, kv.n_q_heads, kv.head_dim, device=dev)
+        self.out_d = torch.empty(k, L, B, kv.n_q_heads, kv.head_dim, device=dev)
+        self.logits = torch.empty(B, k + 1, vocab, dtype=torch.bfloat16, device=dev)
+        self.draft_tokens = torch.zeros(B, k, dtype=torch.int32, device=dev)
+        self.target = torch.empty(B, k + 1, dtype=torch.int32, device=dev)
+        self.n_accepted = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.next_token = torch.empty(B, dtype=torch.int32, device=dev)
+        self.entropy = torch.empty(k, device=dev)           # of sequence 0's drafted tokens
+        self.state = torch.tensor([1.0, 4.0], device=dev)   # tracked mean entropy of accepted / rejected tokens
+        self.cand = torch.arange(1, k + 1, dtype=torch.int32, device=dev)
+        self.k_star = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.p = torch.empty(k, device=dev)
+        self.score = torch.empty(k, device=dev)
+        self.ws_v = binding.alloc_workspace(binding.workspace_bytes(binding.WS_VERIFY, kv, cfg.n_q, self.max_ctx), dev)
+        self.ws_d = binding.alloc_workspace(binding.workspace_bytes(binding.WS_DRAFT, kv, k_total=cfg.k_total + k), dev)
+        self.graph = None
+
+    def _verify(self, ctx):
+        binding.spec_verify_attn(self.kv, self.case.q_verify, ctx, self.max_ctx, self.cfg.stat_window,
+                                 out=self.out_v, stats=self.stats, workspace=self.ws_v, want_lse=False)
+
+    def _select(self):
+        c = self.cfg
+        binding.spec_select_recall(self.stats, self.committed, c.k_sink, c.k_recent, c.k_total,
+                                   indices=self.indices, n_indices=self.n_idx)
+
+    def prime(self):
+        """The index of the first round, from a verification pass over the last rows before the
+        committed length (what a prefill leaves behind), and the first round's lengths."""
+        self._verify(self.committed)
+        self._select()
+        binding.spec_advance_lengths(self.committed, None, self.k, self.ctx_verify, self.cur_len)
+
+    def round(self):
+        for j in range(self.k):
+            binding.spec_sparse_draft_attn(self.kv, self.case.q_draft[j], self.indices, self.n_idx, self.committed,
+                                           self.cur_len[j], self.k, out=self.out_d[j], workspace=self.ws_d,
+                                           want_lse=False)
+        self._verify(self.ctx_verify)
+        binding.spec_accept_greedy(self.logits, self.draft_tokens, target=self.target,
+                                   n_accepted=self.n_accepted, next_token=self.next_token)
+        binding.spec_token_entropy(self.logits[0, :self.k], entropy=self.entropy)
+        binding.spec_controller_update(self.state, self.entropy, self.n_accepted[:1], self.beta)
+        binding.spec_controller_select(self.state, self.entropy, self.cand, self.c_d, self.c_v,
+                                       k_star=self.k_star, p=self.p, score=self.score)
+        binding.spec_advance_lengths(self.committed, self.n_accepted, self.k, self.ctx_verify, self.cur_len)
+        self._select()
+
+    def capture(self):
+        self.prime()
+        saved = (self.committed.clone(), self.ctx_verify.clone(), self.cur_len.clone(), self.state.clone())
+        self.round()  # warm-up outside the capture
+        torch.cuda.synchronize()
+        self.committed.copy_(saved[0])
+        self.ctx_verify.copy_(saved[1])
+        self.cur_len.copy_(saved[2])
+        self.state.copy_(saved[3])
+        self._verify(self.committed)  # the warm-up round replaced the statistic and the index: rebuild them
+        self._select()
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.round()
+
+    def replay(self):
+        self.graph.replay()
