@@ -140,8 +140,11 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
  * tcgen05 kernel for groups of up to 8 heads whose shape fits its cache, else by the generic
  * kernels.  spec_select_recall then runs with n_kv_heads = n_q_heads, and the draft call takes
  * SPEC_DRAFT_INDICES_PER_QUERY_HEAD.
+ *
+ * SPEC_VERIFY_OUT_BF16: `out` points to bf16 elements of the same shape (the fp32 result rounded to
+ * nearest even: what a bf16 output projection consumes); lse and stats stay fp32.
  */
-enum { SPEC_VERIFY_ACCUMULATE_STATS = 1, SPEC_VERIFY_STATS_PER_QUERY_HEAD = 2 };
+enum { SPEC_VERIFY_ACCUMULATE_STATS = 1, SPEC_VERIFY_STATS_PER_QUERY_HEAD = 2, SPEC_VERIFY_OUT_BF16 = 4 };
 int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
                         int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
                         float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,
@@ -294,10 +297,11 @@ int spec_controller_select(const float* state, const float* entropy, int32_t n,
  * spec_sparse_draft_attn with option flags.  SPEC_DRAFT_INDICES_PER_QUERY_HEAD: Eq. 5 as printed,
  * every attention head gathers its own index set: indices is int32 [n_layers, batch, n_q_heads,
  * k_total] and n_indices int32 [n_layers, batch, n_q_heads]; K and V rows still come from the
- * head's KV head (hq / group).  The gathered bytes grow by the group size.  flags == 0 is
- * spec_sparse_draft_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
+ * head's KV head (hq / group).  The gathered bytes grow by the group size.
+ * SPEC_DRAFT_OUT_BF16: `out` points to bf16 elements (fp32 result rounded to nearest even).
+ * flags == 0 is spec_sparse_draft_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
  */
-enum { SPEC_DRAFT_INDICES_PER_QUERY_HEAD = 1 };
+enum { SPEC_DRAFT_INDICES_PER_QUERY_HEAD = 1, SPEC_DRAFT_OUT_BF16 = 2 };
 int spec_sparse_draft_attn_ex(const spec_kv_t* kv, const void* q, const int32_t* indices,
                               const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
                               const int32_t* cur_len, int32_t max_tail, float* out, float* lse,

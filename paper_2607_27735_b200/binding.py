@@ -22,6 +22,8 @@ VERIFY_TCGEN05_CACHED_2PASS = 5
 VERIFY_ACCUMULATE_STATS = 1  # flag of spec_verify_attn_ex: add to the statistic instead of replacing it
 VERIFY_STATS_PER_QUERY_HEAD = 2  # flag of spec_verify_attn_ex: one score per attention head
 DRAFT_INDICES_PER_QUERY_HEAD = 1  # flag of spec_sparse_draft_attn_ex: one index set per attention head
+VERIFY_OUT_BF16 = 4  # flag of spec_verify_attn_ex: bf16 attention output
+DRAFT_OUT_BF16 = 2  # flag of spec_sparse_draft_attn_ex: bf16 attention output
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
@@ -136,7 +138,8 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 
 def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
-                     stat_stride=None, workspace=None, want_lse=True, accumulate=False, per_head=False):
+                     stat_stride=None, workspace=None, want_lse=True, accumulate=False, per_head=False,
+                     out_bf16=False):
     """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``.
     ``accumulate`` adds this call's statistic to the given ``stats``; ``per_head`` keeps one score per
     attention head (``stats`` is ``[L, B, n_q_heads, stride]``); both go through spec_verify_attn_ex."""
@@ -146,8 +149,9 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
     s = _kv_struct(kv)
     if stat_stride is None:
         stat_stride = (max_ctx_len + 63) // 64 * 64 if stats is None else stats.shape[-1]
+    out_dtype = torch.bfloat16 if out_bf16 else torch.float32
     if out is None:
-        out = torch.empty(L, B, n_q, Hq, D, dtype=torch.float32, device=dev)
+        out = torch.empty(L, B, n_q, Hq, D, dtype=out_dtype, device=dev)
     if lse is None and want_lse:
         lse = torch.empty(L, B, n_q, Hq, dtype=torch.float32, device=dev)
     if stats is None:
@@ -158,13 +162,14 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
     if accumulate and stats is None:
         raise ValueError("accumulate needs the stats tensor that holds the running sums")
     args = (ctypes.byref(s), _dev(q, torch.bfloat16, "q"), n_q, _dev(ctx_len, torch.int32, "ctx_len"),
-            max_ctx_len, stat_window, _dev(out, torch.float32, "out"),
+            max_ctx_len, stat_window, _dev(out, out_dtype, "out"),
             None if lse is None else _dev(lse, torch.float32, "lse"),
             _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel())
     if stats.shape[2] != (kv.n_q_heads if per_head else kv.n_kv_heads):
         raise ValueError("stats: wrong head count for this mode")
-    if accumulate or per_head:
-        flags = (VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0)
+    if accumulate or per_head or out_bf16:
+        flags = ((VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0) |
+                 (VERIFY_OUT_BF16 if out_bf16 else 0))
         rc = lib.spec_verify_attn_ex(*args, flags, _stream())
     else:
         rc = lib.spec_verify_attn(*args, _stream())
@@ -228,7 +233,7 @@ def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, 
 
 
 def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_tail, out=None,
-                           lse=None, workspace=None, want_lse=True, per_head=False):
+                           lse=None, workspace=None, want_lse=True, per_head=False, out_bf16=False):
     """Eq. 5 sparse draft attention; returns ``(out, lse, workspace)``.  ``per_head``: ``indices`` is
     ``[L, B, n_q_heads, k_total]``, one set per attention head (spec_sparse_draft_attn_ex)."""
     lib = load()
@@ -236,8 +241,9 @@ def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_t
     dev = q.device
     s = _kv_struct(kv)
     k_total = indices.shape[-1]
+    out_dtype = torch.bfloat16 if out_bf16 else torch.float32
     if out is None:
-        out = torch.empty(L, B, Hq, D, dtype=torch.float32, device=dev)
+        out = torch.empty(L, B, Hq, D, dtype=out_dtype, device=dev)
     if lse is None and want_lse:
         lse = torch.empty(L, B, Hq, dtype=torch.float32, device=dev)
     if workspace is None:
@@ -247,11 +253,12 @@ def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_t
     args = (ctypes.byref(s), _dev(q, torch.bfloat16, "q"), _dev(indices, torch.int32, "indices"),
             _dev(n_indices, torch.int32, "n_indices"), k_total,
             _dev(tail_start, torch.int32, "tail_start"), _dev(cur_len, torch.int32, "cur_len"),
-            max_tail, _dev(out, torch.float32, "out"),
+            max_tail, _dev(out, out_dtype, "out"),
             None if lse is None else _dev(lse, torch.float32, "lse"), workspace.data_ptr(),
             workspace.numel())
-    if per_head:
-        rc = lib.spec_sparse_draft_attn_ex(*args, DRAFT_INDICES_PER_QUERY_HEAD, _stream())
+    if per_head or out_bf16:
+        flags = (DRAFT_INDICES_PER_QUERY_HEAD if per_head else 0) | (DRAFT_OUT_BF16 if out_bf16 else 0)
+        rc = lib.spec_sparse_draft_attn_ex(*args, flags, _stream())
     else:
         rc = lib.spec_sparse_draft_attn(*args, _stream())
     if rc != 0:

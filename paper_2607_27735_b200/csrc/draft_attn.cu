@@ -633,7 +633,10 @@ draft_cluster_kernel(DraftArgs a, DraftShape shp, int* __restrict__ status)
         }
         const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + r;
         const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-        *(reinterpret_cast<float2*>(a.out + row * D) + dp) = make_float2(o0 * inv, o1 * inv);
+        if (a.out_bf16)
+            *(reinterpret_cast<uint32_t*>(reinterpret_cast<__nv_bfloat16*>(a.out) + row * D) + dp) = pack_bf16(o0 * inv, o1 * inv);
+        else
+            *(reinterpret_cast<float2*>(a.out + row * D) + dp) = make_float2(o0 * inv, o1 * inv);
         if (a.lse && dp == 0) a.lse[row] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.69314718055994530942f : -INFINITY;
     }
     DSTAMP(7);

@@ -89,7 +89,8 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
                         int64_t stat_stride, void* workspace, size_t workspace_bytes, uint32_t flags,
                         void* cuda_stream)
 {
-    if (flags & ~(uint32_t)(SPEC_VERIFY_ACCUMULATE_STATS | SPEC_VERIFY_STATS_PER_QUERY_HEAD)) return SPEC_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(SPEC_VERIFY_ACCUMULATE_STATS | SPEC_VERIFY_STATS_PER_QUERY_HEAD | SPEC_VERIFY_OUT_BF16))
+        return SPEC_ERR_INVALID_ARG;
     VerifyArgs a;
     const int rc = make_view(kv, &a.kv);
     if (rc != SPEC_OK) return rc;
@@ -115,6 +116,7 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
     a.workspace_bytes = workspace_bytes;
     a.stat_accumulate = (flags & SPEC_VERIFY_ACCUMULATE_STATS) ? 1 : 0;
     a.stat_per_head = (flags & SPEC_VERIFY_STATS_PER_QUERY_HEAD) ? 1 : 0;
+    a.out_bf16 = (flags & SPEC_VERIFY_OUT_BF16) ? 1 : 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int impl = g_verify_impl.load();
     if (impl != SPEC_VERIFY_GENERIC) {
@@ -164,11 +166,12 @@ int spec_sparse_draft_attn_ex(const spec_kv_t* kv, const void* q, const int32_t*
                               const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream)
 {
-    if (flags & ~(uint32_t)SPEC_DRAFT_INDICES_PER_QUERY_HEAD) return SPEC_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(SPEC_DRAFT_INDICES_PER_QUERY_HEAD | SPEC_DRAFT_OUT_BF16)) return SPEC_ERR_INVALID_ARG;
     DraftArgs a;
     const int rc = make_view(kv, &a.kv);
     if (rc != SPEC_OK) return rc;
     a.head_div = 1;
+    a.out_bf16 = (flags & SPEC_DRAFT_OUT_BF16) ? 1 : 0;
     if (flags & SPEC_DRAFT_INDICES_PER_QUERY_HEAD) {
         // every attention head is a problem of its own (group size 1) that reads the rows of its
         // KV head: the kernels see n_q_heads "KV heads" and divide the head index for the cache

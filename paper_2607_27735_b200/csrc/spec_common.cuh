@@ -54,6 +54,12 @@ __device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, in
            slot * kv.slot_stride;
 }
 
+// Two fp32 values as one packed bf16 pair (x in the low half), round to nearest even.
+__device__ __forceinline__ uint32_t pack_bf16(float x, float y)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(x, y);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
@@ -92,6 +98,7 @@ struct VerifyArgs {
     size_t workspace_bytes;
     int stat_accumulate;  // add this call's statistic to what stats[] holds instead of overwriting it
     int stat_per_head;    // stats is [layers, batch, n_q_heads, stride]: one score per attention head
+    int out_bf16;         // `out` points to bf16 elements (round to nearest even) instead of fp32
 };
 
 size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);
@@ -116,6 +123,7 @@ struct DraftArgs {
     size_t workspace_bytes;
     int head_div;  // K/V of problem head h are read from cache head h / head_div (1 unless every
                    // attention head carries its own index set)
+    int out_bf16;  // `out` points to bf16 elements (round to nearest even) instead of fp32
 };
 size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
 int draft_launch(const DraftArgs& a, cudaStream_t stream);

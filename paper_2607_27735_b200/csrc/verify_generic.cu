@@ -289,7 +289,9 @@ __global__ void verify_out_combine_kernel(VerifyArgs a, int n_splits, const floa
     const int h = prob % a.kv.n_kv_heads;
     const int64_t lb = prob / a.kv.n_kv_heads;
     const int j = r / G, g = r - j * G;
-    a.out[((lb * a.n_q + j) * a.kv.n_q_heads + h * G + g) * D + d] = s;
+    const int64_t o = ((lb * a.n_q + j) * a.kv.n_q_heads + h * G + g) * D + d;
+    if (a.out_bf16) reinterpret_cast<__nv_bfloat16*>(a.out)[o] = __float2bfloat16_rn(s);
+    else a.out[o] = s;
 }
 
 template <int D>

@@ -289,7 +289,8 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
         VerifyArgs pb = a;  // rows [nA, n_q) against the whole context; their statistic goes to scratch
         pb.n_q = sp.nB;
         pb.q = a.q + sp.nA * row_elems;
-        pb.out = a.out + sp.nA * row_elems;
+        pb.out = a.out_bf16 ? reinterpret_cast<float*>(reinterpret_cast<__nv_bfloat16*>(a.out) + sp.nA * row_elems)
+                            : a.out + sp.nA * row_elems;
         pb.lse = a.lse ? a.lse + (int64_t)sp.nA * a.kv.n_q_heads : nullptr;
         pb.first_stat_row = a.first_stat_row > sp.nA ? a.first_stat_row - sp.nA : 0;
         pb.stats = second;

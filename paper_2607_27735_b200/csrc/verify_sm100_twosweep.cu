@@ -649,7 +649,11 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                 const int r = e / (kD / 4), d4 = e - r * (kD / 4);
                 const int j = r / G, g = r - j * G;
                 const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
-                reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
+                if (p.a.out_bf16)
+                    reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.a.out) + row * kD)[d4] =
+                        make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+                else
+                    reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
             }
             return true;
         };
