@@ -50,7 +50,7 @@ enum {
     SPEC_ERR_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < spec_workspace_bytes(...) */
     SPEC_ERR_CUDA = -4,                /* a CUDA runtime/driver call failed at launch time */
     SPEC_ERR_TIMEOUT = -5,             /* status word: a bounded device-side wait ran out */
-    SPEC_ERR_BAD_INDEX = -6            /* status word: a recall index was out of range */
+    SPEC_ERR_BAD_INDEX = -6            /* status word: a recall index, page-table entry or length was out of range */
 };
 
 /* Which entry point a workspace is sized for. */
@@ -104,7 +104,8 @@ typedef struct {
  *   q        bf16 [n_layers, batch, n_q, n_q_heads, head_dim]
  *   n_q      k+1, 1..32, with n_q * (n_q_heads/n_kv_heads) <= 128
  *   ctx_len  int32 [batch], each n_q <= ctx_len[b] <= max_ctx_len; INCLUDES the n_q rows, whose
- *            K/V are already in the cache
+ *            K/V are already in the cache.  A value outside that range is clamped into it on the
+ *            device and sets SPEC_ERR_BAD_INDEX in the status word (no access leaves the buffers)
  *   max_ctx_len  host upper bound of ctx_len (sizes the launch)
  *   stat_window  W of Eq. 3; 0 means 16
  *   out      fp32 [n_layers, batch, n_q, n_q_heads, head_dim]
@@ -189,10 +190,17 @@ int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers
  *              only the status word, which this call never clears (one launch per call, no
  *              memset): zero it once after allocation; an error stays until
  *              spec_read_status() returns it.
- * An index outside [0, cur_len[b]) is skipped and sets SPEC_ERR_BAD_INDEX in the status word.
+ * An index outside [0, cur_len[b]), or a page-table entry outside [0, n_pages), is skipped and
+ * sets SPEC_ERR_BAD_INDEX in the status word; so does a cur_len[b] beyond max_pages * page_size
+ * (clamped to it) and a tail longer than max_tail (the rows beyond max_tail are dropped).
  * The one device-side wait (the first CTA of a cluster waiting for the partial results of the
  * others) is bounded; if it runs out the status word gets SPEC_ERR_TIMEOUT.
  * A problem with an empty key set yields out = 0, lse = -inf.
+ * Limits: n_q_heads / n_kv_heads <= 8 (SPEC_ERR_UNSUPPORTED_SHAPE otherwise; with
+ * SPEC_DRAFT_INDICES_PER_QUERY_HEAD every head is its own group of one, so any ratio works);
+ * n_pages * page_stride < 2^35 elements (one layer's K below 64 GiB).
+ * Stream order: the call reads all of its inputs only after every earlier kernel of the stream
+ * has completed, unless SPEC_DRAFT_EARLY_GATHER is given (spec_sparse_draft_attn_ex).
  */
 int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* indices,
                            const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
@@ -214,8 +222,11 @@ int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* in
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress, with that device current); make that first call before starting any
  *     stream capture on the device.
+ *   - `cuda_stream` must belong to the device that is current at the call (the array's address is
+ *     looked up for the current device).
  *   - All calls on a device share the one array, and it keeps the previous call's contents;
- *     every call re-zeroes the control words it depends on, on `cuda_stream`.  Two calls that
+ *     every call re-zeroes the control words it depends on, on `cuda_stream`; the status word is
+ *     kept until spec_noalloc_read_status() returns it.  Two calls that
  *     may overlap on the GPU (different streams, no ordering) race on it: serialise them.
  *   - spec_noalloc_read_status() is spec_read_status() on that array for the current device.
  */
@@ -284,9 +295,14 @@ int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t
  * tokens, ctx_verify[b] = committed[b] + k + 1 (the ctx_len of its verification pass, rows included)
  * and cur_len[j][b] = committed[b] + j + 1 for j < k (the cur_len of its j-th drafting step, whose
  * tail starts at committed[b]).  ctx_verify and cur_len (int32 [k][batch]) may be NULL.
+ * max_len > 0 is the number of tokens a sequence's cache can hold (the max_ctx_len later calls are
+ * sized for): a sequence whose next round would not fit (committed + k + 1 > max_len) is held at
+ * max_len - k - 1 instead and SPEC_ERR_BAD_INDEX is recorded in the status word at the head of
+ * `workspace` (any workspace of this library; NULL: not recorded).  max_len == 0: no bound.
  */
 int spec_advance_lengths(int32_t* committed, const int32_t* n_accepted, int32_t batch, int32_t k,
-                         int32_t* ctx_verify, int32_t* cur_len, void* cuda_stream);
+                         int32_t max_len, void* workspace, int32_t* ctx_verify, int32_t* cur_len,
+                         void* cuda_stream);
 int spec_controller_update(float* state, const float* entropy, int32_t k,
                            const int32_t* n_accepted, float beta, void* cuda_stream);
 int spec_controller_select(const float* state, const float* entropy, int32_t n,
@@ -299,9 +315,17 @@ int spec_controller_select(const float* state, const float* entropy, int32_t n,
  * k_total] and n_indices int32 [n_layers, batch, n_q_heads]; K and V rows still come from the
  * head's KV head (hq / group).  The gathered bytes grow by the group size.
  * SPEC_DRAFT_OUT_BF16: `out` points to bf16 elements (fp32 result rounded to nearest even).
+ * SPEC_DRAFT_EARLY_GATHER: the kernel is launched so that it may start while the preceding kernel
+ * of the stream is still running, and it reads indices, n_indices, tail_start, cur_len, the page
+ * table and the recalled K/V rows BEFORE that kernel has finished; only q, the rows of the dense
+ * tail and the outputs wait for the stream's earlier work.  Give the flag only when those
+ * early-read arguments were complete before the preceding kernel of the stream STARTED: true for
+ * every call of a drafting round but the first one that follows the producers of the index sets and
+ * the lengths (selection, the length bookkeeping), since nothing changes them during a round.
+ * Without the flag the call starts after all earlier work of the stream, like any kernel.
  * flags == 0 is spec_sparse_draft_attn.  Unknown flag bits: SPEC_ERR_INVALID_ARG.
  */
-enum { SPEC_DRAFT_INDICES_PER_QUERY_HEAD = 1, SPEC_DRAFT_OUT_BF16 = 2 };
+enum { SPEC_DRAFT_INDICES_PER_QUERY_HEAD = 1, SPEC_DRAFT_OUT_BF16 = 2, SPEC_DRAFT_EARLY_GATHER = 4 };
 int spec_sparse_draft_attn_ex(const spec_kv_t* kv, const void* q, const int32_t* indices,
                               const int32_t* n_indices, int32_t k_total, const int32_t* tail_start,
                               const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
@@ -326,6 +350,12 @@ int spec_read_status(const void* workspace, void* cuda_stream);
 /* Chooses the verification kernel (process-wide; SPEC_VERIFY_AUTO picks the tcgen05 kernel
  * when the shape allows it).  Returns the previous setting, or SPEC_ERR_INVALID_ARG. */
 int spec_set_verify_impl(int impl);
+
+/* Device-side waits (a CTA waiting for another CTA's partial result, for a copy, for the tensor
+ * cores) give up after this many SM clocks, set SPEC_ERR_TIMEOUT in the status word and let the
+ * kernel drain and return.  Default 2e9 (about a second).  Process-wide; applies to calls made
+ * after it.  Returns the previous limit, or SPEC_ERR_INVALID_ARG for cycles < 1. */
+int64_t spec_set_wait_limit_cycles(int64_t cycles);
 
 /* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC,
  * SPEC_VERIFY_TCGEN05_TWOSWEEP, SPEC_VERIFY_TCGEN05_CACHED or SPEC_VERIFY_TCGEN05_CACHED_2PASS; 0 before the

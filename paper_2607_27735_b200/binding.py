@@ -24,6 +24,8 @@ VERIFY_STATS_PER_QUERY_HEAD = 2  # flag of spec_verify_attn_ex: one score per at
 DRAFT_INDICES_PER_QUERY_HEAD = 1  # flag of spec_sparse_draft_attn_ex: one index set per attention head
 VERIFY_OUT_BF16 = 4  # flag of spec_verify_attn_ex: bf16 attention output
 DRAFT_OUT_BF16 = 2  # flag of spec_sparse_draft_attn_ex: bf16 attention output
+DRAFT_EARLY_GATHER = 4  # flag of spec_sparse_draft_attn_ex: index sets, lengths and recalled rows are older than the
+#                         preceding kernel of the stream, so the gather may start before that kernel has finished
 
 EXPORTS = [
     "spec_verify_attn", "spec_select_recall", "spec_sparse_draft_attn", "spec_workspace_bytes",
@@ -31,7 +33,7 @@ EXPORTS = [
     "spec_strerror", "spec_version", "spec_verify_attn_noalloc", "spec_noalloc_scratch_bytes",
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
     "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
-    "spec_sparse_draft_attn_ex", "spec_advance_lengths",
+    "spec_sparse_draft_attn_ex", "spec_advance_lengths", "spec_set_wait_limit_cycles",
 ]
 
 
@@ -85,13 +87,15 @@ def load() -> ctypes.CDLL:
         lib.spec_token_entropy.argtypes = [vp, i32, i32, i32, i64, vp, vp]
         lib.spec_token_argmax.argtypes = [vp, i32, i32, i32, i64, vp, vp, vp]
         lib.spec_accept_greedy.argtypes = [vp, i32, i32, i32, i32, i64, vp, vp, vp, vp, vp, vp]
-        lib.spec_advance_lengths.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        lib.spec_advance_lengths.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
         lib.spec_controller_update.argtypes = [vp, vp, i32, vp, f32, vp]
         lib.spec_controller_select.argtypes = [vp, vp, i32, vp, i32, f32, f32, vp, vp, vp, vp]
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
         lib.spec_workspace_bytes.restype = ctypes.c_size_t
         lib.spec_read_status.argtypes = [vp, vp]
         lib.spec_set_verify_impl.argtypes = [ctypes.c_int]
+        lib.spec_set_wait_limit_cycles.argtypes = [ctypes.c_int64]
+        lib.spec_set_wait_limit_cycles.restype = ctypes.c_int64
         lib.spec_launch_count.restype = ctypes.c_int64
         lib.spec_strerror.argtypes = [ctypes.c_int]
         lib.spec_strerror.restype = ctypes.c_char_p
@@ -233,9 +237,11 @@ def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, 
 
 
 def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_tail, out=None,
-                           lse=None, workspace=None, want_lse=True, per_head=False, out_bf16=False):
+                           lse=None, workspace=None, want_lse=True, per_head=False, out_bf16=False,
+                           early_gather=False):
     """Eq. 5 sparse draft attention; returns ``(out, lse, workspace)``.  ``per_head``: ``indices`` is
-    ``[L, B, n_q_heads, k_total]``, one set per attention head (spec_sparse_draft_attn_ex)."""
+    ``[L, B, n_q_heads, k_total]``, one set per attention head (spec_sparse_draft_attn_ex).
+    ``early_gather``: the caller's promise behind SPEC_DRAFT_EARLY_GATHER (see the header)."""
     lib = load()
     L, B, Hq, D = q.shape
     dev = q.device
@@ -256,8 +262,9 @@ def spec_sparse_draft_attn(kv, q, indices, n_indices, tail_start, cur_len, max_t
             max_tail, _dev(out, out_dtype, "out"),
             None if lse is None else _dev(lse, torch.float32, "lse"), workspace.data_ptr(),
             workspace.numel())
-    if per_head or out_bf16:
-        flags = (DRAFT_INDICES_PER_QUERY_HEAD if per_head else 0) | (DRAFT_OUT_BF16 if out_bf16 else 0)
+    if per_head or out_bf16 or early_gather:
+        flags = ((DRAFT_INDICES_PER_QUERY_HEAD if per_head else 0) | (DRAFT_OUT_BF16 if out_bf16 else 0) |
+                 (DRAFT_EARLY_GATHER if early_gather else 0))
         rc = lib.spec_sparse_draft_attn_ex(*args, flags, _stream())
     else:
         rc = lib.spec_sparse_draft_attn(*args, _stream())
@@ -333,12 +340,14 @@ def spec_accept_greedy(logits, draft, n_draft=None, target=None, n_accepted=None
     return target, n_accepted, next_token
 
 
-def spec_advance_lengths(committed, n_accepted, k, ctx_verify=None, cur_len=None):
+def spec_advance_lengths(committed, n_accepted, k, ctx_verify=None, cur_len=None, max_len=0, workspace=None):
     """committed += n_accepted + 1 on the device (``n_accepted=None``: unchanged), then the lengths of the
-    next round: ``ctx_verify`` [batch] and ``cur_len`` [k, batch] (both optional, int32)."""
+    next round: ``ctx_verify`` [batch] and ``cur_len`` [k, batch] (both optional, int32).  ``max_len`` > 0
+    holds a sequence whose next round would not fit the cache and records that in ``workspace``."""
     rc = load().spec_advance_lengths(
         _dev(committed, torch.int32, "committed"),
         None if n_accepted is None else _dev(n_accepted, torch.int32, "n_accepted"), committed.numel(), k,
+        int(max_len), None if workspace is None else workspace.data_ptr(),
         None if ctx_verify is None else _dev(ctx_verify, torch.int32, "ctx_verify"),
         None if cur_len is None else _dev(cur_len, torch.int32, "cur_len"), _stream())
     if rc != 0:
@@ -377,6 +386,11 @@ def spec_controller_select(state, entropy, cand, c_d, c_v, k_star=None, p=None, 
 
 def read_status(workspace) -> int:
     return int(load().spec_read_status(workspace.data_ptr(), _stream()))
+
+
+def set_wait_limit_cycles(cycles: int) -> int:
+    """Sets the bound of the device-side waits in SM clocks; returns the previous one."""
+    return int(load().spec_set_wait_limit_cycles(int(cycles)))
 
 
 def set_verify_impl(impl: int) -> int:

@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libspec_attn.so")
 SOURCES = ["spec_api.cu", "verify_generic.cu", "verify_sm100.cu", "verify_sm100_twosweep.cu",
-           "verify_sm100_cached.cu", "select_recall.cu", "draft_attn.cu", "spec_noalloc.cu",
+           "verify_sm100_cached.cu", "select_recall.cu", "draft_stream.cu", "spec_noalloc.cu",
            "length_ctrl.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),

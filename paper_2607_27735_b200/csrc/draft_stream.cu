@@ -1,0 +1,444 @@
+// Sparse draft attention of Eq. 5, streaming variant: every warp walks its own 16-key chunks of
+// the recalled rows through a private ring of shared-memory stages, so that the gather (16-byte
+// cp.async copies straight from the dense cache by index) of the chunks ahead runs under the
+// tensor-core work of the current one, and no block-wide barrier sits in the loop.  Several
+// small CTAs share an SM, which keeps gathers in flight on every SM for the whole call.
+//
+// Per chunk (16 keys x head_dim), in registers, with the G <= 8 query heads of the group packed
+// into the M dimension of mma.sync m16n8k16:
+//   S = Q K^T      A = Q (rows 0..7 = heads, rows 8..15 zero), B = K rows as they lie in memory;
+//   online softmax per head (running max with a lazy rescale, running sum);
+//   O += P V       A = [P_hi ; P_lo] (rows 0..7 the bf16 rounding of P, rows 8..15 its remainder:
+//                  the second half of the M dimension is free, so the split costs no extra MMA),
+//                  B = V rows through ldmatrix.trans.
+// The warps of a CTA merge their (max, sum, O) through shared memory, the CTAs of a cluster
+// (one cluster per (layer, sequence, KV head)) deposit theirs in the cluster's first CTA with
+// asynchronous distributed-shared-memory stores counted on an mbarrier; it merges them in rank
+// order, so the result is deterministic.  One launch per call, no global scratch.
+#include "spec_common.cuh"
+#include "draft_common.cuh"
+
+namespace spec {
+
+namespace {
+
+using namespace draft;
+
+constexpr int kChunk = 16;
+constexpr uint32_t kNoRow = 0xffffffffu;
+
+template <int D>
+struct Geo {
+    static constexpr int ROWB = D * 2 + 16;          // bytes per shared-memory row: 16 B of padding spread the banks
+    static constexpr int STAGE = 2 * kChunk * ROWB;  // a chunk's K rows, then its V rows
+};
+
+// Shared memory of one CTA: [NW warps][ST stages][STAGE] | row offsets uint32 [per] |
+// per-warp (max, sum) float2 [NW][8] | deposit barrier (16 B) | deposit area float [cs][G * (D + 2)]
+template <int D>
+__host__ __device__ inline size_t stream_smem_bytes(int G, int nw, int st, int per, int cs)
+{
+    return (size_t)nw * st * Geo<D>::STAGE + (size_t)per * 4 + (size_t)nw * 8 * 8 + 16 + (size_t)cs * G * (D + 2) * 4;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D, int NW, int ST>
+__global__ void __launch_bounds__(NW * 32)
+draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
+{
+    constexpr int ROWB = Geo<D>::ROWB, STAGE = Geo<D>::STAGE;
+    constexpr int NT = NW * 32;
+    constexpr int KS = D / 16;  // 16-wide steps of the head dimension
+    constexpr float kLog2e = 1.4426950408889634f;
+    extern __shared__ __align__(16) uint8_t smem[];
+    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+    const int per = shp.per, PS = G * (D + 2);
+    uint8_t* stages = smem;
+    uint32_t* rowoff = reinterpret_cast<uint32_t*>(smem + (size_t)NW * ST * STAGE);
+    float2* wml = reinterpret_cast<float2*>(rowoff + per);        // [NW][8]
+    uint64_t* dep_bar = reinterpret_cast<uint64_t*>(wml + NW * 8);
+    float* comb = reinterpret_cast<float*>(dep_bar + 2);          // [cs][PS]: O rows [G][D], maxima [G], sums [G]
+
+    const int CS = gridDim.x, rank = blockIdx.x, h = blockIdx.y;
+    const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
+    const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = lane >> 2, quad = lane & 3;
+
+    // The next kernel of the stream may start while this one runs (programmatic dependent launch).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (CS > 1) {
+        if (rank == 0 && tid == 0) {
+            mbar_init(smem_addr(dep_bar), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            mbar_arrive_expect_tx(smem_addr(dep_bar), (uint32_t)(CS - 1) * PS * 4);
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
+    // Without the early-gather promise the launch is an ordinary one: all earlier work is complete.
+    bool waited = !a.early_gather;
+
+    const int n_rec = min(max(__ldg(a.n_indices + prob), 0), a.k_total);
+    const int ts = __ldg(a.tail_start + b);
+    int cl = __ldg(a.cur_len + b);
+    const int64_t cap = (int64_t)a.kv.max_pages * a.kv.page_size;
+    if (cl > cap) {  // a length beyond the cache: clamp, so that no row address leaves it
+        if (tid == 0) set_status(status, SPEC_ERR_BAD_INDEX);
+        cl = (int)cap;
+    }
+    int n_tail = max(cl - ts, 0);
+    if (n_tail > a.max_tail) {  // the launch was sized for max_tail rows: the rest is dropped, and reported
+        if (tid == 0) set_status(status, SPEC_ERR_BAD_INDEX);
+        n_tail = a.max_tail;
+    }
+    const int n = n_rec + n_tail;
+    const int k0 = min(n, rank * per), k1 = min(n, k0 + per);
+    const int nch = (k1 - k0 + kChunk - 1) / kChunk;
+    const int first_tail = max(n_rec, k0) - k0;  // local rows [first_tail, k1 - k0) come from the dense tail
+
+    // ---- resolve the rows of this CTA's share once: position -> offset of the row in 16-byte units ----
+    const int hm = a.head_div > 1 ? h / a.head_div : h;  // the cache head this problem's rows come from
+    {
+        const int32_t* idx = a.indices + prob * a.k_total;
+        const int32_t* ptab = a.kv.page_table ? a.kv.page_table + (int64_t)b * a.kv.max_pages : nullptr;
+        for (int lr = tid; lr < nch * kChunk; lr += NT) {
+            uint32_t off = kNoRow;
+            if (k0 + lr < k1) {
+                const int li = k0 + lr;
+                const int pos = li < n_rec ? __ldg(idx + li) : ts + (li - n_rec);
+                if (pos < 0 || pos >= cl) {
+                    set_status(status, SPEC_ERR_BAD_INDEX);
+                } else {
+                    const int page = page_of(a.kv, pos);
+                    const int slot_in = pos - page * a.kv.page_size;
+                    const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
+                    if (phys < 0 || phys >= a.kv.n_pages) set_status(status, SPEC_ERR_BAD_INDEX);
+                    else off = (uint32_t)((phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride) >> 3);
+                }
+            }
+            rowoff[lr] = off;
+        }
+    }
+    __syncthreads();
+
+    // ---- per-warp pipeline over the chunks warp, warp + NW, ... of the share ----
+    // one instruction copies 16-byte pieces of 32 / (2 * PIECES) rows: the K pieces and the V pieces of each
+    constexpr int PIECES = D / 8, RPI = 32 / (2 * PIECES);
+    const int piece = lane % PIECES, is_v = (lane / PIECES) & 1, rsub = lane / (2 * PIECES);
+    const __nv_bfloat16* gbase = (is_v ? a.kv.v : a.kv.k) + layer * a.kv.layer_stride + hm * a.kv.head_stride + piece * 8;
+    uint8_t* wst = stages + (size_t)warp * ST * STAGE;
+    const uint32_t dst_lane = (is_v ? kChunk * ROWB : 0) + rsub * ROWB + piece * 16;
+
+    auto issue = [&](int c, int stage) {  // gather chunk c (local index) into a stage; always one commit group
+        if (c < nch) {
+            if (!waited && c * kChunk + kChunk > first_tail && first_tail < k1 - k0) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");  // rows of the dense tail are written by the stream
+                waited = true;
+            }
+            const uint32_t mine = rowoff[c * kChunk + (lane & 15)];
+            uint8_t* dst = wst + stage * STAGE + dst_lane;
+#pragma unroll
+            for (int r = 0; r < kChunk; r += RPI) {
+                const uint32_t o = __shfl_sync(0xffffffffu, mine, r + rsub);
+                cp_async16(dst + r * ROWB, gbase + ((int64_t)(o == kNoRow ? 0u : o) << 3), o == kNoRow ? 0u : 16u);
+            }
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int s = 0; s < ST; ++s) issue(warp + s * NW, s);
+
+    if (!waited && tid < G)  // Q is written by an earlier kernel of the stream: ask L2 for its lines meanwhile
+        prefetch_l2(a.q + (((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + tid) * D, D * 2);
+    if (!waited) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // Q is written by the stream
+        waited = true;
+    }
+    // A fragments of Q (heads x d): the thread holds head grp at d = 16 ks + 2 quad + {0, 1} and + {8, 9}
+    uint32_t qa[KS][2];
+    {
+        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + grp;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + row * D);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qa[ks][0] = grp < G ? __ldg(qrow + ks * 8 + quad) : 0u;
+            qa[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
+        }
+    }
+
+    const float sc = a.kv.scale * kLog2e;
+    float M = kNegBig, L = 0.f;
+    float o[D / 8][4];
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+
+    int stage = 0;
+    for (int c = warp; c < nch; c += NW) {
+        cp_async_wait<ST - 1>();
+        __syncwarp();
+        const uint8_t* ksm = wst + stage * STAGE;
+        const uint8_t* vsm = ksm + kChunk * ROWB;
+        // ---- S = Q K^T: keys 0..7 and 8..15 of the chunk are the two 8-wide column blocks ----
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};  // four accumulation chains
+            const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB + ((lane >> 3) & 1) * 16;
+#pragma unroll
+            for (int ks = 0; ks < KS; ks += 2) {
+                uint32_t kf[4], kg[4];
+                ldmatrix_x4(kf, kp + ks * 32);
+                ldmatrix_x4(kg, kp + ks * 32 + 32);
+                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, kf[0], kf[1]);
+                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, kf[2], kf[3]);
+                mma_bf16_16816(t0, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[0], kg[1]);
+                mma_bf16_16816(t1, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[2], kg[3]);
+            }
+            s0[0] += t0[0];
+            s0[1] += t0[1];
+            s1[0] += t1[0];
+            s1[1] += t1[1];
+        }
+        // the thread's four keys: 2 quad, 2 quad + 1, 8 + 2 quad, 9 + 2 quad; masked rows carry no offset
+        const uint2 va = *reinterpret_cast<const uint2*>(rowoff + c * kChunk + 2 * quad);
+        const uint2 vb = *reinterpret_cast<const uint2*>(rowoff + c * kChunk + 8 + 2 * quad);
+        float sv[4];
+        sv[0] = va.x != kNoRow ? s0[0] * sc : kNegBig;
+        sv[1] = va.y != kNoRow ? s0[1] * sc : kNegBig;
+        sv[2] = vb.x != kNoRow ? s1[0] * sc : kNegBig;
+        sv[3] = vb.y != kNoRow ? s1[1] * sc : kNegBig;
+        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        // the running maximum moves only when some head's chunk maximum beats it by 2^8 (warp-uniform branch)
+        if (__any_sync(0xffffffffu, mx > M + 8.f)) {
+            const float Mn = fmaxf(M, mx);
+            const float alpha = ex2f(M - Mn);
+            M = Mn;
+            L *= alpha;
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i) {
+                o[i][0] *= alpha;
+                o[i][1] *= alpha;
+                o[i][2] *= alpha;
+                o[i][3] *= alpha;
+            }
+        }
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = sv[i] > 0.5f * kNegBig ? ex2f(sv[i] - M) : 0.f;
+        L += (p[0] + p[1]) + (p[2] + p[3]);
+        // [P_hi ; P_lo] as the A operand: rows 0..7 the bf16 rounding, rows 8..15 the remainder
+        uint32_t ah0, al0, ah1, al1;
+        {
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(p[0], p[1]), h23 = __floats2bfloat162_rn(p[2], p[3]);
+            ah0 = *reinterpret_cast<const uint32_t*>(&h01);
+            ah1 = *reinterpret_cast<const uint32_t*>(&h23);
+            al0 = pack_bf16(p[0] - __low2float(h01), p[1] - __high2float(h01));
+            al1 = pack_bf16(p[2] - __low2float(h23), p[3] - __high2float(h23));
+        }
+        // ---- O += [P_hi ; P_lo] V ----
+        {
+            const uint8_t* vp = vsm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + ((lane >> 4) & 1) * 16;
+#pragma unroll
+            for (int nb = 0; nb < KS; ++nb) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(vf, vp + nb * 32);
+                mma_bf16_16816(o[2 * nb], ah0, al0, ah1, al1, vf[0], vf[1]);
+                mma_bf16_16816(o[2 * nb + 1], ah0, al0, ah1, al1, vf[2], vf[3]);
+            }
+        }
+        __syncwarp();  // every lane is done with the stage before it is refilled
+        issue(c + ST * NW, stage);
+        stage = stage + 1 == ST ? 0 : stage + 1;
+    }
+    cp_async_wait<0>();
+    L += __shfl_xor_sync(0xffffffffu, L, 1);
+    L += __shfl_xor_sync(0xffffffffu, L, 2);
+
+    // ---- the warps of the CTA: (max, sum, O) through shared memory (each warp's own first stage) ----
+    __syncwarp();
+    {
+        float* ow = reinterpret_cast<float*>(wst);  // [8 heads][D]
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i)
+            *reinterpret_cast<float2*>(ow + grp * D + i * 8 + 2 * quad) = make_float2(o[i][0] + o[i][2], o[i][1] + o[i][3]);
+        if (quad == 0) wml[warp * 8 + grp] = make_float2(M, L);
+    }
+    __syncthreads();
+    // every CTA of the cluster knows by now that the first CTA's deposit barrier is armed
+    if (CS > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const bool remote = rank != 0;
+    float* mine = comb + rank * PS;
+    const uint32_t mine_r = remote ? map_to_rank(smem_addr(mine), 0) : 0u;
+    const uint32_t bar_r = remote ? map_to_rank(smem_addr(dep_bar), 0) : 0u;
+    auto put = [&](int i, float v) {
+        if (remote) st_async_f32(mine_r + 4 * i, v, bar_r);
+        else mine[i] = v;
+    };
+    for (int e = tid; e < G * D; e += NT) {
+        const int r = e / D, d = e - r * D;
+        float Mc = kNegBig;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) Mc = fmaxf(Mc, wml[w * 8 + r].x);
+        float Lc = 0.f, oc = 0.f;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {  // fixed order: deterministic
+            const float2 ml = wml[w * 8 + r];
+            const float wgt = ex2f(ml.x - Mc);
+            Lc += ml.y * wgt;
+            oc += reinterpret_cast<const float*>(stages + (size_t)w * ST * STAGE)[r * D + d] * wgt;
+        }
+        put(e, oc);
+        if (d == 0) {
+            put(G * D + r, Mc);
+            put(G * D + G + r, Lc);
+        }
+    }
+    if (remote) return;
+    if (CS > 1) wait_deposits(smem_addr(dep_bar), a.wait_limit, status);
+    __syncthreads();  // this CTA's own slot
+    merge_and_store<D, NT>(a, comb, CS, G, layer, b, h, tid);
+}
+
+template <int D, int NW, int ST>
+int launch_inst(const DraftArgs& a, const StreamShape& shp, size_t smem, cudaStream_t stream)
+{
+    auto kern = draft_stream_kernel<D, NW, ST>;
+    if (!opt_in_smem(reinterpret_cast<const void*>(kern), smem)) return SPEC_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(shp.cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = shp.cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // Only a call that carries the early-gather promise may start under the preceding kernel; any
+    // other call is an ordinary launch, so whatever follows it finds that kernel's predecessors complete.
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.early_gather ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kern, a, shp, static_cast<int*>(a.workspace)) != cudaSuccess) {
+        cudaGetLastError();
+        return SPEC_ERR_CUDA;
+    }
+    count_launch(1);
+    return SPEC_OK;
+}
+
+template <int D>
+int launch_shape(const DraftArgs& a, const StreamShape& shp, cudaStream_t stream)
+{
+    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+    const size_t smem = stream_smem_bytes<D>(G, shp.nw, shp.st, shp.per, shp.cs);
+    if (smem > kSmemLimit) return SPEC_ERR_UNSUPPORTED_SHAPE;
+#define SPEC_INST(W_, S_) \
+    if (shp.nw == W_ && shp.st == S_) return launch_inst<D, W_, S_>(a, shp, smem, stream);
+    SPEC_INST(4, 2)
+    SPEC_INST(4, 3)
+    SPEC_INST(8, 1)
+    SPEC_INST(8, 2)
+    SPEC_INST(8, 3)
+#undef SPEC_INST
+    return SPEC_ERR_UNSUPPORTED_SHAPE;
+}
+
+}  // namespace
+
+// How a call is split: CTAs per cluster (one cluster per (layer, sequence, KV head)), keys per CTA,
+// warps per CTA and stages per warp.
+//  - Few problems (a per-layer call at batch 1): the call is a chain of latencies, so every chunk
+//    should be in flight at once on as many SMs as a cluster reaches, and the CTAs of three
+//    consecutive calls should fit the GPU together (a call's early gather runs under the calls
+//    before it): 8 warps x 3 stages, one CTA per SM, clusters of 8, or of 6 where three calls of
+//    8-CTA clusters would not fit and a warp still gets about three chunks.
+//  - Many problems: several small CTAs per SM whose gathers overlap each other's arithmetic; the
+//    split is the one a simple cost model likes best (waves of CTAs x the longer of "bytes an SM
+//    pulls at about 48 GB/s" and "trips to memory of one warp").
+bool stream_plan(const KvView& kv, int head_dim, int n_keys_max, StreamShape* out)
+{
+    const long probs = (long)kv.n_layers * kv.batch * kv.n_kv_heads;
+    const int G = kv.n_q_heads / kv.n_kv_heads;
+    const int keys = n_keys_max > 0 ? n_keys_max : 1;
+    const int chunks = (keys + kChunk - 1) / kChunk;
+    const int nsm = sm_count();
+    const size_t stage = head_dim == 128 ? Geo<128>::STAGE : Geo<64>::STAGE;
+    auto smem_of = [&](int cs, int nw, int st, int per) {
+        return (size_t)nw * st * stage + (size_t)per * 4 + (size_t)nw * 64 + 16 + (size_t)cs * G * (head_dim + 2) * 4;
+    };
+    if (probs * draft::kMaxCluster <= nsm) {
+        int cs = draft::kMaxCluster;
+        if (3 * probs * 8 > nsm && 3 * probs * 6 <= nsm && chunks <= 6 * 8 * 3) cs = 6;
+        while (cs > 1 && (chunks + cs - 1) / cs < 8) --cs;  // at least a chunk per warp
+        const int per = (chunks + cs - 1) / cs * kChunk;
+        int st = 3;
+        while (st > 1 && smem_of(cs, 8, st, per) > draft::kSmemLimit) --st;
+        if (smem_of(cs, 8, st, per) > draft::kSmemLimit) return false;
+        *out = StreamShape{cs, per, 8, st};
+        return true;
+    }
+    static const int kCombos[4][2] = {{4, 2}, {4, 3}, {8, 2}, {8, 3}};
+    double best = 1e30;
+    StreamShape bs = {0, 0, 0, 0};
+    for (int cs = 1; cs <= draft::kMaxCluster; ++cs) {
+        const int cc = (chunks + cs - 1) / cs;  // chunks per CTA
+        const int per = cc * kChunk;
+        for (const auto& nwst : kCombos) {
+            const int nw = nwst[0], st = nwst[1];
+            const size_t smem = smem_of(cs, nw, st, per);
+            if (smem > draft::kSmemLimit) continue;
+            int occ = (int)((228 * 1024) / (smem + 1024));
+            occ = occ < 1 ? 1 : occ;
+            if (occ * nw > 48) occ = 48 / nw;  // registers: about 140 per thread
+            const long ctas = probs * cs;
+            const long slots = (long)nsm * occ;
+            const long waves = (ctas + slots - 1) / slots;
+            const int wc = (cc + nw - 1) / nw;     // chunks per warp
+            const int rounds = (wc + st - 1) / st;  // latency-bound trips to memory per warp
+            const double sm_ctas = ctas >= slots ? occ : (double)ctas / nsm > 1.0 ? (double)ctas / nsm : 1.0;
+            const double bytes_us = sm_ctas * cc * (double)stage / 48.0e3;
+            const double trips_us = rounds * 1.3 + wc * 0.18;
+            const double t = waves * (bytes_us > trips_us ? bytes_us : trips_us) + 0.25 * cs + 0.02 * nw;
+            if (t < best) {
+                best = t;
+                bs = StreamShape{cs, per, nw, st};
+            }
+        }
+    }
+    if (bs.cs == 0) return false;
+    *out = bs;
+    return true;
+}
+
+int draft_stream_launch(const DraftArgs& a, const StreamShape& shp, cudaStream_t stream)
+{
+    if (a.kv.head_dim == 128) return launch_shape<128>(a, shp, stream);
+    if (a.kv.head_dim == 64) return launch_shape<64>(a, shp, stream);
+    return SPEC_ERR_UNSUPPORTED_SHAPE;
+}
+
+size_t draft_workspace(const KvView&, int) { return kStatusBytes; }
+
+int draft_launch(const DraftArgs& a, cudaStream_t stream)
+{
+    const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+    if (G > draft::kMaxGroup) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    if (a.workspace_bytes < kStatusBytes) return SPEC_ERR_WORKSPACE_TOO_SMALL;
+    // row offsets travel as 32-bit counts of 16-byte units: a layer's K (or V) must stay below 64 GiB
+    if ((int64_t)a.kv.n_pages * a.kv.page_stride >= ((int64_t)1 << 35)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    StreamShape shp;
+    if (!stream_plan(a.kv, a.kv.head_dim, a.k_total + a.max_tail, &shp)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    return draft_stream_launch(a, shp, stream);
+}
+
+}  // namespace spec

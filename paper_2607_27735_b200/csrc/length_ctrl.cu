@@ -292,11 +292,15 @@ __global__ void controller_select_kernel(const float* __restrict__ state, const 
 // verification context of a round with k drafted tokens, and the draft step lengths.
 __global__ void advance_lengths_kernel(int32_t* __restrict__ committed, const int32_t* __restrict__ n_accepted,
                                        int batch, int k, int32_t* __restrict__ ctx_verify,
-                                       int32_t* __restrict__ cur_len)
+                                       int32_t* __restrict__ cur_len, int max_len, int* __restrict__ status)
 {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
-    const int t = committed[b] + (n_accepted ? min(max(n_accepted[b], 0), k) + 1 : 0);
+    int t = committed[b] + (n_accepted ? min(max(n_accepted[b], 0), k) + 1 : 0);
+    if (max_len > 0 && t + k + 1 > max_len) {  // the next round would leave the cache: hold the sequence and say so
+        t = max(max_len - k - 1, 0);
+        if (status) atomicCAS(status, 0, SPEC_ERR_BAD_INDEX);
+    }
     committed[b] = t;
     if (ctx_verify) ctx_verify[b] = t + k + 1;
     if (cur_len)
@@ -323,9 +327,6 @@ int rows_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t ro
     int cs = 8;
     while (cs > 1 && (long)n_rows * cs > 2L * sm_count()) cs /= 2;
     while (cs > 1 && vocab < cs * 8 * kEntThreads) cs /= 2;
-#ifdef SPEC_TRACE
-    if (const char* e = getenv("SPEC_ENT_CS")) cs = atoi(e);
-#endif
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cs, n_rows);
     cfg.blockDim = dim3(kEntThreads);
@@ -364,10 +365,10 @@ int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_
     return SPEC_OK;
 }
 
-int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int32_t* ctx_verify,
+int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int max_len, int* status, int32_t* ctx_verify,
                            int32_t* cur_len, cudaStream_t stream)
 {
-    advance_lengths_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(committed, n_accepted, batch, k, ctx_verify, cur_len);
+    advance_lengths_kernel<<<(batch + 127) / 128, 128, 0, stream>>>(committed, n_accepted, batch, k, ctx_verify, cur_len, max_len, status);
     if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
     count_launch(1);
     return SPEC_OK;

@@ -15,7 +15,6 @@ constexpr int kD = 128;               // head_dim of the fast path
 constexpr int kSlotBytes = 32768;     // one K or V tile: 2 halves x 128 rows x 128 B (SW128)
 constexpr int kThreads = 384;
 constexpr int kRing = 4;              // partial buffers are recycled every kRing units
-constexpr long long kTimeoutCycles = 2000ll * 1000ll * 1000ll;  // about a second of SM clocks
 constexpr uint64_t kEvictFirst = 0x12F0000000000000ull;
 constexpr uint64_t kEvictLast = 0x14F0000000000000ull;
 constexpr int kTmemCols = 512;
@@ -35,8 +34,7 @@ struct FastParams {
     int n_pages;
     int n_cache;                      // S tiles the TMEM cache holds (cached variant)
     int q_bufs;                       // Q buffers in shared memory (cached variant: 1)
-    long long* trace;
-    int dbg;                          // development knobs (trace builds only)
+    long long wait_limit;             // SM clocks after which a device-side wait gives up
     // divisions of get_seg() as multiply-high + shift (x / d = umulhi(x, mul) >> sh for 0 <= x < 2^31;
     // sh < 0 marks d == 1): by units per layer, by head groups per sequence, by CTAs per head, by the
     // group size G
@@ -183,22 +181,11 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t saddr)
 
 // ---------------------------------------------------------------------------------------------
 
-#ifdef SPEC_TRACE
-// Development aid (not compiled by default): per-CTA, per-role clock64 stamps in the workspace.
-#define TRACE(role, slot) do { if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 60) \
-    p.trace[((int64_t)blockIdx.x * 4 + (role)) * 64 + trace_n[role]++] = ((long long)(slot) << 48) | (clock64() & 0xffffffffffffll); } while (0)
-#define TRACEV(role, slot, val) do { if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 60) \
-    p.trace[((int64_t)blockIdx.x * 4 + (role)) * 64 + trace_n[role]++] = ((long long)(slot) << 48) | ((long long)(val) & 0xffffffffffffll); } while (0)
-#define TCLK() clock64()
-#else
-#define TRACE(role, slot) do { } while (0)
-#define TRACEV(role, slot, val) do { } while (0)
-#define TCLK() 0ll
-#endif
 
 struct Ctl {
     volatile int* abort_flag;  // shared
     int* status;               // global status word (+ diagnostics in the following ints)
+    long long limit;           // SM clocks a wait may take
 };
 
 static __device__ __noinline__ void report_timeout(const Ctl& c, int where)
@@ -219,7 +206,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const C
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*c.abort_flag) return false;
-            if (clock64() - t0 > kTimeoutCycles) {
+            if (clock64() - t0 > c.limit) {
                 report_timeout(c, where);
                 return false;
             }
@@ -237,7 +224,7 @@ __device__ __forceinline__ bool counter_wait(const int* ctr, int target, const C
         __nanosleep(32);
         if ((++spins & 63u) == 0) {
             if (*c.abort_flag) return false;
-            if (clock64() - t0 > kTimeoutCycles) {
+            if (clock64() - t0 > c.limit) {
                 report_timeout(c, where);
                 return false;
             }
@@ -270,7 +257,11 @@ __device__ __forceinline__ Seg get_seg(const FastParams& p, int unit, int head_l
     const int rem = unit - s.layer * per_layer;
     s.b = fast_div(p, 1, rem);
     s.h = (rem - s.b * p.NHG) * p.HG + head_local;
-    s.T = p.a.ctx_len[s.b];
+    // a length outside [n_q, max_ctx_len] is clamped (the launch, the score cache and the output rows
+    // were sized for that range) and reported
+    const int t_in = p.a.ctx_len[s.b];
+    s.T = min(max(t_in, p.a.n_q), p.a.max_ctx_len);
+    if (t_in != s.T) set_status(p.status, SPEC_ERR_BAD_INDEX);
     const int nb = (s.T + kTile - 1) / kTile;
     s.t0 = fast_div(p, 2, rank * nb);        // rank < SMs, nb < 2^20: the products stay far below 2^31
     s.t1 = fast_div(p, 2, (rank + 1) * nb);

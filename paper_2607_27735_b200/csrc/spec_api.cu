@@ -2,7 +2,11 @@
 // stream.  No device allocation, no synchronisation (except spec_read_status).
 #include <atomic>
 #include <cmath>
+#include <map>
+#include <mutex>
+#include <utility>
 
+#include "draft_common.cuh"
 #include "spec_common.cuh"
 #include "verify_sm100.cuh"
 
@@ -14,18 +18,40 @@ static std::atomic<int> g_last_verify_impl{0};
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Everything remembered about a device is kept per device ordinal: one process may drive several.
+constexpr int kMaxDevices = 64;
+
 int sm_count()
 {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            cached = n;
-        else
-            return 148;
+    static std::atomic<int> cached[kMaxDevices];
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+    n = cached[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+        cached[dev].store(n, std::memory_order_relaxed);
     }
-    return cached;
+    return n;
+}
+
+static std::atomic<long long> g_wait_limit{2000ll * 1000ll * 1000ll};  // about a second of SM clocks
+long long wait_limit() { return g_wait_limit.load(std::memory_order_relaxed); }
+
+bool draft::opt_in_smem(const void* kernel, size_t smem)
+{
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, size_t> configured;  // (kernel, device) -> largest size opted in
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    size_t& have = configured[std::make_pair(kernel, dev)];
+    if (smem <= have) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    have = smem;
+    return true;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -166,12 +192,15 @@ int spec_sparse_draft_attn_ex(const spec_kv_t* kv, const void* q, const int32_t*
                               const int32_t* cur_len, int32_t max_tail, float* out, float* lse,
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream)
 {
-    if (flags & ~(uint32_t)(SPEC_DRAFT_INDICES_PER_QUERY_HEAD | SPEC_DRAFT_OUT_BF16)) return SPEC_ERR_INVALID_ARG;
+    if (flags & ~(uint32_t)(SPEC_DRAFT_INDICES_PER_QUERY_HEAD | SPEC_DRAFT_OUT_BF16 | SPEC_DRAFT_EARLY_GATHER))
+        return SPEC_ERR_INVALID_ARG;
     DraftArgs a;
     const int rc = make_view(kv, &a.kv);
     if (rc != SPEC_OK) return rc;
     a.head_div = 1;
     a.out_bf16 = (flags & SPEC_DRAFT_OUT_BF16) ? 1 : 0;
+    a.early_gather = (flags & SPEC_DRAFT_EARLY_GATHER) ? 1 : 0;
+    a.wait_limit = wait_limit();
     if (flags & SPEC_DRAFT_INDICES_PER_QUERY_HEAD) {
         // every attention head is a problem of its own (group size 1) that reads the rows of its
         // KV head: the kernels see n_q_heads "KV heads" and divide the head index for the cache
@@ -255,11 +284,12 @@ int spec_accept_greedy(const void* logits, int32_t dtype, int32_t batch, int32_t
 }
 
 int spec_advance_lengths(int32_t* committed, const int32_t* n_accepted, int32_t batch, int32_t k,
-                         int32_t* ctx_verify, int32_t* cur_len, void* cuda_stream)
+                         int32_t max_len, void* workspace, int32_t* ctx_verify, int32_t* cur_len,
+                         void* cuda_stream)
 {
-    if (!committed || batch < 0 || k < 0) return SPEC_ERR_INVALID_ARG;
+    if (!committed || batch < 0 || k < 0 || max_len < 0) return SPEC_ERR_INVALID_ARG;
     if (batch == 0) return SPEC_OK;
-    return advance_lengths_launch(committed, n_accepted, batch, k, ctx_verify, cur_len,
+    return advance_lengths_launch(committed, n_accepted, batch, k, max_len, static_cast<int*>(workspace), ctx_verify, cur_len,
                                   static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -305,6 +335,12 @@ int spec_set_verify_impl(int impl)
 
 int spec_last_verify_impl(void) { return g_last_verify_impl.load(); }
 
+int64_t spec_set_wait_limit_cycles(int64_t cycles)
+{
+    if (cycles < 1) return SPEC_ERR_INVALID_ARG;
+    return g_wait_limit.exchange(cycles);
+}
+
 int64_t spec_launch_count(void) { return g_launches.load(); }
 
 const char* spec_strerror(int code)
@@ -316,7 +352,7 @@ const char* spec_strerror(int code)
         case SPEC_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case SPEC_ERR_CUDA: return "CUDA error";
         case SPEC_ERR_TIMEOUT: return "device-side wait timed out";
-        case SPEC_ERR_BAD_INDEX: return "recall index out of range";
+        case SPEC_ERR_BAD_INDEX: return "recall index, page-table entry or length out of range";
         default: return "unknown error";
     }
 }

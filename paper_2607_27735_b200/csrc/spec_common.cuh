@@ -44,12 +44,19 @@ __device__ __forceinline__ int page_of(const KvView& kv, int pos)
     return kv.page_sh < 0 ? pos : (int)(__umulhi((uint32_t)pos, kv.page_mul) >> kv.page_sh);
 }
 
-__device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, int b, int pos, int h)
+// Offset of a cache row.  A page-table entry outside [0, n_pages) is replaced by page 0 (the access stays
+// inside the cache) and, when a status word is given, reported there as SPEC_ERR_BAD_INDEX.
+__device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, int b, int pos, int h,
+                                                 int* status = nullptr)
 {
     const int page = page_of(kv, pos);
     const int slot = pos - page * kv.page_size;
-    const int64_t phys = kv.page_table ? (int64_t)__ldg(kv.page_table + (int64_t)b * kv.max_pages + page)
-                                       : (int64_t)b * kv.max_pages + page;
+    int64_t phys = kv.page_table ? (int64_t)__ldg(kv.page_table + (int64_t)b * kv.max_pages + page)
+                                 : (int64_t)b * kv.max_pages + page;
+    if (phys < 0 || phys >= kv.n_pages) {
+        if (status) atomicCAS(status, 0, SPEC_ERR_BAD_INDEX);
+        phys = 0;
+    }
     return layer * kv.layer_stride + phys * kv.page_stride + h * kv.head_stride +
            slot * kv.slot_stride;
 }
@@ -101,6 +108,16 @@ struct VerifyArgs {
     int out_bf16;         // `out` points to bf16 elements (round to nearest even) instead of fp32
 };
 
+// Context length of sequence b as the kernels use it: a value outside [n_q, max_ctx_len] (the range the
+// launch, the workspace and the score rows were sized for) is clamped into it and reported.
+__device__ __forceinline__ int clamped_ctx_len(const VerifyArgs& a, int b)
+{
+    const int t = a.ctx_len[b];
+    const int T = min(max(t, a.n_q), a.max_ctx_len);
+    if (T != t) set_status(static_cast<int*>(a.workspace), SPEC_ERR_BAD_INDEX);
+    return T;
+}
+
 size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);
 int verify_generic_launch(const VerifyArgs& a, cudaStream_t stream);
 
@@ -124,6 +141,10 @@ struct DraftArgs {
     int head_div;  // K/V of problem head h are read from cache head h / head_div (1 unless every
                    // attention head carries its own index set)
     int out_bf16;  // `out` points to bf16 elements (round to nearest even) instead of fp32
+    int early_gather;      // the caller promised that the index sets, lengths and recalled rows were complete
+                           // before the preceding kernel of the stream started: they are read before this
+                           // kernel's dependency on that kernel is resolved
+    long long wait_limit;  // SM clocks after which a device-side wait gives up (SPEC_ERR_TIMEOUT)
 };
 size_t draft_workspace(const KvView& kv, int k_total_plus_tail);
 int draft_launch(const DraftArgs& a, cudaStream_t stream);
@@ -132,7 +153,7 @@ int rows_launch(const void* logits, int dtype, int n_rows, int vocab, int64_t ro
                 int32_t* token, cudaStream_t stream);
 int accept_launch(const int32_t* target, const int32_t* draft, const int32_t* n_draft, int batch, int k1,
                   int32_t* n_accepted, int32_t* next_token, cudaStream_t stream);
-int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int32_t* ctx_verify,
+int advance_lengths_launch(int32_t* committed, const int32_t* n_accepted, int batch, int k, int max_len, int* status, int32_t* ctx_verify,
                            int32_t* cur_len, cudaStream_t stream);
 int controller_update_launch(float* state, const float* entropy, int k, const int32_t* n_accepted, float beta,
                              cudaStream_t stream);
@@ -141,6 +162,7 @@ int controller_select_launch(const float* state, const float* entropy, int n, co
                              cudaStream_t stream);
 
 void count_launch(int n = 1);
-int sm_count();
+int sm_count();            // of the current device
+long long wait_limit();    // SM clocks a device-side wait may take (spec_set_wait_limit_cycles)
 
 }  // namespace spec

@@ -56,11 +56,14 @@ int spec_verify_attn_noalloc(const spec_kv_t* kv, const void* q, int32_t n_q, co
     const int rc = scratch_address(&scratch);
     if (rc != SPEC_OK) return rc;
     // The array keeps whatever the previous call left (possibly laid out for another shape): the
-    // status word and the cross-CTA counters that follow it (at most two per (layer, sequence,
-    // KV head) plus one) must start at zero.
-    size_t head = spec::kStatusBytes + (2 * (size_t)kv->n_layers * kv->batch * kv->n_kv_heads + 1) * sizeof(int) + 256;
-    if (head > need) head = need;
-    if (cudaMemsetAsync(scratch, 0, head, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return SPEC_ERR_CUDA;
+    // cross-CTA counters behind the status block (at most two per (layer, sequence, KV head) plus
+    // one) must start at zero.  The status word itself is left alone, so that an error nobody has
+    // read yet survives until spec_noalloc_read_status(), as with a caller's workspace.
+    size_t head = (2 * (size_t)kv->n_layers * kv->batch * kv->n_kv_heads + 1) * sizeof(int) + 256;
+    if (spec::kStatusBytes + head > need) head = need > spec::kStatusBytes ? need - spec::kStatusBytes : 0;
+    if (head > 0 && cudaMemsetAsync(static_cast<char*>(scratch) + spec::kStatusBytes, 0, head,
+                                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return SPEC_ERR_CUDA;
     return spec_verify_attn(kv, q, n_q, ctx_len, max_ctx_len, stat_window, out, lse, stats, stat_stride, scratch,
                             kStaticScratchBytes, cuda_stream);
 }

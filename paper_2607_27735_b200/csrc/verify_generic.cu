@@ -52,14 +52,14 @@ Layout make_layout(const KvView& kv, int n_q, int max_ctx_len)
 template <int D>
 __device__ __forceinline__ void score_tile(const KvView& kv, int layer, int b, int h,
                                            const float* __restrict__ Qs, float* __restrict__ S,
-                                           int R, int G, int n_q, int T, int key0)
+                                           int R, int G, int n_q, int T, int key0, int* status)
 {
     const int key_l = threadIdx.x % kTK;
     const int rg = threadIdx.x / kTK;  // 0 or 1
     const int key = key0 + key_l;
     const bool valid = key < T;
     const uint4* krow = nullptr;
-    if (valid) krow = reinterpret_cast<const uint4*>(kv.k + kv_row_offset(kv, layer, b, key, h));
+    if (valid) krow = reinterpret_cast<const uint4*>(kv.k + kv_row_offset(kv, layer, b, key, h, status));
     for (int r0 = rg * 4; r0 < R; r0 += 8) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         if (valid) {
@@ -123,7 +123,7 @@ verify_lse_partial_kernel(VerifyArgs a, int n_splits, float2* __restrict__ ml_pa
     float* l_run = m_run + R;
     const int split = blockIdx.x, h = blockIdx.y;
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
-    const int T = a.ctx_len[b];
+    const int T = clamped_ctx_len(a, b);
     int t0, t1;
     split_range(T, n_splits, split, t0, t1);
     load_q<D>(a, layer, b, h, R, G, Qs);
@@ -134,7 +134,7 @@ verify_lse_partial_kernel(VerifyArgs a, int n_splits, float2* __restrict__ ml_pa
     __syncthreads();
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     for (int t = t0; t < t1; ++t) {
-        score_tile<D>(a.kv, layer, b, h, Qs, S, R, G, a.n_q, T, t * kTK);
+        score_tile<D>(a.kv, layer, b, h, Qs, S, R, G, a.n_q, T, t * kTK, static_cast<int*>(a.workspace));
         __syncthreads();
         for (int r = warp; r < R; r += kThreads / 32) {
             float v[kTK / 32];
@@ -203,7 +203,7 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
     const int split = blockIdx.x, h = blockIdx.y;
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
     const int64_t prob = (int64_t)blockIdx.z * a.kv.n_kv_heads + h;
-    const int T = a.ctx_len[b];
+    const int T = clamped_ctx_len(a, b);
     int t0, t1;
     split_range(T, n_splits, split, t0, t1);
     load_q<D>(a, layer, b, h, R, G, Qs);
@@ -219,7 +219,7 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
 
     for (int t = t0; t < t1; ++t) {
         const int key0 = t * kTK;
-        score_tile<D>(a.kv, layer, b, h, Qs, S, R, G, a.n_q, T, key0);
+        score_tile<D>(a.kv, layer, b, h, Qs, S, R, G, a.n_q, T, key0, static_cast<int*>(a.workspace));
         __syncthreads();
         for (int idx = threadIdx.x; idx < R * kTK; idx += kThreads) {
             const int r = idx / kTK, kl = idx - r * kTK;
@@ -248,7 +248,7 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
                 if (kl + kk < nk) {
-                    const __nv_bfloat16* vrow = a.kv.v + kv_row_offset(a.kv, layer, b, key0 + kl + kk, h);
+                    const __nv_bfloat16* vrow = a.kv.v + kv_row_offset(a.kv, layer, b, key0 + kl + kk, h, static_cast<int*>(a.workspace));
                     const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(vrow) + dp);
                     v0[kk] = bf16_lo(w);
                     v1[kk] = bf16_hi(w);

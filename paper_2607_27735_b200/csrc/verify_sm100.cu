@@ -33,7 +33,7 @@ struct Plan {
     bool cached;
     int HG, cph, n_units, N, n_slots, p_bufs, box_rows, boxes, n_cache;
     size_t smem_bytes;
-    size_t ctr_off, ctr_bytes, ml_off, o_off, total, trace_off;
+    size_t ctr_off, ctr_bytes, ml_off, o_off, total;
 };
 
 int box_rows_for(int page_size)
@@ -111,9 +111,6 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         // barriers and small arrays; the rest is the K/V tile ring
         pl->p_bufs = 2;
         fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544;
-#ifdef SPEC_TRACE
-        fixed += 1536;  // stamps of the development trace
-#endif
         slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
         if (slots > 8) slots = 8;
         // more P buffers (up to four) where they cost no K/V slot: the P V product of a tile then has two tiles
@@ -151,11 +148,6 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
     pl->o_off = off;
     off += (size_t)kRing * pl->HG * pl->cph * R * kD * sizeof(float);
     pl->total = (off + 255) & ~(size_t)255;
-    pl->trace_off = 0;
-#ifdef SPEC_TRACE
-    pl->trace_off = pl->total;
-    pl->total += (size_t)nsm * 4 * 64 * sizeof(long long);
-#endif
     return true;
 }
 
@@ -226,9 +218,9 @@ __global__ void shorten_ctx_kernel(const int32_t* ctx_len, int by, int32_t* out)
 
 // stats <- (first part's value where it wrote one) + second part's value
 __global__ void add_stats_kernel(float* stats, int64_t stat_stride, const float* second, int64_t second_stride,
-                                 const int32_t* ctx_len, int nB, int n_kv_heads, int accumulate)
+                                 const int32_t* ctx_len, int max_ctx_len, int nB, int n_kv_heads, int accumulate)
 {
-    const int T = ctx_len[0];
+    const int T = min(max(ctx_len[0], 0), max_ctx_len);  // the two verification kernels report a length out of range
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < (int64_t)n_kv_heads * T;
          i += (int64_t)gridDim.x * blockDim.x) {
         const int h = (int)(i / T), key = (int)(i - (int64_t)h * T);
@@ -299,7 +291,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
         pb.workspace_bytes = sp.main_bytes;
         rc = verify_sm100_launch(pb, 2, stream, nullptr);
         if (rc != SPEC_OK) return rc;
-        add_stats_kernel<<<sm_count(), 256, 0, stream>>>(a.stats, a.stat_stride, second, sp.stat_stride, a.ctx_len, sp.nB,
+        add_stats_kernel<<<sm_count(), 256, 0, stream>>>(a.stats, a.stat_stride, second, sp.stat_stride, a.ctx_len, a.max_ctx_len, sp.nB,
                                                          a.kv.n_kv_heads, a.stat_accumulate);
         count_launch(1);
         if (cudaGetLastError() != cudaSuccess) return SPEC_ERR_CUDA;
@@ -340,12 +332,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.status = reinterpret_cast<int*>(ws);
     fp.n_pages = n_pages;
     fp.n_cache = pl.n_cache;
-    fp.trace = nullptr;
-    fp.dbg = 0;
-#ifdef SPEC_TRACE
-    fp.trace = reinterpret_cast<long long*>(ws + a.workspace_bytes - (size_t)sm_count() * 4 * 64 * sizeof(long long));  // tail of the caller's buffer
-    if (const char* e = std::getenv("SPEC_DBG")) fp.dbg = std::atoi(e);
-#endif
+    fp.wait_limit = wait_limit();
     // no memset: the workspace arrives zeroed and the kernel's last CTA re-zeroes the counters
     if (used_variant) *used_variant = pl.cached ? 2 : 1;
     const int grid = pl.cph * pl.HG;

@@ -38,16 +38,6 @@ namespace sm100 {
 
 namespace {
 
-#ifdef SPEC_TRACE
-// Development trace: stamps collect in shared memory and reach the workspace at the end (a global
-// store per stamp would sit in front of the stamped warp's next barrier); the clock is read by a
-// volatile asm with a memory clobber so that it keeps its place among the waits it brackets.
-#define CTRACE(role, slot) do { long long t_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(t_) :: "memory"); \
-    if (p.trace && (threadIdx.x & 31) == 0 && trace_n[role] < 48) \
-    trace_s[(role) * 48 + trace_n[role]++] = ((long long)(slot) << 48) | (t_ & 0xffffffffffffll); } while (0)
-#else
-#define CTRACE(role, slot) do { } while (0)
-#endif
 
 constexpr int kMaxCache = 32;
 constexpr int kLsePubMax = 48;  // CTAs per head up to which the publisher warp alone combines the LSE partials
@@ -161,12 +151,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 12288);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    Ctl ctl{abort_flag, p.status};
-#ifdef SPEC_TRACE
-    int trace_n[4] = {0, 0, 0, 0};
-    long long* trace_s = reinterpret_cast<long long*>(misc + 12544);
-    for (int i = threadIdx.x; i < 192; i += blockDim.x) trace_s[i] = 0;
-#endif
+    Ctl ctl{abort_flag, p.status, p.wait_limit};
 
     if (threadIdx.x < kMaxCache) {  // one region's pair of barriers per thread
         mbar_init(B.s_full + 8 * threadIdx.x, 1);
@@ -256,7 +241,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         for (int u = 0; u < U && ok; ++u) {
             const Seg sg = get_seg(p, u, head_local, rank);
             if (sg.t1 <= sg.t0) continue;
-            CTRACE(0, 1);
             const uint32_t qb = 0, qph = qn & 1;
             ++qn;
             ok = mbar_wait(B.q_empty + 8 * qb, qph ^ 1, ctl, 2);
@@ -269,16 +253,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
             __syncwarp();
             for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t);
-            CTRACE(0, 2);
-#ifdef SPEC_TRACE
-            if (p.dbg & 32) {  // experiment: hold the V prefetch until half of the head's CTAs published P1
-                bool got = true;
-                if (lane == 0) got = counter_wait(p.counters + u * p.HG + head_local, p.cph / 2, ctl, 3);
-                if (!__shfl_sync(0xffffffffu, got ? 1 : 0, 0)) break;
-            }
-#endif
             for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_v, sg, t);
-            CTRACE(0, 3);
         }
         if (!ok) {  // let copies in flight land before the CTA's shared memory is released
             const long long t0 = clock64();
@@ -351,12 +326,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 }
                 tc_commit(B.s_full + 8 * c);
                 tc_commit(B.slot_empty + 8 * s);
-#ifdef SPEC_TRACE
-                if (p.dbg & 16) {
-                    mbar_wait(B.slot_empty + 8 * s, (slot / p.n_slots) & 1, ctl, 18);
-                    CTRACE(1, 4);
-                }
-#endif
                 if (qq.t == qq.t1 - 1) tc_commit(B.q_empty + 8 * qq.qb);  // last use of this Q buffer
                 if (++qq.t == qq.t1) seek(qq);
             };
@@ -417,7 +386,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 if ((++spins & 63u) == 0) {
                     if (spins == 64) t_idle = clock64();
                     if (*ctl.abort_flag) ok = false;
-                    else if (clock64() - t_idle > kTimeoutCycles) {
+                    else if (clock64() - t_idle > ctl.limit) {
                         report_timeout(ctl, 16);
                         ok = false;
                     }
@@ -512,7 +481,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (lane == 0) ok = counter_wait(p.counters + U * p.HG + unit * p.HG + head_local, p.cph, ctl, 30);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-            CTRACE(3, 1);
             const Seg sg = get_seg(p, unit, head_local, rank);
             const int E4 = R * kD / 4;
             const int lo = fast_div(p, 2, rank * E4), hi = fast_div(p, 2, (rank + 1) * E4);  // products far below 2^31
@@ -546,7 +514,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 else
                     reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
             }
-            CTRACE(3, 2);
         }
     } else {
         // =========================== softmax warpgroups ===========================
@@ -597,7 +564,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             const Seg sg = get_seg(p, unit, head_local, rank);
             const int n_t = sg.t1 - sg.t0;
             const bool nonempty = n_t > 0;
-            if (warp == 4) CTRACE(2, 1);
             // ------------------------------ P1 ------------------------------
             float m[NH], l[NH];
 #pragma unroll
@@ -646,7 +612,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 for (int i = 0; i < NH; ++i) l[i] += ex2(sc[i] - m[i]);
             }
             if (!ok) break;
-            if (warp == 4) CTRACE(2, 2);
             // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem:
             // a butterfly that halves the columns a lane carries at every step (see ml_step)
             {
@@ -685,7 +650,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
             ok = group_sync(B.sm_sync, sync_n, ctl, 27);
             if (!ok) break;
-            if (warp == 4) CTRACE(2, 3);
             if (nonempty) {
                 // ------------------------------ P2a: P V with the CTA-local normaliser ------------------
                 // P~ = exp2(S - lse_local) needs nothing from other CTAs, so V streams and the tensor
@@ -788,11 +752,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 tc_fence_before();
                 pv_idx += n_t;
                 slot_base += 2 * n_t;
-                if (warp == 4) CTRACE(2, 4);
                 // ---- the row LSE and the rescale factors, combined by the publisher warp meanwhile ----
                 ok = mbar_wait(B.lse_ready, unit & 1, ctl, 31);
                 if (!ok) break;
-                if (warp == 4) CTRACE(2, 5);
                 if (!LP) {  // many CTAs per head: too many partials for one warp, all softmax threads fold them
                     if (lane == 0) ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 33);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;  // lane 0's acquire, then warp-wide
@@ -840,7 +802,6 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 ok = group_sync(B.sm_sync, sync_n, ctl, 22);  // every warp is done with the P V pass
                 if (!ok) break;
                 tc_fence_after();  // the P~ stores of the other warps, ordered by the barrier
-                if (warp == 4) CTRACE(2, 6);
                 // ------------------------------ P2b: the Eq. 3 statistic ------------------------------
                 // second visit of the cached tiles, which hold P~ = exp2(S - lse_local) by now (masked
                 // entries are 0): weighted with exp2(lse_local - LSE) per row they are the exactly
@@ -924,21 +885,15 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 ok = mbar_wait(B.lse_ready, unit & 1, ctl, 32);  // keeps step with the publisher warp (see there)
                 if (!ok) break;
             }
-            if (warp == 4) CTRACE(2, 7);
             // ---- this unit's accumulator: rescale and hand to the reducers ----
             ok = epilogue(unit, nonempty);
             if (!ok) break;
-            if (warp == 4) CTRACE(2, 8);
         }
     }
 
     // ---- teardown ----
     tc_fence_before();
     __syncthreads();
-#ifdef SPEC_TRACE
-    if (p.trace)
-        for (int i = threadIdx.x; i < 192; i += blockDim.x) p.trace[(int64_t)blockIdx.x * 256 + i] = trace_s[i];
-#endif
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -970,11 +925,14 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    static bool pdl_ok = true;  // a driver that refuses it is asked only once
+    static bool pdl_refused[64] = {};  // per device: a driver that refuses the attribute is asked only once
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    const bool pdl_ok = !pdl_refused[dev];
     cudaError_t err = pdl_ok ? cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp) : cudaErrorNotSupported;
     if (err != cudaSuccess) {
         if (pdl_ok) cudaGetLastError();
-        pdl_ok = false;
+        pdl_refused[dev] = true;
         attr[0].id = cudaLaunchAttributeCooperative;
         attr[0].val.cooperative = 1;
         err = cudaLaunchKernelEx(&cfg, kern, tk, tv, tq, fp);

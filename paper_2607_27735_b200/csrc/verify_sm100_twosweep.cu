@@ -159,10 +159,7 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 512 + 3072 + 8 * 64 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    Ctl ctl{abort_flag, p.status};
-#ifdef SPEC_TRACE
-    int trace_n[4] = {0, 0, 0, 0};
-#endif
+    Ctl ctl{abort_flag, p.status, p.wait_limit};
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.n_slots; ++i) {
@@ -233,7 +230,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
             return true;
         };
         for (int round = 0; round <= U && ok; ++round) {
-            TRACE(0, 1);
             if (round < U) {
                 const Seg sg = get_seg(p, round, head_local, rank);
                 if (sg.t1 > sg.t0) {
@@ -251,7 +247,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t, kEvictLast);
                 }
             }
-            TRACE(0, 2);
             if (round >= 1 && ok) {
                 const Seg sg = get_seg(p, round - 1, head_local, rank);
                 for (int t = sg.t0; t < sg.t1 && ok; ++t) {
@@ -360,11 +355,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
         bool ok = true;
         int prev_lse_idx = 0;
         bool prev_nonempty = false;
-        long long w_sfull = 0, w_pempty = 0, w_stat = 0;
         for (int round = 0; round <= U && ok; ++round) {
             bool cur_nonempty = false;
-            if (warp == 2) { TRACEV(1, 1, w_sfull); TRACEV(1, 2, w_pempty); TRACEV(1, 3, w_stat); w_sfull = w_pempty = w_stat = 0; }
-            if (warp == 2) TRACE(2, 1);
             if (round < U) {
                 // ------------------------------ P1 ------------------------------
                 const Seg sg = get_seg(p, round, head_local, rank);
@@ -379,10 +371,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     const uint32_t sb = qk_idx & 1, sbph = (qk_idx >> 1) & 1;
                     ++qk_idx;
                     ++slot_idx;
-                    const long long tw0 = TCLK();
                     ok = mbar_wait(B.s_full + 8 * sb, sbph, ctl, 20);
                     if (!ok) break;
-                    w_sfull += TCLK() - tw0;
                     tc_fence_after();
                     uint32_t v[NH];
                     load_cols<NH>(t_lane + (sb ? kColS1 : kColS0) + c0, v);
@@ -422,7 +412,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     for (int i = 0; i < NH; ++i) l[i] += ex2(sc[i] - m[i]);
                 }
                 if (!ok) break;
-                if (warp == 2) { TRACE(2, 2); TRACEV(1, 4, w_sfull); w_sfull = 0; }
                 // reduce (m, l) over the 32 key lanes of this warp, then over the 4 warps via smem
 #pragma unroll
                 for (int i = 0; i < NH; ++i) {
@@ -460,7 +449,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     atomicAdd(p.counters + round * p.HG + head_local, 1);
                 }
             }
-            if (warp == 2) TRACE(2, 3);
             if (round >= 1 && ok) {
                 // ------------------------------ P2 ------------------------------
                 const Seg sg = get_seg(p, round - 1, head_local, rank);
@@ -470,7 +458,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     ok = mbar_wait(B.lse_full + 8 * lb, lph, ctl, 21);
                     if (!ok) break;
                     const float4* lse4 = reinterpret_cast<const float4*>(lse_s + lb * 128 + c0);
-                    if (warp == 2) TRACE(2, 4);
                     for (int t = sg.t0; t < sg.t1 && ok; ++t) {
                         const uint32_t sb = qk_idx & 1, sbph = (qk_idx >> 1) & 1;
                         ++qk_idx;
@@ -479,10 +466,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                         ++slot_idx;                       // V slot
                         const uint32_t pb = pv_idx % p.p_bufs, pph = (pv_idx / p.p_bufs) & 1;
                         ++pv_idx;
-                        const long long tw0 = TCLK();
                         ok = mbar_wait(B.s_full + 8 * sb, sbph, ctl, 22);
                         if (!ok) break;
-                        w_sfull += TCLK() - tw0;
                         tc_fence_after();
                         uint32_t v[NH];
                         load_cols<NH>(t_lane + (sb ? kColS1 : kColS0) + c0, v);
@@ -513,10 +498,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                         float st = 0.f;
 #pragma unroll
                         for (int i = 0; i < NH; ++i) st += (c0 + i >= stat_r0) ? pr[i] : 0.f;
-                        const long long tw1 = TCLK();
                         ok = mbar_wait(B.p_empty + 8 * pb, pph ^ 1, ctl, 23);
                         if (!ok) break;
-                        w_pempty += TCLK() - tw1;
                         // [P_hi | P_lo]^T as the B operand, rows contiguous (MN-major, 128-byte swizzle):
                         // 16-byte chunk j (rows 8j..8j+7 of the concatenation) of key k lives at
                         // (j/8)*16384 + k*128 + ((j%8) ^ (k%8))*16
@@ -571,10 +554,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                             __syncwarp();
                             if (lane == 0) mbar_arrive(B.stat_full + 8 * sq);
                         } else {
-                            const long long tw2 = TCLK();
                             ok = mbar_wait(B.stat_full + 8 * sq, sqph, ctl, 28);
                             if (!ok) break;
-                            w_stat += TCLK() - tw2;
                             if (key < sg.T) {
                                 float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
                                 const float v = st + stat_tmp[sq * 128 + key_l];
@@ -585,7 +566,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     if (!ok) break;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(B.lse_empty + 8 * lb);
-                    if (warp == 2) TRACE(2, 5);
                     // ---- epilogue: O^T (d on lanes, rows on columns) -> partial [r][d] ----
                     ok = mbar_wait(B.o_full, o_phase, ctl, 25);
                     if (!ok) break;
@@ -615,7 +595,6 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
             }
             if (cur_nonempty) prev_lse_idx = lse_n++;
             prev_nonempty = cur_nonempty;
-            if (warp == 2) TRACE(2, 6);
         }
     } else {
         // =========================== aux warps: LSE combine, O reduction ===========================
@@ -665,10 +644,8 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                 if (sg.t1 > sg.t0) {
                     const uint32_t lb = lse_n & 1, lph = (lse_n >> 1) & 1;
                     ++lse_n;
-                    if (warp == 10) TRACE(3, 1);
                     ok = counter_wait(p.counters + unit * p.HG + head_local, p.cph, ctl, 31);
                     if (!ok) break;
-                    if (warp == 10) TRACE(3, 2);
                     __threadfence();
                     ok = mbar_wait(B.lse_empty + 8 * lb, lph ^ 1, ctl, 32);
                     if (!ok) break;
@@ -702,11 +679,9 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                     ok = group_sync(B.aux_sync, sync_n, ctl, 33);
                     if (!ok) break;
                     if (tid == 0) mbar_arrive(B.lse_full + 8 * lb);
-                    if (warp == 10) TRACE(3, 3);
                 }
             }
             if (round >= 2) ok = reduce_unit(round - 2);
-            if (warp == 10) TRACE(3, 4);
         }
     }
 

@@ -73,18 +73,24 @@ class SpecStepRunner:
 
     def draft_phase(self):
         c = self.cfg
+        # The index sets and every step's lengths are complete before the phase begins, so every call
+        # but the first (whose predecessor in the stream may be their producer) may gather early.
+        first = True
         for j in range(c.draft_steps):
             if self.fold:
                 binding.spec_sparse_draft_attn(
                     self.kv, self.q_draft[j], self.indices, self.n_idx, self.tail_start,
                     self.cur_lens[j], c.draft_steps, out=self.out_d[j], workspace=self.ws_d,
-                    want_lse=False, per_head=self.per_head)
+                    want_lse=False, per_head=self.per_head, early_gather=not first)
+                first = False
                 continue
             for l in range(self.L):
                 binding.spec_sparse_draft_attn(
                     self._layers[l], self.q_draft[j, l:l + 1], self.indices[l:l + 1],
                     self.n_idx[l:l + 1], self.tail_start, self.cur_lens[j], c.draft_steps,
-                    out=self.out_d[j, l:l + 1], workspace=self.ws_d, want_lse=False, per_head=self.per_head)
+                    out=self.out_d[j, l:l + 1], workspace=self.ws_d, want_lse=False, per_head=self.per_head,
+                    early_gather=not first)
+                first = False
 
     def step(self):
         self.verify_phase()
@@ -209,13 +215,15 @@ class SpecLoopRunner:
         committed length (what a prefill leaves behind), and the first round's lengths."""
         self._verify(self.committed)
         self._select()
-        binding.spec_advance_lengths(self.committed, None, self.k, self.ctx_verify, self.cur_len)
+        binding.spec_advance_lengths(self.committed, None, self.k, self.ctx_verify, self.cur_len,
+                                     max_len=self.max_ctx, workspace=self.ws_v)
 
     def round(self):
         for j in range(self.k):
+            # step 0 follows the kernels that wrote the index sets and the lengths; the later steps do not
             binding.spec_sparse_draft_attn(self.kv, self.case.q_draft[j], self.indices, self.n_idx, self.committed,
                                            self.cur_len[j], self.k, out=self.out_d[j], workspace=self.ws_d,
-                                           want_lse=False)
+                                           want_lse=False, early_gather=j > 0)
         self._verify(self.ctx_verify)
         binding.spec_accept_greedy(self.logits, self.draft_tokens, target=self.target,
                                    n_accepted=self.n_accepted, next_token=self.next_token)
@@ -223,7 +231,8 @@ class SpecLoopRunner:
         binding.spec_controller_update(self.state, self.entropy, self.n_accepted[:1], self.beta)
         binding.spec_controller_select(self.state, self.entropy, self.cand, self.c_d, self.c_v,
                                        k_star=self.k_star, p=self.p, score=self.score)
-        binding.spec_advance_lengths(self.committed, self.n_accepted, self.k, self.ctx_verify, self.cur_len)
+        binding.spec_advance_lengths(self.committed, self.n_accepted, self.k, self.ctx_verify, self.cur_len,
+                                     max_len=self.max_ctx, workspace=self.ws_v)
         self._select()
 
     def capture(self):

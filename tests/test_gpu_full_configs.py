@@ -103,10 +103,10 @@ def test_cfg2_8b_32k_full_step_sampled_heads():
     assert hits / 3 > 0.9
 
 
-@pytest.mark.parametrize("k", [1, 16])
-def test_cfg3_128k_speculation_length_sweep_ends(k):
-    """131072-token context, 4 of the 32 layers; k = 16 gives 68 rows per KV head and a window
-    longer than W."""
+@pytest.mark.parametrize("k", [1, 2, 8, 16])
+def test_cfg3_128k_speculation_length_sweep(k):
+    """131072-token context, 4 of the 32 layers, the workload's sweep of speculation lengths (k = 4
+    runs in the drift test below); k = 16 gives 68 rows per KV head and a window longer than W."""
     cfg = dataclasses.replace(inputs.baseline_configs(k)["cfg3_8b_128k"], n_layers=4)
     run_config(cfg, [(0, 0, 1), (3, 0, 6)])
 
