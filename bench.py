@@ -320,7 +320,8 @@ def run_gpu(args):
         import dataclasses
         cfg = dataclasses.replace(cfg, seed=cfg.seed + 101 * rank)
     case = inputs.make_case(cfg, device=dev)
-    run = runner.SpecStepRunner(case, fold_layers=args.fold_layers, per_head=args.per_head)
+    run = runner.SpecStepRunner(case, fold_layers=args.fold_layers, per_head=args.per_head,
+                                fused_hist=args.fused_hist)
     counts = run.capture()
     launches_per_step = sum(counts)
 
@@ -434,6 +435,8 @@ def run_gpu(args):
         fold = L if args.fold_layers else 1
         line["roofline"]["traffic"] = t["verify"] * fold
         line["draft_roofline"]["traffic"] = t["draft"] * fold
+    if args.fused_hist:
+        line["config"]["select_first_pass"] = "fused into the verification kernel"
     if args.per_head:
         line["config"]["index_sets"] = "per attention head"
         line["roofline"]["traffic"] = None
@@ -467,6 +470,9 @@ def main():
     ap.add_argument("--per-head", action="store_true",
                     help="one score and one index set per attention head (Eq. 3 / Eq. 5 as printed) instead of "
                          "per KV head: the draft gathers group-size times the rows")
+    ap.add_argument("--fused-hist", action="store_true",
+                    help="the verification kernel counts the selection's first radix pass (top 11 bits of every "
+                         "score) while it writes the statistic; the selection skips that sweep")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()

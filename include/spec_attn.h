@@ -152,6 +152,23 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
                         uint32_t flags, void* cuda_stream);
 
 /*
+ * spec_verify_attn_ex that also hands the selection its first radix pass (Eq. 4 picks the largest
+ * scores; the selection kernel finds the K-th largest by a radix select on the scores' fp32 bit
+ * patterns, whose first pass is a histogram of the top 11 bits).  score_hist: uint32
+ * [n_layers, batch, heads, 2048] (heads = n_kv_heads, or n_q_heads with
+ * SPEC_VERIFY_STATS_PER_QUERY_HEAD), ZERO-FILLED once after allocation; this call ADDS, for every
+ * score stats[.., i] it writes (i < ctx_len[b]), one count to bin (bit pattern >> 21) of the
+ * value written.  spec_select_recall_hist consumes the counts and clears them, so a
+ * verify / select pair leaves the array zero again.  The score-cache kernel counts while it writes
+ * the statistic (one fire-and-forget reduction per key); every other verification path runs a short
+ * sweep over the finished statistic instead.  score_hist == NULL is spec_verify_attn_ex.
+ */
+int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                          int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
+                          float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,
+                          uint32_t flags, uint32_t* score_hist, void* cuda_stream);
+
+/*
  * Recall selection (Eq. 4).  For each problem with T' = sel_len[b]:
  *   T' <= k_total : indices = 0..T'-1, n = T'.
  *   otherwise     : sink [0,k_sink) U the k_mid = k_total-k_sink-k_recent positions of
@@ -171,6 +188,21 @@ int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers
                        int32_t n_kv_heads, const int32_t* sel_len, int32_t k_sink,
                        int32_t k_recent, int32_t k_total, int32_t* indices, int32_t* n_indices,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * spec_select_recall fed with the counts of spec_verify_attn_hist.  score_hist: uint32
+ * [n_layers, batch, n_kv_heads, 2048] as that call left it; hist_len: int32 [batch], the ctx_len of
+ * that call (the counts cover positions [0, hist_len[b]) of stats).  The kernel removes the
+ * positions outside the candidate span from the counts, skips its own first sweep over the
+ * scores, and writes zeros back to score_hist.  The result is the same, bit for bit, as
+ * spec_select_recall on the same stats.  A sequence with sel_len[b] > hist_len[b] falls back to
+ * the full sweep.  score_hist and hist_len are both NULL (= spec_select_recall) or both given.
+ */
+int spec_select_recall_hist(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
+                            int32_t n_kv_heads, const int32_t* sel_len, int32_t k_sink,
+                            int32_t k_recent, int32_t k_total, int32_t* indices, int32_t* n_indices,
+                            uint32_t* score_hist, const int32_t* hist_len, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream);
 
 /*
  * Sparse draft attention (Eq. 5; Sec. 3.1 "Sparse Drafting Stage").  One query per sequence.

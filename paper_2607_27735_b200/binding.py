@@ -34,6 +34,7 @@ EXPORTS = [
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
     "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
     "spec_sparse_draft_attn_ex", "spec_advance_lengths", "spec_set_wait_limit_cycles",
+    "spec_verify_attn_hist", "spec_select_recall_hist",
 ]
 
 
@@ -73,6 +74,10 @@ def load() -> ctypes.CDLL:
                                          i64, vp, ctypes.c_size_t, vp]
         lib.spec_verify_attn_ex.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
                                             i64, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
+        lib.spec_verify_attn_hist.argtypes = [ctypes.POINTER(_KV), vp, i32, vp, i32, i32, vp, vp, vp,
+                                              i64, vp, ctypes.c_size_t, ctypes.c_uint32, vp, vp]
+        lib.spec_select_recall_hist.argtypes = [vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp,
+                                                ctypes.c_size_t, vp]
         lib.spec_sparse_draft_attn_ex.argtypes = [ctypes.POINTER(_KV), vp, vp, vp, i32, vp, vp, i32,
                                                   vp, vp, vp, ctypes.c_size_t, ctypes.c_uint32, vp]
         lib.spec_select_recall.argtypes = [vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp,
@@ -143,8 +148,10 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
                      stat_stride=None, workspace=None, want_lse=True, accumulate=False, per_head=False,
-                     out_bf16=False):
+                     out_bf16=False, score_hist=None):
     """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``.
+    ``score_hist`` (uint32-as-int32 ``[L, B, heads, 2048]``, zero before the first use) receives the
+    selection's first radix pass (spec_verify_attn_hist).
     ``accumulate`` adds this call's statistic to the given ``stats``; ``per_head`` keeps one score per
     attention head (``stats`` is ``[L, B, n_q_heads, stride]``); both go through spec_verify_attn_ex."""
     lib = load()
@@ -171,9 +178,13 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
             _dev(stats, torch.float32, "stats"), stat_stride, workspace.data_ptr(), workspace.numel())
     if stats.shape[2] != (kv.n_q_heads if per_head else kv.n_kv_heads):
         raise ValueError("stats: wrong head count for this mode")
-    if accumulate or per_head or out_bf16:
-        flags = ((VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0) |
-                 (VERIFY_OUT_BF16 if out_bf16 else 0))
+    flags = ((VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0) |
+             (VERIFY_OUT_BF16 if out_bf16 else 0))
+    if score_hist is not None:
+        if score_hist.shape != stats.shape[:3] + (2048,):
+            raise ValueError("score_hist: expected [L, B, heads, 2048]")
+        rc = lib.spec_verify_attn_hist(*args, flags, _dev(score_hist, torch.int32, "score_hist"), _stream())
+    elif flags:
         rc = lib.spec_verify_attn_ex(*args, flags, _stream())
     else:
         rc = lib.spec_verify_attn(*args, _stream())
@@ -217,8 +228,10 @@ def noalloc_read_status() -> int:
     return int(load().spec_noalloc_read_status(_stream()))
 
 
-def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, n_indices=None):
-    """Eq. 4 recall selection; returns ``(indices, n_indices)``."""
+def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, n_indices=None,
+                       score_hist=None, hist_len=None):
+    """Eq. 4 recall selection; returns ``(indices, n_indices)``.  ``score_hist`` / ``hist_len``: the
+    counts a verification call left (spec_select_recall_hist); they are cleared."""
     lib = load()
     L, B, Hkv, stride = stats.shape
     dev = stats.device
@@ -226,11 +239,18 @@ def spec_select_recall(stats, sel_len, k_sink, k_recent, k_total, indices=None, 
         indices = torch.empty(L, B, Hkv, k_total, dtype=torch.int32, device=dev)
     if n_indices is None:
         n_indices = torch.empty(L, B, Hkv, dtype=torch.int32, device=dev)
-    rc = lib.spec_select_recall(
-        _dev(stats, torch.float32, "stats"), stride, L, B, Hkv,
-        _dev(sel_len, torch.int32, "sel_len"), k_sink, k_recent, k_total,
-        _dev(indices, torch.int32, "indices"), _dev(n_indices, torch.int32, "n_indices"), None, 0,
-        _stream())
+    if score_hist is not None:
+        rc = lib.spec_select_recall_hist(
+            _dev(stats, torch.float32, "stats"), stride, L, B, Hkv,
+            _dev(sel_len, torch.int32, "sel_len"), k_sink, k_recent, k_total,
+            _dev(indices, torch.int32, "indices"), _dev(n_indices, torch.int32, "n_indices"),
+            _dev(score_hist, torch.int32, "score_hist"), _dev(hist_len, torch.int32, "hist_len"), None, 0, _stream())
+    else:
+        rc = lib.spec_select_recall(
+            _dev(stats, torch.float32, "stats"), stride, L, B, Hkv,
+            _dev(sel_len, torch.int32, "sel_len"), k_sink, k_recent, k_total,
+            _dev(indices, torch.int32, "indices"), _dev(n_indices, torch.int32, "n_indices"), None, 0,
+            _stream())
     if rc != 0:
         raise SpecError(rc, "spec_select_recall")
     return indices, n_indices

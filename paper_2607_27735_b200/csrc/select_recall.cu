@@ -3,6 +3,9 @@
 // fp32 bit pattern orders like the value and the K_mid-th largest is found by a three-pass
 // radix select (11 + 11 + 10 bits) on the bit patterns; an ordered compaction then emits, in
 // ascending position, everything above the threshold plus the lowest-position ties.
+// The first pass's histogram (top 11 bits) may arrive from the verification kernel, which counts
+// every score it writes: the positions outside the candidate span are taken out again here, the
+// sweep over the scores is skipped, and the counts are cleared for the next round.
 #include "spec_common.cuh"
 
 namespace spec {
@@ -10,7 +13,8 @@ namespace spec {
 namespace {
 
 constexpr int kThreads = 1024;
-constexpr int kBins = 2048;
+constexpr int kBins = kScoreBins;
+static_assert(kBins == 2 * kThreads, "two bins per thread");
 constexpr int kItems = 8;  // consecutive candidates per thread in the compaction sweep
 
 // Exclusive block-wide prefix sum of one int per thread; `total` gets the block sum.
@@ -42,10 +46,11 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& t
     return warp_tmp[warp] + inc - x;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)  // two CTAs per SM: 32 registers per thread
 select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int batch, int n_kv_heads,
                      const int32_t* __restrict__ sel_len, int k_sink, int k_recent, int k_total,
-                     int32_t* __restrict__ indices, int32_t* __restrict__ n_indices)
+                     int32_t* __restrict__ indices, int32_t* __restrict__ n_indices,
+                     uint32_t* __restrict__ hist_g, const int32_t* __restrict__ hist_len)
 {
     __shared__ int hist[kBins];
     __shared__ int warp_tmp[33];
@@ -53,10 +58,33 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
 
     const int64_t prob = blockIdx.x;
     const int b = (int)((prob / n_kv_heads) % batch);
+    const int tid = threadIdx.x;
+    // counts handed over by the verification kernel: requested first (two bins per thread), taken and
+    // cleared whatever happens below
+    uint32_t h0 = 0, h1 = 0;
+    uint32_t* hg = hist_g ? hist_g + prob * kBins : nullptr;
+    if (hg) {
+        h0 = hg[tid];
+        h1 = hg[tid + kThreads];
+    }
     const int T = sel_len[b];
+    const int HL = hg ? hist_len[b] : 0;
     int32_t* out = indices + prob * k_total;
     const uint32_t* st = reinterpret_cast<const uint32_t*>(stats + prob * stat_stride);
-    const int tid = threadIdx.x;
+    // they cover positions [0, hist_len): usable if the candidate span lies inside.  The positions outside
+    // the span that were counted (sink, recent window, rows beyond the committed length: a few dozen)
+    // are fetched now and taken out of the counts below.
+    const bool have_hist = hg && T <= HL && T > k_total;
+    uint32_t excl = 0xffffffffu;
+    if (have_hist && tid < k_sink + (HL - (T - k_recent)))
+        excl = __ldg(st + (tid < k_sink ? tid : T - k_recent + (tid - k_sink))) >> 21;
+    if (hg) {
+        hist[tid] = (int)h0;
+        hist[tid + kThreads] = (int)h1;
+        hg[tid] = 0u;
+        hg[tid + kThreads] = 0u;
+        __syncthreads();
+    }
 
     if (T <= k_total) {  // everything fits: keep every position
         for (int i = tid; i < k_total; i += kThreads) out[i] = i < T ? i : -1;
@@ -76,11 +104,19 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
         const int nb = pass == 2 ? 1024 : 2048;
-        for (int i = tid; i < kBins; i += kThreads) hist[i] = 0;
-        __syncthreads();
-        for (int i = lo + tid; i < hi; i += kThreads) {
-            const uint32_t u = __ldg(st + i);
-            if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+        if (pass == 0 && have_hist) {
+            if (excl != 0xffffffffu) atomicSub(&hist[excl], 1);
+            for (int i = tid + kThreads; i < lo + (HL - hi); i += kThreads) {  // (more than 1024 positions outside)
+                const int pos = i < lo ? i : hi + (i - lo);
+                atomicSub(&hist[__ldg(st + pos) >> 21], 1);
+            }
+        } else {
+            for (int i = tid; i < kBins; i += kThreads) hist[i] = 0;
+            __syncthreads();
+            for (int i = lo + tid; i < hi; i += kThreads) {
+                const uint32_t u = __ldg(st + i);
+                if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+            }
         }
         __syncthreads();
         // walk the buckets from the largest digit down: thread t owns reversed bins 2t, 2t+1
@@ -143,15 +179,40 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     }
 }
 
+// Top-11-bit counts of stats[prob][0 : len[b]) for the verification kernels that do not count while
+// they write the statistic.
+__global__ void __launch_bounds__(256)
+score_hist_kernel(const float* __restrict__ stats, int64_t stat_stride, int batch, int heads,
+                  const int32_t* __restrict__ len, int max_len, uint32_t* __restrict__ hist)
+{
+    const int64_t prob = blockIdx.y;
+    const int b = (int)((prob / heads) % batch);
+    const int T = min(max(len[b], 0), max_len);
+    const uint32_t* st = reinterpret_cast<const uint32_t*>(stats + prob * stat_stride);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < T; i += gridDim.x * blockDim.x)
+        atomicAdd(hist + prob * kBins + (__ldg(st + i) >> 21), 1u);
+}
+
 }  // namespace
 
 int select_launch(const float* stats, int64_t stat_stride, int n_layers, int batch, int n_kv_heads,
                   const int32_t* sel_len, int k_sink, int k_recent, int k_total, int32_t* indices,
-                  int32_t* n_indices, cudaStream_t stream)
+                  int32_t* n_indices, uint32_t* hist, const int32_t* hist_len, cudaStream_t stream)
 {
     const long probs = (long)n_layers * batch * n_kv_heads;
     select_recall_kernel<<<(unsigned)probs, kThreads, 0, stream>>>(
-        stats, stat_stride, batch, n_kv_heads, sel_len, k_sink, k_recent, k_total, indices, n_indices);
+        stats, stat_stride, batch, n_kv_heads, sel_len, k_sink, k_recent, k_total, indices, n_indices, hist, hist_len);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
+}
+
+int score_hist_launch(const float* stats, int64_t stat_stride, long probs, int batch, int heads, const int32_t* len,
+                      int max_len, uint32_t* hist, cudaStream_t stream)
+{
+    if (probs > 65535) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    const int bx = max_len > 256 * 16 ? 16 : (max_len + 255) / 256;
+    score_hist_kernel<<<dim3(bx > 0 ? bx : 1, (unsigned)probs), 256, 0, stream>>>(stats, stat_stride, batch, heads, len,
+                                                                                 max_len, hist);
     count_launch(1);
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;
 }

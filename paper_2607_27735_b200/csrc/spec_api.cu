@@ -115,6 +115,15 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
                         int64_t stat_stride, void* workspace, size_t workspace_bytes, uint32_t flags,
                         void* cuda_stream)
 {
+    return spec_verify_attn_hist(kv, q, n_q, ctx_len, max_ctx_len, stat_window, out, lse, stats, stat_stride, workspace,
+                                 workspace_bytes, flags, nullptr, cuda_stream);
+}
+
+int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
+                          int32_t max_ctx_len, int32_t stat_window, float* out, float* lse, float* stats,
+                          int64_t stat_stride, void* workspace, size_t workspace_bytes, uint32_t flags,
+                          uint32_t* score_hist, void* cuda_stream)
+{
     if (flags & ~(uint32_t)(SPEC_VERIFY_ACCUMULATE_STATS | SPEC_VERIFY_STATS_PER_QUERY_HEAD | SPEC_VERIFY_OUT_BF16))
         return SPEC_ERR_INVALID_ARG;
     VerifyArgs a;
@@ -143,7 +152,10 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
     a.stat_accumulate = (flags & SPEC_VERIFY_ACCUMULATE_STATS) ? 1 : 0;
     a.stat_per_head = (flags & SPEC_VERIFY_STATS_PER_QUERY_HEAD) ? 1 : 0;
     a.out_bf16 = (flags & SPEC_VERIFY_OUT_BF16) ? 1 : 0;
+    a.hist = score_hist;  // the score-cache kernel counts in its statistic pass; the others get a sweep afterwards
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const long hist_probs = (long)kv->n_layers * kv->batch * (a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads);
+    const int hist_heads = a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads;
     const int impl = g_verify_impl.load();
     if (impl != SPEC_VERIFY_GENERIC) {
         int used = 0;
@@ -152,6 +164,9 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
             g_last_verify_impl.store(used == 3   ? SPEC_VERIFY_TCGEN05_CACHED_2PASS
                                      : used == 2 ? SPEC_VERIFY_TCGEN05_CACHED
                                                  : SPEC_VERIFY_TCGEN05_TWOSWEEP);
+            if (score_hist && used != 2)
+                return score_hist_launch(stats, stat_stride, hist_probs, kv->batch, hist_heads, ctx_len, max_ctx_len,
+                                         score_hist, stream);
             return SPEC_OK;
         }
         // an explicit tcgen05 request fails loudly; AUTO falls through to the generic kernels only
@@ -160,7 +175,10 @@ int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const i
     }
     if (workspace_bytes < verify_generic_workspace(a.kv, n_q, max_ctx_len)) return SPEC_ERR_WORKSPACE_TOO_SMALL;
     g_last_verify_impl.store(SPEC_VERIFY_GENERIC);
-    return verify_generic_launch(a, stream);
+    const int rc3 = verify_generic_launch(a, stream);
+    if (rc3 != SPEC_OK || !score_hist) return rc3;
+    return score_hist_launch(stats, stat_stride, hist_probs, kv->batch, hist_heads, ctx_len, max_ctx_len, score_hist,
+                             stream);
 }
 
 int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
@@ -168,14 +186,24 @@ int spec_select_recall(const float* stats, int64_t stat_stride, int32_t n_layers
                        int32_t k_total, int32_t* indices, int32_t* n_indices, void* workspace,
                        size_t workspace_bytes, void* cuda_stream)
 {
+    return spec_select_recall_hist(stats, stat_stride, n_layers, batch, n_kv_heads, sel_len, k_sink, k_recent, k_total,
+                                   indices, n_indices, nullptr, nullptr, workspace, workspace_bytes, cuda_stream);
+}
+
+int spec_select_recall_hist(const float* stats, int64_t stat_stride, int32_t n_layers, int32_t batch,
+                            int32_t n_kv_heads, const int32_t* sel_len, int32_t k_sink, int32_t k_recent,
+                            int32_t k_total, int32_t* indices, int32_t* n_indices, uint32_t* score_hist,
+                            const int32_t* hist_len, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
     (void)workspace;
     (void)workspace_bytes;
+    if ((score_hist != nullptr) != (hist_len != nullptr)) return SPEC_ERR_INVALID_ARG;
     if (!stats || !sel_len || !indices || !n_indices) return SPEC_ERR_INVALID_ARG;
     if (n_layers < 1 || batch < 1 || n_kv_heads < 1 || stat_stride < 1) return SPEC_ERR_INVALID_ARG;
     if (k_sink < 0 || k_recent < 0 || k_total < 1 || k_sink + (int64_t)k_recent > k_total)
         return SPEC_ERR_INVALID_ARG;
     return select_launch(stats, stat_stride, n_layers, batch, n_kv_heads, sel_len, k_sink, k_recent,
-                         k_total, indices, n_indices, static_cast<cudaStream_t>(cuda_stream));
+                         k_total, indices, n_indices, score_hist, hist_len, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int spec_sparse_draft_attn(const spec_kv_t* kv, const void* q, const int32_t* indices,

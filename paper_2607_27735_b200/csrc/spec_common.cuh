@@ -88,6 +88,7 @@ __device__ __forceinline__ float warp_sum(float x)
 __device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 
 constexpr int kStatusBytes = 256;  // head of every workspace: status word + padding
+constexpr int kScoreBins = 2048;   // histogram of the top 11 bits of a score's fp32 pattern (first radix pass of Eq. 4)
 
 // ---- launchers (defined in the kernel files; all enqueue on `stream`, none synchronises) ----
 struct VerifyArgs {
@@ -106,6 +107,7 @@ struct VerifyArgs {
     int stat_accumulate;  // add this call's statistic to what stats[] holds instead of overwriting it
     int stat_per_head;    // stats is [layers, batch, n_q_heads, stride]: one score per attention head
     int out_bf16;         // `out` points to bf16 elements (round to nearest even) instead of fp32
+    uint32_t* hist;       // not null: += counts of the final scores' top 11 bits, [problems][kScoreBins]
 };
 
 // Context length of sequence b as the kernels use it: a value outside [n_q, max_ctx_len] (the range the
@@ -123,7 +125,10 @@ int verify_generic_launch(const VerifyArgs& a, cudaStream_t stream);
 
 int select_launch(const float* stats, int64_t stat_stride, int n_layers, int batch, int n_kv_heads,
                   const int32_t* sel_len, int k_sink, int k_recent, int k_total, int32_t* indices,
-                  int32_t* n_indices, cudaStream_t stream);
+                  int32_t* n_indices, uint32_t* hist, const int32_t* hist_len, cudaStream_t stream);
+// counts the top 11 bits of stats[prob][0 : len[b]) into hist[prob][kScoreBins] (kernels that do not fuse it)
+int score_hist_launch(const float* stats, int64_t stat_stride, long probs, int batch, int heads, const int32_t* len,
+                      int max_len, uint32_t* hist, cudaStream_t stream);
 
 struct DraftArgs {
     KvView kv;

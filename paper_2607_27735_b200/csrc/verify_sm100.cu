@@ -276,6 +276,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
         pa.ctx_len = ctx_a;
         pa.first_stat_row = a.first_stat_row < sp.nA ? a.first_stat_row : sp.nA;
         pa.workspace_bytes = sp.main_bytes;
+        pa.hist = nullptr;  // the histogram is of the summed statistic: counted after the closing add
         int rc = verify_sm100_launch(pa, 2, stream, nullptr);
         if (rc != SPEC_OK) return rc;
         VerifyArgs pb = a;  // rows [nA, n_q) against the whole context; their statistic goes to scratch
@@ -288,6 +289,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
         pb.stats = second;
         pb.stat_stride = sp.stat_stride;
         pb.stat_accumulate = 0;
+        pb.hist = nullptr;
         pb.workspace_bytes = sp.main_bytes;
         rc = verify_sm100_launch(pb, 2, stream, nullptr);
         if (rc != SPEC_OK) return rc;

@@ -147,6 +147,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128] global row LSE (log2 domain)
     float* loc_s = reinterpret_cast<float*>(misc + 1024 + 512);           // [128] CTA-local row LSE
     float* fac_s = reinterpret_cast<float*>(misc + 2048);                 // [128] exp2(local - global)
+    uint32_t* hist_s = reinterpret_cast<uint32_t*>(misc + 2560);          // [1024] packed 16-bit counts of score bins, 4 KB
     float2* red = reinterpret_cast<float2*>(misc + 8192);                 // [kSW warps][NC] (m, l), <= 4 KB
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 12288);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -183,6 +184,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     // zero the Q buffers once: rows R..N-1 are padding the TMA never writes
     for (int i = threadIdx.x; i < q_bytes / 16; i += kBlock)
         *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
+    if (p.a.hist)
+        for (int i = threadIdx.x; i < kScoreBins / 2; i += kBlock) hist_s[i] = 0u;
     for (int r = R + threadIdx.x; r < 128; r += kBlock) {  // padded rows: P = 0
         lse_s[r] = 1.0e30f;
         loc_s[r] = 1.0e30f;
@@ -871,13 +874,38 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             for (int g = 0; g < 8; ++g) {
                                 if (g < G) {
                                     float* dst = p.a.stats + (sg.prob * G + g) * p.a.stat_stride + key;
-                                    *dst = p.a.stat_accumulate ? *dst + sth[g] : sth[g];
+                                    const float val = p.a.stat_accumulate ? *dst + sth[g] : sth[g];
+                                    *dst = val;
+                                    if (p.a.hist) atomicAdd(p.a.hist + (sg.prob * G + g) * kScoreBins + (__float_as_uint(val) >> 21), 1u);
                                 }
                             }
                         }
                     } else if (key < sg.T) {
                         float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
-                        *dst = p.a.stat_accumulate ? *dst + st : st;
+                        const float val = p.a.stat_accumulate ? *dst + st : st;
+                        *dst = val;
+                        // first radix pass of the selection, fused: count the score's top 11 bits in this
+                        // CTA's shared-memory histogram (two 16-bit counters per word: a CTA holds at most
+                        // 4096 keys of a head)
+                        if (p.a.hist) {
+                            const uint32_t bin = __float_as_uint(val) >> 21;
+                            atomicAdd(hist_s + (bin >> 1), 1u << ((bin & 1u) * 16));
+                        }
+                    }
+                }
+                if (!PH && p.a.hist) {
+                    // the CTA's counts of this head join the global ones: one reduction per bin that is not
+                    // empty (a few dozen), and the shared-memory copy is clear again for the next unit
+                    ok = group_sync(B.sm_sync, sync_n, ctl, 28);
+                    if (!ok) break;
+                    uint32_t* hg = p.a.hist + sg.prob * kScoreBins;
+                    for (int w = tid_s; w < kScoreBins / 2; w += 128 * CG) {
+                        const uint32_t v = hist_s[w];
+                        if (v) {
+                            hist_s[w] = 0u;
+                            if (v & 0xffffu) atomicAdd(hg + 2 * w, v & 0xffffu);
+                            if (v >> 16) atomicAdd(hg + 2 * w + 1, v >> 16);
+                        }
                     }
                 }
             }

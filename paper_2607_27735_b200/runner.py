@@ -21,11 +21,13 @@ from . import binding
 
 
 class SpecStepRunner:
-    def __init__(self, case, fold_layers: bool = False, want_lse: bool = False, per_head: bool = False):
+    def __init__(self, case, fold_layers: bool = False, want_lse: bool = False, per_head: bool = False,
+                 fused_hist: bool = False):
         cfg, kv = case.cfg, case.kv
         self.case, self.cfg, self.kv = case, cfg, kv
         self.fold = fold_layers
         self.per_head = per_head  # one score and one index set per attention head (Eq. 3 / Eq. 5 as printed)
+        self.fused_hist = fused_hist  # the verification kernel counts the selection's first radix pass
         n_sets = kv.n_q_heads if per_head else kv.n_kv_heads
         dev = kv.k.device
         L, B = kv.n_layers, kv.batch
@@ -37,6 +39,7 @@ class SpecStepRunner:
         self.stats = torch.zeros(L, B, n_sets, self.stat_stride, device=dev)
         self.indices = torch.empty(L, B, n_sets, cfg.k_total, dtype=torch.int32, device=dev)
         self.n_idx = torch.empty(L, B, n_sets, dtype=torch.int32, device=dev)
+        self.hist = torch.zeros(L, B, n_sets, 2048, dtype=torch.int32, device=dev) if fused_hist else None
         self.out_d = torch.empty(max(cfg.draft_steps, 1), L, B, kv.n_q_heads, kv.head_dim, device=dev)
         self.q_verify = case.q_verify
         self.q_draft = case.q_draft
@@ -57,19 +60,21 @@ class SpecStepRunner:
             binding.spec_verify_attn(self.kv, self.q_verify, self.ctx_len, self.max_ctx,
                                      self.cfg.stat_window, out=self.out_v, lse=self.lse_v,
                                      stats=self.stats, workspace=self.ws_v, want_lse=False,
-                                     per_head=self.per_head)
+                                     per_head=self.per_head, score_hist=self.hist)
             return
         for l in range(self.L):
             binding.spec_verify_attn(
                 self._layers[l], self.q_verify[l:l + 1], self.ctx_len, self.max_ctx,
                 self.cfg.stat_window, out=self.out_v[l:l + 1],
                 lse=None if self.lse_v is None else self.lse_v[l:l + 1],
-                stats=self.stats[l:l + 1], workspace=self.ws_v, want_lse=False, per_head=self.per_head)
+                stats=self.stats[l:l + 1], workspace=self.ws_v, want_lse=False, per_head=self.per_head,
+                score_hist=None if self.hist is None else self.hist[l:l + 1])
 
     def select_phase(self):
         c = self.cfg
         binding.spec_select_recall(self.stats, self.ctx_len, c.k_sink, c.k_recent, c.k_total,
-                                   indices=self.indices, n_indices=self.n_idx)
+                                   indices=self.indices, n_indices=self.n_idx, score_hist=self.hist,
+                                   hist_len=None if self.hist is None else self.ctx_len)
 
     def draft_phase(self):
         c = self.cfg
