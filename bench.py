@@ -27,10 +27,15 @@ METRIC = "us_per_spec_step"
 UNIT = "us"
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/, for the per-layer launches of the headline workload.  A launch
-# that folds L layers moves L times as much (traffic grows in proportion to the keys streamed).
+# summarised under profiles/ (not measured inside this run: ncu cannot run under the timed
+# region), for the per-layer launches of the headline workload, with the file and the source
+# revision each figure was captured at.  A launch that folds L layers moves L times as much
+# (traffic grows in proportion to the keys streamed).
 NCU_TRAFFIC = {
-    "cfg2_8b_32k": {"verify": 134.39e6 + 3.77e6, "draft": 8.51e6},
+    "cfg2_8b_32k": {
+        "verify": (134.38e6 + 3.77e6, "ncu, profiles/verify_cached_cfg2_32k.md"),
+        "draft": (8.51e6, "ncu, profiles/draft_stream_cfg2_budget2048.md"),
+    },
 }
 
 
@@ -127,23 +132,28 @@ def config_json(cfg, n_gpus: int) -> dict:
 # CPU oracle legs
 
 
-def oracle_step_seconds(cfg, sample_layers: int):
-    """Times the oracle on `sample_layers` layers of the workload (host cores)."""
+def oracle_step_seconds(cfg, sample_layers: int, case=None):
+    """Times the oracle on `sample_layers` layers of the workload (host cores).  `case`: a CPU copy of
+    those layers of the workload the GPU arm ran (same bits), else they are drawn here.  Returns the
+    seconds, the threads used and the oracle's results (for the parity figures of the bench line)."""
     import torch
 
     import oracle
     from paper_2607_27735_b200 import inputs
 
-    case = inputs.make_case(cfg, device="cpu", n_layers=sample_layers)
+    if case is None:
+        case = inputs.make_case(cfg, device="cpu", n_layers=sample_layers)
     kv = case.kv
     t0 = time.perf_counter()
     out, lse, stats = oracle.verify_attn(kv, case.q_verify, case.ctx_len, cfg.stat_window)
     idx, n = oracle.select_recall(stats.float(), case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total)
+    drafts = []
     for j in range(cfg.draft_steps):
-        oracle.sparse_draft_attn(kv, case.q_draft[j].contiguous(), idx, n, case.ctx_len,
-                                 (case.ctx_len + j + 1).int())
+        d, _ = oracle.sparse_draft_attn(kv, case.q_draft[j].contiguous(), idx, n, case.ctx_len,
+                                        (case.ctx_len + j + 1).int())
+        drafts.append(d)
     dt = time.perf_counter() - t0
-    return dt, oracle.threads()
+    return dt, oracle.threads(), dict(out=out, stats=stats, idx=idx, n=n, drafts=drafts)
 
 
 def run_reference(args):
@@ -152,11 +162,11 @@ def run_reference(args):
     if rank != 0:
         return
     cfg = pick_config(args.config, args.layers)
-    sample_layers = 1
+    sample_layers = min(2, cfg.n_layers)  # at least as many (layer, sequence, head) problems as host threads
     times = []
     cores = 1
     for i in range(args.warmup + args.steps):
-        dt, cores = oracle_step_seconds(cfg, sample_layers)
+        dt, cores, _ = oracle_step_seconds(cfg, sample_layers)
         if i >= args.warmup:
             times.append(dt)
     scale = cfg.n_layers / sample_layers
@@ -297,6 +307,92 @@ def controller_bench(cfg, dev, peak):
     return out
 
 
+
+def timed_phases(run, steps, warmup=3):
+    """Replays a captured step `steps` times; returns (step_us, [verify_us, select_us, draft_us])."""
+    import torch
+    for _ in range(warmup):
+        run.replay()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    for s_ in range(steps):
+        run.replay(evs[s_])
+    torch.cuda.synchronize()
+    total = evs[0][0].elapsed_time(evs[-1][3]) * 1e3 / steps
+    phases = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) * 1e3 / steps for i in range(3)]
+    return total, phases
+
+
+def other_workloads(peak, dev, layers=4, steps=5):
+    """After the timed region: the other baseline workloads at their full context / batch / page layout,
+    cut to `layers` layers each (layers are independent and identically shaped), one launch per layer."""
+    import dataclasses
+
+    import torch
+
+    from paper_2607_27735_b200 import binding, inputs, runner
+    out = {}
+    jobs = [("cfg3_8b_128k", 1), ("cfg3_8b_128k", 8), ("cfg3_8b_128k", 16), ("cfg4_ragged_paged", None),
+            ("cfg5_32b_64k", None)]
+    impl_names = {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
+                  5: "tcgen05 score-cache, rows in two passes"}
+    for name, k in jobs:
+        full = inputs.baseline_configs(k if k is not None else 8)[name]
+        cfg = dataclasses.replace(full, n_layers=layers)
+        case = inputs.make_case(cfg, device=dev)
+        run = runner.SpecStepRunner(case)
+        counts = run.capture()
+        total, ph = timed_phases(run, steps)
+        vb = run.verify_kv_bytes_per_layer()
+        db = sum(run.draft_kv_bytes_per_layer_step(j) for j in range(cfg.draft_steps)) * layers
+        v_us = ph[0] / layers
+        d_us = ph[2] / max(1, counts[2])
+        key = name + (f"_k{k}" if k is not None else "")
+        out[key] = {
+            "layers": f"{layers} of {full.n_layers} layers",
+            "verify_us_per_layer": v_us, "verify_GBs": vb / v_us / 1e3, "verify_frac": vb / v_us / 1e3 / peak,
+            "select_us": ph[1], "draft_us_per_call": d_us, "draft_GBs": db / ph[2] / 1e3,
+            "draft_frac": db / ph[2] / 1e3 / peak, "verify_impl": impl_names.get(binding.last_verify_impl()),
+            "status": [binding.read_status(run.ws_v), binding.read_status(run.ws_d)],
+        }
+        del run, case
+        torch.cuda.empty_cache()
+    return out
+
+
+def parity_figures(case, run, ref, n_layers):
+    """Max-abs differences between the GPU arm's results for layers [0, n_layers) and the oracle's on the
+    same bits (`ref` comes from the CPU-baseline leg, which runs the oracle on exactly those layers), and
+    the agreement of the index sets."""
+    import torch
+
+    import oracle
+    cfg = case.cfg
+    T = int(case.ctx_len.max())
+    out_err = (run.out_v[:n_layers].cpu().double() - ref["out"]).abs().max().item()
+    st_err = (run.stats[:n_layers, :, :, :T].cpu().double() - ref["stats"][..., :T]).abs().max().item()
+    d_err = max((run.out_d[j, :n_layers].cpu().double() - ref["drafts"][j]).abs().max().item()
+                for j in range(cfg.draft_steps))
+    # recall indices: bit-exact on the GPU's own score array; end to end against the oracle's scores
+    g_stats = run.stats[:n_layers].cpu()
+    o_idx, o_n = oracle.select_recall(g_stats, case.ctx_len.cpu(), cfg.k_sink, cfg.k_recent, cfg.k_total)
+    g_idx = run.indices[:n_layers].cpu()
+    exact = bool(torch.equal(g_idx, o_idx) and torch.equal(run.n_idx[:n_layers].cpu(), o_n))
+    overlaps = []
+    e_idx = ref["idx"]
+    for l in range(n_layers):
+        for b in range(cfg.batch):
+            for h in range(cfg.n_kv_heads):
+                a, c = set(g_idx[l, b, h].tolist()), set(e_idx[l, b, h].tolist())
+                a.discard(-1)
+                c.discard(-1)
+                overlaps.append(len(a & c) / max(1, len(c)))
+    return {"checked": f"layers 0..{n_layers - 1} of the timed workload, every sequence and head, against the fp64 oracle",
+            "tolerance_max_abs": 2e-3, "verify_out_max_abs": out_err, "score_max_abs": st_err,
+            "draft_out_max_abs": d_err, "indices_bit_exact_on_gpu_scores": exact,
+            "end_to_end_index_overlap_min": min(overlaps), "end_to_end_index_overlap_mean": sum(overlaps) / len(overlaps)}
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -384,11 +480,36 @@ def run_gpu(args):
     draft_gbs = draft_bytes / (phase_ms[2] * 1e-3) / 1e9 if phase_ms[2] > 0 else None
 
     cpu_layers = min(2, L)
+    parity = None
     if args.no_cpu_baseline:
         cpu_dt, cores = float("nan"), 0
     else:
-        cpu_dt, cores = oracle_step_seconds(cfg, cpu_layers)
+        import dataclasses
+        run.replay()  # the resident step once more, so that the buffers hold one whole step's results
+        torch.cuda.synchronize()
+        sub = dataclasses.replace(case, kv=case.kv.layer_slice(0, cpu_layers).cpu(),
+                                  q_verify=case.q_verify[:cpu_layers].cpu(),
+                                  q_draft=case.q_draft[:, :cpu_layers].cpu(), ctx_len=case.ctx_len.cpu())
+        oracle_step_seconds(cfg, cpu_layers, sub)  # untimed: pages in the data and starts the threads
+        cpu_dt, cores, ref = oracle_step_seconds(cfg, cpu_layers, sub)
+        if not args.per_head:
+            parity = parity_figures(case, run, ref, cpu_layers)
     cpu_us = cpu_dt * (L / cpu_layers) * 1e6
+
+    folded = None
+    if not args.fold_layers and not args.no_folded and L > 1:
+        # the kernels' own roofline: all layers of a phase in one launch (independent problems)
+        frun = runner.SpecStepRunner(case, fold_layers=True, per_head=args.per_head)
+        fcounts = frun.capture()
+        _, fph = timed_phases(frun, max(3, min(args.steps, 10)))
+        fv = run.verify_kv_bytes_per_layer() * L
+        folded = {"note": "all layers of a phase in one launch: independent problems, not a decoder's dependency chain",
+                  "verify_us_per_layer": fph[0] / L, "verify_GBs": fv / fph[0] / 1e3, "verify_frac": fv / fph[0] / 1e3 / peak,
+                  "draft_us_per_launch": fph[2] / max(1, fcounts[2]), "draft_GBs": draft_bytes / fph[2] / 1e3,
+                  "draft_frac": draft_bytes / fph[2] / 1e3 / peak, "select_us": fph[1], "step_us": sum(fph)}
+        del frun
+        torch.cuda.empty_cache()
+    workloads = None
 
     line = {
         "metric": METRIC, "value": step_ms * 1e3, "unit": UNIT, "n_gpus": world,
@@ -419,13 +540,15 @@ def run_gpu(args):
             "share_of_step_time": phase_ms[2] / step_ms,
         },
         "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{cpu_layers} of {L} layers, time scaled x{L / cpu_layers:g}"},
+                         "sample": f"{cpu_layers} of {L} layers (the bits of the GPU arm's layers 0..{cpu_layers - 1}), "
+                                   f"second of two runs, time scaled x{L / cpu_layers:g}"},
         "e2e": {"value": e2e_ms * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
                 "note": "Q in from pinned host memory, attention outputs back to host every step (the "
                         "drafting Q and the verification outputs travel on a second stream under the "
                         "phases that do not need them); the dense KV cache stays resident by the "
                         "method's definition"},
+        "parity": parity, "folded": folded, "workloads": workloads,
         "gpu_launches": launches_per_step * args.steps,
         "launches_per_step": {"verify": counts[0], "select": counts[1], "draft": counts[2]},
         "clocks": clocks,
@@ -433,8 +556,10 @@ def run_gpu(args):
     t = NCU_TRAFFIC.get(cfg.name)
     if t and cfg.n_layers == pick_config(args.config).n_layers:
         fold = L if args.fold_layers else 1
-        line["roofline"]["traffic"] = t["verify"] * fold
-        line["draft_roofline"]["traffic"] = t["draft"] * fold
+        line["roofline"]["traffic"] = t["verify"][0] * fold
+        line["roofline"]["traffic_source"] = t["verify"][1]
+        line["draft_roofline"]["traffic"] = t["draft"][0] * fold
+        line["draft_roofline"]["traffic_source"] = t["draft"][1]
     if args.fused_hist:
         line["config"]["select_first_pass"] = "fused into the verification kernel"
     if args.per_head:
@@ -445,6 +570,12 @@ def run_gpu(args):
         line["recall"] = drift_recall(case, run, args.recall_steps)
     if not args.no_controller:
         line["controller"] = controller_bench(cfg, dev, peak)
+    if args.workloads and args.layers == 0 and not args.per_head and not args.fold_layers:
+        del run
+        torch.cuda.empty_cache()
+        line["workloads"] = other_workloads(peak, dev)
+    line["roofline"]["us_per_launch_x_sm_mhz"] = (verify_us * clocks["sm_mhz"]
+                                                  if clocks and clocks.get("sm_mhz") else None)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -470,6 +601,9 @@ def main():
     ap.add_argument("--per-head", action="store_true",
                     help="one score and one index set per attention head (Eq. 3 / Eq. 5 as printed) instead of "
                          "per KV head: the draft gathers group-size times the rows")
+    ap.add_argument("--no-folded", action="store_true", help="skip the layer-folded measurement")
+    ap.add_argument("--no-workloads", dest="workloads", action="store_false",
+                    help="skip the other baseline workloads (4 layers each) that the default run reports beside the step")
     ap.add_argument("--fused-hist", action="store_true",
                     help="the verification kernel counts the selection's first radix pass (top 11 bits of every "
                          "score) while it writes the statistic; the selection skips that sweep")
