@@ -84,11 +84,12 @@ def _kv_struct(kv):
     return s, (k, v, pt)
 
 
-def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None, per_head=False):
+def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None, per_head=False, group_max=False):
     """Full-context verification attention and the Eq. 3 statistic.
 
     Returns ``(out fp64 [L,B,n_q,Hq,D], lse fp64 [L,B,n_q,Hq], stats fp64 [L,B,Hkv,stat_stride])``;
-    with ``per_head`` the statistic is kept per attention head: ``[L,B,Hq,stat_stride]``.
+    with ``per_head`` the statistic is kept per attention head: ``[L,B,Hq,stat_stride]``; with
+    ``group_max`` it is the largest per-head score of the group at every key (``[L,B,Hkv,stat_stride]``).
     """
     lib = _load()
     s, keep = _kv_struct(kv)
@@ -105,7 +106,8 @@ def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None, per_head=False
         ctypes.byref(s), ctypes.c_void_p(q.data_ptr()), ctypes.c_int(n_q),
         ctypes.c_void_p(ctx_len.data_ptr()), ctypes.c_int(stat_window),
         ctypes.c_void_p(out.data_ptr()), ctypes.c_void_p(lse.data_ptr()),
-        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stat_stride), ctypes.c_int(1 if per_head else 0),
+        ctypes.c_void_p(stats.data_ptr()), ctypes.c_int64(stat_stride),
+        ctypes.c_int(2 if group_max else (1 if per_head else 0)),
     )
     if rc != 0:
         raise ValueError("oracle_verify_attn: invalid arguments")

@@ -99,7 +99,9 @@ static double logit(const oracle_kv_t *kv, const uint16_t *qrow, int layer, int 
  */
 /* per_head = 0: stats [L, B, Hkv, stat_stride], the score summed over the query heads of a KV head
  * (the reading used by the hot path).  per_head = 1: stats [L, B, Hq, stat_stride], one score per
- * attention head, Eq. 3 as printed ("per-head" indices). */
+ * attention head, Eq. 3 as printed ("per-head" indices).  per_head = 2: stats [L, B, Hkv,
+ * stat_stride], the LARGEST of the group's per-head scores at every key (the other way to fold the
+ * group into one score per KV head; its mass is no longer G * min(W, n_q), see the pins). */
 int oracle_verify_attn_ex(const oracle_kv_t *kv, const uint16_t *q, int n_q, const int32_t *ctx_len,
                           int stat_window, double *out, double *lse, double *stats,
                           int64_t stat_stride, int per_head)
@@ -119,16 +121,19 @@ int oracle_verify_attn_ex(const oracle_kv_t *kv, const uint16_t *q, int n_q, con
             for (int h = 0; h < Hkv; ++h) {
                 const int64_t T = ctx_len[b];
                 double *p = (double *)malloc(sizeof(double) * (size_t)T);
-                for (int g = 0; g < (per_head ? G : 1); ++g) {
-                    double *z = per_head ? stats + (((int64_t)layer * B + b) * Hq + h * G + g) * stat_stride
+                /* max over the group: the per-head scores are kept here and folded at the end */
+                double *zg = per_head == 2 ? (double *)calloc((size_t)G * (size_t)T, sizeof(double)) : NULL;
+                for (int g = 0; g < (per_head == 1 ? G : 1); ++g) {
+                    double *z = per_head == 1 ? stats + (((int64_t)layer * B + b) * Hq + h * G + g) * stat_stride
                                          : stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
                     for (int64_t i = 0; i < T; ++i) z[i] = 0.0;
                 }
                 for (int j = 0; j < n_q; ++j)
                     for (int g = 0; g < G; ++g) {
                         const int qh = h * G + g;
-                        double *st = per_head ? stats + (((int64_t)layer * B + b) * Hq + qh) * stat_stride
-                                              : stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
+                        double *st = per_head == 1 ? stats + (((int64_t)layer * B + b) * Hq + qh) * stat_stride
+                                     : per_head == 2 ? zg + (int64_t)g * T
+                                                     : stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
                         const int64_t pos = T - n_q + j; /* last visible key */
                         const int64_t row = (((int64_t)layer * B + b) * n_q + j) * Hq + qh;
                         const uint16_t *qrow = q + row * D;
@@ -152,6 +157,16 @@ int oracle_verify_attn_ex(const oracle_kv_t *kv, const uint16_t *q, int n_q, con
                         }
                         if (lse) lse[row] = m + log(denom);
                     }
+                if (zg) {
+                    double *z = stats + (((int64_t)layer * B + b) * Hkv + h) * stat_stride;
+                    for (int64_t i = 0; i < T; ++i) {
+                        double best = zg[i];
+                        for (int g = 1; g < G; ++g)
+                            if (zg[(int64_t)g * T + i] > best) best = zg[(int64_t)g * T + i];
+                        z[i] = best;
+                    }
+                    free(zg);
+                }
                 free(p);
             }
     return 0;

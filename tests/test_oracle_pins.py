@@ -495,3 +495,44 @@ def test_per_head_draft_with_shared_sets_is_the_group_draft():
     qv = q.view(1, 1, 1, 8, -1).contiguous()
     ver, _, _ = oracle.verify_attn(kv_plus, qv, case.ctx_len, 16)
     assert (dense - ver[:, :, 0]).abs().max().item() < 1e-12
+
+
+# ---- max instead of sum over the query heads of a group (the other way to fold a GQA group) ----
+
+def test_group_max_statistic_bounds_closed_form_and_mass():
+    """oracle.verify_attn(group_max=True): the largest per-head Eq. 3 score of the group at every key.
+    Pins: it is the elementwise maximum of the (separately pinned) per-head scores; it lies between
+    sum / G and sum; with one head per group it is the summed form bit for bit; on identical keys
+    every head gives the same probabilities 1 / (pos + 1), so the closed form is the per-head one;
+    and its mass over the keys lies in [min(W, n_q), G min(W, n_q)] and is NOT G min(W, n_q) in
+    general, which is why the hot path sums (the sum keeps "every row adds 1 per head")."""
+    from paper_2607_27735_b200 import inputs
+    cfg = inputs.small_config(ctx=(220, 300), batch=2, n_q=5, n_q_heads=8, n_kv_heads=2, planted=3, seed=41)
+    case = inputs.make_case(cfg)
+    G = 4
+    out, lse, st_sum = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16)
+    out_m, lse_m, st_max = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16, group_max=True)
+    _, _, st_h = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16, per_head=True)
+    assert torch.equal(out, out_m) and torch.equal(lse, lse_m)
+    L, B, Hq, S = st_h.shape
+    assert torch.equal(st_h.view(L, B, 2, G, S).max(dim=3).values, st_max)
+    assert (st_max <= st_sum + 1e-15).all() and (st_max >= st_sum / G - 1e-15).all()
+    for b in range(B):
+        T = int(case.ctx_len[b])
+        mass = st_max[:, b, :, :T].sum(-1)
+        assert (mass >= cfg.n_q - 1e-9).all() and (mass <= G * cfg.n_q + 1e-9).all()
+        assert (mass < G * cfg.n_q - 1e-3).all()  # heads disagree on these inputs: strictly below the sum's mass
+    # one head per group: nothing to fold
+    c1 = inputs.make_case(inputs.small_config(ctx=(150, 150), n_q=3, n_q_heads=2, n_kv_heads=2, seed=42))
+    assert torch.equal(oracle.verify_attn(c1.kv, c1.q_verify, c1.ctx_len, 16)[2],
+                       oracle.verify_attn(c1.kv, c1.q_verify, c1.ctx_len, 16, group_max=True)[2])
+    # identical keys: p = 1 / (pos + 1) for every head, so max over heads = one head's score
+    T, n_q, W = 40, 6, 4
+    c2 = inputs.make_case(inputs.small_config(ctx=(T, T), n_q=n_q, n_q_heads=6, n_kv_heads=2, planted=0, seed=43))
+    c2.kv.k[:] = c2.kv.k[:, :, :, :1, :]  # every slot holds the first slot's key
+    _, _, st2 = oracle.verify_attn(c2.kv, c2.q_verify, c2.ctx_len, W, group_max=True)
+    want = torch.zeros(T, dtype=torch.float64)
+    for j in range(n_q - W, n_q):
+        pos = T - n_q + j
+        want[:pos + 1] += 1.0 / (pos + 1)
+    assert (st2[0, 0] - want).abs().max().item() < 1e-12
