@@ -142,10 +142,17 @@ int spec_verify_attn(const spec_kv_t* kv, const void* q, int32_t n_q, const int3
  * kernels.  spec_select_recall then runs with n_kv_heads = n_q_heads, and the draft call takes
  * SPEC_DRAFT_INDICES_PER_QUERY_HEAD.
  *
+ * SPEC_VERIFY_STATS_GROUP_MAX: stats keeps its per-KV-head shape, but a key's score is the LARGEST
+ * of its group's per-head scores (each the Eq. 3 sum over that head's window rows) instead of their
+ * sum: the other way to fold a grouped-query group into one ranking.  Each head's mass is 1 per
+ * window row, so the summed form has mass G per row and this one anything between 1 and G.  Same
+ * kernels and limits as SPEC_VERIFY_STATS_PER_QUERY_HEAD; the two flags exclude each other.
+ *
  * SPEC_VERIFY_OUT_BF16: `out` points to bf16 elements of the same shape (the fp32 result rounded to
  * nearest even: what a bf16 output projection consumes); lse and stats stay fp32.
  */
-enum { SPEC_VERIFY_ACCUMULATE_STATS = 1, SPEC_VERIFY_STATS_PER_QUERY_HEAD = 2, SPEC_VERIFY_OUT_BF16 = 4 };
+enum { SPEC_VERIFY_ACCUMULATE_STATS = 1, SPEC_VERIFY_STATS_PER_QUERY_HEAD = 2, SPEC_VERIFY_OUT_BF16 = 4,
+       SPEC_VERIFY_STATS_GROUP_MAX = 8 };
 int spec_verify_attn_ex(const spec_kv_t* kv, const void* q, int32_t n_q, const int32_t* ctx_len,
                         int32_t max_ctx_len, int32_t stat_window, float* out, float* lse,
                         float* stats, int64_t stat_stride, void* workspace, size_t workspace_bytes,

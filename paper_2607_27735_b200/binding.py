@@ -23,6 +23,7 @@ VERIFY_ACCUMULATE_STATS = 1  # flag of spec_verify_attn_ex: add to the statistic
 VERIFY_STATS_PER_QUERY_HEAD = 2  # flag of spec_verify_attn_ex: one score per attention head
 DRAFT_INDICES_PER_QUERY_HEAD = 1  # flag of spec_sparse_draft_attn_ex: one index set per attention head
 VERIFY_OUT_BF16 = 4  # flag of spec_verify_attn_ex: bf16 attention output
+VERIFY_STATS_GROUP_MAX = 8  # flag of spec_verify_attn_ex: fold the group's per-head scores by max, not sum
 DRAFT_OUT_BF16 = 2  # flag of spec_sparse_draft_attn_ex: bf16 attention output
 DRAFT_EARLY_GATHER = 4  # flag of spec_sparse_draft_attn_ex: index sets, lengths and recalled rows are older than the
 #                         preceding kernel of the stream, so the gather may start before that kernel has finished
@@ -148,7 +149,7 @@ def alloc_workspace(nbytes: int, device) -> torch.Tensor:
 
 def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=None, stats=None,
                      stat_stride=None, workspace=None, want_lse=True, accumulate=False, per_head=False,
-                     out_bf16=False, score_hist=None):
+                     out_bf16=False, score_hist=None, group_max=False):
     """Verification attention + Eq. 3 statistic; returns ``(out, lse, stats, workspace)``.
     ``score_hist`` (uint32-as-int32 ``[L, B, heads, 2048]``, zero before the first use) receives the
     selection's first radix pass (spec_verify_attn_hist).
@@ -179,7 +180,7 @@ def spec_verify_attn(kv, q, ctx_len, max_ctx_len, stat_window=16, out=None, lse=
     if stats.shape[2] != (kv.n_q_heads if per_head else kv.n_kv_heads):
         raise ValueError("stats: wrong head count for this mode")
     flags = ((VERIFY_ACCUMULATE_STATS if accumulate else 0) | (VERIFY_STATS_PER_QUERY_HEAD if per_head else 0) |
-             (VERIFY_OUT_BF16 if out_bf16 else 0))
+             (VERIFY_OUT_BF16 if out_bf16 else 0) | (VERIFY_STATS_GROUP_MAX if group_max else 0))
     if score_hist is not None:
         if score_hist.shape != stats.shape[:3] + (2048,):
             raise ValueError("score_hist: expected [L, B, heads, 2048]")

@@ -124,8 +124,10 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
                           int64_t stat_stride, void* workspace, size_t workspace_bytes, uint32_t flags,
                           uint32_t* score_hist, void* cuda_stream)
 {
-    if (flags & ~(uint32_t)(SPEC_VERIFY_ACCUMULATE_STATS | SPEC_VERIFY_STATS_PER_QUERY_HEAD | SPEC_VERIFY_OUT_BF16))
+    if (flags & ~(uint32_t)(SPEC_VERIFY_ACCUMULATE_STATS | SPEC_VERIFY_STATS_PER_QUERY_HEAD | SPEC_VERIFY_OUT_BF16 |
+                            SPEC_VERIFY_STATS_GROUP_MAX))
         return SPEC_ERR_INVALID_ARG;
+    if ((flags & SPEC_VERIFY_STATS_PER_QUERY_HEAD) && (flags & SPEC_VERIFY_STATS_GROUP_MAX)) return SPEC_ERR_INVALID_ARG;
     VerifyArgs a;
     const int rc = make_view(kv, &a.kv);
     if (rc != SPEC_OK) return rc;
@@ -151,6 +153,7 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
     a.workspace_bytes = workspace_bytes;
     a.stat_accumulate = (flags & SPEC_VERIFY_ACCUMULATE_STATS) ? 1 : 0;
     a.stat_per_head = (flags & SPEC_VERIFY_STATS_PER_QUERY_HEAD) ? 1 : 0;
+    a.stat_group_max = (flags & SPEC_VERIFY_STATS_GROUP_MAX) ? 1 : 0;
     a.out_bf16 = (flags & SPEC_VERIFY_OUT_BF16) ? 1 : 0;
     a.hist = score_hist;  // the score-cache kernel counts in its statistic pass; the others get a sweep afterwards
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -106,6 +106,7 @@ struct VerifyArgs {
     size_t workspace_bytes;
     int stat_accumulate;  // add this call's statistic to what stats[] holds instead of overwriting it
     int stat_per_head;    // stats is [layers, batch, n_q_heads, stride]: one score per attention head
+    int stat_group_max;   // stats is per KV head, but the group's per-head scores are folded by max instead of sum
     int out_bf16;         // `out` points to bf16 elements (round to nearest even) instead of fp32
     uint32_t* hist;       // not null: += counts of the final scores' top 11 bits, [problems][kScoreBins]
 };

@@ -228,7 +228,16 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
         }
         __syncthreads();
         if (threadIdx.x < kTK && key0 + threadIdx.x < T) {
-            if (a.stat_per_head) {  // one score per attention head: rows j * G + g with the same g
+            if (a.stat_group_max) {  // per KV head, the largest of the group's per-head scores
+                float best = 0.f;
+                for (int g = 0; g < G; ++g) {
+                    float cs = 0.f;
+                    for (int r = stat_r0 + g; r < R; r += G) cs += S[r * kSP + threadIdx.x];
+                    best = g == 0 ? cs : fmaxf(best, cs);
+                }
+                float* dst = a.stats + prob * a.stat_stride + key0 + threadIdx.x;
+                *dst = a.stat_accumulate ? *dst + best : best;
+            } else if (a.stat_per_head) {  // one score per attention head: rows j * G + g with the same g
                 for (int g = 0; g < G; ++g) {
                     float cs = 0.f;
                     for (int r = stat_r0 + g; r < R; r += G) cs += S[r * kSP + threadIdx.x];

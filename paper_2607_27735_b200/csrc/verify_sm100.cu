@@ -253,7 +253,7 @@ size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
 
 int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant)
 {
-    if (a.stat_per_head) {
+    if (a.stat_per_head || a.stat_group_max) {
         // only the score-cache kernel keeps one score per attention head, for groups of up to 8;
         // everything else goes to the generic kernels
         const int G = a.kv.n_q_heads / a.kv.n_kv_heads;

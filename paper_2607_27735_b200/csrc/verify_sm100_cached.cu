@@ -869,7 +869,17 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             sth[1] += sth[3];
                         }
                         if (ph_fast && G == 1) sth[0] += sth[1];
-                        if (key < sg.T) {
+                        if (key < sg.T && p.a.stat_group_max) {
+                            // one score per KV head: the largest of the group's per-head scores
+                            float best = sth[0];
+#pragma unroll
+                            for (int g = 1; g < 8; ++g)
+                                if (g < G) best = fmaxf(best, sth[g]);
+                            float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
+                            const float val = p.a.stat_accumulate ? *dst + best : best;
+                            *dst = val;
+                            if (p.a.hist) atomicAdd(p.a.hist + sg.prob * kScoreBins + (__float_as_uint(val) >> 21), 1u);
+                        } else if (key < sg.T) {
 #pragma unroll
                             for (int g = 0; g < 8; ++g) {
                                 if (g < G) {
@@ -978,7 +988,7 @@ int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& 
 int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                   int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    const bool lp = fp.cph <= kLsePubMax, ph = fp.a.stat_per_head != 0;
+    const bool lp = fp.cph <= kLsePubMax, ph = fp.a.stat_per_head != 0 || fp.a.stat_group_max != 0;
 #define SPEC_CASE(n, nc, cg)                                                                              \
     case n:                                                                                               \
         if (ph) return lp ? launch_cfg<nc, cg, true, true>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
