@@ -265,10 +265,10 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     // ---- the warps of the CTA: (max, sum, O) through shared memory (each warp's own first stage) ----
     __syncwarp();
     {
-        float* ow = reinterpret_cast<float*>(wst);  // [8 heads][D]
+        float* ow = reinterpret_cast<float*>(wst);  // [8 heads][D + 8]: the padding keeps the heads on different banks
 #pragma unroll
         for (int i = 0; i < D / 8; ++i)
-            *reinterpret_cast<float2*>(ow + grp * D + i * 8 + 2 * quad) = make_float2(o[i][0] + o[i][2], o[i][1] + o[i][3]);
+            *reinterpret_cast<float2*>(ow + grp * (D + 8) + i * 8 + 2 * quad) = make_float2(o[i][0] + o[i][2], o[i][1] + o[i][3]);
         if (quad == 0) wml[warp * 8 + grp] = make_float2(M, L);
     }
     __syncthreads();
@@ -293,7 +293,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
             const float2 ml = wml[w * 8 + r];
             const float wgt = ex2f(ml.x - Mc);
             Lc += ml.y * wgt;
-            oc += reinterpret_cast<const float*>(stages + (size_t)w * ST * STAGE)[r * D + d] * wgt;
+            oc += reinterpret_cast<const float*>(stages + (size_t)w * ST * STAGE)[r * (D + 8) + d] * wgt;
         }
         put(e, oc);
         if (d == 0) {
