@@ -349,6 +349,7 @@ int launch_shape(const DraftArgs& a, const StreamShape& shp, cudaStream_t stream
     SPEC_INST(8, 1)
     SPEC_INST(8, 2)
     SPEC_INST(8, 3)
+    SPEC_INST(12, 2)
 #undef SPEC_INST
     return SPEC_ERR_UNSUPPORTED_SHAPE;
 }
@@ -385,6 +386,8 @@ bool stream_plan(const KvView& kv, int head_dim, int n_keys_max, StreamShape* ou
         while (st > 1 && smem_of(cs, 8, st, per) > draft::kSmemLimit) --st;
         if (smem_of(cs, 8, st, per) > draft::kSmemLimit) return false;
         *out = StreamShape{cs, per, 8, st};
+        // more chunks than 8 warps x 3 stages hold at once: 12 warps x 2 stages finish the share in fewer trips
+        if (per / kChunk > 24 && smem_of(cs, 12, 2, per) <= draft::kSmemLimit) *out = StreamShape{cs, per, 12, 2};
         return true;
     }
     static const int kCombos[4][2] = {{4, 2}, {4, 3}, {8, 2}, {8, 3}};
