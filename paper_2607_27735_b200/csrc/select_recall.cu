@@ -16,6 +16,7 @@ constexpr int kThreads = 1024;
 constexpr int kBins = kScoreBins;
 static_assert(kBins == 2 * kThreads, "two bins per thread");
 constexpr int kItems = 8;  // consecutive candidates per thread in the compaction sweep
+constexpr int kCap = 4096; // candidates of the first pass's threshold bin kept in shared memory
 
 // Exclusive block-wide prefix sum of one int per thread; `total` gets the block sum.
 __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& total)
@@ -46,6 +47,21 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& t
     return warp_tmp[warp] + inc - x;
 }
 
+// Calls f(bits) for every candidate of [lo, hi): eight loads per thread are in flight before the first
+// is used (a loop of one load and one atomic per trip would pay the memory latency on every trip).
+template <typename F>
+__device__ __forceinline__ void sweep(const uint32_t* __restrict__ st, int lo, int hi, F f)
+{
+    for (int base = lo + threadIdx.x; base < hi; base += 8 * kThreads) {
+        uint32_t u[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) u[k] = base + k * kThreads < hi ? __ldg(st + base + k * kThreads) : 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (base + k * kThreads < hi) f(u[k]);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 2)  // two CTAs per SM: 32 registers per thread
 select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int batch, int n_kv_heads,
                      const int32_t* __restrict__ sel_len, int k_sink, int k_recent, int k_total,
@@ -54,7 +70,8 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
 {
     __shared__ int hist[kBins];
     __shared__ int warp_tmp[33];
-    __shared__ int sh_bucket, sh_above;
+    __shared__ int sh_bucket, sh_above, sh_count, list_n;
+    __shared__ uint32_t list[kCap];
 
     const int64_t prob = blockIdx.x;
     const int b = (int)((prob / n_kv_heads) % batch);
@@ -101,6 +118,8 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     // ---- radix select: bit pattern `thr` of the k_mid-th largest candidate ----
     uint32_t prefix = 0, mask = 0;
     int need = k_mid;  // how many to take among candidates matching the decided prefix
+    int n_list = 0;
+    bool use_list = false;
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
         const int nb = pass == 2 ? 1024 : 2048;
@@ -113,9 +132,15 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
         } else {
             for (int i = tid; i < kBins; i += kThreads) hist[i] = 0;
             __syncthreads();
-            for (int i = lo + tid; i < hi; i += kThreads) {
-                const uint32_t u = __ldg(st + i);
-                if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+            if (pass > 0 && use_list) {  // the candidates that share the first digit sit in shared memory
+                for (int i = tid; i < n_list; i += kThreads) {
+                    const uint32_t u = list[i];
+                    if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+                }
+            } else {
+                sweep(st, lo, hi, [&](uint32_t u) {
+                    if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
+                });
             }
         }
         __syncthreads();
@@ -128,54 +153,67 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
         if (ex < need && need <= ex + c0) {
             sh_bucket = nb - 1 - j0;
             sh_above = ex;
+            sh_count = c0;
         } else if (ex + c0 < need && need <= ex + c0 + c1) {
             sh_bucket = nb - 1 - j1;
             sh_above = ex + c0;
+            sh_count = c1;
         }
         __syncthreads();
         prefix |= (uint32_t)sh_bucket << shift;
         mask |= (uint32_t)(nb - 1) << shift;
         need -= sh_above;
         __syncthreads();
+        if (pass == 0 && sh_count <= kCap) {
+            // One sweep collects the candidates of the threshold's bin (usually a few hundred of the tens
+            // of thousands); the two remaining digits are then decided on that list instead of by two
+            // more sweeps over all scores.  A bin too full for the list (flat scores) keeps the sweeps.
+            if (tid == 0) list_n = 0;
+            __syncthreads();
+            sweep(st, lo, hi, [&](uint32_t u) {
+                if ((u & mask) == prefix) {
+                    const int at = atomicAdd(&list_n, 1);
+                    if (at < kCap) list[at] = u;
+                }
+            });
+            __syncthreads();
+            n_list = list_n;
+            use_list = n_list <= kCap;
+        }
     }
     const uint32_t thr = prefix;  // take every candidate > thr and the first `need` equal to it
 
     // ---- ordered compaction over the candidate span ----
-    int written = 0, eq_seen = 0;
+    // One block scan per trip: the counts of "above the threshold" (high half) and "equal to it" (low
+    // half) travel in one word; a candidate's slot is (candidates above it so far) + (equal ones so far,
+    // capped at the number still needed).
+    int gt_seen = 0, eq_seen = 0;
     for (int base = lo; base < hi; base += kThreads * kItems) {
         const int i0 = base + tid * kItems;
         uint32_t u[kItems];
-        int n_eq = 0;
+        int packed = 0;
 #pragma unroll
         for (int k = 0; k < kItems; ++k) {
             u[k] = (i0 + k < hi) ? __ldg(st + i0 + k) : 0u;
-            n_eq += (i0 + k < hi && u[k] == thr) ? 1 : 0;
+            if (i0 + k < hi) packed += u[k] > thr ? (1 << 16) : (u[k] == thr ? 1 : 0);
         }
-        int eq_total;
-        int eq_rank = eq_seen + block_exclusive_scan(n_eq, warp_tmp, eq_total);
-        int n_take = 0;
-        unsigned take_mask = 0;
+        int total;
+        const int ex = block_exclusive_scan(packed, warp_tmp, total);
+        int gt = gt_seen + (ex >> 16), eq = eq_seen + (ex & 0xffff);
 #pragma unroll
         for (int k = 0; k < kItems; ++k) {
             if (i0 + k < hi) {
-                bool take = u[k] > thr;
-                if (u[k] == thr) {
-                    take = eq_rank < need;
-                    ++eq_rank;
-                }
-                if (take) {
-                    take_mask |= 1u << k;
-                    ++n_take;
+                if (u[k] > thr) {
+                    out[k_sink + gt + min(eq, need)] = i0 + k;
+                    ++gt;
+                } else if (u[k] == thr) {
+                    if (eq < need) out[k_sink + gt + eq] = i0 + k;
+                    ++eq;
                 }
             }
         }
-        int take_total;
-        int dst = written + block_exclusive_scan(n_take, warp_tmp, take_total);
-#pragma unroll
-        for (int k = 0; k < kItems; ++k)
-            if (take_mask & (1u << k)) out[k_sink + dst++] = i0 + k;
-        written += take_total;
-        eq_seen += eq_total;
+        gt_seen += total >> 16;
+        eq_seen += total & 0xffff;
     }
 }
 

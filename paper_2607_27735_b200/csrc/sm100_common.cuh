@@ -258,15 +258,18 @@ __device__ __forceinline__ Seg get_seg(const FastParams& p, int unit, int head_l
     s.b = fast_div(p, 1, rem);
     s.h = (rem - s.b * p.NHG) * p.HG + head_local;
     // a length outside [n_q, max_ctx_len] is clamped (the launch, the score cache and the output rows
-    // were sized for that range) and reported
-    const int t_in = p.a.ctx_len[s.b];
-    s.T = min(max(t_in, p.a.n_q), p.a.max_ctx_len);
-    if (t_in != s.T) set_status(p.status, SPEC_ERR_BAD_INDEX);
+    // were sized for that range); the TMA producer warp reports it (check_len)
+    s.T = min(max(p.a.ctx_len[s.b], p.a.n_q), p.a.max_ctx_len);
     const int nb = (s.T + kTile - 1) / kTile;
     s.t0 = fast_div(p, 2, rank * nb);        // rank < SMs, nb < 2^20: the products stay far below 2^31
     s.t1 = fast_div(p, 2, (rank + 1) * nb);
     s.prob = ((int64_t)s.layer * p.a.kv.batch + s.b) * p.a.kv.n_kv_heads + s.h;
     return s;
+}
+
+__device__ __forceinline__ void check_len(const FastParams& p, const Seg& s)
+{
+    if (p.a.ctx_len[s.b] != s.T) set_status(p.status, SPEC_ERR_BAD_INDEX);
 }
 
 // launchers of the two kernel variants (host)

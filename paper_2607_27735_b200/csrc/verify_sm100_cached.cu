@@ -243,6 +243,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         };
         for (int u = 0; u < U && ok; ++u) {
             const Seg sg = get_seg(p, u, head_local, rank);
+            if (lane == 0) check_len(p, sg);
             if (sg.t1 <= sg.t0) continue;
             const uint32_t qb = 0, qph = qn & 1;
             ++qn;

@@ -232,6 +232,7 @@ verify_twosweep_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
         for (int round = 0; round <= U && ok; ++round) {
             if (round < U) {
                 const Seg sg = get_seg(p, round, head_local, rank);
+                if (lane == 0) check_len(p, sg);
                 if (sg.t1 > sg.t0) {
                     const uint32_t qb = qn & 1, qph = (qn >> 1) & 1;
                     ++qn;
