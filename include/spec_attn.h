@@ -401,6 +401,17 @@ int64_t spec_set_wait_limit_cycles(int64_t cycles);
  * first call). */
 int spec_last_verify_impl(void);
 
+/*
+ * How a call of this shape would be split (host-side planning only: nothing is launched, no GPU is
+ * needed; without a current device the plan assumes 148 SMs).  which = SPEC_WS_VERIFY: out =
+ * {kernel (0 = generic kernels, 1 = tcgen05 two-sweep, 2 = tcgen05 score-cache, 3 = score-cache on two
+ * halves of the rows), KV heads per unit, CTAs per head, units, score columns N, score tiles the
+ * tensor-memory cache holds, K/V tile slots, P buffers}.  which = SPEC_WS_DRAFT (k_total = budget
+ * + longest tail): out = {CTAs per cluster, keys per CTA, warps per CTA, stages per warp, 0...}.
+ */
+int spec_describe_plan(int which, const spec_kv_t* kv, int32_t n_q, int32_t max_ctx_len,
+                       int32_t k_total, int32_t out[8]);
+
 /* Number of kernels this library has launched since load (host-side counter). */
 int64_t spec_launch_count(void);
 

@@ -35,7 +35,7 @@ EXPORTS = [
     "spec_noalloc_read_status", "spec_token_entropy", "spec_controller_update", "spec_controller_select",
     "spec_token_argmax", "spec_accept_greedy", "spec_verify_attn_ex",
     "spec_sparse_draft_attn_ex", "spec_advance_lengths", "spec_set_wait_limit_cycles",
-    "spec_verify_attn_hist", "spec_select_recall_hist",
+    "spec_verify_attn_hist", "spec_select_recall_hist", "spec_describe_plan",
 ]
 
 
@@ -99,6 +99,7 @@ def load() -> ctypes.CDLL:
         lib.spec_workspace_bytes.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32]
         lib.spec_workspace_bytes.restype = ctypes.c_size_t
         lib.spec_read_status.argtypes = [vp, vp]
+        lib.spec_describe_plan.argtypes = [ctypes.c_int, ctypes.POINTER(_KV), i32, i32, i32, ctypes.POINTER(i32 * 8)]
         lib.spec_set_verify_impl.argtypes = [ctypes.c_int]
         lib.spec_set_wait_limit_cycles.argtypes = [ctypes.c_int64]
         lib.spec_set_wait_limit_cycles.restype = ctypes.c_int64
@@ -407,6 +408,16 @@ def spec_controller_select(state, entropy, cand, c_d, c_v, k_star=None, p=None, 
 
 def read_status(workspace) -> int:
     return int(load().spec_read_status(workspace.data_ptr(), _stream()))
+
+
+def describe_plan(which: int, kv_struct, n_q: int = 1, max_ctx_len: int = 1, k_total: int = 1):
+    """Host-side split of a call (spec_describe_plan); ``kv_struct`` is a ``binding._KV`` (no tensors needed,
+    so this works without a GPU).  Returns the eight integers as a list."""
+    out = (ctypes.c_int32 * 8)()
+    rc = load().spec_describe_plan(which, ctypes.byref(kv_struct), n_q, max_ctx_len, k_total, ctypes.byref(out))
+    if rc != 0:
+        raise SpecError(rc, "spec_describe_plan")
+    return list(out)
 
 
 def set_wait_limit_cycles(cycles: int) -> int:

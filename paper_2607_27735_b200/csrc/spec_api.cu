@@ -366,6 +366,32 @@ int spec_set_verify_impl(int impl)
 
 int spec_last_verify_impl(void) { return g_last_verify_impl.load(); }
 
+int spec_describe_plan(int which, const spec_kv_t* kv, int32_t n_q, int32_t max_ctx_len, int32_t k_total,
+                       int32_t out[8])
+{
+    if (!out) return SPEC_ERR_INVALID_ARG;
+    for (int i = 0; i < 8; ++i) out[i] = 0;
+    KvView v;
+    const int rc = make_view(kv, &v);
+    if (rc != SPEC_OK) return rc;
+    if (which == SPEC_WS_VERIFY) {
+        if (n_q < 1 || n_q > 32 || max_ctx_len < n_q) return SPEC_ERR_INVALID_ARG;
+        verify_sm100_describe(v, n_q, max_ctx_len, out);
+        return SPEC_OK;
+    }
+    if (which == SPEC_WS_DRAFT) {
+        if (k_total < 1) return SPEC_ERR_INVALID_ARG;
+        StreamShape s;
+        if (!stream_plan(v, v.head_dim, k_total, &s)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+        out[0] = s.cs;
+        out[1] = s.per;
+        out[2] = s.nw;
+        out[3] = s.st;
+        return SPEC_OK;
+    }
+    return SPEC_ERR_INVALID_ARG;
+}
+
 int64_t spec_set_wait_limit_cycles(int64_t cycles)
 {
     if (cycles < 1) return SPEC_ERR_INVALID_ARG;

@@ -238,6 +238,19 @@ bool verify_sm100_supported(const KvView& kv, int n_q, int variant)
     return kv.slot_stride >= kD;
 }
 
+void verify_sm100_describe(const KvView& kv, int n_q, int max_ctx_len, int32_t out[8])
+{
+    for (int i = 0; i < 8; ++i) out[i] = 0;
+    Plan pl;
+    SplitPlan sp;
+    int kind = 0;
+    if (make_split_plan(kv, n_q, max_ctx_len, &sp) && make_plan(kv, sp.nA, max_ctx_len, 2, &pl)) kind = 3;
+    else if (make_plan(kv, n_q, max_ctx_len, 0, &pl)) kind = pl.cached ? 2 : 1;
+    if (!kind || kv.slot_stride < kD) return;
+    const int v[8] = {kind, pl.HG, pl.cph, pl.n_units, pl.N, pl.n_cache, pl.n_slots, pl.p_bufs};
+    for (int i = 0; i < 8; ++i) out[i] = v[i];
+}
+
 size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
 {
     // the same bytes serve either variant: take the larger of the two plans
