@@ -11,7 +11,7 @@ namespace spec {
 namespace sm100 {
 
 constexpr int kTile = 128;            // keys per tile = UMMA M
-constexpr int kD = 128;               // head_dim of the fast path
+constexpr int kD = 128;               // head_dim the tiles are laid out for (head_dim 64 uses the lower half)
 constexpr int kSlotBytes = 32768;     // one K or V tile: 2 halves x 128 rows x 128 B (SW128)
 constexpr int kThreads = 384;
 constexpr int kRing = 4;              // partial buffers are recycled every kRing units
@@ -24,12 +24,13 @@ struct FastParams {
     VerifyArgs a;
     int HG, NHG, cph, n_units, N, R, G;
     int n_slots, p_bufs;
+    int D;                            // head_dim: 128, or 64 (score-cache kernel only)
     int box_rows, boxes;              // TMA boxes per 64-wide half of a tile
     float scale_log2;
     int* counters;                    // [2][n_units * HG]: P1 partials done, O partials done; then one
                                       // "CTAs finished" word.  All zero between calls.
     float2* ml_part;                  // [kRing][HG][cph][R]
-    float* o_part;                    // [kRing][HG][cph][R][kD]
+    float* o_part;                    // [kRing][HG][cph][R][kD] (columns >= head_dim unused)
     int* status;
     int n_pages;
     int n_cache;                      // S tiles the TMEM cache holds (cached variant)

@@ -47,7 +47,8 @@ int box_rows_for(int page_size)
 bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl)
 {
     const int G = kv.n_q_heads / kv.n_kv_heads, R = n_q * G;
-    if (kv.head_dim != kD || R > 128 || G > 256 || n_q > 256) return false;
+    // head_dim 64 runs on the score-cache kernel only (one 64-wide half per tile, V padded with zero rows)
+    if (!(kv.head_dim == kD || (kv.head_dim == 64 && variant != 1)) || R > 128 || G > 256 || n_q > 256) return false;
     const int box_rows = box_rows_for(kv.page_size);
     if (box_rows == 0) return false;
     const int nsm = sm_count();
@@ -76,7 +77,7 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         cached = best_hg != 0;
     }
     if (!cached) {
-        if (variant == 2) return false;
+        if (variant == 2 || kv.head_dim != kD) return false;
         double best = -1.0;
         for (int hg = 1; hg <= kv.n_kv_heads; ++hg) {
             if (kv.n_kv_heads % hg) continue;
@@ -155,7 +156,7 @@ bool encode_kv_map(CUtensorMap* map, const void* base, const KvView& kv, int n_p
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)kv.page_size, (cuuint64_t)kv.n_kv_heads,
+    const cuuint64_t dims[5] = {(cuuint64_t)kv.head_dim, (cuuint64_t)kv.page_size, (cuuint64_t)kv.n_kv_heads,
                                 (cuuint64_t)n_pages, (cuuint64_t)kv.n_layers};
     const cuuint64_t strides[4] = {(cuuint64_t)kv.slot_stride * 2, (cuuint64_t)kv.head_stride * 2,
                                    (cuuint64_t)kv.page_stride * 2, (cuuint64_t)kv.layer_stride * 2};
@@ -173,9 +174,9 @@ bool encode_q_map(CUtensorMap* map, const void* q, const KvView& kv, int n_q, in
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)kv.n_q_heads,
+    const cuuint64_t dims[3] = {(cuuint64_t)kv.head_dim, (cuuint64_t)kv.n_q_heads,
                                 (cuuint64_t)kv.n_layers * kv.batch * n_q};
-    const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)kv.n_q_heads * kD * 2};
+    const cuuint64_t strides[2] = {(cuuint64_t)kv.head_dim * 2, (cuuint64_t)kv.n_q_heads * kv.head_dim * 2};
     const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)n_q};
     const cuuint32_t estr[3] = {1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, estr,
@@ -235,7 +236,7 @@ bool verify_sm100_supported(const KvView& kv, int n_q, int variant)
 {
     Plan pl;
     if (!make_plan(kv, n_q, kTile, variant == 2 ? 0 : variant, &pl)) return false;
-    return kv.slot_stride >= kD;
+    return kv.slot_stride >= kv.head_dim;
 }
 
 void verify_sm100_describe(const KvView& kv, int n_q, int max_ctx_len, int32_t out[8])
@@ -246,7 +247,7 @@ void verify_sm100_describe(const KvView& kv, int n_q, int max_ctx_len, int32_t o
     int kind = 0;
     if (make_split_plan(kv, n_q, max_ctx_len, &sp) && make_plan(kv, sp.nA, max_ctx_len, 2, &pl)) kind = 3;
     else if (make_plan(kv, n_q, max_ctx_len, 0, &pl)) kind = pl.cached ? 2 : 1;
-    if (!kind || kv.slot_stride < kD) return;
+    if (!kind || kv.slot_stride < kv.head_dim) return;
     const int v[8] = {kind, pl.HG, pl.cph, pl.n_units, pl.N, pl.n_cache, pl.n_slots, pl.p_bufs};
     for (int i = 0; i < 8; ++i) out[i] = v[i];
 }
@@ -336,6 +337,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.N = pl.N;
     fp.R = a.n_q * G;
     fp.G = G;
+    fp.D = a.kv.head_dim;
     fp.n_slots = pl.n_slots;
     fp.p_bufs = pl.p_bufs;
     fp.box_rows = pl.box_rows;

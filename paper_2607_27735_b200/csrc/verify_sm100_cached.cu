@@ -186,6 +186,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         *reinterpret_cast<uint4*>(sgen + (s_q - sbase) + 16 * i) = make_uint4(0, 0, 0, 0);
     if (p.a.hist)
         for (int i = threadIdx.x; i < kScoreBins / 2; i += kBlock) hist_s[i] = 0u;
+    if (p.D == 64) {  // the upper 64-wide half of every tile slot is never loaded: zero rows of V^T (and of K)
+        for (int i = threadIdx.x; i < p.n_slots * 1024; i += kBlock)
+            *reinterpret_cast<uint4*>(sgen + (s_slots - sbase) + (i >> 10) * kSlotBytes + 16384 + 16 * (i & 1023)) =
+                make_uint4(0, 0, 0, 0);
+    }
     for (int r = R + threadIdx.x; r < 128; r += kBlock) {  // padded rows: P = 0
         lse_s[r] = 1.0e30f;
         loc_s[r] = 1.0e30f;
@@ -213,6 +218,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         uint32_t slot_idx = 0, qn = 0;
         const int boxes = p.boxes, box_rows = p.box_rows;
         const uint32_t box_bytes = box_rows * 128;
+        const int halves = p.D / 64;  // 64-wide halves of the head dimension
         bool ok = true;
         auto load_tile = [&](const CUtensorMap* map, const Seg& sg, int tile) -> bool {
             const uint32_t s = slot_idx % p.n_slots, ph = (slot_idx / p.n_slots) & 1;
@@ -223,9 +229,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             // boxes of this tile that hold at least one key < T (pages past the context may not exist)
             const int key0 = tile * kTile;
             const int n_box = min(boxes, (sg.T - key0 + box_rows - 1) / box_rows);
-            if (lane == 0) mbar_expect_tx(B.slot_full + 8 * s, 2u * n_box * box_bytes);
+            if (lane == 0) mbar_expect_tx(B.slot_full + 8 * s, (uint32_t)halves * n_box * box_bytes);
             __syncwarp();
-            for (int i = lane; i < 2 * n_box; i += 32) {
+            for (int i = lane; i < halves * n_box; i += 32) {
                 const int half = i >= n_box ? 1 : 0, bx = i - half * n_box;  // i < 2 * n_box
                 const int pos = key0 + bx * box_rows;
                 const int page = page_of(p.a.kv, pos), slot_in_page = pos - page * p.a.kv.page_size;
@@ -250,10 +256,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             ok = mbar_wait(B.q_empty + 8 * qb, qph ^ 1, ctl, 2);
             if (!ok) break;
             if (lane == 0) {
-                mbar_expect_tx(B.q_full + 8 * qb, 2u * R * 128);
+                mbar_expect_tx(B.q_full + 8 * qb, (uint32_t)halves * R * 128);
                 const int row0 = (sg.layer * p.a.kv.batch + sg.b) * p.a.n_q;
                 tma_load_3d(s_q + qb * q_bytes, &tm_q, B.q_full + 8 * qb, 0, sg.h * G, row0);
-                tma_load_3d(s_q + qb * q_bytes + N * 128, &tm_q, B.q_full + 8 * qb, 64, sg.h * G, row0);
+                if (halves == 2) tma_load_3d(s_q + qb * q_bytes + N * 128, &tm_q, B.q_full + 8 * qb, 64, sg.h * G, row0);
             }
             __syncwarp();
             for (int t = sg.t0; t < sg.t1 && ok; ++t) ok = load_tile(&tm_k, sg, t);
@@ -324,9 +330,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const uint32_t d_s = tmem_base + col_s + c * N;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t a = desc_kmajor(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
-                    const uint64_t b = desc_kmajor(q_addr + (ks >> 2) * (N * 128) + (ks & 3) * 32);
-                    tc_mma(d_s, a, b, idesc_qk, ks ? 1u : 0u);
+                    if (ks * 16 < p.D) {  // head_dim 64: the first four 16-wide steps
+                        const uint64_t a = desc_kmajor(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
+                        const uint64_t b = desc_kmajor(q_addr + (ks >> 2) * (N * 128) + (ks & 3) * 32);
+                        tc_mma(d_s, a, b, idesc_qk, ks ? 1u : 0u);
+                    }
                 }
                 tc_commit(B.s_full + 8 * c);
                 tc_commit(B.slot_empty + 8 * s);
@@ -491,6 +499,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             const float4* src = reinterpret_cast<const float4*>(
                 p.o_part + ((int64_t)(unit % kRing) * p.HG + head_local) * p.cph * R * kD);
             for (int e = lo + tid; e < hi; e += 32) {
+                const int r = e / (kD / 4), d4 = e - r * (kD / 4);
+                if (d4 * 4 >= p.D) continue;  // head_dim 64: the partial's upper columns are padding
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int k0 = 0; k0 < p.cph; k0 += 16) {  // batches of 16 independent loads
                     float4 x[16];
@@ -509,14 +519,13 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         acc.w += x[u].w;
                     }
                 }
-                const int r = e / (kD / 4), d4 = e - r * (kD / 4);
                 const int j = r / G, g = r - j * G;
                 const int64_t row = (((int64_t)sg.layer * p.a.kv.batch + sg.b) * p.a.n_q + j) * p.a.kv.n_q_heads + sg.h * G + g;
                 if (p.a.out_bf16)
-                    reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.a.out) + row * kD)[d4] =
+                    reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.a.out) + row * p.D)[d4] =
                         make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
                 else
-                    reinterpret_cast<float4*>(p.a.out + row * kD)[d4] = acc;
+                    reinterpret_cast<float4*>(p.a.out + row * p.D)[d4] = acc;
             }
         }
     } else {

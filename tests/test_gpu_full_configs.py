@@ -82,6 +82,7 @@ def run_config(cfg, samples, fold=False):
 def test_cfg1_tiny_every_head():
     cfg = inputs.baseline_configs()["cfg1_tiny"]
     _, _, worst = run_config(cfg, [(0, 0, 0), (0, 0, 1)])
+    assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED  # head_dim 64 on the tcgen05 path
     assert worst["overlap"] > 0.97
 
 

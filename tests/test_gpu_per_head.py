@@ -20,7 +20,7 @@ TOL = 2e-3
     (dict(ctx=(800, 800), n_q=4, n_q_heads=10, n_kv_heads=2), binding.VERIFY_TCGEN05_CACHED),    # groups of 5
     (dict(ctx=(2300, 2300), n_q=7, n_q_heads=6, n_kv_heads=2, n_layers=2), binding.VERIFY_TCGEN05_CACHED),  # groups of 3, window offset
     (dict(ctx=(500, 500), n_q=2, n_q_heads=20, n_kv_heads=2), binding.VERIFY_GENERIC),            # groups of 10
-    (dict(ctx=(600, 600), n_q=4, n_q_heads=8, n_kv_heads=2, head_dim=64), binding.VERIFY_GENERIC),
+    (dict(ctx=(600, 600), n_q=4, n_q_heads=8, n_kv_heads=2, head_dim=64), binding.VERIFY_TCGEN05_CACHED),
 ])
 def test_per_head_path_matches_oracle(shape, expect_impl):
     cfg = inputs.small_config(k_total=160, k_recent=16, draft_steps=2, **shape)

@@ -18,7 +18,7 @@ def kv_struct(n_layers, batch, hq, hkv, d, max_ctx, page=None):
 
 
 VERIFY_CASES = [  # (name, kv, n_q, ctx, expected kernel)
-    ("cfg1", kv_struct(1, 1, 8, 2, 64, 2048), 5, 2048, 0),            # head_dim 64: generic kernels
+    ("cfg1", kv_struct(1, 1, 8, 2, 64, 2048), 5, 2048, 2),            # head_dim 64: lower half of each tile
     ("cfg2", kv_struct(1, 1, 32, 8, 128, 32768 + 128), 9, 32768, 2),
     ("cfg3_k1", kv_struct(1, 1, 32, 8, 128, 131072 + 128), 2, 131072, 2),
     ("cfg3_k8", kv_struct(1, 1, 32, 8, 128, 131072 + 128), 9, 131072, 2),

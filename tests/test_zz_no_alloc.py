@@ -43,7 +43,7 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
 def test_noalloc_reuses_the_scratch_for_another_shape():
     _compare(inputs.small_config(ctx=(300, 1100), n_q=7, batch=3, page_size=16, shuffled_pages=True,
                                  planted=0, q_mode="iid", q_std=0.09, n_q_heads=8, n_kv_heads=2))
-    _compare(inputs.small_config(ctx=(700, 700), n_q=5, head_dim=64, planted=4))  # generic kernels
+    _compare(inputs.small_config(ctx=(700, 700), n_q=5, head_dim=64, planted=4))  # head_dim 64
 
 
 def test_noalloc_refuses_shapes_beyond_the_built_in_scratch():
