@@ -47,6 +47,7 @@ class _KV(ctypes.Structure):
         ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32),
         ("sm_scale", ctypes.c_double),
+        ("kv_fp8", ctypes.c_int32), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -70,18 +71,31 @@ def _cpu(t: torch.Tensor, dtype) -> torch.Tensor:
 
 
 def _kv_struct(kv):
-    k = _cpu(kv.k, torch.bfloat16)
-    v = _cpu(kv.v, torch.bfloat16)
+    fp8 = bool(getattr(kv, "fp8", False))
+    k = _cpu(kv.k, torch.uint8 if fp8 else torch.bfloat16)
+    v = _cpu(kv.v, torch.uint8 if fp8 else torch.bfloat16)
     pt = None
     if kv.page_table is not None:
         pt = _cpu(kv.page_table, torch.int32)
+    ks = vs = None
+    if fp8 and getattr(kv, "k_scale", None) is not None:
+        ks, vs = _cpu(kv.k_scale, torch.float32), _cpu(kv.v_scale, torch.float32)
+        assert ks.shape == (kv.n_layers, kv.n_kv_heads) and vs.shape == ks.shape
     s = _KV(
         k.data_ptr(), v.data_ptr(), kv.layer_stride, kv.page_stride, kv.head_stride,
         kv.slot_stride, kv.n_layers, kv.page_size, pt.data_ptr() if pt is not None else None,
         kv.max_pages, kv.batch, kv.n_q_heads, kv.n_kv_heads, kv.head_dim,
-        float(kv.sm_scale or 0.0),
+        float(kv.sm_scale or 0.0), 1 if fp8 else 0,
+        ks.data_ptr() if ks is not None else None, vs.data_ptr() if vs is not None else None,
     )
-    return s, (k, v, pt)
+    return s, (k, v, pt, ks, vs)
+
+
+def e4m3_to_double(byte: int) -> float:
+    """The oracle's decoder of one e4m3 byte (exposed for the pins)."""
+    lib = _load()
+    lib.oracle_e4m3_to_double.restype = ctypes.c_double
+    return float(lib.oracle_e4m3_to_double(ctypes.c_int(byte)))
 
 
 def verify_attn(kv, q, ctx_len, stat_window=16, stat_stride=None, per_head=False, group_max=False):

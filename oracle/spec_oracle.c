@@ -39,12 +39,18 @@
 #endif
 
 typedef struct {
-    const uint16_t *k, *v; /* bf16 bit patterns */
-    int64_t layer_stride, page_stride, head_stride, slot_stride;
+    const void *k, *v; /* bf16 bit patterns, or fp8 (e4m3) bytes when kv_fp8 is set */
+    int64_t layer_stride, page_stride, head_stride, slot_stride; /* in elements */
     int32_t n_layers, page_size;
     const int32_t *page_table;
     int32_t max_pages, batch, n_q_heads, n_kv_heads, head_dim;
     double sm_scale; /* <= 0 means 1/sqrt(head_dim) */
+    /* 8-bit cache: an element is e4m3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; exponent 0 is
+     * the denormal range m / 8 * 2^-6; no infinities, S.1111.111 is NaN) times a per-(layer, KV head)
+     * scale, k_scale / v_scale [n_layers, n_kv_heads] (NULL: 1).  The attention is then the plain
+     * definition on those dequantised values. */
+    int32_t kv_fp8;
+    const float *k_scale, *v_scale;
 } oracle_kv_t;
 
 static double bf16_to_double(uint16_t bits)
@@ -54,6 +60,29 @@ static double bf16_to_double(uint16_t bits)
     memcpy(&f, &u, sizeof f);
     return (double)f;
 }
+
+static double e4m3_to_double(uint8_t b)
+{
+    const int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* element `off` of K (which = 0) or V (which = 1) of (layer, KV head h), dequantised */
+static double kv_elem(const oracle_kv_t *kv, int which, int layer, int h, int64_t off)
+{
+    const void *base = which ? kv->v : kv->k;
+    if (!kv->kv_fp8) return bf16_to_double(((const uint16_t *)base)[off]);
+    const float *sc = which ? kv->v_scale : kv->k_scale;
+    const double scale = sc ? (double)sc[(int64_t)layer * kv->n_kv_heads + h] : 1.0;
+    return e4m3_to_double(((const uint8_t *)base)[off]) * scale;
+}
+
+/* decoder exposed for the pins */
+double oracle_e4m3_to_double(int byte) { return e4m3_to_double((uint8_t)byte); }
 
 static int64_t kv_row_offset(const oracle_kv_t *kv, int layer, int b, int64_t pos, int h)
 {
@@ -82,9 +111,9 @@ int oracle_threads(void)
 static double logit(const oracle_kv_t *kv, const uint16_t *qrow, int layer, int b, int64_t pos,
                     int h, double scale)
 {
-    const uint16_t *krow = kv->k + kv_row_offset(kv, layer, b, pos, h);
+    const int64_t krow = kv_row_offset(kv, layer, b, pos, h);
     double s = 0.0;
-    for (int d = 0; d < kv->head_dim; ++d) s += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+    for (int d = 0; d < kv->head_dim; ++d) s += bf16_to_double(qrow[d]) * kv_elem(kv, 0, layer, h, krow + d);
     return s * scale;
 }
 
@@ -151,8 +180,8 @@ int oracle_verify_attn_ex(const oracle_kv_t *kv, const uint16_t *q, int n_q, con
                         for (int d = 0; d < D; ++d) o[d] = 0.0;
                         for (int64_t i = 0; i <= pos; ++i) {
                             p[i] /= denom;
-                            const uint16_t *vrow = kv->v + kv_row_offset(kv, layer, b, i, h);
-                            for (int d = 0; d < D; ++d) o[d] += p[i] * bf16_to_double(vrow[d]);
+                            const int64_t vrow = kv_row_offset(kv, layer, b, i, h);
+                            for (int d = 0; d < D; ++d) o[d] += p[i] * kv_elem(kv, 1, layer, h, vrow + d);
                             if (j >= first_stat_row) st[i] += p[i];
                         }
                         if (lse) lse[row] = m + log(denom);
@@ -293,9 +322,9 @@ int oracle_sparse_draft_attn_ex(const oracle_kv_t *kv, const uint16_t *q, const 
                     double *o = out + row * D;
                     for (int d = 0; d < D; ++d) o[d] = 0.0;
                     for (int i = 0; i < n; ++i) {
-                        const uint16_t *vrow = kv->v + kv_row_offset(kv, layer, b, keys[i], h);
+                        const int64_t vrow = kv_row_offset(kv, layer, b, keys[i], h);
                         const double w = p[i] / denom;
-                        for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(vrow[d]);
+                        for (int d = 0; d < D; ++d) o[d] += w * kv_elem(kv, 1, layer, h, vrow + d);
                     }
                     if (lse) lse[row] = n > 0 ? m + log(denom) : -INFINITY;
                 }

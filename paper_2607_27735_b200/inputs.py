@@ -47,17 +47,24 @@ class KVCache:
     head_dim: int
     sm_scale: float = 0.0
     n_pages: int = 0  # physical pages in the pool (0: batch * max_pages)
+    fp8: bool = False  # k, v hold e4m3 bytes (uint8) instead of bf16; strides stay in elements
+    k_scale: Optional[torch.Tensor] = None  # fp32 [L, Hkv]: dequantised value = e4m3 value * scale
+    v_scale: Optional[torch.Tensor] = None
 
     def to(self, device) -> "KVCache":
         pt = None if self.page_table is None else self.page_table.to(device)
-        return dataclasses.replace(self, k=self.k.to(device), v=self.v.to(device), page_table=pt)
+        ks = None if self.k_scale is None else self.k_scale.to(device)
+        vs = None if self.v_scale is None else self.v_scale.to(device)
+        return dataclasses.replace(self, k=self.k.to(device), v=self.v.to(device), page_table=pt, k_scale=ks, v_scale=vs)
 
     def cpu(self) -> "KVCache":
         return self.to("cpu")
 
     def layer_slice(self, lo: int, hi: int) -> "KVCache":
         """View of layers ``[lo, hi)`` (shares storage)."""
-        return dataclasses.replace(self, k=self.k[lo:hi], v=self.v[lo:hi], n_layers=hi - lo)
+        ks = None if self.k_scale is None else self.k_scale[lo:hi].contiguous()
+        vs = None if self.v_scale is None else self.v_scale[lo:hi].contiguous()
+        return dataclasses.replace(self, k=self.k[lo:hi], v=self.v[lo:hi], n_layers=hi - lo, k_scale=ks, v_scale=vs)
 
     def phys_page(self, b: int, page: int) -> int:
         if self.page_table is None:
@@ -310,3 +317,30 @@ def make_logits(rows: int, vocab: int, dtype=torch.bfloat16, seed: int = 0, devi
     view.scatter_add_(1, cols, boost)
     buf = buf.to(dtype).to(device)
     return buf[offset:offset + rows * stride].view(rows, stride)[:, :vocab]
+
+
+def quantize_kv_fp8(kv: KVCache) -> KVCache:
+    """An 8-bit copy of a bf16 cache: e4m3 bytes (same layout, strides in elements) and a power-of-two
+    scale per (layer, KV head) chosen so that the head's largest magnitude lands below 448, the e4m3
+    maximum.  Only a cast and a scale: no attention arithmetic."""
+    L, Hkv = kv.n_layers, kv.n_kv_heads
+
+    def one(x):
+        amax = x.float().abs().amax(dim=(1, 3, 4)).clamp(min=1e-30)            # [L, Hkv] over pages, slots, d
+        scale = torch.exp2(torch.ceil(torch.log2(amax / 448.0))).float()
+        q = (x.float() / scale.view(L, 1, Hkv, 1, 1)).to(torch.float8_e4m3fn).view(torch.uint8)
+        return q.contiguous(), scale.contiguous()
+
+    k8, ks = one(kv.k)
+    v8, vs = one(kv.v)
+    return dataclasses.replace(kv, k=k8, v=v8, fp8=True, k_scale=ks, v_scale=vs)
+
+
+def dequantize_kv_fp8(kv: KVCache) -> KVCache:
+    """The bf16 cache whose values are exactly the dequantised ones (an e4m3 value times a power of two has
+    four significant bits: representable in bf16 without rounding)."""
+    L, Hkv = kv.n_layers, kv.n_kv_heads
+    k = (kv.k.view(torch.float8_e4m3fn).float() * kv.k_scale.view(L, 1, Hkv, 1, 1)).to(torch.bfloat16)
+    v = (kv.v.view(torch.float8_e4m3fn).float() * kv.v_scale.view(L, 1, Hkv, 1, 1)).to(torch.bfloat16)
+    return dataclasses.replace(kv, k=k, v=v, fp8=False, k_scale=None, v_scale=None)
+

@@ -536,3 +536,45 @@ def test_group_max_statistic_bounds_closed_form_and_mass():
         pos = T - n_q + j
         want[:pos + 1] += 1.0 / (pos + 1)
     assert (st2[0, 0] - want).abs().max().item() < 1e-12
+
+
+# ---- 8-bit (e4m3) KV cache: the same attention on dequantised values ----
+
+def test_e4m3_decoder_matches_the_library_cast():
+    """All 256 byte patterns against torch's float8_e4m3fn (an independent decoder), NaN patterns included."""
+    raw = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    lib = raw.view(torch.float8_e4m3fn).double()
+    for b in range(256):
+        mine = oracle.e4m3_to_double(b)
+        if math.isnan(float(lib[b])):
+            assert math.isnan(mine) and (b & 0x7f) == 0x7f
+        else:
+            assert mine == float(lib[b]), b
+    assert oracle.e4m3_to_double(0x7e) == 448.0 and oracle.e4m3_to_double(0x01) == 2.0 ** -9
+
+
+def test_fp8_cache_is_the_bf16_oracle_on_the_dequantised_cache():
+    """Verification (output, LSE, score) and drafting over an e4m3 cache with per-(layer, head) power-of-two
+    scales equal, bit for bit, the pinned bf16 functions on the cache of dequantised values (which bf16
+    holds exactly), contiguous and paged."""
+    from paper_2607_27735_b200 import inputs
+    for kw in (dict(ctx=(180, 260), batch=2, n_q=5, n_q_heads=8, n_kv_heads=2, n_layers=2, planted=3, seed=51),
+               dict(ctx=(90, 200), batch=3, n_q=3, page_size=16, shuffled_pages=True, planted=0, q_mode="iid",
+                    head_dim=64, seed=52)):
+        cfg = inputs.small_config(k_total=64, k_recent=8, draft_steps=1, **kw)
+        case = inputs.make_case(cfg)
+        kv8 = inputs.quantize_kv_fp8(case.kv)
+        deq = inputs.dequantize_kv_fp8(kv8)
+        assert (kv8.k_scale > 0).all() and torch.equal(torch.log2(kv8.k_scale), torch.log2(kv8.k_scale).round())
+        a = oracle.verify_attn(kv8, case.q_verify, case.ctx_len, 16)
+        b = oracle.verify_attn(deq, case.q_verify, case.ctx_len, 16)
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+        # and it is a different problem from the unquantised one (the cast rounds to 4 significant bits)
+        c = oracle.verify_attn(case.kv, case.q_verify, case.ctx_len, 16)
+        assert (a[0] - c[0]).abs().max().item() > 1e-4
+        idx, n = oracle.select_recall(a[2].float(), case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total)
+        q = case.q_draft[0].contiguous()
+        d8 = oracle.sparse_draft_attn(kv8, q, idx, n, case.ctx_len, case.ctx_len + 1)
+        dd = oracle.sparse_draft_attn(deq, q, idx, n, case.ctx_len, case.ctx_len + 1)
+        assert torch.equal(d8[0], dd[0]) and torch.equal(d8[1], dd[1])
