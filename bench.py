@@ -357,6 +357,55 @@ def other_workloads(peak, dev, layers=4, steps=5):
         }
         del run, case
         torch.cuda.empty_cache()
+    out.update(fp8_draft_workload(peak, dev))
+    return out
+
+
+def fp8_draft_workload(peak, dev, layers=4, steps=5):
+    """The headline shape's drafting phase over an 8-bit (e4m3) copy of the cache: same index sets (built by
+    the bf16 verification), half the gathered bytes.  Per layer-call and with the layers folded."""
+    import dataclasses
+
+    import torch
+
+    from paper_2607_27735_b200 import binding, inputs, runner
+    out = {}
+    full = inputs.baseline_configs(8)["cfg2_8b_32k"]
+    for fold, n_layers in ((False, layers), (True, 32)):
+        cfg = dataclasses.replace(full, n_layers=n_layers)
+        case = inputs.make_case(cfg, device=dev)
+        run = runner.SpecStepRunner(case, fold_layers=fold)
+        run.verify_phase()
+        run.select_phase()
+        torch.cuda.synchronize()
+        kv8 = inputs.quantize_kv_fp8(case.kv)
+        run.kv = kv8
+        run._layers = [kv8.layer_slice(l, l + 1) for l in range(n_layers)]
+        run.draft_phase()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        before = binding.launch_count()
+        with torch.cuda.graph(g):
+            run.draft_phase()
+        n_launch = binding.launch_count() - before
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / steps
+        nbytes = sum(run.draft_kv_bytes_per_layer_step(j) for j in range(cfg.draft_steps)) * n_layers // 2
+        out["cfg2_8b_32k_fp8_draft" + ("_folded" if fold else "")] = {
+            "layers": f"{n_layers} of 32 layers", "kv": "e4m3, one power-of-two scale per (layer, KV head)",
+            "draft_us_per_call": us / n_launch, "draft_bytes_per_call": nbytes // n_launch,
+            "draft_GBs": nbytes / us / 1e3, "draft_frac": nbytes / us / 1e3 / peak,
+            "status": binding.read_status(run.ws_d)}
+        del run, case, kv8, g
+        torch.cuda.empty_cache()
     return out
 
 

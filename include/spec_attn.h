@@ -88,7 +88,22 @@ typedef struct {
     int32_t n_pages;               /* physical pages in the pool (bounds page_table entries);
                                       0 means batch * max_pages */
     float sm_scale;                /* softmax scale; <= 0 means 1/sqrt(head_dim) */
+    int32_t kv_dtype;              /* SPEC_KV_BF16 (0) or SPEC_KV_FP8_E4M3: k and v hold e4m3 bytes (1 sign, 4
+                                      exponent bits with bias 7, 3 mantissa bits, no infinities), same
+                                      addressing rule with strides in elements (= bytes), every stride a
+                                      multiple of 16 */
+    const float* k_scale;          /* SPEC_KV_FP8_E4M3: device fp32 [n_layers, n_kv_heads], an element's value */
+    const float* v_scale;          /* is its e4m3 value times the (layer, KV head) scale; NULL means 1 */
 } spec_kv_t;
+
+/* Element type of the cache.  With SPEC_KV_FP8_E4M3 (the decode step is bound by loading the cache:
+ * Sec. 1, so an 8-bit cache halves the bytes of every call) Q stays bf16 and all results are those of
+ * the same attention on the dequantised values.  Served by the sparse draft attention kernel
+ * (tensor cores on fp16 copies of the rows, which hold e4m3 values exactly; Q is converted to fp16:
+ * exact for magnitudes in [6.1e-5, 65504], absolute error <= 3e-8 below that) and by the generic
+ * verification kernels; the tcgen05 verification kernels take bf16 caches only, so spec_verify_attn
+ * with an 8-bit cache always runs the generic kernels. */
+enum { SPEC_KV_BF16 = 0, SPEC_KV_FP8_E4M3 = 1 };
 
 /*
  * Full-context verification attention + importance score (Sec. 3.1 "Full Verification

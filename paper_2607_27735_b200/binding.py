@@ -55,6 +55,7 @@ class _KV(ctypes.Structure):
         ("max_pages", ctypes.c_int32), ("batch", ctypes.c_int32),
         ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
         ("head_dim", ctypes.c_int32), ("n_pages", ctypes.c_int32), ("sm_scale", ctypes.c_float),
+        ("kv_dtype", ctypes.c_int32), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p),
     ]
 
 
@@ -122,14 +123,22 @@ def _dev(t: torch.Tensor, dtype, name: str) -> int:
     return t.data_ptr()
 
 
+KV_BF16, KV_FP8_E4M3 = 0, 1
+
+
 def _kv_struct(kv) -> _KV:
-    _dev(kv.k, torch.bfloat16, "kv.k")
-    _dev(kv.v, torch.bfloat16, "kv.v")
+    fp8 = bool(getattr(kv, "fp8", False))
+    _dev(kv.k, torch.uint8 if fp8 else torch.bfloat16, "kv.k")
+    _dev(kv.v, torch.uint8 if fp8 else torch.bfloat16, "kv.v")
     pt = None if kv.page_table is None else _dev(kv.page_table, torch.int32, "kv.page_table")
+    ks = vs = None
+    if fp8 and getattr(kv, "k_scale", None) is not None:
+        ks = _dev(kv.k_scale, torch.float32, "kv.k_scale")
+        vs = _dev(kv.v_scale, torch.float32, "kv.v_scale")
     return _KV(kv.k.data_ptr(), kv.v.data_ptr(), kv.layer_stride, kv.page_stride, kv.head_stride,
                kv.slot_stride, kv.n_layers, kv.page_size, pt, kv.max_pages, kv.batch,
                kv.n_q_heads, kv.n_kv_heads, kv.head_dim, int(getattr(kv, "n_pages", 0) or 0),
-               float(kv.sm_scale or 0.0))
+               float(kv.sm_scale or 0.0), KV_FP8_E4M3 if fp8 else KV_BF16, ks, vs)
 
 
 def _stream() -> int:

@@ -27,20 +27,39 @@ using namespace draft;
 constexpr int kChunk = 16;
 constexpr uint32_t kNoRow = 0xffffffffu;
 
-template <int D>
+template <int D, bool F8>
 struct Geo {
-    static constexpr int ROWB = D * 2 + 16;          // bytes per shared-memory row: 16 B of padding spread the banks
+    static constexpr int ES = F8 ? 1 : 2;            // bytes per cache element (e4m3 or bf16)
+    static constexpr int ROWB = D * ES + 16;         // bytes per shared-memory row: 16 B of padding spread the banks
     static constexpr int STAGE = 2 * kChunk * ROWB;  // a chunk's K rows, then its V rows
 };
 
 // Shared memory of one CTA: [NW warps][ST stages][STAGE] | row offsets uint32 [per] |
 // per-warp (max, sum) float2 [NW][8] | deposit barrier (16 B) | deposit area float [cs][G * (D + 2)]
-template <int D>
+template <int D, bool F8>
 __host__ __device__ inline size_t stream_smem_bytes(int G, int nw, int st, int per, int cs)
 {
-    return (size_t)nw * st * Geo<D>::STAGE + (size_t)per * 4 + (size_t)nw * 8 * 8 + 16 + (size_t)cs * G * (D + 2) * 4;
+    return (size_t)nw * st * Geo<D, F8>::STAGE + (size_t)per * 4 + (size_t)nw * 8 * 8 + 16 + (size_t)cs * G * (D + 2) * 4;
 }
 
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// two e4m3 bytes (the low 16 bits of `two`) as a packed fp16 pair: exact
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two)
+{
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(two & 0xffffu), __NV_E4M3);
+    return (uint32_t)h.x | ((uint32_t)h.y << 16);
+}
+__device__ __forceinline__ uint32_t pack_f16(float x, float y)
+{
+    const __half2 v = __floats2half2_rn(x, y);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1)
 {
@@ -49,11 +68,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int D, int NW, int ST>
+// F8: the cache holds e4m3 bytes.  The rows are gathered as they are (half the bytes), turned into fp16
+// pairs on their way into the MMA fragments (fp16 holds every e4m3 value), and the two products run as
+// fp16 MMAs; the heads' scales join the softmax scale (K) and the final output (V).
+template <int D, int NW, int ST, bool F8>
 __global__ void __launch_bounds__(NW * 32)
 draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 {
-    constexpr int ROWB = Geo<D>::ROWB, STAGE = Geo<D>::STAGE;
+    constexpr int ROWB = Geo<D, F8>::ROWB, STAGE = Geo<D, F8>::STAGE, ES = Geo<D, F8>::ES;
     constexpr int NT = NW * 32;
     constexpr int KS = D / 16;  // 16-wide steps of the head dimension
     constexpr float kLog2e = 1.4426950408889634f;
@@ -120,7 +142,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
                     const int slot_in = pos - page * a.kv.page_size;
                     const int64_t phys = ptab ? (int64_t)__ldg(ptab + page) : (int64_t)b * a.kv.max_pages + page;
                     if (phys < 0 || phys >= a.kv.n_pages) set_status(status, SPEC_ERR_BAD_INDEX);
-                    else off = (uint32_t)((phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride) >> 3);
+                    else off = (uint32_t)((phys * a.kv.page_stride + (int64_t)slot_in * a.kv.slot_stride) >> (F8 ? 4 : 3));
                 }
             }
             rowoff[lr] = off;
@@ -130,9 +152,11 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 
     // ---- per-warp pipeline over the chunks warp, warp + NW, ... of the share ----
     // one instruction copies 16-byte pieces of 32 / (2 * PIECES) rows: the K pieces and the V pieces of each
-    constexpr int PIECES = D / 8, RPI = 32 / (2 * PIECES);
+    constexpr int PIECES = D * ES / 16, RPI = 32 / (2 * PIECES);
     const int piece = lane % PIECES, is_v = (lane / PIECES) & 1, rsub = lane / (2 * PIECES);
-    const __nv_bfloat16* gbase = (is_v ? a.kv.v : a.kv.k) + layer * a.kv.layer_stride + hm * a.kv.head_stride + piece * 8;
+    const uint8_t* gbase = (F8 ? (is_v ? a.kv.v8 : a.kv.k8)
+                               : reinterpret_cast<const uint8_t*>(is_v ? a.kv.v : a.kv.k)) +
+                           (layer * a.kv.layer_stride + hm * a.kv.head_stride) * ES + piece * 16;
     uint8_t* wst = stages + (size_t)warp * ST * STAGE;
     const uint32_t dst_lane = (is_v ? kChunk * ROWB : 0) + rsub * ROWB + piece * 16;
 
@@ -147,7 +171,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 #pragma unroll
             for (int r = 0; r < kChunk; r += RPI) {
                 const uint32_t o = __shfl_sync(0xffffffffu, mine, r + rsub);
-                cp_async16(dst + r * ROWB, gbase + ((int64_t)(o == kNoRow ? 0u : o) << 3), o == kNoRow ? 0u : 16u);
+                cp_async16(dst + r * ROWB, gbase + ((int64_t)(o == kNoRow ? 0u : o) << 4), o == kNoRow ? 0u : 16u);
             }
         }
         cp_async_commit();
@@ -161,19 +185,29 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         asm volatile("griddepcontrol.wait;" ::: "memory");  // Q is written by the stream
         waited = true;
     }
-    // A fragments of Q (heads x d): the thread holds head grp at d = 16 ks + 2 quad + {0, 1} and + {8, 9}
+    // A fragments of Q (heads x d): the thread holds head grp at d = 16 ks + 2 quad + {0, 1} and + {8, 9}.
+    // F8: the K fragment of a step comes from ONE 4-byte load (d = 16 ks + 4 quad + 0..3), so the step's
+    // sixteen d's are visited in that order and Q follows it: d = 16 ks + 4 quad + {0, 1} and + {2, 3},
+    // as fp16.
     uint32_t qa[KS][2];
     {
         const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + grp;
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + row * D);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            qa[ks][0] = grp < G ? __ldg(qrow + ks * 8 + quad) : 0u;
-            qa[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
+            if (F8) {
+                const uint32_t w0 = grp < G ? __ldg(qrow + ks * 8 + 2 * quad) : 0u;
+                const uint32_t w1 = grp < G ? __ldg(qrow + ks * 8 + 2 * quad + 1) : 0u;
+                qa[ks][0] = pack_f16(bf16_lo(w0), bf16_hi(w0));
+                qa[ks][1] = pack_f16(bf16_lo(w1), bf16_hi(w1));
+            } else {
+                qa[ks][0] = grp < G ? __ldg(qrow + ks * 8 + quad) : 0u;
+                qa[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
+            }
         }
     }
 
-    const float sc = a.kv.scale * kLog2e;
+    const float sc = a.kv.scale * kLog2e * (F8 ? kv_scale_of(a.kv.k_scale, a.kv, layer, hm) : 1.f);
     float M = kNegBig, L = 0.f;
     float o[D / 8][4];
 #pragma unroll
@@ -189,16 +223,32 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
         {
             float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};  // four accumulation chains
-            const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB + ((lane >> 3) & 1) * 16;
+            if (F8) {
+                // key grp (and grp + 8), bytes 16 ks + 4 quad .. + 3: one load per key block and step
+                const uint8_t* kp = ksm + grp * ROWB + 4 * quad;
 #pragma unroll
-            for (int ks = 0; ks < KS; ks += 2) {
-                uint32_t kf[4], kg[4];
-                ldmatrix_x4(kf, kp + ks * 32);
-                ldmatrix_x4(kg, kp + ks * 32 + 32);
-                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, kf[0], kf[1]);
-                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, kf[2], kf[3]);
-                mma_bf16_16816(t0, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[0], kg[1]);
-                mma_bf16_16816(t1, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[2], kg[3]);
+                for (int ks = 0; ks < KS; ks += 2) {
+                    const uint32_t k00 = *reinterpret_cast<const uint32_t*>(kp + ks * 16);
+                    const uint32_t k01 = *reinterpret_cast<const uint32_t*>(kp + 8 * ROWB + ks * 16);
+                    const uint32_t k10 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 16);
+                    const uint32_t k11 = *reinterpret_cast<const uint32_t*>(kp + 8 * ROWB + ks * 16 + 16);
+                    mma_f16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, e4m3x2_to_f16x2(k00), e4m3x2_to_f16x2(k00 >> 16));
+                    mma_f16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, e4m3x2_to_f16x2(k01), e4m3x2_to_f16x2(k01 >> 16));
+                    mma_f16_16816(t0, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, e4m3x2_to_f16x2(k10), e4m3x2_to_f16x2(k10 >> 16));
+                    mma_f16_16816(t1, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, e4m3x2_to_f16x2(k11), e4m3x2_to_f16x2(k11 >> 16));
+                }
+            } else {
+                const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB + ((lane >> 3) & 1) * 16;
+#pragma unroll
+                for (int ks = 0; ks < KS; ks += 2) {
+                    uint32_t kf[4], kg[4];
+                    ldmatrix_x4(kf, kp + ks * 32);
+                    ldmatrix_x4(kg, kp + ks * 32 + 32);
+                    mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, kf[0], kf[1]);
+                    mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, kf[2], kf[3]);
+                    mma_bf16_16816(t0, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[0], kg[1]);
+                    mma_bf16_16816(t1, qa[ks + 1][0], 0u, qa[ks + 1][1], 0u, kg[2], kg[3]);
+                }
             }
             s0[0] += t0[0];
             s0[1] += t0[1];
@@ -234,9 +284,15 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 #pragma unroll
         for (int i = 0; i < 4; ++i) p[i] = sv[i] > 0.5f * kNegBig ? ex2f(sv[i] - M) : 0.f;
         L += (p[0] + p[1]) + (p[2] + p[3]);
-        // [P_hi ; P_lo] as the A operand: rows 0..7 the bf16 rounding, rows 8..15 the remainder
+        // [P_hi ; P_lo] as the A operand: rows 0..7 the 16-bit rounding, rows 8..15 the remainder
         uint32_t ah0, al0, ah1, al1;
-        {
+        if (F8) {
+            const __half2 h01 = __floats2half2_rn(p[0], p[1]), h23 = __floats2half2_rn(p[2], p[3]);
+            ah0 = *reinterpret_cast<const uint32_t*>(&h01);
+            ah1 = *reinterpret_cast<const uint32_t*>(&h23);
+            al0 = pack_f16(p[0] - __low2float(h01), p[1] - __high2float(h01));
+            al1 = pack_f16(p[2] - __low2float(h23), p[3] - __high2float(h23));
+        } else {
             const __nv_bfloat162 h01 = __floats2bfloat162_rn(p[0], p[1]), h23 = __floats2bfloat162_rn(p[2], p[3]);
             ah0 = *reinterpret_cast<const uint32_t*>(&h01);
             ah1 = *reinterpret_cast<const uint32_t*>(&h23);
@@ -244,7 +300,27 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
             al1 = pack_bf16(p[2] - __low2float(h23), p[3] - __high2float(h23));
         }
         // ---- O += [P_hi ; P_lo] V ----
-        {
+        if (F8) {
+            // A transposing 8x8 load works on 2-byte units, so a thread gets, for keys 2 quad and 2 quad + 1,
+            // the byte PAIR d = 2 grp, 2 grp + 1 (of a 16-byte column block): bytes 0 and 2 of the register are
+            // the B fragment of the even d, bytes 1 and 3 of the odd d.  Four column blocks of 8 come out
+            // of one x4 load (32 bytes of every row); the accumulators therefore hold the head dimension in
+            // the order d = 32 j + 16 (t / 2) + 4 quad + (t % 2) + {0, 2} for block 4 j + t (see the store).
+            const uint8_t* vp = vsm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + ((lane >> 4) & 1) * 16;
+#pragma unroll
+            for (int j = 0; j < D / 32; ++j) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(vf, vp + j * 32);
+                mma_f16_16816(o[4 * j + 0], ah0, al0, ah1, al1, e4m3x2_to_f16x2(__byte_perm(vf[0], 0u, 0x4420)),
+                              e4m3x2_to_f16x2(__byte_perm(vf[1], 0u, 0x4420)));
+                mma_f16_16816(o[4 * j + 1], ah0, al0, ah1, al1, e4m3x2_to_f16x2(__byte_perm(vf[0], 0u, 0x4431)),
+                              e4m3x2_to_f16x2(__byte_perm(vf[1], 0u, 0x4431)));
+                mma_f16_16816(o[4 * j + 2], ah0, al0, ah1, al1, e4m3x2_to_f16x2(__byte_perm(vf[2], 0u, 0x4420)),
+                              e4m3x2_to_f16x2(__byte_perm(vf[3], 0u, 0x4420)));
+                mma_f16_16816(o[4 * j + 3], ah0, al0, ah1, al1, e4m3x2_to_f16x2(__byte_perm(vf[2], 0u, 0x4431)),
+                              e4m3x2_to_f16x2(__byte_perm(vf[3], 0u, 0x4431)));
+            }
+        } else {
             const uint8_t* vp = vsm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + ((lane >> 4) & 1) * 16;
 #pragma unroll
             for (int nb = 0; nb < KS; ++nb) {
@@ -266,9 +342,19 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     __syncwarp();
     {
         float* ow = reinterpret_cast<float*>(wst);  // [8 heads][D + 8]: the padding keeps the heads on different banks
+        if (F8) {  // undo the order of the head dimension (see the V product) and apply the head's V scale
+            const float vs = kv_scale_of(a.kv.v_scale, a.kv, layer, hm);
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i)
-            *reinterpret_cast<float2*>(ow + grp * (D + 8) + i * 8 + 2 * quad) = make_float2(o[i][0] + o[i][2], o[i][1] + o[i][3]);
+            for (int i = 0; i < D / 8; ++i) {
+                const int d0 = 32 * (i >> 2) + 16 * ((i >> 1) & 1) + 4 * quad + (i & 1);
+                ow[grp * (D + 8) + d0] = (o[i][0] + o[i][2]) * vs;
+                ow[grp * (D + 8) + d0 + 2] = (o[i][1] + o[i][3]) * vs;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i)
+                *reinterpret_cast<float2*>(ow + grp * (D + 8) + i * 8 + 2 * quad) = make_float2(o[i][0] + o[i][2], o[i][1] + o[i][3]);
+        }
         if (quad == 0) wml[warp * 8 + grp] = make_float2(M, L);
     }
     __syncthreads();
@@ -307,10 +393,10 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     merge_and_store<D, NT>(a, comb, CS, G, layer, b, h, tid);
 }
 
-template <int D, int NW, int ST>
+template <int D, int NW, int ST, bool F8>
 int launch_inst(const DraftArgs& a, const StreamShape& shp, size_t smem, cudaStream_t stream)
 {
-    auto kern = draft_stream_kernel<D, NW, ST>;
+    auto kern = draft_stream_kernel<D, NW, ST, F8>;
     if (!opt_in_smem(reinterpret_cast<const void*>(kern), smem)) return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(shp.cs, a.kv.n_kv_heads, a.kv.n_layers * a.kv.batch);
@@ -336,14 +422,14 @@ int launch_inst(const DraftArgs& a, const StreamShape& shp, size_t smem, cudaStr
     return SPEC_OK;
 }
 
-template <int D>
+template <int D, bool F8>
 int launch_shape(const DraftArgs& a, const StreamShape& shp, cudaStream_t stream)
 {
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
-    const size_t smem = stream_smem_bytes<D>(G, shp.nw, shp.st, shp.per, shp.cs);
+    const size_t smem = stream_smem_bytes<D, F8>(G, shp.nw, shp.st, shp.per, shp.cs);
     if (smem > kSmemLimit) return SPEC_ERR_UNSUPPORTED_SHAPE;
 #define SPEC_INST(W_, S_) \
-    if (shp.nw == W_ && shp.st == S_) return launch_inst<D, W_, S_>(a, shp, smem, stream);
+    if (shp.nw == W_ && shp.st == S_) return launch_inst<D, W_, S_, F8>(a, shp, smem, stream);
     SPEC_INST(4, 2)
     SPEC_INST(4, 3)
     SPEC_INST(8, 1)
@@ -373,7 +459,8 @@ bool stream_plan(const KvView& kv, int head_dim, int n_keys_max, StreamShape* ou
     const int keys = n_keys_max > 0 ? n_keys_max : 1;
     const int chunks = (keys + kChunk - 1) / kChunk;
     const int nsm = sm_count();
-    const size_t stage = head_dim == 128 ? Geo<128>::STAGE : Geo<64>::STAGE;
+    const size_t stage = kv.fp8 ? (head_dim == 128 ? Geo<128, true>::STAGE : Geo<64, true>::STAGE)
+                                : (head_dim == 128 ? Geo<128, false>::STAGE : Geo<64, false>::STAGE);
     auto smem_of = [&](int cs, int nw, int st, int per) {
         return (size_t)nw * st * stage + (size_t)per * 4 + (size_t)nw * 64 + 16 + (size_t)cs * G * (head_dim + 2) * 4;
     };
@@ -425,8 +512,8 @@ bool stream_plan(const KvView& kv, int head_dim, int n_keys_max, StreamShape* ou
 
 int draft_stream_launch(const DraftArgs& a, const StreamShape& shp, cudaStream_t stream)
 {
-    if (a.kv.head_dim == 128) return launch_shape<128>(a, shp, stream);
-    if (a.kv.head_dim == 64) return launch_shape<64>(a, shp, stream);
+    if (a.kv.head_dim == 128) return a.kv.fp8 ? launch_shape<128, true>(a, shp, stream) : launch_shape<128, false>(a, shp, stream);
+    if (a.kv.head_dim == 64) return a.kv.fp8 ? launch_shape<64, true>(a, shp, stream) : launch_shape<64, false>(a, shp, stream);
     return SPEC_ERR_UNSUPPORTED_SHAPE;
 }
 
@@ -438,7 +525,7 @@ int draft_launch(const DraftArgs& a, cudaStream_t stream)
     if (G > draft::kMaxGroup) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.workspace_bytes < kStatusBytes) return SPEC_ERR_WORKSPACE_TOO_SMALL;
     // row offsets travel as 32-bit counts of 16-byte units: a layer's K (or V) must stay below 64 GiB
-    if ((int64_t)a.kv.n_pages * a.kv.page_stride >= ((int64_t)1 << 35)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)a.kv.n_pages * a.kv.page_stride >= ((int64_t)1 << (a.kv.fp8 ? 36 : 35))) return SPEC_ERR_UNSUPPORTED_SHAPE;
     StreamShape shp;
     if (!stream_plan(a.kv, a.kv.head_dim, a.k_total + a.max_tail, &shp)) return SPEC_ERR_UNSUPPORTED_SHAPE;
     return draft_stream_launch(a, shp, stream);

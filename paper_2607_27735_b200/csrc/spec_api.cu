@@ -66,12 +66,19 @@ static int make_view(const spec_kv_t* kv, KvView* out)
     if (kv->n_q_heads % kv->n_kv_heads != 0) return SPEC_ERR_INVALID_ARG;
     if (kv->head_dim != 64 && kv->head_dim != 128) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (!aligned16(kv->k) || !aligned16(kv->v)) return SPEC_ERR_INVALID_ARG;
+    if (kv->kv_dtype != SPEC_KV_BF16 && kv->kv_dtype != SPEC_KV_FP8_E4M3) return SPEC_ERR_INVALID_ARG;
+    const bool fp8 = kv->kv_dtype == SPEC_KV_FP8_E4M3;
     const int64_t strides[4] = {kv->layer_stride, kv->page_stride, kv->head_stride, kv->slot_stride};
     for (int64_t s : strides)
-        if (s < 0 || s % 8 != 0) return SPEC_ERR_INVALID_ARG;
+        if (s < 0 || s % (fp8 ? 16 : 8) != 0) return SPEC_ERR_INVALID_ARG;  // every row starts on 16 bytes
     if (kv->slot_stride < kv->head_dim) return SPEC_ERR_INVALID_ARG;
-    out->k = static_cast<const __nv_bfloat16*>(kv->k);
-    out->v = static_cast<const __nv_bfloat16*>(kv->v);
+    out->fp8 = fp8 ? 1 : 0;
+    out->k = fp8 ? nullptr : static_cast<const __nv_bfloat16*>(kv->k);
+    out->v = fp8 ? nullptr : static_cast<const __nv_bfloat16*>(kv->v);
+    out->k8 = fp8 ? static_cast<const uint8_t*>(kv->k) : nullptr;
+    out->v8 = fp8 ? static_cast<const uint8_t*>(kv->v) : nullptr;
+    out->k_scale = fp8 ? kv->k_scale : nullptr;
+    out->v_scale = fp8 ? kv->v_scale : nullptr;
     out->layer_stride = kv->layer_stride;
     out->page_stride = kv->page_stride;
     out->head_stride = kv->head_stride;
@@ -159,7 +166,7 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const long hist_probs = (long)kv->n_layers * kv->batch * (a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads);
     const int hist_heads = a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads;
-    const int impl = g_verify_impl.load();
+    const int impl = a.kv.fp8 ? (int)SPEC_VERIFY_GENERIC : g_verify_impl.load();  // 8-bit cache: generic kernels
     if (impl != SPEC_VERIFY_GENERIC) {
         int used = 0;
         const int rc2 = verify_sm100_launch(a, sm100_variant(impl), stream, &used);

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -18,6 +19,13 @@ struct KvView {
     const int32_t* page_table;
     int32_t n_layers, page_size, max_pages, batch, n_q_heads, n_kv_heads, head_dim, n_pages;
     float scale;  // resolved softmax scale
+    // 8-bit cache (spec_kv_t::kv_dtype == SPEC_KV_FP8_E4M3): k8 / v8 hold e4m3 bytes and k / v are null;
+    // an element's value is its e4m3 value times k_scale / v_scale [n_layers, n_kv_heads] (null: 1)
+    int32_t fp8;
+    const uint8_t* k8;
+    const uint8_t* v8;
+    const float* k_scale;
+    const float* v_scale;
     // pos / page_size without a division: page = umulhi(pos, page_mul) >> page_sh for 0 <= pos < 2^31
     // (page_mul = ceil(2^(31 + c) / page_size), page_sh = c - 1, c = ceil(log2 page_size));
     // page_sh < 0 marks page_size == 1
@@ -59,6 +67,17 @@ __device__ __forceinline__ int64_t kv_row_offset(const KvView& kv, int layer, in
     }
     return layer * kv.layer_stride + phys * kv.page_stride + h * kv.head_stride +
            slot * kv.slot_stride;
+}
+
+// Two e4m3 bytes (low byte first) as two floats: exact (cvt to fp16 holds every e4m3 value).
+__device__ __forceinline__ float2 e4m3x2_to_float2(uint16_t two)
+{
+    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)two, __NV_E4M3);
+    return __half22float2(*reinterpret_cast<const __half2*>(&h));
+}
+__device__ __forceinline__ float kv_scale_of(const float* scale, const KvView& kv, int layer, int h)
+{
+    return scale ? __ldg(scale + (int64_t)layer * kv.n_kv_heads + h) : 1.f;
 }
 
 // Two fp32 values as one packed bf16 pair (x in the low half), round to nearest even.

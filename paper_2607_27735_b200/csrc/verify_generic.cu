@@ -59,15 +59,30 @@ __device__ __forceinline__ void score_tile(const KvView& kv, int layer, int b, i
     const int key = key0 + key_l;
     const bool valid = key < T;
     const uint4* krow = nullptr;
-    if (valid) krow = reinterpret_cast<const uint4*>(kv.k + kv_row_offset(kv, layer, b, key, h, status));
+    const uint2* krow8 = nullptr;
+    const float scale = kv.scale * (kv.fp8 ? kv_scale_of(kv.k_scale, kv, layer, h) : 1.f);
+    if (valid) {
+        const int64_t off = kv_row_offset(kv, layer, b, key, h, status);
+        if (kv.fp8) krow8 = reinterpret_cast<const uint2*>(kv.k8 + off);
+        else krow = reinterpret_cast<const uint4*>(kv.k + off);
+    }
     for (int r0 = rg * 4; r0 < R; r0 += 8) {
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         if (valid) {
 #pragma unroll 4
             for (int c = 0; c < D / 8; ++c) {
-                const uint4 kk = __ldg(krow + c);
-                const float kf[8] = {bf16_lo(kk.x), bf16_hi(kk.x), bf16_lo(kk.y), bf16_hi(kk.y),
-                                     bf16_lo(kk.z), bf16_hi(kk.z), bf16_lo(kk.w), bf16_hi(kk.w)};
+                float kf[8];
+                if (kv.fp8) {  // eight e4m3 bytes; the head's scale joins the softmax scale
+                    const uint2 kk = __ldg(krow8 + c);
+                    const float2 a0 = e4m3x2_to_float2((uint16_t)kk.x), a1 = e4m3x2_to_float2((uint16_t)(kk.x >> 16));
+                    const float2 a2 = e4m3x2_to_float2((uint16_t)kk.y), a3 = e4m3x2_to_float2((uint16_t)(kk.y >> 16));
+                    kf[0] = a0.x; kf[1] = a0.y; kf[2] = a1.x; kf[3] = a1.y;
+                    kf[4] = a2.x; kf[5] = a2.y; kf[6] = a3.x; kf[7] = a3.y;
+                } else {
+                    const uint4 kk = __ldg(krow + c);
+                    kf[0] = bf16_lo(kk.x); kf[1] = bf16_hi(kk.x); kf[2] = bf16_lo(kk.y); kf[3] = bf16_hi(kk.y);
+                    kf[4] = bf16_lo(kk.z); kf[5] = bf16_hi(kk.z); kf[6] = bf16_lo(kk.w); kf[7] = bf16_hi(kk.w);
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (r0 + i < R) {
@@ -84,7 +99,7 @@ __device__ __forceinline__ void score_tile(const KvView& kv, int layer, int b, i
             const int r = r0 + i;
             if (r < R) {
                 const int pos = T - n_q + r / G;  // last key row r may see
-                S[r * kSP + key_l] = (valid && key <= pos) ? acc[i] * kv.scale : -INFINITY;
+                S[r * kSP + key_l] = (valid && key <= pos) ? acc[i] * scale : -INFINITY;
             }
         }
     }
@@ -216,6 +231,7 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
 #pragma unroll
     for (int i = 0; i < RPT; ++i) acc[i][0] = acc[i][1] = 0.f;
     const int stat_r0 = a.first_stat_row * G;
+    const float v_scale = a.kv.fp8 ? kv_scale_of(a.kv.v_scale, a.kv, layer, h) : 1.f;
 
     for (int t = t0; t < t1; ++t) {
         const int key0 = t * kTK;
@@ -257,10 +273,16 @@ verify_main_kernel(VerifyArgs a, int n_splits, const float* __restrict__ lse_ws,
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
                 if (kl + kk < nk) {
-                    const __nv_bfloat16* vrow = a.kv.v + kv_row_offset(a.kv, layer, b, key0 + kl + kk, h, static_cast<int*>(a.workspace));
-                    const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(vrow) + dp);
-                    v0[kk] = bf16_lo(w);
-                    v1[kk] = bf16_hi(w);
+                    const int64_t voff = kv_row_offset(a.kv, layer, b, key0 + kl + kk, h, static_cast<int*>(a.workspace));
+                    if (a.kv.fp8) {
+                        const float2 vv = e4m3x2_to_float2(__ldg(reinterpret_cast<const uint16_t*>(a.kv.v8 + voff) + dp));
+                        v0[kk] = vv.x * v_scale;
+                        v1[kk] = vv.y * v_scale;
+                    } else {
+                        const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(a.kv.v + voff) + dp);
+                        v0[kk] = bf16_lo(w);
+                        v1[kk] = bf16_hi(w);
+                    }
                 } else {
                     v0[kk] = v1[kk] = 0.f;
                 }

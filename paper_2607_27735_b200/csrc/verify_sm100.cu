@@ -47,6 +47,7 @@ int box_rows_for(int page_size)
 bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl)
 {
     const int G = kv.n_q_heads / kv.n_kv_heads, R = n_q * G;
+    if (kv.fp8) return false;  // the tcgen05 kernels take bf16 caches only
     // head_dim 64 runs on the score-cache kernel only (one 64-wide half per tile, V padded with zero rows)
     if (!(kv.head_dim == kD || (kv.head_dim == 64 && variant != 1)) || R > 128 || G > 256 || n_q > 256) return false;
     const int box_rows = box_rows_for(kv.page_size);

@@ -14,7 +14,7 @@ def kv_struct(n_layers, batch, hq, hkv, d, max_ctx, page=None):
     page_size = page or max_ctx
     max_pages = (max_ctx + page_size - 1) // page_size
     return binding._KV(1 << 20, 1 << 21, batch * max_pages * hkv * page_size * d, hkv * page_size * d, page_size * d, d,
-                       n_layers, page_size, None, max_pages, batch, hq, hkv, d, batch * max_pages, 0.0)
+                       n_layers, page_size, None, max_pages, batch, hq, hkv, d, batch * max_pages, 0.0, 0, None, None)
 
 
 VERIFY_CASES = [  # (name, kv, n_q, ctx, expected kernel)
