@@ -598,6 +598,13 @@ def run_gpu(args):
                         "phases that do not need them); the dense KV cache stays resident by the "
                         "method's definition"},
         "parity": parity, "folded": folded, "workloads": workloads,
+        "paper_context": {
+            "hardware": "1x NVIDIA A40, Hugging Face Transformers eager attention, contexts <= 64K (another machine "
+                        "and software stack: context, not a target)",
+            "index_update_ms_per_iteration_at_60K": 41.1,
+            "end_to_end_speedup_over_autoregressive": "2.79x (Llama-3.1-8B, LongBench v2), 1.55x-2.79x across models",
+            "this_path_here": "selection of all 32 layers at 32K: phases_us.select; the paper prints no kernel-level "
+                              "figure for verification or draft attention"},
         "gpu_launches": launches_per_step * args.steps,
         "launches_per_step": {"verify": counts[0], "select": counts[1], "draft": counts[2]},
         "clocks": clocks,
