@@ -3,6 +3,12 @@
 // fp32 bit pattern orders like the value and the K_mid-th largest is found by a three-pass
 // radix select (11 + 11 + 10 bits) on the bit patterns; an ordered compaction then emits, in
 // ascending position, everything above the threshold plus the lowest-position ties.
+// The scores are swept twice when the threshold's first-digit bin fits in shared memory (the usual
+// case): the second sweep marks every candidate above that bin in a position bitmap and keeps the
+// bin's own candidates (score, position) in a list; the last two digits are decided on the list and
+// the index set is read off the bitmap in position order.  Flat scores (a bin too full for the list)
+// and contexts too long for the bitmap fall back to one sweep per digit plus one for an ordered
+// compaction.
 // The first pass's histogram (top 11 bits) may arrive from the verification kernel, which counts
 // every score it writes: the positions outside the candidate span are taken out again here, the
 // sweep over the scores is skipped, and the counts are cleared for the next round.
@@ -16,7 +22,10 @@ constexpr int kThreads = 1024;
 constexpr int kBins = kScoreBins;
 static_assert(kBins == 2 * kThreads, "two bins per thread");
 constexpr int kItems = 8;  // consecutive candidates per thread in the compaction sweep
-constexpr int kCap = 4096; // candidates of the first pass's threshold bin kept in shared memory
+constexpr int kCap = 6144; // candidates (score, position) kept in shared memory
+constexpr int kMapWords = 4096;  // position bitmap: contexts up to 128 K keys
+static_assert(kMapWords == 4 * kThreads, "at most four bitmap words per thread");
+constexpr size_t kDynSmem = (size_t)(2 * kCap + kMapWords) * 4;
 
 // Exclusive block-wide prefix sum of one int per thread; `total` gets the block sum.
 __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& total)
@@ -47,7 +56,7 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tmp, int& t
     return warp_tmp[warp] + inc - x;
 }
 
-// Calls f(bits) for every candidate of [lo, hi): eight loads per thread are in flight before the first
+// Calls f(bits, position) for every candidate of [lo, hi): eight loads per thread are in flight before the first
 // is used (a loop of one load and one atomic per trip would pay the memory latency on every trip).
 template <typename F>
 __device__ __forceinline__ void sweep(const uint32_t* __restrict__ st, int lo, int hi, F f)
@@ -58,7 +67,7 @@ __device__ __forceinline__ void sweep(const uint32_t* __restrict__ st, int lo, i
         for (int k = 0; k < 8; ++k) u[k] = base + k * kThreads < hi ? __ldg(st + base + k * kThreads) : 0u;
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-            if (base + k * kThreads < hi) f(u[k]);
+            if (base + k * kThreads < hi) f(u[k], base + k * kThreads);
     }
 }
 
@@ -71,7 +80,10 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     __shared__ int hist[kBins];
     __shared__ int warp_tmp[33];
     __shared__ int sh_bucket, sh_above, sh_count, list_n;
-    __shared__ uint32_t list[kCap];
+    extern __shared__ uint32_t dyn_smem[];
+    uint32_t* list = dyn_smem;                                // [kCap] score bit patterns
+    int* lpos = reinterpret_cast<int*>(dyn_smem + kCap);      // [kCap] their positions
+    uint32_t* bitmap = dyn_smem + 2 * kCap;                   // [kMapWords] chosen positions
 
     const int64_t prob = blockIdx.x;
     const int b = (int)((prob / n_kv_heads) % batch);
@@ -120,6 +132,29 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     int need = k_mid;  // how many to take among candidates matching the decided prefix
     int n_list = 0;
     bool use_list = false;
+    const bool map_ok = hi <= kMapWords * 32;
+    const int map_words = map_ok ? (hi + 31) >> 5 : 0;
+    const int wpt = (map_words + kThreads - 1) / kThreads;  // bitmap words per thread (consecutive ones)
+    // walks the buckets of `hist` from the largest digit down (thread t owns reversed bins 2t, 2t+1) and
+    // leaves the one in which the running count reaches `want`; false if the counts do not reach it
+    auto find_bucket = [&](int nb, int want) -> bool {
+        const int j0 = 2 * tid, j1 = 2 * tid + 1;
+        const int c0 = j0 < nb ? hist[nb - 1 - j0] : 0;
+        const int c1 = j1 < nb ? hist[nb - 1 - j1] : 0;
+        int total;
+        const int ex = block_exclusive_scan(c0 + c1, warp_tmp, total);
+        if (ex < want && want <= ex + c0) {
+            sh_bucket = nb - 1 - j0;
+            sh_above = ex;
+            sh_count = c0;
+        } else if (ex + c0 < want && want <= ex + c0 + c1) {
+            sh_bucket = nb - 1 - j1;
+            sh_above = ex + c0;
+            sh_count = c1;
+        }
+        __syncthreads();
+        return total >= want;
+    };
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
         const int nb = pass == 2 ? 1024 : 2048;
@@ -137,43 +172,52 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
                     const uint32_t u = list[i];
                     if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
                 }
+            } else if (pass == 0) {
+                // The first trip (8 K candidates) is counted in full; the bin in which ITS count reaches
+                // k_mid bounds the threshold's bin from below, so the remaining trips count only what
+                // lies at or above it: a few percent of the candidates instead of all of them (the
+                // counts below the threshold's bin are never looked at).
+                const int mid = min(hi, lo + 8 * kThreads);
+                sweep(st, lo, mid, [&](uint32_t u, int) { atomicAdd(&hist[u >> 21], 1); });
+                if (mid < hi) {
+                    __syncthreads();
+                    const uint32_t floor_bin = find_bucket(nb, need) ? (uint32_t)sh_bucket : 0u;
+                    sweep(st, mid, hi, [&](uint32_t u, int) {
+                        if ((u >> 21) >= floor_bin) atomicAdd(&hist[u >> 21], 1);
+                    });
+                }
             } else {
-                sweep(st, lo, hi, [&](uint32_t u) {
+                sweep(st, lo, hi, [&](uint32_t u, int) {
                     if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & (nb - 1)], 1);
                 });
             }
         }
         __syncthreads();
-        // walk the buckets from the largest digit down: thread t owns reversed bins 2t, 2t+1
-        const int j0 = 2 * tid, j1 = 2 * tid + 1;
-        const int c0 = j0 < nb ? hist[nb - 1 - j0] : 0;
-        const int c1 = j1 < nb ? hist[nb - 1 - j1] : 0;
-        int total;
-        const int ex = block_exclusive_scan(c0 + c1, warp_tmp, total);
-        if (ex < need && need <= ex + c0) {
-            sh_bucket = nb - 1 - j0;
-            sh_above = ex;
-            sh_count = c0;
-        } else if (ex + c0 < need && need <= ex + c0 + c1) {
-            sh_bucket = nb - 1 - j1;
-            sh_above = ex + c0;
-            sh_count = c1;
-        }
-        __syncthreads();
+        find_bucket(nb, need);
         prefix |= (uint32_t)sh_bucket << shift;
         mask |= (uint32_t)(nb - 1) << shift;
         need -= sh_above;
+        const int in_bucket = sh_count;
         __syncthreads();
-        if (pass == 0 && sh_count <= kCap) {
+        if (pass == 0 && in_bucket <= kCap) {
             // One sweep collects the candidates of the threshold's bin (usually a few hundred of the tens
-            // of thousands); the two remaining digits are then decided on that list instead of by two
-            // more sweeps over all scores.  A bin too full for the list (flat scores) keeps the sweeps.
+            // of thousands) with their positions and marks everything above that bin in the position
+            // bitmap; the two remaining digits are then decided on the list instead of by two more
+            // sweeps over all scores.  A bin too full for the list (flat scores) keeps the sweeps.
             if (tid == 0) list_n = 0;
+            for (int i = tid; i < map_words; i += kThreads) bitmap[i] = 0u;
             __syncthreads();
-            sweep(st, lo, hi, [&](uint32_t u) {
-                if ((u & mask) == prefix) {
+            const uint32_t bucket = prefix >> 21;
+            sweep(st, lo, hi, [&](uint32_t u, int pos) {
+                const uint32_t bin = u >> 21;
+                if (bin == bucket) {
                     const int at = atomicAdd(&list_n, 1);
-                    if (at < kCap) list[at] = u;
+                    if (at < kCap) {
+                        list[at] = u;
+                        lpos[at] = pos;
+                    }
+                } else if (bin > bucket && map_ok) {
+                    atomicOr(&bitmap[pos >> 5], 1u << (pos & 31));
                 }
             });
             __syncthreads();
@@ -183,7 +227,61 @@ select_recall_kernel(const float* __restrict__ stats, int64_t stat_stride, int b
     }
     const uint32_t thr = prefix;  // take every candidate > thr and the first `need` equal to it
 
-    // ---- ordered compaction over the candidate span ----
+    bool off_map = use_list && map_ok;
+    int n_eq = 0;
+    int* eqpos = hist;  // the tie positions reuse the histogram's storage
+    if (off_map) {
+        // list entries above the threshold join the bitmap; the ties (bit pattern equal to the
+        // threshold) are set aside
+        if (tid == 0) list_n = 0;
+        __syncthreads();
+        for (int i = tid; i < n_list; i += kThreads) {
+            const uint32_t u = list[i];
+            const int pos = lpos[i];
+            if (u > thr) {
+                atomicOr(&bitmap[pos >> 5], 1u << (pos & 31));
+            } else if (u == thr) {
+                const int at = atomicAdd(&list_n, 1);
+                if (at < kBins) eqpos[at] = pos;
+            }
+        }
+        __syncthreads();
+        n_eq = list_n;
+        off_map = n_eq <= kBins;  // (thousands of equal scores: the ordered compaction below handles them)
+    }
+    if (off_map) {
+        // ---- the index set off the bitmap ----
+        // the ties are ranked by position among themselves and the lowest `need` join
+        for (int i = tid; i < n_eq; i += kThreads) {
+            const int pos = eqpos[i];
+            int rank = 0;
+            if (n_eq > need)
+                for (int j = 0; j < n_eq; ++j) rank += eqpos[j] < pos ? 1 : 0;
+            if (rank < need) atomicOr(&bitmap[pos >> 5], 1u << (pos & 31));
+        }
+        __syncthreads();
+        uint32_t w[4];
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            w[k] = (k < wpt && wpt * tid + k < map_words) ? bitmap[wpt * tid + k] : 0u;
+            cnt += __popc(w[k]);
+        }
+        int total;
+        int at = k_sink + block_exclusive_scan(cnt, warp_tmp, total);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t m = w[k];
+            while (m) {
+                const int bit = __ffs(m) - 1;
+                m &= m - 1;
+                out[at++] = (wpt * tid + k) * 32 + bit;
+            }
+        }
+        return;
+    }
+
+    // ---- ordered compaction over the candidate span (flat scores or very long contexts) ----
     // One block scan per trip: the counts of "above the threshold" (high half) and "equal to it" (low
     // half) travel in one word; a candidate's slot is (candidates above it so far) + (equal ones so far,
     // capped at the number still needed).
@@ -238,7 +336,16 @@ int select_launch(const float* stats, int64_t stat_stride, int n_layers, int bat
                   int32_t* n_indices, uint32_t* hist, const int32_t* hist_len, cudaStream_t stream)
 {
     const long probs = (long)n_layers * batch * n_kv_heads;
-    select_recall_kernel<<<(unsigned)probs, kThreads, 0, stream>>>(
+    static bool opted_in[64] = {};  // per device: the kernel's dynamic shared memory exceeds the default limit
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPEC_ERR_CUDA;
+    if (!opted_in[dev]) {
+        if (cudaFuncSetAttribute(select_recall_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem) !=
+            cudaSuccess)
+            return SPEC_ERR_CUDA;
+        opted_in[dev] = true;
+    }
+    select_recall_kernel<<<(unsigned)probs, kThreads, kDynSmem, stream>>>(
         stats, stat_stride, batch, n_kv_heads, sel_len, k_sink, k_recent, k_total, indices, n_indices, hist, hist_len);
     count_launch(1);
     return cudaGetLastError() == cudaSuccess ? SPEC_OK : SPEC_ERR_CUDA;

@@ -194,6 +194,23 @@ def test_select_bit_exact_random_and_tied_scores(T, k_sink, k_recent, k_total):
     check_select(tiny, sel_len, k_sink, k_recent, k_total)
 
 
+@pytest.mark.parametrize("T,n_tied", [
+    (20000, 40), (20000, 1500), (20000, 3000), (20000, 9000), (131072 + 64, 40), (140000, 40), (140000, 3000),
+])
+def test_select_ties_at_the_threshold_and_long_contexts(T, n_tied):
+    """The threshold's score repeated n_tied times (a handful: ranked by position in shared memory;
+    thousands: the ordered compaction), and contexts on both sides of the position bitmap's reach."""
+    g = torch.Generator(device="cuda").manual_seed(T + n_tied)
+    L, B, H = 1, 2, 2
+    k_sink, k_recent, k_total = 4, 64, 2048
+    sel_len = torch.tensor([T, T - 7], dtype=torch.int32, device="cuda")
+    stats = torch.rand(L, B, H, T, generator=g, device="cuda") ** 6
+    kth = stats[..., k_sink:T - k_recent - 7].topk(k_total - k_sink - k_recent, dim=-1).values[..., -1:]
+    where = torch.rand(L, B, H, T, generator=g, device="cuda").argsort(dim=-1)[..., :n_tied]
+    stats.scatter_(-1, where, kth.expand(L, B, H, n_tied).contiguous())
+    check_select(stats, sel_len, k_sink, k_recent, k_total)
+
+
 def test_select_on_gpu_statistic_and_end_to_end_overlap():
     cfg = inputs.baseline_configs()["cfg1_tiny"]
     case = inputs.make_case(cfg, device="cuda")
