@@ -26,6 +26,9 @@ K3 = 8  # speculation length of the third workload (--k3)
 METRIC = "us_per_spec_step"
 UNIT = "us"
 
+IMPL_NAMES = {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
+              5: "tcgen05 score-cache, rows in two passes"}
+
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/ (not measured inside this run: ncu cannot run under the timed
 # region), for the per-layer launches of the headline workload, with the file and the source
@@ -334,8 +337,7 @@ def other_workloads(peak, dev, layers=4, steps=5):
     out = {}
     jobs = [("cfg3_8b_128k", 1), ("cfg3_8b_128k", 8), ("cfg3_8b_128k", 16), ("cfg4_ragged_paged", None),
             ("cfg5_32b_64k", None)]
-    impl_names = {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
-                  5: "tcgen05 score-cache, rows in two passes"}
+    impl_names = IMPL_NAMES
     for name, k in jobs:
         full = inputs.baseline_configs(k if k is not None else 8)[name]
         cfg = dataclasses.replace(full, n_layers=layers)
@@ -383,6 +385,27 @@ def fp8_draft_workload(peak, dev, layers=4, steps=5):
         run._layers = [kv8.layer_slice(l, l + 1) for l in range(n_layers)]
         run.draft_phase()
         torch.cuda.synchronize()
+        v_us = v_impl = None
+        if not fold:
+            # verification over the 8-bit cache: its workspace also holds the bf16 expansion of a layer
+            saved = (run.ws_v, run.out_v.clone(), run.stats.clone())
+            run.ws_v = binding.alloc_workspace(
+                binding.workspace_bytes(binding.WS_VERIFY, run._layers[0], cfg.n_q, run.max_ctx), dev)
+            for _ in range(2):
+                run.verify_phase()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                run.verify_phase()
+            e1.record()
+            torch.cuda.synchronize()
+            v_us = e0.elapsed_time(e1) * 1e3 / steps / n_layers
+            v_impl = IMPL_NAMES.get(binding.last_verify_impl(), "?")
+            v_status = binding.read_status(run.ws_v)
+            run.ws_v = saved[0]
+            run.out_v.copy_(saved[1])
+            run.stats.copy_(saved[2])
         g = torch.cuda.CUDAGraph()
         before = binding.launch_count()
         with torch.cuda.graph(g):
@@ -404,6 +427,10 @@ def fp8_draft_workload(peak, dev, layers=4, steps=5):
             "draft_us_per_call": us / n_launch, "draft_bytes_per_call": nbytes // n_launch,
             "draft_GBs": nbytes / us / 1e3, "draft_frac": nbytes / us / 1e3 / peak,
             "status": binding.read_status(run.ws_d)}
+        if v_us is not None:
+            out["cfg2_8b_32k_fp8_draft"].update({
+                "verify_us_per_layer": v_us, "verify_impl": v_impl + " on a bf16 expansion of the layer",
+                "verify_status": v_status})
         del run, case, kv8, g
         torch.cuda.empty_cache()
     return out
@@ -567,8 +594,7 @@ def run_gpu(args):
         "data": "synthetic", "config": config_json(cfg, world),
         "phases_us": {"verify": phase_ms[0] * 1e3, "select": phase_ms[1] * 1e3,
                       "draft": phase_ms[2] * 1e3},
-        "verify_impl": {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
-                        5: "tcgen05 score-cache, rows in two passes"}.get(
+        "verify_impl": IMPL_NAMES.get(
             binding.last_verify_impl()),
         "roofline": {
             "kernel": "verification attention + Eq.3 statistic (per-layer launch)",

@@ -100,9 +100,14 @@ typedef struct {
  * Sec. 1, so an 8-bit cache halves the bytes of every call) Q stays bf16 and all results are those of
  * the same attention on the dequantised values.  Served by the sparse draft attention kernel
  * (tensor cores on fp16 copies of the rows, which hold e4m3 values exactly; Q is converted to fp16:
- * exact for magnitudes in [6.1e-5, 65504], absolute error <= 3e-8 below that) and by the generic
- * verification kernels; the tcgen05 verification kernels take bf16 caches only, so spec_verify_attn
- * with an 8-bit cache always runs the generic kernels. */
+ * exact for magnitudes in [6.1e-5, 65504], absolute error <= 3e-8 below that).  Verification: the pages
+ * the contexts reach are expanded to bf16 (exact, scales left out) in the tail of the workspace and
+ * streamed by the tensor-core score-cache kernel, which multiplies K's scale into the softmax scale and
+ * V's into the output; spec_workspace_bytes(SPEC_WS_VERIFY, ...) of an 8-bit cache therefore includes
+ * 4 bytes per cache element of the view (K and V).  A workspace without that room (at least the size
+ * for the same view as bf16), a layout whose pages or layers interleave, a per-attention-head or
+ * group-max statistic, or a shape outside the score-cache kernel runs the generic FP32 kernels on the
+ * bytes instead (correct, many times slower). */
 enum { SPEC_KV_BF16 = 0, SPEC_KV_FP8_E4M3 = 1 };
 
 /*

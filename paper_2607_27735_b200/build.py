@@ -16,7 +16,7 @@ OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libspec_attn.so")
 SOURCES = ["spec_api.cu", "verify_generic.cu", "verify_sm100.cu", "verify_sm100_twosweep.cu",
            "verify_sm100_cached.cu", "select_recall.cu", "draft_stream.cu", "spec_noalloc.cu",
-           "length_ctrl.cu"]
+           "length_ctrl.cu", "kv_expand.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
               "-I", CSRC]

@@ -98,6 +98,25 @@ static int make_view(const spec_kv_t* kv, KvView* out)
     return SPEC_OK;
 }
 
+// The bf16 twin of an 8-bit view: same strides, page table and scales, data pointers filled in by the caller.
+static KvView bf16_twin(const KvView& kv)
+{
+    KvView t = kv;
+    t.fp8 = 0;
+    t.k8 = nullptr;
+    t.v8 = nullptr;
+    return t;
+}
+
+// Workspace of a verification call over an 8-bit cache: [0, base) as for any call (base = the larger of the
+// generic kernels' and the tensor-core kernels' needs on the bf16 twin), then the twin's K and V.
+static size_t fp8_verify_base(const KvView& kv, int n_q, int max_ctx_len)
+{
+    const size_t g = verify_generic_workspace(kv, n_q, max_ctx_len);
+    const size_t f = verify_sm100_workspace(bf16_twin(kv), n_q, max_ctx_len);
+    return ((g > f ? g : f) + 255) & ~(size_t)255;
+}
+
 static int sm100_variant(int impl)
 {
     return impl == SPEC_VERIFY_TCGEN05_TWOSWEEP ? 1 : (impl == SPEC_VERIFY_TCGEN05_CACHED ? 2 : 0);
@@ -166,10 +185,32 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const long hist_probs = (long)kv->n_layers * kv->batch * (a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads);
     const int hist_heads = a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads;
-    const int impl = a.kv.fp8 ? (int)SPEC_VERIFY_GENERIC : g_verify_impl.load();  // 8-bit cache: generic kernels
-    if (impl != SPEC_VERIFY_GENERIC) {
+    const int impl = g_verify_impl.load();
+    // 8-bit cache: expanded to bf16 in the tail of the workspace (when the caller sized it with
+    // spec_workspace_bytes and the layout allows) and streamed by the score-cache kernel, which applies the
+    // scales; otherwise the generic kernels read the bytes directly
+    VerifyArgs twin = a;
+    bool fast_ok = !a.kv.fp8;
+    if (a.kv.fp8 && impl != SPEC_VERIFY_GENERIC && kv_expand_supported(a.kv)) {
+        const size_t base = fp8_verify_base(a.kv, n_q, max_ctx_len);
+        const size_t elems = (size_t)kv_expand_elems(a.kv);
+        if (workspace_bytes >= base + 4 * elems) {
+            __nv_bfloat16* k16 = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + base);
+            twin.kv = bf16_twin(a.kv);
+            twin.kv.k = k16;
+            twin.kv.v = k16 + elems;
+            twin.workspace_bytes = base;
+            fast_ok = verify_sm100_can_run(twin, sm100_variant(impl));
+            if (fast_ok) {
+                const int rc1 = kv_expand_launch(a.kv, k16, k16 + elems, ctx_len, max_ctx_len,
+                                                 static_cast<int*>(workspace), stream);
+                if (rc1 != SPEC_OK) return rc1;
+            }
+        }
+    }
+    if (impl != SPEC_VERIFY_GENERIC && fast_ok) {
         int used = 0;
-        const int rc2 = verify_sm100_launch(a, sm100_variant(impl), stream, &used);
+        const int rc2 = verify_sm100_launch(twin, sm100_variant(impl), stream, &used);
         if (rc2 == SPEC_OK) {
             g_last_verify_impl.store(used == 3   ? SPEC_VERIFY_TCGEN05_CACHED_2PASS
                                      : used == 2 ? SPEC_VERIFY_TCGEN05_CACHED
@@ -273,6 +314,9 @@ size_t spec_workspace_bytes(int which, const spec_kv_t* kv, int32_t n_q, int32_t
     if (make_view(kv, &v) != SPEC_OK) return 0;
     if (which == SPEC_WS_VERIFY) {
         if (n_q < 1 || n_q > 32 || max_ctx_len < n_q) return 0;
+        // 8-bit cache: room for its bf16 copy behind the usual workspace (4 bytes per cache element of the view)
+        if (v.fp8 && kv_expand_supported(v))
+            return fp8_verify_base(v, n_q, max_ctx_len) + 4 * (size_t)kv_expand_elems(v);
         size_t g = verify_generic_workspace(v, n_q, max_ctx_len);
         size_t f = verify_sm100_workspace(v, n_q, max_ctx_len);
         return g > f ? g : f;

@@ -141,6 +141,13 @@ __device__ __forceinline__ int clamped_ctx_len(const VerifyArgs& a, int b)
 }
 
 size_t verify_generic_workspace(const KvView& kv, int n_q, int max_ctx_len);
+
+// 8-bit cache -> bf16 copy with the same strides (kv_expand.cu): elements per tensor, whether the view's
+// layout allows it, and the launch (pages up to each sequence's context only; scales are not applied)
+int64_t kv_expand_elems(const KvView& kv);
+bool kv_expand_supported(const KvView& kv);
+int kv_expand_launch(const KvView& kv, __nv_bfloat16* k_out, __nv_bfloat16* v_out, const int32_t* ctx_len,
+                     int max_ctx_len, int* status, cudaStream_t stream);
 int verify_generic_launch(const VerifyArgs& a, cudaStream_t stream);
 
 int select_launch(const float* stats, int64_t stat_stride, int n_layers, int batch, int n_kv_heads,

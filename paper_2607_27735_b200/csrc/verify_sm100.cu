@@ -266,8 +266,28 @@ size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
     return best;
 }
 
+// Whether verify_sm100_launch would accept these arguments (same decisions, nothing launched).
+bool verify_sm100_can_run(const VerifyArgs& a, int variant)
+{
+    const bool scaled = a.kv.k_scale || a.kv.v_scale;
+    if (scaled && (a.stat_per_head || a.stat_group_max)) return false;  // no such instance of the kernel
+    if (a.stat_per_head || a.stat_group_max) {
+        const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
+        Plan pl;
+        if (variant == 1 || G > 8 || !make_plan(a.kv, a.n_q, a.max_ctx_len, 2, &pl)) return false;
+        variant = 2;
+    }
+    SplitPlan sp;
+    if (variant == 0 && make_split_plan(a.kv, a.n_q, a.max_ctx_len, &sp)) return a.workspace_bytes >= sp.total;
+    Plan pl;
+    if (!make_plan(a.kv, a.n_q, a.max_ctx_len, variant, &pl)) return false;
+    if ((a.kv.k_scale || a.kv.v_scale) && !pl.cached) return false;
+    return a.workspace_bytes >= pl.total;
+}
+
 int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant)
 {
+    if ((a.kv.k_scale || a.kv.v_scale) && (a.stat_per_head || a.stat_group_max)) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.stat_per_head || a.stat_group_max) {
         // only the score-cache kernel keeps one score per attention head, for groups of up to 8;
         // everything else goes to the generic kernels
@@ -317,6 +337,8 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     }
     Plan pl;
     if (!make_plan(a.kv, a.n_q, a.max_ctx_len, variant, &pl)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    // per-(layer, KV head) scales (an 8-bit cache expanded to bf16): only the score-cache kernel applies them
+    if ((a.kv.k_scale || a.kv.v_scale) && !pl.cached) return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.workspace_bytes < pl.total) return SPEC_ERR_WORKSPACE_TOO_SMALL;
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     const int n_pages = a.kv.n_pages;

@@ -103,7 +103,7 @@ struct CBars {  // mbarrier addresses (shared space)
 // LP: the publisher warp combines the LSE partials (few CTAs per head); otherwise the softmax warps do.
 // PH: one Eq. 3 score per attention head (stats [.., n_q_heads, stride]) instead of per KV head,
 // for groups of at most 8 heads (a short statistic pass when the group size divides 8).
-template <int NC, int CG, bool LP, bool PH>
+template <int NC, int CG, bool LP, bool PH, bool SC>
 __global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_q, const FastParams p)
@@ -539,7 +539,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const int stat_r0 = p.a.first_stat_row * G;
         const bool ph_fast = (8 % G) == 0;  // per-head statistic: column i of a 16-column chunk is head i mod 8 mod G
-        const float cs = p.scale_log2;
+        const float cs0 = p.scale_log2;
+        float vsc = 1.f;  // SC: scale of this unit's V
         constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
         uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, sfull_par = 0;
         bool ok = true;
@@ -563,7 +564,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     const int r = c0 + i;
                     if (r < R)
                         p.o_part[obase + (int64_t)r * kD + key_l] =
-                            (__uint_as_float(v[i]) + __uint_as_float(w[i])) * fac_s[r];
+                            (__uint_as_float(v[i]) + __uint_as_float(w[i])) * (SC ? fac_s[r] * vsc : fac_s[r]);
                 }
             } else {
                 for (int i = tid_s; i < R * kD; i += 128 * CG) p.o_part[obase + i] = 0.f;
@@ -577,6 +578,14 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             const Seg sg = get_seg(p, unit, head_local, rank);
             const int n_t = sg.t1 - sg.t0;
             const bool nonempty = n_t > 0;
+            // SC (an 8-bit cache expanded to bf16 without its scales): K's per-(layer, KV head) scale joins
+            // the softmax scale, V's the output
+            float cs = cs0;
+            if (SC) {
+                const int64_t sh = (int64_t)sg.layer * p.a.kv.n_kv_heads + sg.h;
+                if (p.a.kv.k_scale) cs *= __ldg(p.a.kv.k_scale + sh);
+                vsc = p.a.kv.v_scale ? __ldg(p.a.kv.v_scale + sh) : 1.f;
+            }
             // ------------------------------ P1 ------------------------------
             float m[NH], l[NH];
 #pragma unroll
@@ -949,11 +958,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
-template <int NC, int CG, bool LP, bool PH>
+template <int NC, int CG, bool LP, bool PH, bool SC>
 int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    auto kern = verify_cached_kernel<NC, CG, LP, PH>;
+    auto kern = verify_cached_kernel<NC, CG, LP, PH, SC>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -999,12 +1008,18 @@ int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMa
                   int grid, size_t smem_bytes, cudaStream_t stream)
 {
     const bool lp = fp.cph <= kLsePubMax, ph = fp.a.stat_per_head != 0 || fp.a.stat_group_max != 0;
-#define SPEC_CASE(n, nc, cg)                                                                              \
-    case n:                                                                                               \
-        if (ph) return lp ? launch_cfg<nc, cg, true, true>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
-                          : launch_cfg<nc, cg, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
-        return lp ? launch_cfg<nc, cg, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream)             \
-                  : launch_cfg<nc, cg, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+    // per-(layer, KV head) scales: instances of their own (the bf16 instances carry no code for them),
+    // built for the per-KV-head statistic only
+    const bool sc = fp.a.kv.k_scale != nullptr || fp.a.kv.v_scale != nullptr;
+    if (sc && ph) return SPEC_ERR_UNSUPPORTED_SHAPE;
+#define SPEC_CASE(n, nc, cg)                                                                                     \
+    case n:                                                                                                      \
+        if (sc) return lp ? launch_cfg<nc, cg, true, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
+                          : launch_cfg<nc, cg, false, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
+        if (ph) return lp ? launch_cfg<nc, cg, true, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
+                          : launch_cfg<nc, cg, false, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
+        return lp ? launch_cfg<nc, cg, true, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream)             \
+                  : launch_cfg<nc, cg, false, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
     switch (fp.N) {  // (columns per warpgroup, warpgroups)
         SPEC_CASE(16, 8, 2)
         SPEC_CASE(32, 8, 4)

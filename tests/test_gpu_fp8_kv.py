@@ -1,5 +1,6 @@
-"""8-bit (e4m3) KV cache as a second workload of the path: verification (generic kernels), selection and
-the sparse draft kernel's fp8 instance against the oracle on the same bytes and scales, within the
+"""8-bit (e4m3) KV cache as a second workload of the path: verification (the score-cache kernel on a bf16
+expansion of the cache, with the scales applied in the kernel; the generic kernels on the bytes), selection
+and the sparse draft kernel's fp8 instance against the oracle on the same bytes and scales, within the
 2e-3 bar of the bf16 path."""
 import pytest
 import torch
@@ -31,15 +32,25 @@ def test_fp8_cache_path_matches_the_oracle(shape):
     kv8_cpu = kv8.cpu()
     ctx = case.ctx_len
     T = int(ctx.max())
-    out, lse, stats, ws = binding.spec_verify_attn(kv8, case.q_verify, ctx, T)
-    assert binding.read_status(ws) == 0
-    assert binding.last_verify_impl() == binding.VERIFY_GENERIC  # the tcgen05 kernels take bf16 caches only
-    o_out, o_lse, o_stats = oracle.verify_attn(kv8_cpu, case.q_verify.cpu(), ctx.cpu(), 16, stats.shape[-1])
-    assert (out.cpu().double() - o_out).abs().max().item() <= TOL
-    assert (lse.cpu().double() - o_lse).abs().max().item() <= TOL
-    for b in range(cfg.batch):
-        t = int(ctx[b])
-        assert (stats[:, b, :, :t].cpu().double() - o_stats[:, b, :, :t]).abs().max().item() <= TOL
+    o_out = o_lse = o_stats = None
+    for impl in (binding.VERIFY_GENERIC, binding.VERIFY_AUTO):
+        binding.set_verify_impl(impl)
+        try:
+            out, lse, stats, ws = binding.spec_verify_attn(kv8, case.q_verify, ctx, T)
+        finally:
+            binding.set_verify_impl(binding.VERIFY_AUTO)
+        assert binding.read_status(ws) == 0
+        if impl == binding.VERIFY_GENERIC:
+            assert binding.last_verify_impl() == binding.VERIFY_GENERIC
+        else:  # every shape of this list fits the score-cache kernel
+            assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+        if o_out is None:
+            o_out, o_lse, o_stats = oracle.verify_attn(kv8_cpu, case.q_verify.cpu(), ctx.cpu(), 16, stats.shape[-1])
+        assert (out.cpu().double() - o_out).abs().max().item() <= TOL
+        assert (lse.cpu().double() - o_lse).abs().max().item() <= TOL
+        for b in range(cfg.batch):
+            t = int(ctx[b])
+            assert (stats[:, b, :, :t].cpu().double() - o_stats[:, b, :, :t]).abs().max().item() <= TOL
     idx, n = binding.spec_select_recall(stats, ctx, cfg.k_sink, cfg.k_recent, cfg.k_total)
     o_idx, o_n = oracle.select_recall(stats.cpu(), ctx.cpu(), cfg.k_sink, cfg.k_recent, cfg.k_total)
     assert torch.equal(idx.cpu(), o_idx) and torch.equal(n.cpu(), o_n)
@@ -52,6 +63,36 @@ def test_fp8_cache_path_matches_the_oracle(shape):
         assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL, step
         fin = torch.isfinite(r_lse)
         assert ((d_lse.cpu().double() - r_lse)[fin]).abs().max().item() <= TOL
+
+
+def test_fp8_verify_with_scales_that_are_not_powers_of_two_and_a_short_workspace():
+    """The expansion to bf16 leaves the scales out (a scaled value need not be a bf16 value) and the kernel
+    applies them per (layer, KV head); a workspace without room for the expansion falls back to the
+    generic kernels."""
+    import dataclasses
+    cfg = inputs.small_config(ctx=(700, 1900), n_q=9, batch=2, n_layers=2, n_q_heads=8, n_kv_heads=2,
+                              page_size=16, shuffled_pages=True)
+    case = inputs.make_case(cfg, device="cuda")
+    kv8 = inputs.quantize_kv_fp8(case.kv)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    kv8 = dataclasses.replace(
+        kv8, k_scale=kv8.k_scale * (0.7 + 0.6 * torch.rand(kv8.k_scale.shape, generator=g, device="cuda")),
+        v_scale=kv8.v_scale * (0.7 + 0.6 * torch.rand(kv8.v_scale.shape, generator=g, device="cuda")))
+    ctx = case.ctx_len
+    o_out, o_lse, o_stats = oracle.verify_attn(kv8.cpu(), case.q_verify.cpu(), ctx.cpu(), 16, 1900)
+    full = binding.workspace_bytes(binding.WS_VERIFY, kv8, cfg.n_q, 1900)
+    base = binding.workspace_bytes(binding.WS_VERIFY, case.kv, cfg.n_q, 1900)
+    assert full > base
+    for nbytes, want in ((full, binding.VERIFY_TCGEN05_CACHED), (base, binding.VERIFY_GENERIC)):
+        ws = binding.alloc_workspace(nbytes, "cuda")
+        out, lse, stats, _ = binding.spec_verify_attn(kv8, case.q_verify, ctx, 1900, workspace=ws)
+        assert binding.read_status(ws) == 0
+        assert binding.last_verify_impl() == want
+        assert (out.cpu().double() - o_out).abs().max().item() <= TOL
+        assert (lse.cpu().double() - o_lse).abs().max().item() <= TOL
+        for b in range(cfg.batch):
+            t = int(ctx[b])
+            assert (stats[:, b, :, :t].cpu().double() - o_stats[:, b, :, :t]).abs().max().item() <= TOL
 
 
 def test_fp8_draft_per_head_sets_and_bf16_output():
