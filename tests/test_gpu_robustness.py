@@ -97,6 +97,36 @@ def test_generic_verify_reports_a_bad_page_entry():
         binding.set_verify_impl(prev)
 
 
+def test_verify_over_an_8bit_cache_reports_bad_lengths_and_page_entries():
+    """The expansion of an 8-bit cache into the workspace follows the same rules: a page-table entry
+    outside the pool is replaced and reported, a length beyond the host bound is clamped, and nothing is
+    written outside the workspace's tail."""
+    cfg = inputs.small_config(ctx=(500, 700), n_q=5, batch=2, page_size=16, shuffled_pages=True, planted=0)
+    case = inputs.make_case(cfg, device="cuda")
+    kv8 = inputs.quantize_kv_fp8(case.kv)
+    T = int(case.ctx_len.max())
+    longest = int(case.ctx_len.argmax())
+    need = binding.workspace_bytes(binding.WS_VERIFY, kv8, cfg.n_q, T)
+    pad = 4096
+    guard = torch.zeros(need + 2 * pad, dtype=torch.uint8, device="cuda")
+    guard[:pad] = 0x5a
+    guard[-pad:] = 0x5a
+    ws = guard[pad:-pad]
+    assert ws.data_ptr() % 256 == 0
+    ref = binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, T, workspace=ws)
+    assert binding.read_status(ws) == 0 and binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+    bad = dataclasses.replace(kv8, page_table=kv8.page_table.clone())
+    bad.page_table[longest, 3] = kv8.page_table.numel() + 5
+    out, _, _, _ = binding.spec_verify_attn(bad, case.q_verify, case.ctx_len, T, workspace=ws)
+    assert binding.read_status(ws) == BAD_INDEX and torch.isfinite(out).all()
+    assert torch.equal(out[0, 1 - longest], ref[0][0, 1 - longest])  # the other sequence is unaffected
+    too_long = case.ctx_len.clone()
+    too_long[longest] = T + 1
+    out, _, _, _ = binding.spec_verify_attn(kv8, case.q_verify, too_long, T, workspace=ws)
+    assert binding.read_status(ws) == BAD_INDEX and torch.isfinite(out).all()
+    assert (guard[:pad] == 0x5a).all() and (guard[-pad:] == 0x5a).all()
+
+
 def test_advance_lengths_holds_a_sequence_at_the_capacity():
     committed = torch.tensor([100, 990, 500], dtype=torch.int32, device="cuda")
     m = torch.tensor([3, 4, 0], dtype=torch.int32, device="cuda")
