@@ -5,6 +5,7 @@ page layout, layer count and budget from a seeded generator; the draws are bound
 oracle finishes each case in about a second.  The fixed lists in test_gpu_parity.py aim at known
 edges; this file looks for the ones nobody thought of (ragged batches with units that are empty
 for some CTAs, odd group sizes, budgets around the cluster and round boundaries)."""
+import dataclasses
 import random
 
 import pytest
@@ -39,14 +40,21 @@ def draw_shape(seed):
                 seed=100 + seed)
 
 
-@pytest.mark.parametrize("seed", range(32))
-def test_random_shape_end_to_end(seed):
+def run_shape(seed, eight_bit):
     shape = draw_shape(seed)
     if shape["planted"] == 0:
         shape.update(q_mode="iid", q_std=0.3)
     cfg = inputs.small_config(name=f"fuzz{seed}", **shape)
     case = inputs.make_case(cfg, device="cuda")
     kv, ctx = case.kv, case.ctx_len
+    if eight_bit:
+        # e4m3 bytes with one scale per (layer, KV head); every second case scales that are not powers of two
+        kv = inputs.quantize_kv_fp8(kv)
+        if seed % 2:
+            g = torch.Generator(device="cuda").manual_seed(seed)
+            kv = dataclasses.replace(
+                kv, k_scale=kv.k_scale * (0.7 + 0.6 * torch.rand(kv.k_scale.shape, generator=g, device="cuda")),
+                v_scale=kv.v_scale * (0.7 + 0.6 * torch.rand(kv.v_scale.shape, generator=g, device="cuda")))
     # verify + statistic
     out, lse, stats, ws = binding.spec_verify_attn(kv, case.q_verify, ctx, int(ctx.max()))
     assert binding.read_status(ws) == 0, shape
@@ -70,3 +78,13 @@ def test_random_shape_end_to_end(seed):
         assert (d_out.cpu().double() - r_out).abs().max().item() <= TOL, shape
         fin = torch.isfinite(r_lse)
         assert ((d_lse.cpu().double() - r_lse)[fin]).abs().max().item() <= TOL, shape
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shape_end_to_end(seed):
+    run_shape(seed, eight_bit=False)
+
+
+@pytest.mark.parametrize("seed", range(40, 56))
+def test_random_shape_8bit_cache(seed):
+    run_shape(seed, eight_bit=True)
