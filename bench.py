@@ -363,7 +363,7 @@ def other_workloads(peak, dev, layers=4, steps=5):
     return out
 
 
-def fp8_draft_workload(peak, dev, layers=4, steps=5):
+def fp8_draft_workload(peak, dev, layers=4, steps=5, folded=True):
     """The headline shape's drafting phase over an 8-bit (e4m3) copy of the cache: same index sets (built by
     the bf16 verification), half the gathered bytes.  Per layer-call and with the layers folded."""
     import dataclasses
@@ -373,7 +373,7 @@ def fp8_draft_workload(peak, dev, layers=4, steps=5):
     from paper_2607_27735_b200 import binding, inputs, runner
     out = {}
     full = inputs.baseline_configs(8)["cfg2_8b_32k"]
-    for fold, n_layers in ((False, layers), (True, 32)):
+    for fold, n_layers in ((False, layers), (True, 32)) if folded else ((False, layers),):
         cfg = dataclasses.replace(full, n_layers=n_layers)
         case = inputs.make_case(cfg, device=dev)
         run = runner.SpecStepRunner(case, fold_layers=fold)
@@ -689,11 +689,19 @@ def main():
     ap.add_argument("--fused-hist", action="store_true",
                     help="the verification kernel counts the selection's first radix pass (top 11 bits of every "
                          "score) while it writes the statistic; the selection skips that sweep")
+    ap.add_argument("--fp8-only", action="store_true",
+                    help="run only the 8-bit-cache workload of the headline shape (2 layers) and print its figures "
+                         "(a small command for profiler captures; not a bench line)")
     ap.add_argument("--fold-layers", action="store_true",
                     help="issue verify/draft for all layers in one launch (kernel-roofline view)")
     args = ap.parse_args()
     global K3
     K3 = args.k3
+    if args.fp8_only:
+        import torch
+        print(json.dumps(fp8_draft_workload(measured_peaks()[0], torch.device("cuda:0"), layers=2, steps=10,
+                                            folded=False)))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
