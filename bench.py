@@ -27,7 +27,8 @@ METRIC = "us_per_spec_step"
 UNIT = "us"
 
 IMPL_NAMES = {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
-              5: "tcgen05 score-cache, rows in two passes"}
+              5: "tcgen05 score-cache, rows in two passes",
+              6: "tcgen05 score-cache on a bf16 expansion of the cache"}
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/ (not measured inside this run: ncu cannot run under the timed
@@ -387,7 +388,7 @@ def fp8_draft_workload(peak, dev, layers=4, steps=5, folded=True):
         torch.cuda.synchronize()
         v_us = v_impl = None
         if not fold:
-            # verification over the 8-bit cache: its workspace also holds the bf16 expansion of a layer
+            # verification over the 8-bit cache (the workspace is sized for this view)
             saved = (run.ws_v, run.out_v.clone(), run.stats.clone())
             run.ws_v = binding.alloc_workspace(
                 binding.workspace_bytes(binding.WS_VERIFY, run._layers[0], cfg.n_q, run.max_ctx), dev)
@@ -429,7 +430,8 @@ def fp8_draft_workload(peak, dev, layers=4, steps=5, folded=True):
             "status": binding.read_status(run.ws_d)}
         if v_us is not None:
             out["cfg2_8b_32k_fp8_draft"].update({
-                "verify_us_per_layer": v_us, "verify_impl": v_impl + " on a bf16 expansion of the layer",
+                "verify_us_per_layer": v_us, "verify_impl": v_impl + " (tiles expanded to fp16 in shared memory)",
+                "verify_bytes_per_layer": 32768 * 8 * 128 * 2, "verify_frac": 32768 * 8 * 128 * 2 / v_us / 1e3 / peak,
                 "verify_status": v_status})
         del run, case, kv8, g
         torch.cuda.empty_cache()

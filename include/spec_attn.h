@@ -63,8 +63,11 @@ enum {
     SPEC_VERIFY_TCGEN05 = 2,          /* tcgen05, either variant; unsupported shapes are an error */
     SPEC_VERIFY_TCGEN05_TWOSWEEP = 3, /* K swept twice (second sweep from L2), any context length */
     SPEC_VERIFY_TCGEN05_CACHED = 4,   /* score tiles cached in tensor memory, K and V read once */
-    SPEC_VERIFY_TCGEN05_CACHED_2PASS = 5 /* reported only (spec_last_verify_impl): AUTO ran the score-cache kernel
-                                            on two halves of the rows because all rows did not fit the cache */
+    SPEC_VERIFY_TCGEN05_CACHED_2PASS = 5, /* reported only (spec_last_verify_impl): AUTO ran the score-cache kernel
+                                             on two halves of the rows because all rows did not fit the cache */
+    SPEC_VERIFY_TCGEN05_CACHED_EXPANDED = 6 /* reported only: an 8-bit cache was first expanded to bf16 in the
+                                               workspace (the score-cache kernel could not read its bytes itself:
+                                               head_dim 64) */
 };
 
 /*
@@ -100,14 +103,17 @@ typedef struct {
  * Sec. 1, so an 8-bit cache halves the bytes of every call) Q stays bf16 and all results are those of
  * the same attention on the dequantised values.  Served by the sparse draft attention kernel
  * (tensor cores on fp16 copies of the rows, which hold e4m3 values exactly; Q is converted to fp16:
- * exact for magnitudes in [6.1e-5, 65504], absolute error <= 3e-8 below that).  Verification: the pages
- * the contexts reach are expanded to bf16 (exact, scales left out) in the tail of the workspace and
- * streamed by the tensor-core score-cache kernel, which multiplies K's scale into the softmax scale and
- * V's into the output; spec_workspace_bytes(SPEC_WS_VERIFY, ...) of an 8-bit cache therefore includes
- * 4 bytes per cache element of the view (K and V).  A workspace without that room (at least the size
- * for the same view as bf16), a layout whose pages or layers interleave, a per-attention-head or
- * group-max statistic, or a shape outside the score-cache kernel runs the generic FP32 kernels on the
- * bytes instead (correct, many times slower). */
+ * exact for magnitudes in [6.1e-5, 65504], absolute error <= 3e-8 below that).  Verification at
+ * head_dim 128: the tensor-core score-cache kernel streams the bytes and expands each tile to fp16 in
+ * shared memory (exact), with fp16 copies of Q (same range as above) and of the probabilities (two
+ * fp16 terms: relative error below 2^-21), K's scale multiplied into the softmax scale and V's into the
+ * output.  At head_dim 64 the pages the contexts reach are first expanded to bf16 (exact, scales left
+ * out) in the tail of the workspace and streamed by the same kernel's bf16 instances;
+ * spec_workspace_bytes(SPEC_WS_VERIFY, ...) of an 8-bit cache therefore includes 4 bytes per cache
+ * element of the view (K and V).  A workspace without that room (at least the size for the same view
+ * as bf16), a layout whose pages or layers interleave, a per-attention-head or group-max statistic,
+ * or a shape outside the score-cache kernel runs the generic FP32 kernels on the bytes instead
+ * (correct, many times slower). */
 enum { SPEC_KV_BF16 = 0, SPEC_KV_FP8_E4M3 = 1 };
 
 /*
@@ -417,8 +423,8 @@ int spec_set_verify_impl(int impl);
 int64_t spec_set_wait_limit_cycles(int64_t cycles);
 
 /* Which kernel the last spec_verify_attn call of this process used (SPEC_VERIFY_GENERIC,
- * SPEC_VERIFY_TCGEN05_TWOSWEEP, SPEC_VERIFY_TCGEN05_CACHED or SPEC_VERIFY_TCGEN05_CACHED_2PASS; 0 before the
- * first call). */
+ * SPEC_VERIFY_TCGEN05_TWOSWEEP, SPEC_VERIFY_TCGEN05_CACHED, SPEC_VERIFY_TCGEN05_CACHED_2PASS or
+ * SPEC_VERIFY_TCGEN05_CACHED_EXPANDED; 0 before the first call). */
 int spec_last_verify_impl(void);
 
 /*

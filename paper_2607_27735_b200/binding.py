@@ -19,6 +19,8 @@ WS_VERIFY, WS_SELECT, WS_DRAFT = 0, 1, 2
 VERIFY_AUTO, VERIFY_GENERIC, VERIFY_TCGEN05, VERIFY_TCGEN05_TWOSWEEP, VERIFY_TCGEN05_CACHED = 0, 1, 2, 3, 4
 VERIFY_TCGEN05_CACHED_2PASS = 5
 # ^ reported by last_verify_impl() only: the score-cache kernel on two halves of the rows
+VERIFY_TCGEN05_CACHED_EXPANDED = 6
+# ^ reported only: an 8-bit cache expanded to bf16 in the workspace first (head_dim 64)
 VERIFY_ACCUMULATE_STATS = 1  # flag of spec_verify_attn_ex: add to the statistic instead of replacing it
 VERIFY_STATS_PER_QUERY_HEAD = 2  # flag of spec_verify_attn_ex: one score per attention head
 DRAFT_INDICES_PER_QUERY_HEAD = 1  # flag of spec_sparse_draft_attn_ex: one index set per attention head

@@ -24,6 +24,7 @@ struct FastParams {
     VerifyArgs a;
     int HG, NHG, cph, n_units, N, R, G;
     int n_slots, p_bufs;
+    int n_raw;                        // 8-bit cache read directly: raw 16 KB stages in front of the operand slots (else 0)
     int D;                            // head_dim: 128, or 64 (score-cache kernel only)
     int box_rows, boxes;              // TMA boxes per 64-wide half of a tile
     float scale_log2;

@@ -186,12 +186,16 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
     const long hist_probs = (long)kv->n_layers * kv->batch * (a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads);
     const int hist_heads = a.stat_per_head ? kv->n_q_heads : kv->n_kv_heads;
     const int impl = g_verify_impl.load();
-    // 8-bit cache: expanded to bf16 in the tail of the workspace (when the caller sized it with
-    // spec_workspace_bytes and the layout allows) and streamed by the score-cache kernel, which applies the
-    // scales; otherwise the generic kernels read the bytes directly
+    // 8-bit cache: the score-cache kernel reads the bytes itself where its F8 instances apply; else the
+    // cache is expanded to bf16 in the tail of the workspace (when the caller sized it with
+    // spec_workspace_bytes and the layout allows) and streamed by the kernel's scaled instances; else the
+    // generic kernels read the bytes
     VerifyArgs twin = a;
-    bool fast_ok = !a.kv.fp8;
-    if (a.kv.fp8 && impl != SPEC_VERIFY_GENERIC && kv_expand_supported(a.kv)) {
+    bool fast_ok = !a.kv.fp8, expanded = false;
+    if (a.kv.fp8 && impl != SPEC_VERIFY_GENERIC &&
+        verify_sm100_can_run(a, sm100_variant(impl))) {
+        fast_ok = true;
+    } else if (a.kv.fp8 && impl != SPEC_VERIFY_GENERIC && kv_expand_supported(a.kv)) {
         const size_t base = fp8_verify_base(a.kv, n_q, max_ctx_len);
         const size_t elems = (size_t)kv_expand_elems(a.kv);
         if (workspace_bytes >= base + 4 * elems) {
@@ -201,6 +205,7 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
             twin.kv.v = k16 + elems;
             twin.workspace_bytes = base;
             fast_ok = verify_sm100_can_run(twin, sm100_variant(impl));
+            expanded = fast_ok;
             if (fast_ok) {
                 const int rc1 = kv_expand_launch(a.kv, k16, k16 + elems, ctx_len, max_ctx_len,
                                                  static_cast<int*>(workspace), stream);
@@ -212,7 +217,8 @@ int spec_verify_attn_hist(const spec_kv_t* kv, const void* q, int32_t n_q, const
         int used = 0;
         const int rc2 = verify_sm100_launch(twin, sm100_variant(impl), stream, &used);
         if (rc2 == SPEC_OK) {
-            g_last_verify_impl.store(used == 3   ? SPEC_VERIFY_TCGEN05_CACHED_2PASS
+            g_last_verify_impl.store(expanded    ? SPEC_VERIFY_TCGEN05_CACHED_EXPANDED
+                                     : used == 3 ? SPEC_VERIFY_TCGEN05_CACHED_2PASS
                                      : used == 2 ? SPEC_VERIFY_TCGEN05_CACHED
                                                  : SPEC_VERIFY_TCGEN05_TWOSWEEP);
             if (score_hist && used != 2)

@@ -31,7 +31,7 @@ EncodeTiledFn encode_fn()
 
 struct Plan {
     bool cached;
-    int HG, cph, n_units, N, n_slots, p_bufs, box_rows, boxes, n_cache;
+    int HG, cph, n_units, N, n_slots, p_bufs, box_rows, boxes, n_cache, n_raw;
     size_t smem_bytes;
     size_t ctr_off, ctr_bytes, ml_off, o_off, total;
 };
@@ -47,7 +47,9 @@ int box_rows_for(int page_size)
 bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl)
 {
     const int G = kv.n_q_heads / kv.n_kv_heads, R = n_q * G;
-    if (kv.fp8) return false;  // the tcgen05 kernels take bf16 caches only
+    pl->n_raw = 0;
+    // an 8-bit cache is read by the score-cache kernel only (its F8 instances), at head_dim 128
+    if (kv.fp8 && (variant == 1 || kv.head_dim != kD)) return false;
     // head_dim 64 runs on the score-cache kernel only (one 64-wide half per tile, V padded with zero rows)
     if (!(kv.head_dim == kD || (kv.head_dim == 64 && variant != 1)) || R > 128 || G > 256 || n_q > 256) return false;
     const int box_rows = box_rows_for(kv.page_size);
@@ -78,7 +80,7 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         cached = best_hg != 0;
     }
     if (!cached) {
-        if (variant == 2 || kv.head_dim != kD) return false;
+        if (variant == 2 || kv.head_dim != kD || kv.fp8) return false;
         double best = -1.0;
         for (int hg = 1; hg <= kv.n_kv_heads; ++hg) {
             if (kv.n_kv_heads % hg) continue;
@@ -112,7 +114,8 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
         // one Q buffer, two P buffers ([hi | lo] rows, 8-row blocks: 2N * 256 B each), 12.25 KB of
         // barriers and small arrays; the rest is the K/V tile ring
         pl->p_bufs = 2;
-        fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544;
+        pl->n_raw = kv.fp8 ? 3 : 0;  // 8-bit cache: three raw stages of 16 KB in front of the slots
+        fixed = 1024 /*alignment slack*/ + (size_t)N * 256 + 2 * (size_t)(2 * N * 256) + 12544 + (size_t)pl->n_raw * 16384;
         slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
         if (slots > 8) slots = 8;
         // more P buffers (up to four) where they cost no K/V slot: the P V product of a tile then has two tiles
@@ -125,6 +128,20 @@ bool make_plan(const KvView& kv, int n_q, int max_ctx_len, int variant, Plan* pl
             pl->p_bufs = 1;
             fixed -= (size_t)(2 * N * 256);
             slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
+        }
+        if (kv.fp8) {
+            // 8-bit cache: the raw stages already hold whole tiles in flight, so three operand slots do;
+            // P buffers first (the P V product of a tile hides behind the next tiles' softmax work)
+            slots = 0;
+            for (int pb = 3; pb >= 1 && slots < 3; --pb) {
+                for (int nr = 3; nr >= 2 && slots < 3; --nr) {
+                    fixed = 1024 + (size_t)N * 256 + (size_t)pb * (2 * N * 256) + 12544 + (size_t)nr * 16384;
+                    slots = fixed < cap ? (int)((cap - fixed) / kSlotBytes) : 0;
+                    if (slots > 8) slots = 8;
+                    pl->p_bufs = pb;
+                    pl->n_raw = nr;
+                }
+            }
         }
     } else {
         const size_t p_bytes = (size_t)((2 * N + 63) / 64) * 16384;
@@ -168,6 +185,24 @@ bool encode_kv_map(CUtensorMap* map, const void* base, const KvView& kv, int n_p
     for (int i = 0; i < 4; ++i) st[i] = strides[i] ? strides[i] : 16;
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, st, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 8-bit cache: a box is box_rows whole rows of 128 bytes, unswizzled (the softmax warps expand it)
+bool encode_kv_map_u8(CUtensorMap* map, const void* base, const KvView& kv, int n_pages, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[5] = {(cuuint64_t)kv.head_dim, (cuuint64_t)kv.page_size, (cuuint64_t)kv.n_kv_heads,
+                                (cuuint64_t)n_pages, (cuuint64_t)kv.n_layers};
+    const cuuint64_t strides[4] = {(cuuint64_t)kv.slot_stride, (cuuint64_t)kv.head_stride, (cuuint64_t)kv.page_stride,
+                                   (cuuint64_t)kv.layer_stride};
+    const cuuint32_t box[5] = {128, (cuuint32_t)box_rows, 1, 1, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    cuuint64_t st[4];
+    for (int i = 0; i < 4; ++i) st[i] = strides[i] ? strides[i] : 16;
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 5, const_cast<void*>(base), dims, st, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -269,7 +304,7 @@ size_t verify_sm100_workspace(const KvView& kv, int n_q, int max_ctx_len)
 // Whether verify_sm100_launch would accept these arguments (same decisions, nothing launched).
 bool verify_sm100_can_run(const VerifyArgs& a, int variant)
 {
-    const bool scaled = a.kv.k_scale || a.kv.v_scale;
+    const bool scaled = a.kv.k_scale || a.kv.v_scale || a.kv.fp8;
     if (scaled && (a.stat_per_head || a.stat_group_max)) return false;  // no such instance of the kernel
     if (a.stat_per_head || a.stat_group_max) {
         const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
@@ -287,7 +322,8 @@ bool verify_sm100_can_run(const VerifyArgs& a, int variant)
 
 int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, int* used_variant)
 {
-    if ((a.kv.k_scale || a.kv.v_scale) && (a.stat_per_head || a.stat_group_max)) return SPEC_ERR_UNSUPPORTED_SHAPE;
+    if ((a.kv.k_scale || a.kv.v_scale || a.kv.fp8) && (a.stat_per_head || a.stat_group_max))
+        return SPEC_ERR_UNSUPPORTED_SHAPE;
     if (a.stat_per_head || a.stat_group_max) {
         // only the score-cache kernel keeps one score per attention head, for groups of up to 8;
         // everything else goes to the generic kernels
@@ -343,9 +379,15 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     const int G = a.kv.n_q_heads / a.kv.n_kv_heads;
     const int n_pages = a.kv.n_pages;
     CUtensorMap tk, tv, tq;
-    if (!encode_kv_map(&tk, a.kv.k, a.kv, n_pages, pl.box_rows) ||
-        !encode_kv_map(&tv, a.kv.v, a.kv, n_pages, pl.box_rows) || !encode_q_map(&tq, a.q, a.kv, a.n_q, G))
+    if (a.kv.fp8) {
+        if (!encode_kv_map_u8(&tk, a.kv.k8, a.kv, n_pages, pl.box_rows) ||
+            !encode_kv_map_u8(&tv, a.kv.v8, a.kv, n_pages, pl.box_rows))
+            return SPEC_ERR_CUDA;
+    } else if (!encode_kv_map(&tk, a.kv.k, a.kv, n_pages, pl.box_rows) ||
+               !encode_kv_map(&tv, a.kv.v, a.kv, n_pages, pl.box_rows)) {
         return SPEC_ERR_CUDA;
+    }
+    if (!encode_q_map(&tq, a.q, a.kv, a.n_q, G)) return SPEC_ERR_CUDA;
     char* ws = static_cast<char*>(a.workspace);
     FastParams fp;
     fp.a = a;
@@ -362,6 +404,7 @@ int verify_sm100_launch(const VerifyArgs& a, int variant, cudaStream_t stream, i
     fp.G = G;
     fp.D = a.kv.head_dim;
     fp.n_slots = pl.n_slots;
+    fp.n_raw = pl.n_raw;
     fp.p_bufs = pl.p_bufs;
     fp.box_rows = pl.box_rows;
     fp.boxes = pl.boxes;

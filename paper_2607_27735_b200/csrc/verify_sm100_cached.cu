@@ -93,9 +93,20 @@ __device__ __forceinline__ void ml_step(float (&m)[NHT], float (&l)[NHT], int la
     }
 }
 
+// Four e4m3 bytes as two packed fp16 pairs (bytes 0, 1 and bytes 2, 3): exact, subnormals included.
+// (The same by integer instructions - the byte's low seven bits shifted into bits 7..13 of an fp16 give the
+// value times 2^-8 - measured slower: the softmax warps are bound by instruction issue, and that takes four
+// instructions per pair instead of one.)
+__device__ __forceinline__ void e4m3x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t& hi)
+{
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(w));
+}
+
 struct CBars {  // mbarrier addresses (shared space)
     uint32_t slot_full, slot_empty, q_full, q_empty, s_full, s_free, p_full, p_empty, o_full, o_empty, sm_sync,
-        pub_p1, pub_o, lse_ready;
+        pub_p1, pub_o, lse_ready, raw_full, raw_empty, q_ready;
 };
 
 // NC = score columns per softmax warpgroup, CG = number of such warpgroups (N = NC * CG):
@@ -103,7 +114,14 @@ struct CBars {  // mbarrier addresses (shared space)
 // LP: the publisher warp combines the LSE partials (few CTAs per head); otherwise the softmax warps do.
 // PH: one Eq. 3 score per attention head (stats [.., n_q_heads, stride]) instead of per KV head,
 // for groups of at most 8 heads (a short statistic pass when the group size divides 8).
-template <int NC, int CG, bool LP, bool PH, bool SC>
+// SC: per-(layer, KV head) scales of K and V (an 8-bit cache, expanded to bf16 beforehand or here).
+// F8: the cache holds e4m3 bytes.  TMA brings a tile's bytes (16 KB) into a ring of raw stages; the
+// softmax warps expand a tile one or two places ahead into the operand slot while the tensor cores
+// work on the current one (cvt.rn.f16x2.e4m3x2: every e4m3 value is an fp16 value).  Both products then run on
+// fp16 operands: Q is converted once per unit in shared memory, P~ is split into an fp16 rounding of
+// 2^14 P~ and the fp16 rounding of 2^11 times its remainder (the two accumulator halves are added with
+// that weight in the epilogue); the powers of two join the scales.
+template <int NC, int CG, bool LP, bool PH, bool SC, bool F8>
 __global__ void __launch_bounds__(128 + 128 * CG, 1)
 verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                      const __grid_constant__ CUtensorMap tm_q, const FastParams p)
@@ -122,7 +140,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const int p_bytes = 2 * N * 256;                   // one P buffer: [hi | lo] rows, 8-row blocks x 128 keys x 16 B
 
     const uint32_t s_slots = sbase;
-    const uint32_t s_q = s_slots + p.n_slots * kSlotBytes;
+    const uint32_t s_raw = s_slots + p.n_slots * kSlotBytes;  // F8: n_raw stages of 16 KB
+    const uint32_t s_q = s_raw + (F8 ? p.n_raw * 16384 : 0);
     const uint32_t s_p = s_q + q_bytes;                // one Q buffer: the next unit's Q lands after this unit's last QK^T
     const uint32_t s_misc = s_p + p.p_bufs * p_bytes;
     uint8_t* misc = sgen + (s_misc - sbase);
@@ -143,6 +162,9 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         B.pub_p1 = o; o += 8;   // the last softmax warp stored this CTA's (max, sum) partial
         B.pub_o = o; o += 8;    // every softmax warp stored its share of the output partial
         B.lse_ready = o; o += 8;  // the publisher warp left the row LSE and the rescale factors in shared memory
+        B.raw_full = o; o += 32;  // F8: a tile's bytes have landed in a raw stage
+        B.raw_empty = o; o += 32; // F8: every softmax warp has expanded its part of the stage
+        B.q_ready = o; o += 8;    // F8: Q is fp16 in shared memory
     }
     float* lse_s = reinterpret_cast<float*>(misc + 1024);                 // [128] global row LSE (log2 domain)
     float* loc_s = reinterpret_cast<float*>(misc + 1024 + 512);           // [128] CTA-local row LSE
@@ -160,8 +182,12 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     } else if (threadIdx.x < kMaxCache + 8) {
         const int i = threadIdx.x - kMaxCache;
         if (i < p.n_slots) {
-            mbar_init(B.slot_full + 8 * i, 1);
+            mbar_init(B.slot_full + 8 * i, F8 ? kSW : 1);  // F8: filled by the softmax warps, not by TMA
             mbar_init(B.slot_empty + 8 * i, 1);
+        }
+        if (F8 && i < 4) {
+            mbar_init(B.raw_full + 8 * i, 1);
+            mbar_init(B.raw_empty + 8 * i, kSW);
         }
         if (i < 2) {
             mbar_init(B.q_full + 8 * i, 1);
@@ -178,6 +204,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         mbar_init(B.pub_p1, 1);
         mbar_init(B.pub_o, kSW);
         mbar_init(B.lse_ready, 1);
+        if (F8) mbar_init(B.q_ready, kSW);
         *abort_flag = 0;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -221,6 +248,32 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         const int halves = p.D / 64;  // 64-wide halves of the head dimension
         bool ok = true;
         auto load_tile = [&](const CUtensorMap* map, const Seg& sg, int tile) -> bool {
+            if (F8) {
+                // the tile's bytes (128 per key) go to a raw stage; the softmax warps expand them into a slot
+                const uint32_t r = slot_idx % p.n_raw, rph = (slot_idx / p.n_raw) & 1;
+                ++slot_idx;
+                bool got = true;
+                if (lane == 0) got = mbar_wait(B.raw_empty + 8 * r, rph ^ 1, ctl, 3);
+                if (!__shfl_sync(0xffffffffu, got ? 1 : 0, 0)) return false;
+                const int key0 = tile * kTile;
+                const int n_box = min(boxes, (sg.T - key0 + box_rows - 1) / box_rows);
+                if (lane == 0) mbar_expect_tx(B.raw_full + 8 * r, (uint32_t)n_box * box_bytes);
+                __syncwarp();
+                for (int bx = lane; bx < n_box; bx += 32) {
+                    const int pos = key0 + bx * box_rows;
+                    const int page = page_of(p.a.kv, pos), slot_in_page = pos - page * p.a.kv.page_size;
+                    int phys = p.a.kv.page_table ? __ldg(p.a.kv.page_table + (int64_t)sg.b * p.a.kv.max_pages + page)
+                                                 : sg.b * p.a.kv.max_pages + page;
+                    if (phys < 0 || phys >= p.n_pages) {
+                        set_status(p.status, SPEC_ERR_BAD_INDEX);
+                        phys = 0;
+                    }
+                    tma_load_5d(s_raw + r * 16384 + bx * box_bytes, map, B.raw_full + 8 * r, 0, slot_in_page, sg.h, phys,
+                                sg.layer, kEvictFirst);
+                }
+                __syncwarp();
+                return true;
+            }
             const uint32_t s = slot_idx % p.n_slots, ph = (slot_idx / p.n_slots) & 1;
             ++slot_idx;
             bool got = true;
@@ -272,9 +325,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     } else if (warp == 1) {
         // =========================== MMA issuer ===========================
         if (lane == 0) {
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
+            // operand formats (bits 7-9 and 10-12): 1 = bf16, 0 = fp16 (F8: both products on fp16 operands)
+            const uint32_t ab_fmt = F8 ? 0u : ((1u << 7) | (1u << 10));
+            const uint32_t idesc_qk = (1u << 4) | ab_fmt | ((uint32_t)(N >> 3) << 17) | ((128u >> 4) << 24);
             // O^T += V^T [P_hi | P_lo]^T : A = V^T and B = P^T both MN-major, N = 2 * rows
-            const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+            const uint32_t idesc_pv = (1u << 4) | ab_fmt | (1u << 15) | (1u << 16) |
                                       ((uint32_t)((2 * N) >> 3) << 17) | ((128u >> 4) << 24);
             // Two independent queues, issued in whichever order their inputs become ready: the
             // QK^T tiles of unit u+1 may overtake the P V tiles of unit u that still wait for P.
@@ -315,7 +370,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const int c = qq.t - qq.t0;
                 const uint32_t slot = qq.slot_base + c;
                 const uint32_t s = slot % p.n_slots, sph = (slot / p.n_slots) & 1;
-                if (c == 0 && !mbar_test_wait(B.q_full + 8 * qq.qb, qq.qph)) return false;
+                if (c == 0 && !mbar_test_wait(F8 ? B.q_ready : B.q_full + 8 * qq.qb, qq.qph)) return false;
                 if (!mbar_test_wait(B.slot_full + 8 * s, sph)) return false;
                 return mbar_test_wait(B.s_free + 8 * c, ((sfree_par >> c) & 1) ^ 1);
             };
@@ -541,6 +596,91 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         const bool ph_fast = (8 % G) == 0;  // per-head statistic: column i of a 16-column chunk is head i mod 8 mod G
         const float cs0 = p.scale_log2;
         float vsc = 1.f;  // SC: scale of this unit's V
+        // F8: powers of two that travel with the operands (see the kernel's header)
+        constexpr float kPExp = 16384.f;         // P~ is held times 2^14
+        constexpr float kLoExp = 2048.f;         // the remainder of its fp16 rounding times 2^11
+        uint32_t g_conv = 0, g_total = 0;        // F8: tiles expanded so far / in this launch (K and V of every unit)
+        const uint32_t f8_ahead = F8 ? (uint32_t)min(p.n_slots - 2, 2) : 0u;  // tiles expanded ahead of the one in use
+        int q_next = 0;                          // F8: first unit whose Q is not converted yet
+        uint32_t qn_s = 0;                       // F8: Q buffers seen (phase of q_full / q_ready)
+        if (F8) {
+            for (int u = 0; u < U; ++u) {
+                const Seg s2 = get_seg(p, u, head_local, rank);
+                g_total += 2u * (uint32_t)max(s2.t1 - s2.t0, 0);
+            }
+        }
+        // F8: expands raw tile g (in the order the producer loads them) into operand slot g % n_slots.
+        // A thread of the softmax warps takes 16-byte pieces of the tile's 1024: piece q of row r holds
+        // d = 16 q .. 16 q + 15, i.e. the 16-byte chunks 2 (q % 4) and 2 (q % 4) + 1 of row r in the 64-wide
+        // half q / 4 (rows of 128 B, chunks swizzled with the row's low three bits).
+        auto convert_tile = [&](uint32_t g) -> bool {
+            const uint32_t r = g % p.n_raw, rph = (g / p.n_raw) & 1;
+            const uint32_t s = g % p.n_slots, sph = (g / p.n_slots) & 1;
+            if (!mbar_wait(B.raw_full + 8 * r, rph, ctl, 40)) return false;
+            if (!mbar_wait(B.slot_empty + 8 * s, sph ^ 1, ctl, 41)) return false;
+            const uint8_t* raw = sgen + (s_raw - sbase) + r * 16384;
+            uint8_t* slot = sgen + (s_slots - sbase) + s * kSlotBytes;
+            constexpr int kIter = (1024 + 128 * CG - 1) / (128 * CG);
+            uint4 in[kIter];
+#pragma unroll
+            for (int k = 0; k < kIter; ++k) {  // every load of the thread is in flight before the first is used
+                const int i = tid_s + k * 128 * CG;
+                // eight consecutive threads take eight consecutive rows and eight different pieces: their
+                // loads and both of their stores then fall on eight different 16-byte bank groups
+                const int l = i & 7, blk = i >> 3, row = 8 * (blk >> 3) + l, q = (l + blk) & 7;
+                if (i < 1024) in[k] = *reinterpret_cast<const uint4*>(raw + row * 128 + q * 16);
+            }
+#pragma unroll
+            for (int k = 0; k < kIter; ++k) {
+                const int i = tid_s + k * 128 * CG;
+                if (i < 1024) {
+                    const int l = i & 7, blk = i >> 3, row = 8 * (blk >> 3) + l, q = (l + blk) & 7;
+                    uint32_t o[8];
+                    e4m3x4_to_f16x4(in[k].x, o[0], o[1]);
+                    e4m3x4_to_f16x4(in[k].y, o[2], o[3]);
+                    e4m3x4_to_f16x4(in[k].z, o[4], o[5]);
+                    e4m3x4_to_f16x4(in[k].w, o[6], o[7]);
+                    uint8_t* dst = slot + (q >> 2) * 16384 + row * 128;
+                    const int c0 = (q & 3) * 2, sw = row & 7;
+                    *reinterpret_cast<uint4*>(dst + ((c0 ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(dst + (((c0 + 1) ^ sw) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(B.slot_full + 8 * s);
+                mbar_arrive(B.raw_empty + 8 * r);
+            }
+            return true;
+        };
+        auto ensure_converted = [&](uint32_t g_need) -> bool {
+            while (g_conv <= g_need && g_conv < g_total) {
+                if (!convert_tile(g_conv)) return false;
+                ++g_conv;
+            }
+            return true;
+        };
+        // F8: Q of every unit up to `unit` as fp16, in place (a 16-bit element stays where it is, so the
+        // swizzle does not matter); exact for magnitudes in [6.1e-5, 65504]
+        auto ensure_q = [&](int unit) -> bool {
+            for (; q_next <= unit && q_next < U; ++q_next) {
+                const Seg s2 = get_seg(p, q_next, head_local, rank);
+                if (s2.t1 <= s2.t0) continue;
+                if (!mbar_wait(B.q_full, qn_s & 1, ctl, 42)) return false;
+                ++qn_s;
+                uint32_t* qw = reinterpret_cast<uint32_t*>(sgen + (s_q - sbase));
+                for (int i = tid_s; i < q_bytes / 4; i += 128 * CG) {
+                    const uint32_t w = qw[i];
+                    const __half2 h = __floats2half2_rn(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+                    qw[i] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(B.q_ready);
+            }
+            return true;
+        };
         constexpr float kNegBig = -1.0e30f;      // finite stand-in for -inf: keeps ex2 arguments NaN-free
         uint32_t pv_idx = 0, slot_base = 0, o_phase = 0, sync_n = 0, sfull_par = 0;
         bool ok = true;
@@ -564,7 +704,8 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                     const int r = c0 + i;
                     if (r < R)
                         p.o_part[obase + (int64_t)r * kD + key_l] =
-                            (__uint_as_float(v[i]) + __uint_as_float(w[i])) * (SC ? fac_s[r] * vsc : fac_s[r]);
+                            (F8 ? fmaf(__uint_as_float(w[i]), 1.f / kLoExp, __uint_as_float(v[i]))
+                                : __uint_as_float(v[i]) + __uint_as_float(w[i])) * (SC ? fac_s[r] * vsc : fac_s[r]);
                 }
             } else {
                 for (int i = tid_s; i < R * kD; i += 128 * CG) p.o_part[obase + i] = 0.f;
@@ -586,6 +727,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 if (p.a.kv.k_scale) cs *= __ldg(p.a.kv.k_scale + sh);
                 vsc = p.a.kv.v_scale ? __ldg(p.a.kv.v_scale + sh) : 1.f;
             }
+            if (F8) {
+                vsc *= 1.f / kPExp;
+                ok = ensure_q(unit);
+                if (!ok) break;
+            }
             // ------------------------------ P1 ------------------------------
             float m[NH], l[NH];
 #pragma unroll
@@ -595,6 +741,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
             for (int c = 0; c < n_t && ok; ++c) {
                 const int t = sg.t0 + c;
+                if (F8) {
+                    ok = ensure_converted(slot_base + c + f8_ahead);
+                    if (!ok) break;
+                }
                 ok = mbar_wait(B.s_full + 8 * c, (sfull_par >> c) & 1, ctl, 20);
                 if (!ok) break;
                 sfull_par ^= 1u << c;
@@ -694,15 +844,20 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         const uint32_t pvi = pv_idx + c;
                         const uint32_t pb = pvi % p.p_bufs;
                         const int key = t * kTile + key_l;
+                        if (F8) {  // V tile c + 2 (or the next unit's first K tiles) becomes an operand meanwhile
+                            ok = ensure_converted(slot_base + n_t + c + f8_ahead);
+                            if (!ok) break;
+                        }
                         tc_wait_ld();
                         float pr[NH];
 #pragma unroll
                         for (int i = 0; i < NH; i += 4) {
                             const float4 ls = loc4[i >> 2];
-                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, -ls.x));
-                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, -ls.y));
-                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, -ls.z));
-                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, -ls.w));
+                            // F8: 2^14 P~ (the fp16 parts below then stay normal numbers down to 2^-28)
+                            pr[i + 0] = ex2(fmaf(__uint_as_float(v[i + 0]), cs, F8 ? 14.f - ls.x : -ls.x));
+                            pr[i + 1] = ex2(fmaf(__uint_as_float(v[i + 1]), cs, F8 ? 14.f - ls.y : -ls.y));
+                            pr[i + 2] = ex2(fmaf(__uint_as_float(v[i + 2]), cs, F8 ? 14.f - ls.z : -ls.z));
+                            pr[i + 3] = ex2(fmaf(__uint_as_float(v[i + 3]), cs, F8 ? 14.f - ls.w : -ls.w));
                         }
                         if (c + 1 < n_t) {  // next tile's columns: in flight during the rest of this tile
 #pragma unroll
@@ -744,6 +899,16 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                                 // conversion instructions): hi keeps the top 16 bits, lo the top 16 bits of the
                                 // exact remainder, so p - (hi + lo) < 2^-14 p
                                 const uint32_t ua = __float_as_uint(pr[nb * 8 + 2 * q]), ub = __float_as_uint(pr[nb * 8 + 2 * q + 1]);
+                                if (F8) {
+                                    // fp16 rounding of 2^14 P~ and the fp16 rounding of 2^11 times what it left over
+                                    const __half2 h = __floats2half2_rn(__uint_as_float(ua), __uint_as_float(ub));
+                                    const float2 hf = __half22float2(h);
+                                    const __half2 l = __floats2half2_rn((__uint_as_float(ua) - hf.x) * kLoExp,
+                                                                        (__uint_as_float(ub) - hf.y) * kLoExp);
+                                    hi[q] = *reinterpret_cast<const uint32_t*>(&h);
+                                    lo[q] = *reinterpret_cast<const uint32_t*>(&l);
+                                    continue;
+                                }
                                 hi[q] = __byte_perm(ua, ub, 0x7632);
                                 const float ra = __uint_as_float(ua) - __uint_as_float(ua & 0xffff0000u);
                                 const float rb = __uint_as_float(ub) - __uint_as_float(ub & 0xffff0000u);
@@ -820,6 +985,10 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             p.a.lse[row] = lse2 * 0.69314718055994530942f;
                         }
                     }
+                }
+                if (F8) {  // the next unit's Q has landed by now: its K Q^T can start as the statistic pass frees regions
+                    ok = ensure_q(unit + 1);
+                    if (!ok) break;
                 }
                 ok = group_sync(B.sm_sync, sync_n, ctl, 22);  // every warp is done with the P V pass
                 if (!ok) break;
@@ -911,6 +1080,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         }
                     } else if (key < sg.T) {
                         float* dst = p.a.stats + sg.prob * p.a.stat_stride + key;
+                        if (F8) st *= 1.f / kPExp;  // the cache holds 2^14 P~
                         const float val = p.a.stat_accumulate ? *dst + st : st;
                         *dst = val;
                         // first radix pass of the selection, fused: count the score's top 11 bits in this
@@ -958,11 +1128,11 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     if (!*abort_flag) reset_counters_if_last(p, reinterpret_cast<int*>(const_cast<uint32_t*>(tmem_slot)));
 }
 
-template <int NC, int CG, bool LP, bool PH, bool SC>
+template <int NC, int CG, bool LP, bool PH, bool SC, bool F8>
 int launch_cfg(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tq, const FastParams& fp,
                int grid, size_t smem_bytes, cudaStream_t stream)
 {
-    auto kern = verify_cached_kernel<NC, CG, LP, PH, SC>;
+    auto kern = verify_cached_kernel<NC, CG, LP, PH, SC, F8>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
         return SPEC_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
@@ -1011,15 +1181,18 @@ int launch_cached(const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMa
     // per-(layer, KV head) scales: instances of their own (the bf16 instances carry no code for them),
     // built for the per-KV-head statistic only
     const bool sc = fp.a.kv.k_scale != nullptr || fp.a.kv.v_scale != nullptr;
-    if (sc && ph) return SPEC_ERR_UNSUPPORTED_SHAPE;
-#define SPEC_CASE(n, nc, cg)                                                                                     \
-    case n:                                                                                                      \
-        if (sc) return lp ? launch_cfg<nc, cg, true, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
-                          : launch_cfg<nc, cg, false, false, true>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
-        if (ph) return lp ? launch_cfg<nc, cg, true, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
-                          : launch_cfg<nc, cg, false, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
-        return lp ? launch_cfg<nc, cg, true, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream)             \
-                  : launch_cfg<nc, cg, false, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
+    const bool f8 = fp.a.kv.fp8 != 0;  // 8-bit cache read directly (always an SC instance)
+    if ((sc || f8) && ph) return SPEC_ERR_UNSUPPORTED_SHAPE;
+#define SPEC_CASE(n, nc, cg)                                                                                            \
+    case n:                                                                                                             \
+        if (f8) return lp ? launch_cfg<nc, cg, true, false, true, true>(tk, tv, tq, fp, grid, smem_bytes, stream)       \
+                          : launch_cfg<nc, cg, false, false, true, true>(tk, tv, tq, fp, grid, smem_bytes, stream);     \
+        if (sc) return lp ? launch_cfg<nc, cg, true, false, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
+                          : launch_cfg<nc, cg, false, false, true, false>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
+        if (ph) return lp ? launch_cfg<nc, cg, true, true, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream)      \
+                          : launch_cfg<nc, cg, false, true, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);    \
+        return lp ? launch_cfg<nc, cg, true, false, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream)             \
+                  : launch_cfg<nc, cg, false, false, false, false>(tk, tv, tq, fp, grid, smem_bytes, stream);
     switch (fp.N) {  // (columns per warpgroup, warpgroups)
         SPEC_CASE(16, 8, 2)
         SPEC_CASE(32, 8, 4)

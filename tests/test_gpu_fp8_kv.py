@@ -1,7 +1,7 @@
-"""8-bit (e4m3) KV cache as a second workload of the path: verification (the score-cache kernel on a bf16
-expansion of the cache, with the scales applied in the kernel; the generic kernels on the bytes), selection
-and the sparse draft kernel's fp8 instance against the oracle on the same bytes and scales, within the
-2e-3 bar of the bf16 path."""
+"""8-bit (e4m3) KV cache as a second workload of the path: verification (the score-cache kernel reading the
+bytes at head_dim 128, the same kernel on a bf16 expansion of the cache at head_dim 64, the generic
+kernels on the bytes), selection and the sparse draft kernel's fp8 instance against the oracle on the
+same bytes and scales, within the 2e-3 bar of the bf16 path."""
 import pytest
 import torch
 
@@ -43,7 +43,8 @@ def test_fp8_cache_path_matches_the_oracle(shape):
         if impl == binding.VERIFY_GENERIC:
             assert binding.last_verify_impl() == binding.VERIFY_GENERIC
         else:  # every shape of this list fits the score-cache kernel
-            assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+            assert binding.last_verify_impl() == (binding.VERIFY_TCGEN05_CACHED_EXPANDED if cfg.head_dim == 64
+                                                  else binding.VERIFY_TCGEN05_CACHED)
         if o_out is None:
             o_out, o_lse, o_stats = oracle.verify_attn(kv8_cpu, case.q_verify.cpu(), ctx.cpu(), 16, stats.shape[-1])
         assert (out.cpu().double() - o_out).abs().max().item() <= TOL
@@ -65,13 +66,15 @@ def test_fp8_cache_path_matches_the_oracle(shape):
         assert ((d_lse.cpu().double() - r_lse)[fin]).abs().max().item() <= TOL
 
 
-def test_fp8_verify_with_scales_that_are_not_powers_of_two_and_a_short_workspace():
-    """The expansion to bf16 leaves the scales out (a scaled value need not be a bf16 value) and the kernel
-    applies them per (layer, KV head); a workspace without room for the expansion falls back to the
-    generic kernels."""
+@pytest.mark.parametrize("head_dim", [128, 64])
+def test_fp8_verify_with_scales_that_are_not_powers_of_two_and_a_short_workspace(head_dim):
+    """The kernel applies the scales per (layer, KV head): the expanded copies (fp16 tiles in shared memory
+    at head_dim 128, a bf16 copy in the workspace at head_dim 64) leave them out, because a scaled value
+    need not be a 16-bit value.  At head_dim 64 a workspace without room for the copy falls back to the
+    generic kernels; at head_dim 128 the plain workspace is enough."""
     import dataclasses
     cfg = inputs.small_config(ctx=(700, 1900), n_q=9, batch=2, n_layers=2, n_q_heads=8, n_kv_heads=2,
-                              page_size=16, shuffled_pages=True)
+                              page_size=16, shuffled_pages=True, head_dim=head_dim)
     case = inputs.make_case(cfg, device="cuda")
     kv8 = inputs.quantize_kv_fp8(case.kv)
     g = torch.Generator(device="cuda").manual_seed(5)
@@ -83,7 +86,9 @@ def test_fp8_verify_with_scales_that_are_not_powers_of_two_and_a_short_workspace
     full = binding.workspace_bytes(binding.WS_VERIFY, kv8, cfg.n_q, 1900)
     base = binding.workspace_bytes(binding.WS_VERIFY, case.kv, cfg.n_q, 1900)
     assert full > base
-    for nbytes, want in ((full, binding.VERIFY_TCGEN05_CACHED), (base, binding.VERIFY_GENERIC)):
+    wants = ((full, binding.VERIFY_TCGEN05_CACHED), (base, binding.VERIFY_TCGEN05_CACHED)) if head_dim == 128 else \
+            ((full, binding.VERIFY_TCGEN05_CACHED_EXPANDED), (base, binding.VERIFY_GENERIC))
+    for nbytes, want in wants:
         ws = binding.alloc_workspace(nbytes, "cuda")
         out, lse, stats, _ = binding.spec_verify_attn(kv8, case.q_verify, ctx, 1900, workspace=ws)
         assert binding.read_status(ws) == 0

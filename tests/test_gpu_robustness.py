@@ -97,11 +97,14 @@ def test_generic_verify_reports_a_bad_page_entry():
         binding.set_verify_impl(prev)
 
 
-def test_verify_over_an_8bit_cache_reports_bad_lengths_and_page_entries():
-    """The expansion of an 8-bit cache into the workspace follows the same rules: a page-table entry
-    outside the pool is replaced and reported, a length beyond the host bound is clamped, and nothing is
-    written outside the workspace's tail."""
-    cfg = inputs.small_config(ctx=(500, 700), n_q=5, batch=2, page_size=16, shuffled_pages=True, planted=0)
+@pytest.mark.parametrize("head_dim", [128, 64])
+def test_verify_over_an_8bit_cache_reports_bad_lengths_and_page_entries(head_dim):
+    """Both ways of reading an 8-bit cache (tiles expanded in shared memory at head_dim 128, pages expanded
+    into the workspace at head_dim 64) follow the same rules: a page-table entry outside the pool is
+    replaced and reported, a length beyond the host bound is clamped, and nothing is written outside the
+    workspace."""
+    cfg = inputs.small_config(ctx=(500, 700), n_q=5, batch=2, page_size=16, shuffled_pages=True, planted=0,
+                              head_dim=head_dim)
     case = inputs.make_case(cfg, device="cuda")
     kv8 = inputs.quantize_kv_fp8(case.kv)
     T = int(case.ctx_len.max())
@@ -114,7 +117,9 @@ def test_verify_over_an_8bit_cache_reports_bad_lengths_and_page_entries():
     ws = guard[pad:-pad]
     assert ws.data_ptr() % 256 == 0
     ref = binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, T, workspace=ws)
-    assert binding.read_status(ws) == 0 and binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+    assert binding.read_status(ws) == 0
+    assert binding.last_verify_impl() == (binding.VERIFY_TCGEN05_CACHED if head_dim == 128
+                                          else binding.VERIFY_TCGEN05_CACHED_EXPANDED)
     bad = dataclasses.replace(kv8, page_table=kv8.page_table.clone())
     bad.page_table[longest, 3] = kv8.page_table.numel() + 5
     out, _, _, _ = binding.spec_verify_attn(bad, case.q_verify, case.ctx_len, T, workspace=ws)
