@@ -50,6 +50,22 @@ def test_headline_shape_is_two_units_of_four_heads():
     assert binding.describe_plan(binding.WS_VERIFY, kv, 9, 32768)[:6] == [2, 4, 37, 2, 48, 8]
 
 
+def test_8bit_cache_plans():
+    """The score-cache kernel takes an 8-bit cache at head_dim 128 with three operand slots (its raw stages
+    hold the tiles in flight) and as many P buffers as fit; head_dim 64 is not read directly (the entry
+    point expands it to bf16 first), so the planner reports no tensor-core kernel for that view."""
+    def fp8(kv):
+        return binding._KV(kv.k, kv.v, kv.layer_stride, kv.page_stride, kv.head_stride, kv.slot_stride, kv.n_layers,
+                           kv.page_size, None, kv.max_pages, kv.batch, kv.n_q_heads, kv.n_kv_heads, kv.head_dim,
+                           kv.n_pages, 0.0, binding.KV_FP8_E4M3, None, None)
+    kind, hg, cph, units, n, n_cache, slots, p_bufs = binding.describe_plan(
+        binding.WS_VERIFY, fp8(kv_struct(1, 1, 32, 8, 128, 32768 + 128)), 9, 32768)
+    assert [kind, hg, cph, units, n, n_cache] == [2, 4, 37, 2, 48, 8] and slots == 3 and p_bufs == 3
+    # raw stages (2 x 16 KB), Q, P buffers, slots and the small arrays fit the 227 KB of a CTA
+    assert 1024 + n * 256 + p_bufs * 2 * n * 256 + 12544 + 2 * 16384 + slots * 32768 <= 227 * 1024
+    assert binding.describe_plan(binding.WS_VERIFY, fp8(kv_struct(1, 1, 8, 2, 64, 2048)), 5, 2048)[0] == 0
+
+
 DRAFT_CASES = [  # (name, kv, keys)
     ("cfg2 per layer", kv_struct(1, 1, 32, 8, 128, 32768 + 128), 2056),
     ("cfg2 folded", kv_struct(32, 1, 32, 8, 128, 32768 + 128), 2056),
