@@ -609,41 +609,53 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 g_total += 2u * (uint32_t)max(s2.t1 - s2.t0, 0);
             }
         }
-        // F8: expands raw tile g (in the order the producer loads them) into operand slot g % n_slots.
+        // F8: expands the next raw tile (in the order the producer loads them) into the next operand slot.
         // A thread of the softmax warps takes 16-byte pieces of the tile's 1024: piece q of row r holds
         // d = 16 q .. 16 q + 15, i.e. the 16-byte chunks 2 (q % 4) and 2 (q % 4) + 1 of row r in the 64-wide
         // half q / 4 (rows of 128 B, chunks swizzled with the row's low three bits).
-        auto convert_tile = [&](uint32_t g) -> bool {
-            const uint32_t r = g % p.n_raw, rph = (g / p.n_raw) & 1;
-            const uint32_t s = g % p.n_slots, sph = (g / p.n_slots) & 1;
+        uint32_t cv_r = 0, cv_rph = 0, cv_s = 0, cv_sph = 0;  // ring positions of the next tile to expand (no division per tile)
+        // The thread's pieces, the same for every tile: source offset in the raw stage (low half) and offset of
+        // the first of the two 16-byte chunks in the slot (high half; the second is its neighbour, offset ^ 16).
+        // Eight consecutive threads take eight consecutive rows and eight different pieces: their loads and
+        // both of their stores then fall on eight different 16-byte bank groups.
+        constexpr int kIter = (1024 + 128 * CG - 1) / (128 * CG);
+        uint32_t cv_off[kIter];
+#pragma unroll
+        for (int k = 0; k < kIter; ++k) {
+            const int i = tid_s + k * 128 * CG;
+            const int l = i & 7, blk = i >> 3, row = 8 * (blk >> 3) + l, q = (l + blk) & 7;
+            const int c0 = (q & 3) * 2, sw = row & 7;
+            cv_off[k] = (uint32_t)(row * 128 + q * 16) | ((uint32_t)((q >> 2) * 16384 + row * 128 + ((c0 ^ sw) << 4)) << 16);
+        }
+        auto convert_tile = [&]() -> bool {
+            const uint32_t r = cv_r, rph = cv_rph, s = cv_s, sph = cv_sph;
+            if (++cv_r == (uint32_t)p.n_raw) {
+                cv_r = 0;
+                cv_rph ^= 1;
+            }
+            if (++cv_s == (uint32_t)p.n_slots) {
+                cv_s = 0;
+                cv_sph ^= 1;
+            }
             if (!mbar_wait(B.raw_full + 8 * r, rph, ctl, 40)) return false;
             if (!mbar_wait(B.slot_empty + 8 * s, sph ^ 1, ctl, 41)) return false;
             const uint8_t* raw = sgen + (s_raw - sbase) + r * 16384;
             uint8_t* slot = sgen + (s_slots - sbase) + s * kSlotBytes;
-            constexpr int kIter = (1024 + 128 * CG - 1) / (128 * CG);
             uint4 in[kIter];
 #pragma unroll
-            for (int k = 0; k < kIter; ++k) {  // every load of the thread is in flight before the first is used
-                const int i = tid_s + k * 128 * CG;
-                // eight consecutive threads take eight consecutive rows and eight different pieces: their
-                // loads and both of their stores then fall on eight different 16-byte bank groups
-                const int l = i & 7, blk = i >> 3, row = 8 * (blk >> 3) + l, q = (l + blk) & 7;
-                if (i < 1024) in[k] = *reinterpret_cast<const uint4*>(raw + row * 128 + q * 16);
-            }
+            for (int k = 0; k < kIter; ++k)  // every load of the thread is in flight before the first is used
+                if (tid_s + k * 128 * CG < 1024) in[k] = *reinterpret_cast<const uint4*>(raw + (cv_off[k] & 0xffffu));
 #pragma unroll
             for (int k = 0; k < kIter; ++k) {
-                const int i = tid_s + k * 128 * CG;
-                if (i < 1024) {
-                    const int l = i & 7, blk = i >> 3, row = 8 * (blk >> 3) + l, q = (l + blk) & 7;
+                if (tid_s + k * 128 * CG < 1024) {
                     uint32_t o[8];
                     e4m3x4_to_f16x4(in[k].x, o[0], o[1]);
                     e4m3x4_to_f16x4(in[k].y, o[2], o[3]);
                     e4m3x4_to_f16x4(in[k].z, o[4], o[5]);
                     e4m3x4_to_f16x4(in[k].w, o[6], o[7]);
-                    uint8_t* dst = slot + (q >> 2) * 16384 + row * 128;
-                    const int c0 = (q & 3) * 2, sw = row & 7;
-                    *reinterpret_cast<uint4*>(dst + ((c0 ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    *reinterpret_cast<uint4*>(dst + (((c0 + 1) ^ sw) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                    uint8_t* dst = slot + (cv_off[k] >> 16);
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(reinterpret_cast<uintptr_t>(dst) ^ 16) = make_uint4(o[4], o[5], o[6], o[7]);
                 }
             }
             fence_proxy_async();
@@ -656,7 +668,7 @@ verify_cached_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         };
         auto ensure_converted = [&](uint32_t g_need) -> bool {
             while (g_conv <= g_need && g_conv < g_total) {
-                if (!convert_tile(g_conv)) return false;
+                if (!convert_tile()) return false;
                 ++g_conv;
             }
             return true;
