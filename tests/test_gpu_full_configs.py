@@ -29,9 +29,14 @@ def one_head_cache(kv, layer, b, h, T):
     v = kv.v[layer, phys, h, slot].cpu().contiguous().view(1, 1, 1, T, kv.head_dim)
     D = kv.head_dim
     G = kv.n_q_heads // kv.n_kv_heads
+    ks = vs = None
+    if kv.fp8:  # e4m3 bytes: the head's scales go with them
+        ks = kv.k_scale[layer:layer + 1, h:h + 1].cpu().contiguous()
+        vs = kv.v_scale[layer:layer + 1, h:h + 1].cpu().contiguous()
     return inputs.KVCache(k=k, v=v, layer_stride=T * D, page_stride=T * D, head_stride=T * D,
                           slot_stride=D, n_layers=1, page_size=T, page_table=None, max_pages=1,
-                          batch=1, n_q_heads=G, n_kv_heads=1, head_dim=D, sm_scale=0.0, n_pages=1)
+                          batch=1, n_q_heads=G, n_kv_heads=1, head_dim=D, sm_scale=0.0, n_pages=1,
+                          fp8=kv.fp8, k_scale=ks, v_scale=vs)
 
 
 def check_samples(case, run, samples):
@@ -84,6 +89,27 @@ def test_cfg1_tiny_every_head():
     _, _, worst = run_config(cfg, [(0, 0, 0), (0, 0, 1)])
     assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED  # head_dim 64 on the tcgen05 path
     assert worst["overlap"] > 0.97
+
+
+def test_cfg2_8bit_cache_full_context_sampled_heads():
+    """The headline shape over an e4m3 copy of the cache (4 of its 32 layers; scales that are not powers of
+    two): the score-cache kernel reads the bytes itself, two units of four heads per layer as over bf16."""
+    cfg = dataclasses.replace(inputs.baseline_configs()["cfg2_8b_32k"], n_layers=4)
+    case = inputs.make_case(cfg, device="cuda")
+    kv8 = inputs.quantize_kv_fp8(case.kv)
+    g = torch.Generator(device="cuda").manual_seed(11)
+    kv8 = dataclasses.replace(
+        kv8, k_scale=kv8.k_scale * (0.8 + 0.4 * torch.rand(kv8.k_scale.shape, generator=g, device="cuda")),
+        v_scale=kv8.v_scale * (0.8 + 0.4 * torch.rand(kv8.v_scale.shape, generator=g, device="cuda")))
+    case8 = dataclasses.replace(case, kv=kv8)
+    run = runner.SpecStepRunner(case8)
+    run.step()
+    assert binding.read_status(run.ws_v) == 0 and binding.read_status(run.ws_d) == 0
+    assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+    worst = check_samples(case8, run, [(0, 0, 0), (2, 0, 3), (3, 0, 7)])
+    assert worst["overlap"] > 0.9
+    mass = run.stats[:, 0, :, :32768].sum(-1)
+    assert (mass - cfg.group * cfg.n_q).abs().max().item() < 0.05
 
 
 def test_cfg2_8b_32k_full_step_sampled_heads():
