@@ -213,14 +213,8 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 #pragma unroll
     for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
-    int stage = 0;
-    for (int c = warp; c < nch; c += NW) {
-        cp_async_wait<ST - 1>();
-        __syncwarp();
-        const uint8_t* ksm = wst + stage * STAGE;
-        const uint8_t* vsm = ksm + kChunk * ROWB;
-        // ---- S = Q K^T: keys 0..7 and 8..15 of the chunk are the two 8-wide column blocks ----
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    // S = Q K^T of the chunk in a stage: keys 0..7 and 8..15 are the two 8-wide column blocks
+    auto qk = [&](const uint8_t* ksm, float (&s0)[4], float (&s1)[4]) {
         {
             float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};  // four accumulation chains
             if (F8) {
@@ -255,35 +249,18 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
             s1[0] += t1[0];
             s1[1] += t1[1];
         }
-        // the thread's four keys: 2 quad, 2 quad + 1, 8 + 2 quad, 9 + 2 quad; masked rows carry no offset
+    };
+    // the chunk's four scores of this thread (keys 2 quad, 2 quad + 1, 8 + 2 quad, 9 + 2 quad), scaled; masked rows carry no offset
+    auto scores = [&](int c, const float (&s0)[4], const float (&s1)[4], float (&sv)[4]) {
         const uint2 va = *reinterpret_cast<const uint2*>(rowoff + c * kChunk + 2 * quad);
         const uint2 vb = *reinterpret_cast<const uint2*>(rowoff + c * kChunk + 8 + 2 * quad);
-        float sv[4];
         sv[0] = va.x != kNoRow ? s0[0] * sc : kNegBig;
         sv[1] = va.y != kNoRow ? s0[1] * sc : kNegBig;
         sv[2] = vb.x != kNoRow ? s1[0] * sc : kNegBig;
         sv[3] = vb.y != kNoRow ? s1[1] * sc : kNegBig;
-        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        // the running maximum moves only when some head's chunk maximum beats it by 2^8 (warp-uniform branch)
-        if (__any_sync(0xffffffffu, mx > M + 8.f)) {
-            const float Mn = fmaxf(M, mx);
-            const float alpha = ex2f(M - Mn);
-            M = Mn;
-            L *= alpha;
-#pragma unroll
-            for (int i = 0; i < D / 8; ++i) {
-                o[i][0] *= alpha;
-                o[i][1] *= alpha;
-                o[i][2] *= alpha;
-                o[i][3] *= alpha;
-            }
-        }
-        float p[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = sv[i] > 0.5f * kNegBig ? ex2f(sv[i] - M) : 0.f;
-        L += (p[0] + p[1]) + (p[2] + p[3]);
+    };
+    // O += [P_hi ; P_lo] V of the chunk in a stage, p = the thread's four probabilities
+    auto pv = [&](const uint8_t* vsm, const float (&p)[4]) {
         // [P_hi ; P_lo] as the A operand: rows 0..7 the 16-bit rounding, rows 8..15 the remainder
         uint32_t ah0, al0, ah1, al1;
         if (F8) {
@@ -330,9 +307,83 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
                 mma_bf16_16816(o[2 * nb + 1], ah0, al0, ah1, al1, vf[2], vf[3]);
             }
         }
-        __syncwarp();  // every lane is done with the stage before it is refilled
-        issue(c + ST * NW, stage);
-        stage = stage + 1 == ST ? 0 : stage + 1;
+    };
+
+    if (nch <= NW * ST) {
+        // Every chunk of this warp is in its own stage already (the usual case of a call per layer): one pass
+        // over all of them - the score blocks of up to ST chunks accumulate side by side, one maximum and one
+        // sum per head, no rescaling, and the P V products of the chunks follow one another.
+        cp_async_wait<0>();
+        __syncwarp();
+        // (the products run for every stage, so that their chains interleave; a stage without a chunk holds
+        // whatever it held, and its scores are replaced, not scaled)
+        float s0[ST][4], s1[ST][4];
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            s0[s][0] = s0[s][1] = s0[s][2] = s0[s][3] = 0.f;
+            s1[s][0] = s1[s][1] = s1[s][2] = s1[s][3] = 0.f;
+        }
+#pragma unroll
+        for (int s = 0; s < ST; ++s) qk(wst + s * STAGE, s0[s], s1[s]);
+        float sv[ST][4];
+        float mx = kNegBig;
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            const int c = warp + s * NW;
+            sv[s][0] = sv[s][1] = sv[s][2] = sv[s][3] = kNegBig;
+            if (c < nch) scores(c, s0[s], s1[s], sv[s]);
+            mx = fmaxf(mx, fmaxf(fmaxf(sv[s][0], sv[s][1]), fmaxf(sv[s][2], sv[s][3])));
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        M = mx;
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            const int c = warp + s * NW;
+            if (c < nch) {
+                float p[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) p[i] = sv[s][i] > 0.5f * kNegBig ? ex2f(sv[s][i] - M) : 0.f;
+                L += (p[0] + p[1]) + (p[2] + p[3]);
+                pv(wst + s * STAGE + kChunk * ROWB, p);
+            }
+        }
+    } else {
+        int stage = 0;
+        for (int c = warp; c < nch; c += NW) {
+            cp_async_wait<ST - 1>();
+            __syncwarp();
+            const uint8_t* ksm = wst + stage * STAGE;
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+            qk(ksm, s0, s1);
+            float sv[4];
+            scores(c, s0, s1, sv);
+            float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            // the running maximum moves only when some head's chunk maximum beats it by 2^8 (warp-uniform branch)
+            if (__any_sync(0xffffffffu, mx > M + 8.f)) {
+                const float Mn = fmaxf(M, mx);
+                const float alpha = ex2f(M - Mn);
+                M = Mn;
+                L *= alpha;
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) {
+                    o[i][0] *= alpha;
+                    o[i][1] *= alpha;
+                    o[i][2] *= alpha;
+                    o[i][3] *= alpha;
+                }
+            }
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = sv[i] > 0.5f * kNegBig ? ex2f(sv[i] - M) : 0.f;
+            L += (p[0] + p[1]) + (p[2] + p[3]);
+            pv(ksm + kChunk * ROWB, p);
+            __syncwarp();  // every lane is done with the stage before it is refilled
+            issue(c + ST * NW, stage);
+            stage = stage + 1 == ST ? 0 : stage + 1;
+        }
     }
     cp_async_wait<0>();
     L += __shfl_xor_sync(0xffffffffu, L, 1);
