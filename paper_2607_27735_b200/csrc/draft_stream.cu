@@ -68,6 +68,15 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// transpose of an 8x8 matrix of 16-bit elements held across the warp (thread (grp, quad) holds row grp,
+// columns 2 quad and 2 quad + 1, before and after)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
+{
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+
 // F8: the cache holds e4m3 bytes.  The rows are gathered as they are (half the bytes), turned into fp16
 // pairs on their way into the MMA fragments (fp16 holds every e4m3 value), and the two products run as
 // fp16 MMAs; the heads' scales join the softmax scale (K) and the final output (V).
@@ -189,9 +198,12 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     // F8: the K fragment of a step comes from ONE 4-byte load (d = 16 ks + 4 quad + 0..3), so the step's
     // sixteen d's are visited in that order and Q follows it: d = 16 ks + 4 quad + {0, 1} and + {2, 3},
     // as fp16.
+    // keys_on_rows (see below): Q is the B operand and its eight columns are the heads 0, 0, 1, 1, 2, 2, 3, 3
+    const bool keys_on_rows = !F8 && G <= 4 && nch <= NW * ST;
+    const int qh = keys_on_rows ? grp >> 1 : grp;  // the head whose row this thread's fragments come from
     uint32_t qa[KS][2];
     {
-        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + grp;
+        const int64_t row = ((int64_t)layer * a.kv.batch + b) * a.kv.n_q_heads + h * G + qh;
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(a.q + row * D);
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
@@ -201,8 +213,8 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
                 qa[ks][0] = pack_f16(bf16_lo(w0), bf16_hi(w0));
                 qa[ks][1] = pack_f16(bf16_lo(w1), bf16_hi(w1));
             } else {
-                qa[ks][0] = grp < G ? __ldg(qrow + ks * 8 + quad) : 0u;
-                qa[ks][1] = grp < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
+                qa[ks][0] = qh < G ? __ldg(qrow + ks * 8 + quad) : 0u;
+                qa[ks][1] = qh < G ? __ldg(qrow + ks * 8 + 4 + quad) : 0u;
             }
         }
     }
@@ -309,7 +321,83 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         }
     };
 
-    if (nch <= NW * ST) {
+    if (keys_on_rows) {
+        // Every chunk of this warp is resident and the group has at most four heads (bf16 cache): the keys take
+        // the MMA's 16 rows instead of the heads.  S^T = K Q^T is ONE m16n8k16 per 16 d (Q's fragments are the
+        // same registers as in the head-major form, now the B operand, with every head in two neighbouring
+        // columns), and O^T = V^T P^T one per 16 d as well, the column pair of a head being the bf16 rounding
+        // of its probabilities and the remainder.  Thread (grp, quad) then owns head `quad` throughout: the
+        // scores of keys grp and grp + 8, its maximum and sum, and O^T for d = 16 j + grp and + 8.  Half the
+        // tensor-core instructions of the head-major form below, whose 16 rows are mostly padding.
+        cp_async_wait<0>();
+        __syncwarp();
+        float st[ST][2];  // scores of keys grp, grp + 8 (both columns of the pair hold the same number)
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulation chains
+            const uint8_t* kp = wst + s * STAGE + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16;
+#pragma unroll
+            for (int ks = 0; ks < KS; ks += 2) {
+                uint32_t ka[4], kb[4];
+                ldmatrix_x4(ka, kp + ks * 32);
+                ldmatrix_x4(kb, kp + ks * 32 + 32);
+                mma_bf16_16816(c0, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
+                mma_bf16_16816(c1, kb[0], kb[1], kb[2], kb[3], qa[ks + 1][0], qa[ks + 1][1]);
+            }
+            st[s][0] = c0[0] + c1[0];
+            st[s][1] = c0[2] + c1[2];
+        }
+        float mx = kNegBig;
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            const int c = warp + s * NW;
+            const bool has = c < nch;  // (a stage without a chunk holds whatever it held: replaced, not scaled)
+            const bool v0 = has && rowoff[(has ? c : 0) * kChunk + grp] != kNoRow;
+            const bool v1 = has && rowoff[(has ? c : 0) * kChunk + 8 + grp] != kNoRow;
+            st[s][0] = v0 ? st[s][0] * sc : kNegBig;
+            st[s][1] = v1 ? st[s][1] * sc : kNegBig;
+            mx = fmaxf(mx, fmaxf(st[s][0], st[s][1]));
+        }
+#pragma unroll
+        for (int o2 = 4; o2 < 32; o2 <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));  // over the key lanes
+        M = mx;
+        float ot[D / 16][4];  // O^T: rows d = 16 j + grp (and + 8), columns (rounding, remainder) of head quad
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) ot[j][0] = ot[j][1] = ot[j][2] = ot[j][3] = 0.f;
+#pragma unroll
+        for (int s = 0; s < ST; ++s) {
+            if (warp + s * NW < nch) {  // warp-uniform
+                const float p0 = st[s][0] > 0.5f * kNegBig ? ex2f(st[s][0] - M) : 0.f;
+                const float p1 = st[s][1] > 0.5f * kNegBig ? ex2f(st[s][1] - M) : 0.f;
+                L += p0 + p1;
+                // source of P^T: rows = keys (0..7 and 8..15), columns 2 quad, 2 quad + 1 = (rounding, remainder)
+                const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
+                const uint32_t x0 = pack_bf16(h0, p0 - h0), x1 = pack_bf16(h1, p1 - h1);
+                // transposed: the B operand (keys 2 quad, 2 quad + 1 of each half; column grp)
+                const uint32_t b0 = movmatrix_trans(x0), b1 = movmatrix_trans(x1);
+                // V^T as the A operand: a transposing load of the chunk's V rows [key][d]
+                const uint8_t* vp = wst + s * STAGE + kChunk * ROWB + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB +
+                                    ((lane >> 3) & 1) * 16;
+#pragma unroll
+                for (int j = 0; j < D / 16; ++j) {
+                    uint32_t vf[4];
+                    ldmatrix_x4_trans(vf, vp + j * 32);
+                    mma_bf16_16816(ot[j], vf[0], vf[1], vf[2], vf[3], b0, b1);
+                }
+            }
+        }
+#pragma unroll
+        for (int o2 = 4; o2 < 32; o2 <<= 1) L += __shfl_xor_sync(0xffffffffu, L, o2);
+        // the warp's result block [head][D + 8] (its own first stage), as the head-major form leaves it
+        __syncwarp();  // every lane is done with stage 0
+        float* ow = reinterpret_cast<float*>(wst);
+#pragma unroll
+        for (int j = 0; j < D / 16; ++j) {
+            ow[quad * (D + 8) + 16 * j + grp] = ot[j][0] + ot[j][1];
+            ow[quad * (D + 8) + 16 * j + 8 + grp] = ot[j][2] + ot[j][3];
+        }
+        if (grp == 0) wml[warp * 8 + quad] = make_float2(M, L);
+    } else if (nch <= NW * ST) {
         // Every chunk of this warp is in its own stage already (the usual case of a call per layer): one pass
         // over all of them - the score blocks of up to ST chunks accumulate side by side, one maximum and one
         // sum per head, no rescaling, and the P V products of the chunks follow one another.
@@ -386,12 +474,11 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         }
     }
     cp_async_wait<0>();
-    L += __shfl_xor_sync(0xffffffffu, L, 1);
-    L += __shfl_xor_sync(0xffffffffu, L, 2);
-
     // ---- the warps of the CTA: (max, sum, O) through shared memory (each warp's own first stage) ----
     __syncwarp();
-    {
+    if (!keys_on_rows) {
+        L += __shfl_xor_sync(0xffffffffu, L, 1);
+        L += __shfl_xor_sync(0xffffffffu, L, 2);
         float* ow = reinterpret_cast<float*>(wst);  // [8 heads][D + 8]: the padding keeps the heads on different banks
         if (F8) {  // undo the order of the head dimension (see the V product) and apply the head's V scale
             const float vs = kv_scale_of(a.kv.v_scale, a.kv, layer, hm);
