@@ -199,7 +199,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     // sixteen d's are visited in that order and Q follows it: d = 16 ks + 4 quad + {0, 1} and + {2, 3},
     // as fp16.
     // keys_on_rows (see below): Q is the B operand and its eight columns are the heads 0, 0, 1, 1, 2, 2, 3, 3
-    const bool keys_on_rows = !F8 && G <= 4 && nch <= NW * ST;
+    const bool keys_on_rows = !F8 && G <= 4;
     const int qh = keys_on_rows ? grp >> 1 : grp;  // the head whose row this thread's fragments come from
     uint32_t qa[KS][2];
     {
@@ -322,20 +322,20 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     };
 
     if (keys_on_rows) {
-        // Every chunk of this warp is resident and the group has at most four heads (bf16 cache): the keys take
-        // the MMA's 16 rows instead of the heads.  S^T = K Q^T is ONE m16n8k16 per 16 d (Q's fragments are the
-        // same registers as in the head-major form, now the B operand, with every head in two neighbouring
-        // columns), and O^T = V^T P^T one per 16 d as well, the column pair of a head being the bf16 rounding
-        // of its probabilities and the remainder.  Thread (grp, quad) then owns head `quad` throughout: the
-        // scores of keys grp and grp + 8, its maximum and sum, and O^T for d = 16 j + grp and + 8.  Half the
-        // tensor-core instructions of the head-major form below, whose 16 rows are mostly padding.
-        cp_async_wait<0>();
-        __syncwarp();
-        float st[ST][2];  // scores of keys grp, grp + 8 (both columns of the pair hold the same number)
+        // Groups of at most four heads over a bf16 cache: the keys take the MMA's 16 rows instead of the heads.
+        // S^T = K Q^T is ONE m16n8k16 per 16 d (Q's fragments are the same registers as in the head-major form,
+        // now the B operand, with every head in two neighbouring columns), and O^T = V^T P^T one per 16 d as
+        // well, the column pair of a head being the bf16 rounding of its probabilities and the remainder.
+        // Thread (grp, quad) then owns head `quad` throughout: the scores of keys grp and grp + 8, its maximum
+        // and sum, and O^T for d = 16 j + grp and + 8.  Half the tensor-core instructions of the head-major
+        // form below, whose 16 rows are mostly padding.
+        float ot[D / 16][4];  // O^T: rows d = 16 j + grp (and + 8), columns (rounding, remainder) of head quad
 #pragma unroll
-        for (int s = 0; s < ST; ++s) {
+        for (int j = 0; j < D / 16; ++j) ot[j][0] = ot[j][1] = ot[j][2] = ot[j][3] = 0.f;
+        // scores of keys grp, grp + 8 of the chunk in a stage (both columns of the pair hold the same number)
+        auto tr_qk = [&](const uint8_t* ksm, float (&st)[2]) {
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulation chains
-            const uint8_t* kp = wst + s * STAGE + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16;
+            const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16;
 #pragma unroll
             for (int ks = 0; ks < KS; ks += 2) {
                 uint32_t ka[4], kb[4];
@@ -344,47 +344,92 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
                 mma_bf16_16816(c0, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
                 mma_bf16_16816(c1, kb[0], kb[1], kb[2], kb[3], qa[ks + 1][0], qa[ks + 1][1]);
             }
-            st[s][0] = c0[0] + c1[0];
-            st[s][1] = c0[2] + c1[2];
-        }
-        float mx = kNegBig;
+            st[0] = c0[0] + c1[0];
+            st[1] = c0[2] + c1[2];
+        };
+        // scaled, masked (a key without a row counts for nothing)
+        auto tr_mask = [&](int c, float (&st)[2]) {
+            st[0] = rowoff[c * kChunk + grp] != kNoRow ? st[0] * sc : kNegBig;
+            st[1] = rowoff[c * kChunk + 8 + grp] != kNoRow ? st[1] * sc : kNegBig;
+        };
+        auto tr_pv = [&](const uint8_t* vsm, float p0, float p1) {
+            // source of P^T: rows = keys (0..7 and 8..15), columns 2 quad, 2 quad + 1 = (rounding, remainder)
+            const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
+            const uint32_t x0 = pack_bf16(h0, p0 - h0), x1 = pack_bf16(h1, p1 - h1);
+            // transposed: the B operand (keys 2 quad, 2 quad + 1 of each half; column grp)
+            const uint32_t b0 = movmatrix_trans(x0), b1 = movmatrix_trans(x1);
+            // V^T as the A operand: a transposing load of the chunk's V rows [key][d]
+            const uint8_t* vp = vsm + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB + ((lane >> 3) & 1) * 16;
 #pragma unroll
-        for (int s = 0; s < ST; ++s) {
-            const int c = warp + s * NW;
-            const bool has = c < nch;  // (a stage without a chunk holds whatever it held: replaced, not scaled)
-            const bool v0 = has && rowoff[(has ? c : 0) * kChunk + grp] != kNoRow;
-            const bool v1 = has && rowoff[(has ? c : 0) * kChunk + 8 + grp] != kNoRow;
-            st[s][0] = v0 ? st[s][0] * sc : kNegBig;
-            st[s][1] = v1 ? st[s][1] * sc : kNegBig;
-            mx = fmaxf(mx, fmaxf(st[s][0], st[s][1]));
-        }
+            for (int j = 0; j < D / 16; ++j) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(vf, vp + j * 32);
+                mma_bf16_16816(ot[j], vf[0], vf[1], vf[2], vf[3], b0, b1);
+            }
+        };
+        if (nch <= NW * ST) {
+            // every chunk of this warp is in its own stage already (the usual case of a call per layer): one pass,
+            // the score blocks of up to ST chunks side by side, one maximum and one sum per head, no rescaling
+            cp_async_wait<0>();
+            __syncwarp();
+            float st[ST][2];
 #pragma unroll
-        for (int o2 = 4; o2 < 32; o2 <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));  // over the key lanes
-        M = mx;
-        float ot[D / 16][4];  // O^T: rows d = 16 j + grp (and + 8), columns (rounding, remainder) of head quad
+            for (int s = 0; s < ST; ++s) tr_qk(wst + s * STAGE, st[s]);  // (for every stage: the chains interleave)
+            float mx = kNegBig;
 #pragma unroll
-        for (int j = 0; j < D / 16; ++j) ot[j][0] = ot[j][1] = ot[j][2] = ot[j][3] = 0.f;
+            for (int s = 0; s < ST; ++s) {
+                const int c = warp + s * NW;
+                if (c < nch) tr_mask(c, st[s]);
+                else st[s][0] = st[s][1] = kNegBig;  // a stage without a chunk holds whatever it held
+                mx = fmaxf(mx, fmaxf(st[s][0], st[s][1]));
+            }
 #pragma unroll
-        for (int s = 0; s < ST; ++s) {
-            if (warp + s * NW < nch) {  // warp-uniform
-                const float p0 = st[s][0] > 0.5f * kNegBig ? ex2f(st[s][0] - M) : 0.f;
-                const float p1 = st[s][1] > 0.5f * kNegBig ? ex2f(st[s][1] - M) : 0.f;
-                L += p0 + p1;
-                // source of P^T: rows = keys (0..7 and 8..15), columns 2 quad, 2 quad + 1 = (rounding, remainder)
-                const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
-                const uint32_t x0 = pack_bf16(h0, p0 - h0), x1 = pack_bf16(h1, p1 - h1);
-                // transposed: the B operand (keys 2 quad, 2 quad + 1 of each half; column grp)
-                const uint32_t b0 = movmatrix_trans(x0), b1 = movmatrix_trans(x1);
-                // V^T as the A operand: a transposing load of the chunk's V rows [key][d]
-                const uint8_t* vp = wst + s * STAGE + kChunk * ROWB + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB +
-                                    ((lane >> 3) & 1) * 16;
+            for (int o2 = 4; o2 < 32; o2 <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));  // over the key lanes
+            M = mx;
 #pragma unroll
-                for (int j = 0; j < D / 16; ++j) {
-                    uint32_t vf[4];
-                    ldmatrix_x4_trans(vf, vp + j * 32);
-                    mma_bf16_16816(ot[j], vf[0], vf[1], vf[2], vf[3], b0, b1);
+            for (int s = 0; s < ST; ++s) {
+                if (warp + s * NW < nch) {  // warp-uniform
+                    const float p0 = st[s][0] > 0.5f * kNegBig ? ex2f(st[s][0] - M) : 0.f;
+                    const float p1 = st[s][1] > 0.5f * kNegBig ? ex2f(st[s][1] - M) : 0.f;
+                    L += p0 + p1;
+                    tr_pv(wst + s * STAGE + kChunk * ROWB, p0, p1);
                 }
             }
+        } else {
+            int stage = 0;
+            for (int c = warp; c < nch; c += NW) {
+                cp_async_wait<ST - 1>();
+                __syncwarp();
+                const uint8_t* ksm = wst + stage * STAGE;
+                float st[2];
+                tr_qk(ksm, st);
+                tr_mask(c, st);
+                float mx = fmaxf(st[0], st[1]);
+#pragma unroll
+                for (int o2 = 4; o2 < 32; o2 <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o2));
+                // the running maximum moves only when some head's chunk maximum beats it by 2^8 (warp-uniform branch)
+                if (__any_sync(0xffffffffu, mx > M + 8.f)) {
+                    const float Mn = fmaxf(M, mx);
+                    const float alpha = ex2f(M - Mn);
+                    M = Mn;
+                    L *= alpha;
+#pragma unroll
+                    for (int j = 0; j < D / 16; ++j) {
+                        ot[j][0] *= alpha;
+                        ot[j][1] *= alpha;
+                        ot[j][2] *= alpha;
+                        ot[j][3] *= alpha;
+                    }
+                }
+                const float p0 = st[0] > 0.5f * kNegBig ? ex2f(st[0] - M) : 0.f;
+                const float p1 = st[1] > 0.5f * kNegBig ? ex2f(st[1] - M) : 0.f;
+                L += p0 + p1;
+                tr_pv(ksm + kChunk * ROWB, p0, p1);
+                __syncwarp();  // every lane is done with the stage before it is refilled
+                issue(c + ST * NW, stage);
+                stage = stage + 1 == ST ? 0 : stage + 1;
+            }
+            cp_async_wait<0>();
         }
 #pragma unroll
         for (int o2 = 4; o2 < 32; o2 <<= 1) L += __shfl_xor_sync(0xffffffffu, L, o2);
