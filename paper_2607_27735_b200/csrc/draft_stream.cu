@@ -199,7 +199,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     // sixteen d's are visited in that order and Q follows it: d = 16 ks + 4 quad + {0, 1} and + {2, 3},
     // as fp16.
     // keys_on_rows (see below): Q is the B operand and its eight columns are the heads 0, 0, 1, 1, 2, 2, 3, 3
-    const bool keys_on_rows = !F8 && G <= 4;
+    const bool keys_on_rows = G <= 4;
     const int qh = keys_on_rows ? grp >> 1 : grp;  // the head whose row this thread's fragments come from
     uint32_t qa[KS][2];
     {
@@ -208,8 +208,8 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
             if (F8) {
-                const uint32_t w0 = grp < G ? __ldg(qrow + ks * 8 + 2 * quad) : 0u;
-                const uint32_t w1 = grp < G ? __ldg(qrow + ks * 8 + 2 * quad + 1) : 0u;
+                const uint32_t w0 = qh < G ? __ldg(qrow + ks * 8 + 2 * quad) : 0u;
+                const uint32_t w1 = qh < G ? __ldg(qrow + ks * 8 + 2 * quad + 1) : 0u;
                 qa[ks][0] = pack_f16(bf16_lo(w0), bf16_hi(w0));
                 qa[ks][1] = pack_f16(bf16_lo(w1), bf16_hi(w1));
             } else {
@@ -322,7 +322,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     };
 
     if (keys_on_rows) {
-        // Groups of at most four heads over a bf16 cache: the keys take the MMA's 16 rows instead of the heads.
+        // Groups of at most four heads: the keys take the MMA's 16 rows instead of the heads.
         // S^T = K Q^T is ONE m16n8k16 per 16 d (Q's fragments are the same registers as in the head-major form,
         // now the B operand, with every head in two neighbouring columns), and O^T = V^T P^T one per 16 d as
         // well, the column pair of a head being the bf16 rounding of its probabilities and the remainder.
@@ -335,14 +335,31 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         // scores of keys grp, grp + 8 of the chunk in a stage (both columns of the pair hold the same number)
         auto tr_qk = [&](const uint8_t* ksm, float (&st)[2]) {
             float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};  // two accumulation chains
-            const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16;
+            if (F8) {
+                // rows grp and grp + 8, bytes 16 ks + 4 quad .. + 3: one 4-byte load per row and step gives the
+                // row's two fragment registers (the step's sixteen d's are visited in that order, as Q's are)
+                const uint8_t* kp = ksm + grp * ROWB + 4 * quad;
 #pragma unroll
-            for (int ks = 0; ks < KS; ks += 2) {
-                uint32_t ka[4], kb[4];
-                ldmatrix_x4(ka, kp + ks * 32);
-                ldmatrix_x4(kb, kp + ks * 32 + 32);
-                mma_bf16_16816(c0, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
-                mma_bf16_16816(c1, kb[0], kb[1], kb[2], kb[3], qa[ks + 1][0], qa[ks + 1][1]);
+                for (int ks = 0; ks < KS; ks += 2) {
+                    const uint32_t k00 = *reinterpret_cast<const uint32_t*>(kp + ks * 16);
+                    const uint32_t k01 = *reinterpret_cast<const uint32_t*>(kp + 8 * ROWB + ks * 16);
+                    const uint32_t k10 = *reinterpret_cast<const uint32_t*>(kp + ks * 16 + 16);
+                    const uint32_t k11 = *reinterpret_cast<const uint32_t*>(kp + 8 * ROWB + ks * 16 + 16);
+                    mma_f16_16816(c0, e4m3x2_to_f16x2(k00), e4m3x2_to_f16x2(k01), e4m3x2_to_f16x2(k00 >> 16),
+                                  e4m3x2_to_f16x2(k01 >> 16), qa[ks][0], qa[ks][1]);
+                    mma_f16_16816(c1, e4m3x2_to_f16x2(k10), e4m3x2_to_f16x2(k11), e4m3x2_to_f16x2(k10 >> 16),
+                                  e4m3x2_to_f16x2(k11 >> 16), qa[ks + 1][0], qa[ks + 1][1]);
+                }
+            } else {
+                const uint8_t* kp = ksm + ((lane & 7) + ((lane >> 3) & 1) * 8) * ROWB + (lane >> 4) * 16;
+#pragma unroll
+                for (int ks = 0; ks < KS; ks += 2) {
+                    uint32_t ka[4], kb[4];
+                    ldmatrix_x4(ka, kp + ks * 32);
+                    ldmatrix_x4(kb, kp + ks * 32 + 32);
+                    mma_bf16_16816(c0, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
+                    mma_bf16_16816(c1, kb[0], kb[1], kb[2], kb[3], qa[ks + 1][0], qa[ks + 1][1]);
+                }
             }
             st[0] = c0[0] + c1[0];
             st[1] = c0[2] + c1[2];
@@ -354,17 +371,46 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         };
         auto tr_pv = [&](const uint8_t* vsm, float p0, float p1) {
             // source of P^T: rows = keys (0..7 and 8..15), columns 2 quad, 2 quad + 1 = (rounding, remainder)
-            const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
-            const uint32_t x0 = pack_bf16(h0, p0 - h0), x1 = pack_bf16(h1, p1 - h1);
+            uint32_t x0, x1;
+            if (F8) {
+                const float h0 = __half2float(__float2half_rn(p0)), h1 = __half2float(__float2half_rn(p1));
+                x0 = pack_f16(h0, p0 - h0);
+                x1 = pack_f16(h1, p1 - h1);
+            } else {
+                const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
+                x0 = pack_bf16(h0, p0 - h0);
+                x1 = pack_bf16(h1, p1 - h1);
+            }
             // transposed: the B operand (keys 2 quad, 2 quad + 1 of each half; column grp)
             const uint32_t b0 = movmatrix_trans(x0), b1 = movmatrix_trans(x1);
             // V^T as the A operand: a transposing load of the chunk's V rows [key][d]
             const uint8_t* vp = vsm + ((lane & 7) + ((lane >> 4) & 1) * 8) * ROWB + ((lane >> 3) & 1) * 16;
+            if (F8) {
+                // The load transposes 2-byte units, so a thread gets, for keys 2 quad and 2 quad + 1 (and + 8), the
+                // byte PAIR d = 2 grp, 2 grp + 1 of a 16-byte column block: bytes 0 and 2 of the register are the
+                // fragment of the even d, bytes 1 and 3 of the odd d.  The even d's take rows 0..7 of the MMA and
+                // the odd ones rows 8..15, so block jj's accumulator holds d = 16 jj + 2 grp (c0, c1) and
+                // d = 16 jj + 2 grp + 1 (c2, c3): see the store.
 #pragma unroll
-            for (int j = 0; j < D / 16; ++j) {
-                uint32_t vf[4];
-                ldmatrix_x4_trans(vf, vp + j * 32);
-                mma_bf16_16816(ot[j], vf[0], vf[1], vf[2], vf[3], b0, b1);
+                for (int j = 0; j < D / 32; ++j) {
+                    uint32_t vf[4];  // keys 0..7 x bytes 0..15, keys 0..7 x bytes 16..31, keys 8..15 x the same
+                    ldmatrix_x4_trans(vf, vp + j * 32);
+                    mma_f16_16816(ot[2 * j], e4m3x2_to_f16x2(__byte_perm(vf[0], 0u, 0x4420)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[0], 0u, 0x4431)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[2], 0u, 0x4420)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[2], 0u, 0x4431)), b0, b1);
+                    mma_f16_16816(ot[2 * j + 1], e4m3x2_to_f16x2(__byte_perm(vf[1], 0u, 0x4420)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[1], 0u, 0x4431)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[3], 0u, 0x4420)),
+                                  e4m3x2_to_f16x2(__byte_perm(vf[3], 0u, 0x4431)), b0, b1);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < D / 16; ++j) {
+                    uint32_t vf[4];
+                    ldmatrix_x4_trans(vf, vp + j * 32);
+                    mma_bf16_16816(ot[j], vf[0], vf[1], vf[2], vf[3], b0, b1);
+                }
             }
         };
         if (nch <= NW * ST) {
@@ -436,10 +482,18 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         // the warp's result block [head][D + 8] (its own first stage), as the head-major form leaves it
         __syncwarp();  // every lane is done with stage 0
         float* ow = reinterpret_cast<float*>(wst);
+        if (F8) {  // rows of a block: even d's then odd d's (see the V product); the head's V scale joins here
+            const float vs = kv_scale_of(a.kv.v_scale, a.kv, layer, hm);
 #pragma unroll
-        for (int j = 0; j < D / 16; ++j) {
-            ow[quad * (D + 8) + 16 * j + grp] = ot[j][0] + ot[j][1];
-            ow[quad * (D + 8) + 16 * j + 8 + grp] = ot[j][2] + ot[j][3];
+            for (int j = 0; j < D / 16; ++j)
+                *reinterpret_cast<float2*>(ow + quad * (D + 8) + 16 * j + 2 * grp) =
+                    make_float2((ot[j][0] + ot[j][1]) * vs, (ot[j][2] + ot[j][3]) * vs);
+        } else {
+#pragma unroll
+            for (int j = 0; j < D / 16; ++j) {
+                ow[quad * (D + 8) + 16 * j + grp] = ot[j][0] + ot[j][1];
+                ow[quad * (D + 8) + 16 * j + 8 + grp] = ot[j][2] + ot[j][3];
+            }
         }
         if (grp == 0) wml[warp * 8 + quad] = make_float2(M, L);
     } else if (nch <= NW * ST) {
