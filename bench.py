@@ -38,7 +38,7 @@ IMPL_NAMES = {1: "generic", 3: "tcgen05 two-sweep", 4: "tcgen05 score-cache",
 NCU_TRAFFIC = {
     "cfg2_8b_32k": {
         "verify": (134.38e6 + 3.77e6, "ncu, profiles/verify_cached_cfg2_32k.md"),
-        "draft": (8.51e6, "ncu, profiles/draft_stream_cfg2_budget2048.md"),
+        "draft": (8.54e6, "ncu, profiles/draft_stream_cfg2_budget2048.md"),
     },
 }
 
