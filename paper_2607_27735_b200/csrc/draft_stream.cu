@@ -16,6 +16,7 @@
 // asynchronous distributed-shared-memory stores counted on an mbarrier; it merges them in rank
 // order, so the result is deterministic.  One launch per call, no global scratch.
 #include "spec_common.cuh"
+#include <type_traits>
 #include "draft_common.cuh"
 
 namespace spec {
@@ -605,25 +606,55 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
         if (remote) st_async_f32(mine_r + 4 * i, v, bar_r);
         else mine[i] = v;
     };
-    for (int e = tid; e < G * D; e += NT) {
-        const int r = e / D, d = e - r * D;
-        float Mc = kNegBig;
+    // V neighbouring d of a head per thread: the warps' weights are computed once for all of them, and a remote
+    // deposit is one vector store (a store into another CTA's shared memory costs the same for 4 to 16 bytes)
+    auto merge_warps = [&](auto vec) {
+        constexpr int V = decltype(vec)::value;
+        for (int i = tid; i < G * (D / V); i += NT) {
+            const int r = i / (D / V), d = V * (i - r * (D / V));
+            float2 ml[NW];
+            float Mc = kNegBig;
 #pragma unroll
-        for (int w = 0; w < NW; ++w) Mc = fmaxf(Mc, wml[w * 8 + r].x);
-        float Lc = 0.f, oc = 0.f;
+            for (int w = 0; w < NW; ++w) {
+                ml[w] = wml[w * 8 + r];
+                Mc = fmaxf(Mc, ml[w].x);
+            }
+            float Lc = 0.f, o[V];
 #pragma unroll
-        for (int w = 0; w < NW; ++w) {  // fixed order: deterministic
-            const float2 ml = wml[w * 8 + r];
-            const float wgt = ex2f(ml.x - Mc);
-            Lc += ml.y * wgt;
-            oc += reinterpret_cast<const float*>(stages + (size_t)w * ST * STAGE)[r * (D + 8) + d] * wgt;
+            for (int k = 0; k < V; ++k) o[k] = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {  // fixed order: deterministic
+                const float wgt = ex2f(ml[w].x - Mc);
+                const float* ov = reinterpret_cast<const float*>(stages + (size_t)w * ST * STAGE) + r * (D + 8) + d;
+                Lc += ml[w].y * wgt;
+                if (V == 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(ov);
+                    o[0] += x.x * wgt;
+                    o[1] += x.y * wgt;
+                    o[V - 2] += x.z * wgt;
+                    o[V - 1] += x.w * wgt;
+                } else {
+                    const float2 x = *reinterpret_cast<const float2*>(ov);
+                    o[0] += x.x * wgt;
+                    o[1] += x.y * wgt;
+                }
+            }
+            if (V == 4) {
+                if (remote) st_async_f32x4(mine_r + 4 * (r * D + d), make_float4(o[0], o[1], o[V - 2], o[V - 1]), bar_r);
+                else *reinterpret_cast<float4*>(mine + r * D + d) = make_float4(o[0], o[1], o[V - 2], o[V - 1]);
+            } else {
+                if (remote) st_async_f32x2(mine_r + 4 * (r * D + d), o[0], o[1], bar_r);
+                else *reinterpret_cast<float2*>(mine + r * D + d) = make_float2(o[0], o[1]);
+            }
+            if (d == 0) {
+                put(G * D + r, Mc);
+                put(G * D + G + r, Lc);
+            }
         }
-        put(e, oc);
-        if (d == 0) {
-            put(G * D + r, Mc);
-            put(G * D + G + r, Lc);
-        }
-    }
+    };
+    // a CTA's slot is G (D + 2) floats: its rows start on 16 bytes for an even G, on 8 bytes otherwise
+    if (G % 2 == 0) merge_warps(std::integral_constant<int, 4>{});
+    else merge_warps(std::integral_constant<int, 2>{});
     if (remote) return;
     if (CS > 1) wait_deposits(smem_addr(dep_bar), a.wait_limit, status);
     __syncthreads();  // this CTA's own slot
