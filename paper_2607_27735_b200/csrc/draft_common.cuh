@@ -118,7 +118,7 @@ __device__ __forceinline__ void wait_deposits(uint32_t bar, long long limit, int
 }
 
 // Merge of the cluster's partial results in the first CTA, in rank order (deterministic), and the
-// store of the normalised output rows.  comb: [cs][G * (D + 2)] = O rows [G][D], maxima [G], sums [G].
+// store of the normalised output rows.  comb: [cs][G * (D + 2)] = O rows [G][D], then (maximum, sum) per head.
 template <int D, int NT>
 __device__ __forceinline__ void merge_and_store(const DraftArgs& a, const float* comb, int CS, int G, int layer, int b,
                                                 int h, int tid)
@@ -126,27 +126,25 @@ __device__ __forceinline__ void merge_and_store(const DraftArgs& a, const float*
     const int PS = G * (D + 2);
     for (int i = tid; i < G * (D / 2); i += NT) {
         const int r = i / (D / 2), dp = i - r * (D / 2);
-        float Mc[kMaxCluster], Lc[kMaxCluster];
-        float2 oc[kMaxCluster];
+        float2 ml[kMaxCluster], oc[kMaxCluster];
 #pragma unroll
         for (int c = 0; c < kMaxCluster; ++c) {  // every load is in flight before the first is used
             if (c < CS) {
                 const float* pc = comb + c * PS;
-                Mc[c] = pc[G * D + r];
-                Lc[c] = pc[G * D + G + r];
+                ml[c] = *(reinterpret_cast<const float2*>(pc + G * D) + r);
                 oc[c] = *(reinterpret_cast<const float2*>(pc + r * D) + dp);
             }
         }
         float M = kNegBig;
 #pragma unroll
         for (int c = 0; c < kMaxCluster; ++c)
-            if (c < CS) M = fmaxf(M, Mc[c]);
+            if (c < CS) M = fmaxf(M, ml[c].x);
         float Lsum = 0.f, o0 = 0.f, o1 = 0.f;
 #pragma unroll
         for (int c = 0; c < kMaxCluster; ++c) {
-            if (c < CS && Lc[c] > 0.f) {
-                const float wgt = ex2f(Mc[c] - M);
-                Lsum += Lc[c] * wgt;
+            if (c < CS && ml[c].y > 0.f) {
+                const float wgt = ex2f(ml[c].x - M);
+                Lsum += ml[c].y * wgt;
                 o0 += oc[c].x * wgt;
                 o1 += oc[c].y * wgt;
             }

@@ -96,7 +96,7 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     uint32_t* rowoff = reinterpret_cast<uint32_t*>(smem + (size_t)NW * ST * STAGE);
     float2* wml = reinterpret_cast<float2*>(rowoff + per);        // [NW][8]
     uint64_t* dep_bar = reinterpret_cast<uint64_t*>(wml + NW * 8);
-    float* comb = reinterpret_cast<float*>(dep_bar + 2);          // [cs][PS]: O rows [G][D], maxima [G], sums [G]
+    float* comb = reinterpret_cast<float*>(dep_bar + 2);          // [cs][PS]: O rows [G][D], then (maximum, sum) per head
 
     const int CS = gridDim.x, rank = blockIdx.x, h = blockIdx.y;
     const int layer = blockIdx.z / a.kv.batch, b = blockIdx.z % a.kv.batch;
@@ -602,10 +602,6 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
     float* mine = comb + rank * PS;
     const uint32_t mine_r = remote ? map_to_rank(smem_addr(mine), 0) : 0u;
     const uint32_t bar_r = remote ? map_to_rank(smem_addr(dep_bar), 0) : 0u;
-    auto put = [&](int i, float v) {
-        if (remote) st_async_f32(mine_r + 4 * i, v, bar_r);
-        else mine[i] = v;
-    };
     // V neighbouring d of a head per thread: the warps' weights are computed once for all of them, and a remote
     // deposit is one vector store (a store into another CTA's shared memory costs the same for 4 to 16 bytes)
     auto merge_warps = [&](auto vec) {
@@ -646,9 +642,9 @@ draft_stream_kernel(DraftArgs a, StreamShape shp, int* __restrict__ status)
                 if (remote) st_async_f32x2(mine_r + 4 * (r * D + d), o[0], o[1], bar_r);
                 else *reinterpret_cast<float2*>(mine + r * D + d) = make_float2(o[0], o[1]);
             }
-            if (d == 0) {
-                put(G * D + r, Mc);
-                put(G * D + G + r, Lc);
+            if (d == 0) {  // (maximum, sum) of the head: one store
+                if (remote) st_async_f32x2(mine_r + 4 * (G * D + 2 * r), Mc, Lc, bar_r);
+                else *reinterpret_cast<float2*>(mine + G * D + 2 * r) = make_float2(Mc, Lc);
             }
         }
     };
