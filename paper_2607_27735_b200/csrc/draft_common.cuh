@@ -42,14 +42,9 @@ __device__ __forceinline__ void cp_async_wait()
 {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-// 4 bytes into the shared memory of another CTA of the cluster; the bytes are counted on that
-// CTA's mbarrier when they have landed (no fence, no cluster barrier needed on either side)
-__device__ __forceinline__ void st_async_f32(uint32_t remote_addr, float v, uint32_t remote_bar)
-{
-    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
-                 ::"r"(remote_addr), "r"(__float_as_uint(v)), "r"(remote_bar) : "memory");
-}
-// the same for two neighbouring floats (the address a multiple of 8)
+// Stores into the shared memory of another CTA of the cluster; the bytes are counted on that CTA's
+// mbarrier when they have landed (no fence, no cluster barrier needed on either side).
+// Two neighbouring floats (the address a multiple of 8):
 __device__ __forceinline__ void st_async_f32x2(uint32_t remote_addr, float v0, float v1, uint32_t remote_bar)
 {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];"
