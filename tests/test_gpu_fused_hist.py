@@ -75,3 +75,26 @@ def test_counts_that_do_not_cover_the_span_fall_back_to_the_sweep():
     o_idx, o_n = oracle.select_recall(stats.cpu(), sel.cpu(), 4, 64, 512)
     assert torch.equal(fused[0].cpu(), o_idx) and torch.equal(fused[1].cpu(), o_n)
     assert int(hist.abs().sum()) == 0
+
+
+@pytest.mark.parametrize("head_dim", [128, 64])
+def test_fused_histogram_over_an_8bit_cache(head_dim):
+    """The same pair over an e4m3 cache: the score-cache kernel's 8-bit instances count in their statistic
+    pass (head_dim 128: tiles expanded in shared memory; head_dim 64: the bf16 expansion in the workspace)."""
+    cfg = inputs.small_config(ctx=(900, 2600), n_q=9, batch=2, n_layers=2, n_q_heads=8, n_kv_heads=2, page_size=16,
+                              shuffled_pages=True, planted=6, k_total=256, k_recent=64, head_dim=head_dim)
+    case = inputs.make_case(cfg, device="cuda")
+    kv8 = inputs.quantize_kv_fp8(case.kv)
+    T = int(case.ctx_len.max())
+    hist = torch.zeros(kv8.n_layers, kv8.batch, kv8.n_kv_heads, 2048, dtype=torch.int32, device="cuda")
+    for rnd in range(2):
+        _, _, stats, ws = binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, T, score_hist=hist)
+        assert binding.read_status(ws) == 0
+        assert binding.last_verify_impl() == (binding.VERIFY_TCGEN05_CACHED if head_dim == 128
+                                              else binding.VERIFY_TCGEN05_CACHED_EXPANDED)
+        assert torch.equal(hist.cpu().to(torch.int64), bins_of(stats, case.ctx_len))
+        plain = binding.spec_select_recall(stats, case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total)
+        fused = binding.spec_select_recall(stats, case.ctx_len, cfg.k_sink, cfg.k_recent, cfg.k_total,
+                                           score_hist=hist, hist_len=case.ctx_len)
+        assert torch.equal(plain[0], fused[0]) and torch.equal(plain[1], fused[1])
+        assert int(hist.abs().sum()) == 0
