@@ -125,3 +125,19 @@ def test_fp8_cache_needs_16_byte_rows():
     with pytest.raises(binding.SpecError) as e:
         binding.spec_verify_attn(bad, case.q_verify, case.ctx_len, 100)
     assert e.value.code == -1
+
+
+def test_fp8_verify_flags_accumulate_and_bf16_output():
+    """The call's flags over an 8-bit cache: a second call with ACCUMULATE doubles the statistic, and the bf16
+    output is the fp32 output rounded to nearest even."""
+    cfg = inputs.small_config(ctx=(1200, 1200), n_q=9, n_q_heads=8, n_kv_heads=2, planted=4)
+    case = inputs.make_case(cfg, device="cuda")
+    kv8 = inputs.quantize_kv_fp8(case.kv)
+    out, lse, stats, ws = binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, 1200)
+    assert binding.last_verify_impl() == binding.VERIFY_TCGEN05_CACHED
+    once = stats.clone()
+    binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, 1200, stats=stats, workspace=ws, accumulate=True)
+    assert binding.read_status(ws) == 0
+    assert torch.equal(stats, once + once)
+    o16, _, _, _ = binding.spec_verify_attn(kv8, case.q_verify, case.ctx_len, 1200, out_bf16=True)
+    assert torch.equal(o16, out.to(torch.bfloat16))
